@@ -1,0 +1,132 @@
+/*
+ * darkattn.h -- C ABI of libdarkattn: random-feature attention for the data-aligned softmax kernel
+ * exp(q^T Sigma k), Sigma = M^T M (DARKFormer, Section 4.1), on NVIDIA B200 (sm_100a).
+ *
+ * What the library computes, per batch b and head h (Q,K in R^{N x d}, V in R^{N x dv},
+ * M_h in R^{r x d}, W in R^{m x r} with Gaussian rows w_l, s = sqrt(scale)):
+ *
+ *   x~      = s * M_h x                      re-embedding x -> Mx (Section 4.1; Appendix C)
+ *   phi(x)_l = exp(w_l . x~ - |x~|^2 / 2)    positive random feature for omega~_l = M^T w_l ~ N(0,Sigma)
+ *                                            (Section 4.1 feature map; Appendix B reparametrisation)
+ *   O_i     = sum_j phi(q_i).phi(k_j) v_j / sum_j phi(q_i).phi(k_j)
+ *                                            evaluated as phi(Q) (phi(K)^T V), never forming N x N
+ *                                            (Section 2, "Efficient Attention via Random Feature Kernels")
+ *   causal: the sums run over j <= i; they are evaluated as a chunked prefix scan.
+ *
+ * The common factor 1/sqrt(m) of the feature map and every stabilising shift of the exponent cancel
+ * in O and are not observable through this interface.
+ *
+ * All tensor arguments are DEVICE pointers to contiguous arrays, last index fastest, base address
+ * aligned to 16 bytes. The caller owns every buffer, including `workspace` and `saved`; the library
+ * allocates no device memory and keeps no pointer after a call returns. Calls are asynchronous on the
+ * given CUDA stream and never synchronise it (except darkattn_last_device_status). Argument errors are
+ * reported on the host before anything is launched. There is no CPU fallback.
+ *
+ *   Q, K, dQ, dK   [B, H, N, d]      desc.dtype
+ *   V, O, dO, dV   [B, H, N, dv]     desc.dtype
+ *   M              [H, r, d]         desc.dtype   (row a of M_h produces coordinate a of M_h x)
+ *   W              [m, r]            desc.dtype   (or [H, m, r] when desc.w_per_head != 0)
+ *   dM             [H, r, d]         float32, OVERWRITTEN (summed over the batch inside the call)
+ */
+#ifndef DARKATTN_H_
+#define DARKATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DARKATTN_OK = 0,
+    DARKATTN_ERR_INVALID_ARG = 1,  /* null pointer, non-positive size, misaligned pointer            */
+    DARKATTN_ERR_UNSUPPORTED = 2,  /* shape / dtype / path combination that no kernel here covers     */
+    DARKATTN_ERR_WORKSPACE = 3,    /* workspace pointer missing although workspace_bytes() > 0        */
+    DARKATTN_ERR_CUDA = 4,         /* a CUDA runtime or driver call failed (see darkattn_last_cuda_error) */
+    DARKATTN_ERR_TIMEOUT = 5,      /* a bounded device-side wait gave up (device status word)         */
+    DARKATTN_ERR_NONFINITE = 6     /* reserved: non-finite normaliser seen by a checking build        */
+} darkattn_status_t;
+
+typedef enum { DARKATTN_F32 = 0, DARKATTN_BF16 = 1 } darkattn_dtype_t;
+
+/* Which kernels carry the work.
+ *   AUTO   : F32 -> SIMT; BF16 -> TENSOR where the shape is covered, else SIMT.
+ *   SIMT   : FP32 FFMA kernels with FP32 accumulation (any shape; the only path that meets the
+ *            1e-4 tolerance, because TF32/BF16 operands round the exponent's argument).
+ *   TENSOR : tcgen05 / TMEM / TMA kernels, BF16 operands, FP32 accumulation (BF16 dtype only;
+ *            DARKATTN_ERR_UNSUPPORTED at plan time if the shape is not covered).               */
+typedef enum { DARKATTN_PATH_AUTO = 0, DARKATTN_PATH_SIMT = 1, DARKATTN_PATH_TENSOR = 2 } darkattn_path_t;
+
+typedef struct {
+    int32_t B, H, N;      /* batch, heads, sequence length (all >= 1)                              */
+    int32_t d;            /* query/key width                                                       */
+    int32_t r;            /* rows of M (r <= d in the paper; any r >= 1 accepted); 0 means r = d   */
+    int32_t m;            /* number of random features                                             */
+    int32_t dv;           /* value width; 0 means dv = d                                           */
+    int32_t dtype;        /* darkattn_dtype_t of Q,K,V,M,W,O,dO,dQ,dK,dV                            */
+    int32_t causal;       /* 0: every key; 1: keys j <= i                                          */
+    int32_t chunk;        /* causal chunk length of the prefix scan; 0 means 128                   */
+    float   scale;        /* multiplies q^T Sigma k; 0 means 1/sqrt(d) (Section 2 footnote: the
+                             scaling is absorbed symmetrically, sqrt(scale) into Mq and into Mk)   */
+    int32_t w_per_head;   /* 0: W [m,r] shared by all heads; 1: W [H,m,r]                          */
+    int32_t path;         /* darkattn_path_t                                                       */
+} darkattn_desc_t;
+
+typedef struct darkattn_plan_s *darkattn_plan_t;
+
+/* Validate a descriptor and fix the kernel selection and the workspace layout. Host only: touches
+ * no GPU state. On success *out owns a small host object; release it with darkattn_destroy.     */
+darkattn_status_t darkattn_plan(const darkattn_desc_t *desc, darkattn_plan_t *out);
+
+/* Bytes of device scratch the caller must pass as `workspace` to forward / backward (the larger of
+ * the two needs). Contents need not be preserved between calls.                                  */
+size_t darkattn_workspace_bytes(darkattn_plan_t plan);
+
+/* Bytes of the forward->backward stash (`saved`). 0 means backward recomputes what it needs and
+ * `saved` may be NULL in both calls.                                                             */
+size_t darkattn_saved_bytes(darkattn_plan_t plan);
+
+/* The path (DARKATTN_PATH_SIMT or DARKATTN_PATH_TENSOR) the plan resolved to.                   */
+int32_t darkattn_plan_path(darkattn_plan_t plan);
+
+/* Number of kernel launches one forward (which = 0) or one backward (which = 1) call enqueues.  */
+int32_t darkattn_plan_launches(darkattn_plan_t plan, int32_t which);
+
+/* O = normalised random-feature attention (formulas at the top of this file).                   */
+darkattn_status_t darkattn_forward(darkattn_plan_t plan, const void *Q, const void *K, const void *V,
+                                   const void *M, const void *W, void *O, void *saved /* nullable */,
+                                   void *workspace, void *cuda_stream);
+
+/* Gradients of L = sum(dO .* O) with respect to Q, K, V and M (the paper learns M by
+ * back-propagation, Section 4; the formulas follow from the chain rule through the definitions at
+ * the top of this file, with every stabilising shift held constant, which is exact because O does
+ * not depend on them). `O` is the forward result for the same inputs (may be NULL: recomputed).  */
+darkattn_status_t darkattn_backward(darkattn_plan_t plan, const void *Q, const void *K, const void *V,
+                                    const void *M, const void *W, const void *O, const void *dO,
+                                    const void *saved /* nullable */, void *dQ, void *dK, void *dV,
+                                    float *dM, void *workspace, void *cuda_stream);
+
+/* Synchronise `cuda_stream`, then read the device status word kept at the start of `workspace`
+ * (written by kernels whose bounded waits gave up). Returns DARKATTN_OK, DARKATTN_ERR_TIMEOUT or
+ * DARKATTN_ERR_CUDA.                                                                             */
+darkattn_status_t darkattn_last_device_status(darkattn_plan_t plan, const void *workspace,
+                                              void *cuda_stream);
+
+void darkattn_destroy(darkattn_plan_t plan);
+const char *darkattn_status_string(darkattn_status_t status);
+/* Text of the last CUDA error this thread's calls into the library ran into ("" if none).       */
+const char *darkattn_last_cuda_error(void);
+
+/* Measure this GPU's throughput of the two ALU resources the feature map leans on, so that the
+ * exponent leg of the roofline has a measured denominator: which = 0 -> ex2.approx.f32 (MUFU),
+ * which = 1 -> FP32 FMA. Launches a register-only kernel on every SM `iters` times on `cuda_stream`,
+ * times it with CUDA events and writes operations per second to *ops_per_second (host pointer).
+ * Synchronises the stream.                                                                        */
+darkattn_status_t darkattn_measure_alu_peak(int32_t which, int32_t iters, double *ops_per_second,
+                                            void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DARKATTN_H_ */

@@ -1,0 +1,95 @@
+// Internal declarations shared by the translation units of libdarkattn.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "darkattn.h"
+
+namespace darkattn {
+
+// Resolved problem description (defaults filled in).
+struct Dims {
+    int B, H, N, d, r, m, dv;
+    int BH;          // B * H
+    int C;           // causal chunk length
+    int nc;          // number of chunks = ceil(N / C)   (1 when not causal)
+    int Npad;        // nc * C when causal, else N
+    int dva;         // dv + 1: values with a ones column appended (its sums are the normaliser)
+    int causal;
+    int bf16;        // storage type of the tensors is bf16
+    int w_per_head;
+    float s;         // sqrt(scale), applied to Mq and to Mk
+};
+
+// Offsets (bytes) into the caller's workspace of the SIMT path's intermediates.
+struct SimtLayout {
+    size_t status;                 // device status word (first 256 bytes)
+    size_t Qf, Kf, Vf, Mf, Wf, Gf; // fp32 copies of bf16 inputs (unused for f32 storage)
+    size_t xtQ, xtK;               // x~            [BH, N, r]
+    size_t nQ, nK;                 // |x~|^2 / 2    [BH, N]
+    size_t fQ, fK;                 // exponents, then features  [BH, Npad, m]
+    size_t cK;                     // per-feature key shift     [BH, m]
+    size_t Va;                     // [V | 1]       [BH, Npad, dva]
+    size_t Sloc;                   // chunk states, then exclusive prefixes [BH, nc, m, dva]
+    size_t P;                      // masked intra-chunk kernel  [BH, nc, C, C]   (causal)
+    size_t num;                    // numerators and normaliser  [BH, Npad, dva]
+    // backward only
+    size_t Ga;                     // [dO/den | -delta/den]      [BH, Npad, dva]
+    size_t dP;                     // [BH, nc, C, C]             (causal)
+    size_t Rloc;                   // reverse states             [BH, nc, m, dva]
+    size_t dA, dBf;                // feature gradients, then E  [BH, Npad, m]
+    size_t dVa;                    // [BH, Npad, dva]
+    size_t esQ, esK;               // rowsum(E)                  [BH, N]
+    size_t dxtQ, dxtK;             // dx~                        [BH, N, r]
+    size_t dXf;                    // fp32 dX before the cast    [BH, N, d]
+    size_t dMp;                    // per-(b,h) dM               [BH, r, d]
+    size_t fwd_bytes, total_bytes;
+};
+
+}  // namespace darkattn
+
+struct darkattn_plan_s {
+    darkattn_desc_t desc;
+    darkattn::Dims dims;
+    int path;                      // resolved DARKATTN_PATH_*
+    darkattn::SimtLayout simt;
+    size_t workspace_bytes;
+    size_t saved_bytes;
+    int launches_fwd, launches_bwd;
+};
+
+namespace darkattn {
+
+void set_cuda_error(cudaError_t e, const char *where);
+
+// SIMT (FP32 FFMA) path
+void simt_make_layout(darkattn_plan_s *plan);
+darkattn_status_t simt_forward(const darkattn_plan_s *plan, const void *Q, const void *K, const void *V,
+                               const void *M, const void *W, void *O, char *ws, cudaStream_t st,
+                               bool keep_for_backward);
+darkattn_status_t simt_backward(const darkattn_plan_s *plan, const void *Q, const void *K, const void *V,
+                                const void *M, const void *W, const void *dO, void *dQ, void *dK,
+                                void *dV, float *dM, char *ws, cudaStream_t st);
+
+// Tensor-core (tcgen05 / TMEM / TMA) path, bf16 operands with fp32 accumulation
+bool tensor_supported(const darkattn_plan_s *plan);
+void tensor_make_layout(darkattn_plan_s *plan);
+darkattn_status_t tensor_forward(const darkattn_plan_s *plan, const void *Q, const void *K, const void *V,
+                                 const void *M, const void *W, void *O, char *ws, cudaStream_t st);
+darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, const void *K, const void *V,
+                                  const void *M, const void *W, const void *dO, void *dQ, void *dK,
+                                  void *dV, float *dM, char *ws, cudaStream_t st);
+
+#define DARKATTN_CUDA_TRY(expr, where)                                   \
+    do {                                                                 \
+        cudaError_t e__ = (expr);                                        \
+        if (e__ != cudaSuccess) {                                        \
+            ::darkattn::set_cuda_error(e__, where);                      \
+            return DARKATTN_ERR_CUDA;                                    \
+        }                                                                \
+    } while (0)
+
+}  // namespace darkattn

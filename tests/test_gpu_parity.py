@@ -1,0 +1,116 @@
+"""Element-wise parity of the CUDA path (through the C ABI) with the float64 oracle."""
+import numpy as np
+import pytest
+
+from oracle import ref
+from paper_2603_04127_b200 import inputs
+from tests.util import TOL, assert_close, run_gpu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2603_04127_b200 import binding as b
+    return b
+
+
+def _oracle(t, wl, scale=None, backward=None):
+    out = {"O": ref.forward(t.Q, t.K, t.V, t.M, t.W, causal=wl.causal, scale=scale)}
+    if wl.backward if backward is None else backward:
+        dQ, dK, dV, dM, _ = ref.backward(t.Q, t.K, t.V, t.M, t.W, t.dO, causal=wl.causal, scale=scale)
+        out.update(dQ=dQ, dK=dK, dV=dV, dM=dM)
+    return out
+
+
+def _compare(got, want, tol, tag):
+    for k in want:
+        assert_close(got[k], want[k], tol, f"{tag}:{k}")
+
+
+def test_c1_fp32_noncausal_forward(binding):
+    wl = inputs.WORKLOADS["c1"]
+    t = inputs.generate(wl)
+    _compare(run_gpu(binding, wl, t), _oracle(t, wl), TOL["f32"], "c1")
+
+
+SMALL = [
+    # name, kwargs: sizes span several 64-wide tiles and ragged tails
+    ("nc_ragged", dict(B=2, H=3, N=200, d=48, m=80, causal=False)),
+    ("nc_lowrank", dict(B=1, H=2, N=130, d=64, m=96, r=24, dv=40, causal=False)),
+    ("causal_ragged", dict(B=2, H=2, N=333, d=32, m=72, causal=True)),
+    ("causal_lowrank", dict(B=1, H=3, N=257, d=64, m=64, r=16, dv=72, causal=True)),
+    ("one_token", dict(B=1, H=1, N=1, d=8, m=8, causal=True)),
+    ("one_chunk", dict(B=1, H=2, N=128, d=64, m=128, causal=True)),
+]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("name,kw", SMALL, ids=[s[0] for s in SMALL])
+def test_small_shapes_forward_backward_simt(binding, name, kw, dtype):
+    wl = inputs.small(name=name, wid=20 + len(name), dtype=dtype, backward=True, **kw)
+    t = inputs.generate(wl)
+    got = run_gpu(binding, wl, t, path=binding.PATH_SIMT)
+    _compare(got, _oracle(t, wl), TOL[dtype], name)
+
+
+@pytest.mark.parametrize("chunk", [16, 64, 256])
+def test_chunk_length_does_not_change_the_result(binding, chunk):
+    wl = inputs.small(name="chunks", wid=31, B=1, H=2, N=300, d=32, m=64, causal=True, dtype="f32")
+    t = inputs.generate(wl)
+    _compare(run_gpu(binding, wl, t, chunk=chunk), _oracle(t, wl), TOL["f32"], f"chunk{chunk}")
+
+
+def test_explicit_scale_and_per_head_projections(binding):
+    wl = inputs.small(name="wph", wid=32, B=2, H=2, N=96, d=16, m=32, causal=True, dtype="f32")
+    t = inputs.generate(wl)
+    rng = np.random.default_rng(5)
+    t.W = rng.standard_normal((2, 32, 16)).astype(np.float32).astype(np.float64)
+    got = run_gpu(binding, wl, t, scale=0.2, w_per_head=True)
+    _compare(got, _oracle(t, wl, scale=0.2), TOL["f32"], "wph")
+
+
+def test_large_norm_inputs_stay_finite(binding):
+    # exponents far outside exp's fp32 range without the stabilising shifts
+    wl = inputs.small(name="bignorm", wid=33, B=1, H=1, N=192, d=32, m=64, causal=False, dtype="f32", backward=False)
+    t = inputs.generate(wl)
+    t.Q *= 6.0
+    t.K *= 6.0
+    got = run_gpu(binding, wl, t)
+    _compare(got, _oracle(t, wl), 5e-4, "bignorm")
+
+
+FULL = {
+    # workload -> (b, h) pairs checked against the oracle at full sequence length
+    "c2": [(0, 0), (3, 7), (7, 11)],
+    "c3": [(0, 0), (3, 15)],
+    "c4": [(0, 0), (0, 7)],
+}
+
+
+@pytest.mark.parametrize("name", list(FULL))
+def test_full_size_forward_sampled_heads(binding, name):
+    wl = inputs.WORKLOADS[name]
+    t = inputs.generate(wl)
+    got = run_gpu(binding, wl, t)["O"]
+    sub = inputs.generate(wl, pairs=FULL[name])
+    want = _oracle(sub, wl)["O"]
+    for i, (b, h) in enumerate(FULL[name]):
+        assert_close(got[b, h], want[i, 0], TOL[wl.dtype], f"{name}[{b},{h}]")
+
+
+def test_c5_training_step(binding):
+    wl = inputs.WORKLOADS["c5"]
+    B, H = wl.B, wl.H
+    t = inputs.generate(wl)
+    got = run_gpu(binding, wl, t)
+    # the gradient of M_h sums over the batch: check two heads over every batch entry
+    for h in (0, H - 1):
+        pairs = [(b, h) for b in range(B)]
+        sub = inputs.generate(wl, pairs=pairs)
+        sub.M = sub.M[h:h + 1]
+        want = _oracle(sub, wl)   # B' = B pairs, H' = 1, so dM sums over them
+        for k in ("O", "dQ", "dK", "dV"):
+            g = np.stack([got[k][b, h] for b in range(B)])[:, None]
+            assert_close(g, want[k], TOL["bf16"], f"c5 head {h}: {k}")
+        assert_close(got["dM"][h], want["dM"][0], TOL["bf16"], f"c5 head {h}: dM")
