@@ -93,6 +93,7 @@ darkattn_status_t darkattn_forward(darkattn_plan_t plan, const void *Q, const vo
     if (plan->workspace_bytes && !workspace) return DARKATTN_ERR_WORKSPACE;
     if (!aligned16(workspace)) return DARKATTN_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    DARKATTN_CUDA_TRY(cudaMemsetAsync(workspace, 0, 256, st), "forward: clear status word");
     if (plan->path == DARKATTN_PATH_TENSOR)
         return tensor_forward(plan, Q, K, V, M, W, O, static_cast<char *>(workspace), st);
     return simt_forward(plan, Q, K, V, M, W, O, static_cast<char *>(workspace), st, false);
@@ -111,6 +112,7 @@ darkattn_status_t darkattn_backward(darkattn_plan_t plan, const void *Q, const v
     if (plan->workspace_bytes && !workspace) return DARKATTN_ERR_WORKSPACE;
     if (!aligned16(workspace)) return DARKATTN_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    DARKATTN_CUDA_TRY(cudaMemsetAsync(workspace, 0, 256, st), "backward: clear status word");
     if (plan->path == DARKATTN_PATH_TENSOR)
         return tensor_backward(plan, Q, K, V, M, W, dO, dQ, dK, dV, dM, static_cast<char *>(workspace), st);
     return simt_backward(plan, Q, K, V, M, W, dO, dQ, dK, dV, dM, static_cast<char *>(workspace), st);

@@ -105,13 +105,15 @@ class Tensors:
     heads: list = field(default_factory=list)   # the (b, h) pairs held, in order, when subsampled
 
 
-def generate(wl: Workload, pairs=None) -> Tensors:
+def generate(wl: Workload, pairs=None, as_batch: bool = False) -> Tensors:
     """Generate the tensors of a workload.
 
     Each (b, h) slice has its own random stream, so a subset of pairs (``pairs`` = list of (b, h))
     reproduces exactly the values the full tensor has at those positions. With ``pairs=None`` the
-    full [B,H,N,*] tensors are returned; otherwise Q,K,V,dO have shape [len(pairs),1,N,*] holding
-    the requested slices in order (M keeps all H heads).
+    full [B,H,N,*] tensors are returned. Otherwise the requested slices are returned in order as a
+    problem of their own: by default with shapes [1, P, N, *] (each pair a head, M gathered to
+    [P, r, d]); with ``as_batch`` (all pairs must name the same head h) with shapes [P, 1, N, *] and
+    M = M[h:h+1], so that a gradient of M sums over the pairs exactly as it sums over the batch.
     """
     B, H, N, d, r, m, dv = wl.dims()
     U = random_orthogonal(d, _rng(wl.wid, "U"))
@@ -139,8 +141,14 @@ def generate(wl: Workload, pairs=None) -> Tensors:
 
     if pairs is None:
         shp = lambda w: (B, H, N, w)
-    else:
+    elif as_batch:
+        hs = {h for _, h in use}
+        assert len(hs) == 1, "as_batch needs pairs of one head"
         shp = lambda w: (len(use), 1, N, w)
+        M = M[[next(iter(hs))]]
+    else:
+        shp = lambda w: (1, len(use), N, w)
+        M = M[[h for _, h in use]]
     Q, K, V = Q.reshape(shp(d)), K.reshape(shp(d)), V.reshape(shp(dv))
     if dO is not None:
         dO = dO.reshape(shp(dv))

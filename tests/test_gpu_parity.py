@@ -51,7 +51,12 @@ def test_small_shapes_forward_backward_simt(binding, name, kw, dtype):
     wl = inputs.small(name=name, wid=20 + len(name), dtype=dtype, backward=True, **kw)
     t = inputs.generate(wl)
     got = run_gpu(binding, wl, t, path=binding.PATH_SIMT)
-    _compare(got, _oracle(t, wl), TOL[dtype], name)
+    want = _oracle(t, wl)
+    if name == "one_token":
+        # O_0 = V_0 whatever Q, K and M are: those gradients are exactly zero, so compare them absolutely
+        for k in ("dQ", "dK", "dM"):
+            assert np.abs(want.pop(k)).max() < 1e-12 and np.abs(got[k]).max() < TOL[dtype]
+    _compare(got, want, TOL[dtype], name)
 
 
 @pytest.mark.parametrize("chunk", [16, 64, 256])
@@ -96,7 +101,7 @@ def test_full_size_forward_sampled_heads(binding, name):
     sub = inputs.generate(wl, pairs=FULL[name])
     want = _oracle(sub, wl)["O"]
     for i, (b, h) in enumerate(FULL[name]):
-        assert_close(got[b, h], want[i, 0], TOL[wl.dtype], f"{name}[{b},{h}]")
+        assert_close(got[b, h], want[0, i], TOL[wl.dtype], f"{name}[{b},{h}]")
 
 
 def test_c5_training_step(binding):
@@ -107,8 +112,7 @@ def test_c5_training_step(binding):
     # the gradient of M_h sums over the batch: check two heads over every batch entry
     for h in (0, H - 1):
         pairs = [(b, h) for b in range(B)]
-        sub = inputs.generate(wl, pairs=pairs)
-        sub.M = sub.M[h:h + 1]
+        sub = inputs.generate(wl, pairs=pairs, as_batch=True)
         want = _oracle(sub, wl)   # B' = B pairs, H' = 1, so dM sums over them
         for k in ("O", "dQ", "dK", "dV"):
             g = np.stack([got[k][b, h] for b in range(B)])[:, None]

@@ -29,9 +29,12 @@ def test_subset_of_pairs_reproduces_full_tensor():
     wl = inputs.small(B=2, H=3, N=8, d=4, m=8, dtype="bf16", causal=True)
     full = inputs.generate(wl)
     sub = inputs.generate(wl, pairs=[(1, 2), (0, 1)])
-    assert np.array_equal(sub.Q[0, 0], full.Q[1, 2]) and np.array_equal(sub.K[1, 0], full.K[0, 1])
-    assert np.array_equal(sub.V[0, 0], full.V[1, 2]) and np.array_equal(sub.dO[1, 0], full.dO[0, 1])
-    assert np.array_equal(sub.M, full.M) and np.array_equal(sub.W, full.W)
+    assert np.array_equal(sub.Q[0, 0], full.Q[1, 2]) and np.array_equal(sub.K[0, 1], full.K[0, 1])
+    assert np.array_equal(sub.V[0, 0], full.V[1, 2]) and np.array_equal(sub.dO[0, 1], full.dO[0, 1])
+    assert np.array_equal(sub.M, full.M[[2, 1]]) and np.array_equal(sub.W, full.W)
+    bat = inputs.generate(wl, pairs=[(0, 1), (1, 1)], as_batch=True)
+    assert bat.Q.shape == (2, 1, 8, 4) and np.array_equal(bat.Q[1, 0], full.Q[1, 1])
+    assert np.array_equal(bat.M, full.M[1:2])
     # bf16 workloads hold bf16-representable values
     assert np.array_equal(inputs.round_to_bf16(full.Q).astype(np.float64), full.Q)
 
