@@ -1,0 +1,311 @@
+#!/usr/bin/env python
+"""Benchmark of the DARK-attention hot path: forward + backward tokens/s at N = 8192 on B200.
+
+One step = one forward and one backward call of the whole hot path (feature maps, chunked causal
+scan, dQ/dK/dV/dM) over one batch of the synthetic workload. Prints ONE JSON line.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload headline]
+
+N > 1 is launched under torch.distributed.run, one rank per GPU; every rank processes its own batch
+(weak scaling) and the per-head gradient of M is all-reduced over NCCL, as in data-parallel training.
+`--impl reference` times the float64 CPU oracle on the host cores (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "DARK-attention fwd+bwd tokens/s"
+UNIT = "tokens/s"
+
+
+def flops_per_token_head(d, r, m, dv, C, causal, backward):
+    """Algorithmic floating-point operations per (token, head); intra-chunk terms count the lower
+    triangle only."""
+    feat = 2 * (2 * d * r + 2 * r * m)                 # both sides: x~ = M x and u = W x~
+    fwd = feat + 4 * m * dv + ((C + 1) * (m + dv) if causal else 0)
+    if not backward:
+        return fwd
+    bwd = feat + 10 * m * dv + ((C + 1) * (3 * m + 2 * dv) if causal else 0) + 4 * m * r + 8 * r * d
+    return fwd + bwd
+
+
+def bytes_per_token_head(d, dv, backward, e=2):
+    fwd = (2 * d + 2 * dv) * e                          # Q, K, V in; O out
+    return fwd + ((4 * d + 4 * dv) * e if backward else 0)   # + Q,K,V,dO in; dQ,dK,dV out (+O)
+
+
+def exps_per_token_head(m, backward):
+    return 2 * m * (2 if backward else 1)
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid):
+        self.uuid, self.rows, self.proc = uuid, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", self.uuid, f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        self.thread.join(timeout=2)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+                for n, v in zip(names, r[4:8]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            except Exception:
+                pass
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        j = json.load(open(p))
+        return {"hbm_gbs": j["hbm_gbs"], "bf16_tflops": j["bf16_tflops"],
+                "bf16_tflops_sustained": j.get("bf16_tflops_sustained", j["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def oracle_step(ref, sub, wl):
+    ref.forward(sub.Q, sub.K, sub.V, sub.M, sub.W, causal=wl.causal)
+    if wl.backward:
+        ref.backward(sub.Q, sub.K, sub.V, sub.M, sub.W, sub.dO, causal=wl.causal)
+
+
+def oracle_sample(wl, inputs, ref):
+    cores = ref.num_threads()
+    B, H = wl.B, wl.H
+    P = max(1, min(cores, B * H, 64))
+    pairs = [((i * 7) % B, (i * 5) % H) for i in range(B * H)]
+    seen, use = set(), []
+    for p in pairs:
+        if p not in seen:
+            seen.add(p); use.append(p)
+        if len(use) == P:
+            break
+    sub = inputs.generate(wl, pairs=use)
+    return sub, use, min(cores, len(use))
+
+
+def run_reference(args, wl):
+    """The oracle, as it stands, on the host cores: each step = forward+backward of a bounded sample."""
+    from oracle import ref
+    from paper_2603_04127_b200 import inputs
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    sub, use, cores = oracle_sample(wl, inputs, ref)
+    for _ in range(args.warmup):
+        oracle_step(ref, sub, wl)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(ref, sub, wl)
+    dt = (time.perf_counter() - t0) / args.steps
+    tokens = len(use) * wl.N / wl.H                    # (token, head) pairs processed / heads per token
+    val = tokens / dt
+    sample = f"{len(use)} of {wl.B * wl.H} (batch, head) pairs at full N={wl.N}, forward+backward, float64"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(wl),
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def workload_config(wl):
+    B, H, N, d, r, m, dv = wl.dims()
+    return {"workload": f"{wl.name}: B={B} H={H} N={N} d={d} r={r} m={m} dv={dv} "
+                        f"{'causal (chunk 128)' if wl.causal else 'non-causal'} "
+                        f"{'forward+backward' if wl.backward else 'forward'} {wl.dtype}",
+            "l2": "inputs larger than L2 (Q,K,V,dO total %.0f MB)" % ((3 * B * H * N * d + B * H * N * dv) * 2 / 1e6)}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="headline")
+    ap.add_argument("--path", type=int, default=0, help="0 auto, 1 SIMT, 2 tensor")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    from paper_2603_04127_b200 import inputs
+    wl = inputs.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2603_04127_b200 import binding
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    B, H, N, d, r, m, dv = wl.dims()
+    # every rank draws its own batch (weak scaling): shift the workload id by the rank
+    wl_rank = inputs.Workload(**{**wl.__dict__, "wid": wl.wid + 100 * rank})
+    t = inputs.generate(wl_rank)
+    dt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
+
+    def host(a):
+        return torch.from_numpy(np.ascontiguousarray(a)).to(dt).pin_memory()
+
+    hQ, hK, hV, hM, hW = (host(x) for x in (t.Q, t.K, t.V, t.M, t.W))
+    hG = host(t.dO) if wl.backward else None
+    Q, K, V, M, W = (x.cuda() for x in (hQ, hK, hV, hM, hW))
+    G = hG.cuda() if wl.backward else None
+    O = torch.empty_like(V)
+    dQ, dK, dV = torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V)
+    dM = torch.empty(M.shape, dtype=torch.float32, device="cuda")
+    hO, hdQ, hdK, hdV = (torch.empty_like(x).pin_memory() for x in (hV, hQ, hK, hV))
+    hdM = torch.empty(M.shape, dtype=torch.float32).pin_memory()
+
+    plan = binding.darkattn_plan(B, H, N, d, m, r=r, dv=dv, dtype=binding.BF16 if wl.dtype == "bf16" else binding.F32,
+                                 causal=wl.causal, path=args.path)
+    ws = plan.alloc_workspace()
+    stream = torch.cuda.current_stream()
+
+    def step():
+        binding.darkattn_forward(plan, Q, K, V, M, W, O, ws, stream=stream)
+        if wl.backward:
+            binding.darkattn_backward(plan, Q, K, V, M, W, O, G, dQ, dK, dV, dM, ws, stream=stream)
+            if world > 1:
+                dist.all_reduce(dM)
+
+    def e2e_step():
+        for dst, src in ((Q, hQ), (K, hK), (V, hV), (M, hM), (W, hW)):
+            dst.copy_(src, non_blocking=True)
+        if wl.backward:
+            G.copy_(hG, non_blocking=True)
+        step()
+        hO.copy_(O, non_blocking=True)
+        if wl.backward:
+            for dst, src in ((hdQ, dQ), (hdK, dK), (hdV, dV), (hdM, dM)):
+                dst.copy_(src, non_blocking=True)
+
+    def timed(fn, steps):
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        ms = torch.tensor([e0.elapsed_time(e1)], device="cuda")
+        if world > 1:
+            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+        return float(ms.item())
+
+    for _ in range(args.warmup):
+        step()
+    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(local).uuid).replace("GPU-", ""))
+    if rank == 0:
+        sampler.start()
+    ms = timed(step, args.steps)
+    clocks = sampler.stop() if rank == 0 else None
+    fwd_ms = timed(lambda: binding.darkattn_forward(plan, Q, K, V, M, W, O, ws, stream=stream), args.steps) / args.steps
+    e2e_steps = max(2, min(args.steps, 5))
+    e2e_step()
+    e2e_ms = timed(e2e_step, e2e_steps) / e2e_steps
+    assert binding.darkattn_last_device_status(plan, ws) == binding.OK
+
+    ms_step = ms / args.steps
+    tokens = B * N
+    value = world * tokens / (ms_step * 1e-3)
+    h2d = sum(x.numel() * x.element_size() for x in (hQ, hK, hV, hM, hW) + ((hG,) if wl.backward else ()))
+    d2h = hO.numel() * hO.element_size() + (sum(x.numel() * x.element_size() for x in (hdQ, hdK, hdV, hdM)) if wl.backward else 0)
+
+    peaks = measured_peaks()
+    th = B * H * N
+    flops = flops_per_token_head(d, r, m, dv, 128, wl.causal, wl.backward) * th
+    nbytes = bytes_per_token_head(d, dv, wl.backward) * th
+    nexp = exps_per_token_head(m, wl.backward) * th
+    ex2_peak = binding.darkattn_measure_alu_peak(0, 10)
+    fma_peak = binding.darkattn_measure_alu_peak(1, 10)
+    legs = {"tensor_us": flops / (peaks["bf16_tflops_sustained"] * 1e12) * 1e6,
+            "exp_us": nexp / ex2_peak * 1e6, "hbm_us": nbytes / (peaks["hbm_gbs"] * 1e9) * 1e6}
+    achieved_tf = flops / (ms_step * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "achieved": achieved_tf, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                "frac": achieved_tf / peaks["bf16_tflops_sustained"], "traffic": None,
+                "kernel": "whole step (forward + backward call)", "peak_source": peaks["source"] + " (sustained)",
+                "legs_us": legs, "ex2_per_s_measured": ex2_peak, "fma_per_s_measured": fma_peak,
+                "forward_ms": fwd_ms, "forward_tokens_per_s": world * tokens / (fwd_ms * 1e-3)}
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype,
+        "data": "synthetic", "config": {**workload_config(wl), "path": {1: "simt", 2: "tensor"}[plan.path]},
+        "clocks": clocks,
+        "e2e": {"value": world * tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h},
+        "gpu_launches": args.steps * (plan.launches(False) + (plan.launches(True) if wl.backward else 0)),
+        "roofline": roofline,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import ref
+        sub, use, cores = oracle_sample(wl, inputs, ref)
+        t0 = time.perf_counter()
+        reps = 2
+        for _ in range(reps):
+            oracle_step(ref, sub, wl)
+        dtc = (time.perf_counter() - t0) / reps
+        out["cpu_baseline"] = {"value": len(use) * N / H / dtc, "unit": UNIT, "cores": cores, "kind": "oracle",
+                               "sample": f"{len(use)} of {B * H} (batch, head) pairs at full N={N}, "
+                                         f"{'forward+backward' if wl.backward else 'forward'}, float64, {reps} repetitions"}
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
