@@ -42,7 +42,7 @@ typedef enum {
     DARKATTN_OK = 0,
     DARKATTN_ERR_INVALID_ARG = 1,  /* null pointer, non-positive size, misaligned pointer            */
     DARKATTN_ERR_UNSUPPORTED = 2,  /* shape / dtype / path combination that no kernel here covers     */
-    DARKATTN_ERR_WORKSPACE = 3,    /* workspace pointer missing although workspace_bytes() > 0        */
+    DARKATTN_ERR_WORKSPACE = 3,    /* workspace missing, or too small a built-in one (forward_static) */
     DARKATTN_ERR_CUDA = 4,         /* a CUDA runtime or driver call failed (see darkattn_last_cuda_error) */
     DARKATTN_ERR_TIMEOUT = 5,      /* a bounded device-side wait gave up (device status word)         */
     DARKATTN_ERR_NONFINITE = 6     /* reserved: non-finite normaliser seen by a checking build        */
@@ -125,6 +125,33 @@ const char *darkattn_last_cuda_error(void);
  * Synchronises the stream.                                                                        */
 darkattn_status_t darkattn_measure_alu_peak(int32_t which, int32_t iters, double *ops_per_second,
                                             void *cuda_stream);
+
+/* Forward pass that needs no workspace from the caller and allocates nothing.
+ *
+ * (The paper has no counterpart to this entry point; it exists for deployment reasons only.)
+ *
+ * Some hosts of this library cannot hand it scratch memory: an inference server that gave the whole
+ * GPU to its own pool at start-up and forbids cudaMalloc afterwards because it stalls every stream,
+ * a plug-in that is passed input and output buffers but has no access to its host's allocator, a
+ * latency-critical loop that must not allocate once it is running. For them this call runs the same
+ * FP32 forward as darkattn_forward on the SIMT path (any dtype, any shape, causal or not), with its
+ * intermediates in an array of DARKATTN_STATIC_SCRATCH_BYTES that is part of the library's device
+ * image: every GPU that loads the library holds that much memory until the process exits.
+ *
+ *  - The caller still passes Q, K, V, M, W (inputs) and O (output), laid out as for darkattn_forward.
+ *  - darkattn_static_scratch_needed(plan) tells how much of the array a plan would use. A plan that
+ *    needs more than DARKATTN_STATIC_SCRATCH_BYTES is refused with DARKATTN_ERR_WORKSPACE before
+ *    anything touches the GPU; use darkattn_forward with a workspace of your own for it.
+ *  - The first call on each device looks up the array's device address (with that device current).
+ *    Make that first call before any stream capture begins.
+ *  - No cudaMalloc, cudaFree or other allocating routine is called, now or later.
+ *  - All calls on a device share the one array, and it keeps the previous call's contents; the call
+ *    clears the words that must start at zero itself. Two calls whose GPU work overlaps (different
+ *    streams, or different host threads) race on the array: serialise them on one stream.         */
+#define DARKATTN_STATIC_SCRATCH_BYTES (16u << 20)
+size_t darkattn_static_scratch_needed(darkattn_plan_t plan);
+darkattn_status_t darkattn_forward_static(darkattn_plan_t plan, const void *Q, const void *K, const void *V,
+                                          const void *M, const void *W, void *O, void *cuda_stream);
 
 #ifdef __cplusplus
 }

@@ -23,7 +23,9 @@ EXPORTS = [
     "darkattn_plan", "darkattn_workspace_bytes", "darkattn_saved_bytes", "darkattn_plan_path",
     "darkattn_plan_launches", "darkattn_forward", "darkattn_backward", "darkattn_last_device_status",
     "darkattn_destroy", "darkattn_status_string", "darkattn_last_cuda_error", "darkattn_measure_alu_peak",
+    "darkattn_static_scratch_needed", "darkattn_forward_static",
 ]
+STATIC_SCRATCH_BYTES = 16 << 20
 
 
 class Desc(ctypes.Structure):
@@ -63,6 +65,10 @@ lib.darkattn_last_cuda_error.argtypes = []
 lib.darkattn_last_cuda_error.restype = ctypes.c_char_p
 lib.darkattn_measure_alu_peak.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(ctypes.c_double), _vp]
 lib.darkattn_measure_alu_peak.restype = ctypes.c_int
+lib.darkattn_static_scratch_needed.argtypes = [_vp]
+lib.darkattn_static_scratch_needed.restype = ctypes.c_size_t
+lib.darkattn_forward_static.argtypes = [_vp] * 8
+lib.darkattn_forward_static.restype = ctypes.c_int
 
 
 class DarkAttnError(RuntimeError):
@@ -158,3 +164,16 @@ def darkattn_measure_alu_peak(which: int, iters: int = 20, stream=None) -> float
     _check(lib.darkattn_measure_alu_peak(which, iters, ctypes.byref(out), _stream(stream)),
            "darkattn_measure_alu_peak")
     return out.value
+
+
+def darkattn_static_scratch_needed(plan: Plan) -> int:
+    return int(lib.darkattn_static_scratch_needed(plan.handle))
+
+
+def darkattn_forward_static(plan: Plan, Q, K, V, M, W, O, stream=None):
+    """Forward pass on the library's built-in scratch array: for callers that cannot allocate device
+    memory. Calls on one device must not overlap; problems that need more than STATIC_SCRATCH_BYTES
+    raise with status ERR_WORKSPACE."""
+    _check(lib.darkattn_forward_static(plan.handle, _ptr(Q), _ptr(K), _ptr(V), _ptr(M), _ptr(W), _ptr(O),
+                                       _stream(stream)), "darkattn_forward_static")
+    return O
