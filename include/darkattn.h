@@ -45,7 +45,7 @@ typedef enum {
     DARKATTN_ERR_WORKSPACE = 3,    /* workspace missing, or too small a built-in one (forward_static) */
     DARKATTN_ERR_CUDA = 4,         /* a CUDA runtime or driver call failed (see darkattn_last_cuda_error) */
     DARKATTN_ERR_TIMEOUT = 5,      /* a bounded device-side wait gave up (device status word)         */
-    DARKATTN_ERR_NONFINITE = 6     /* reserved: non-finite normaliser seen by a checking build        */
+    DARKATTN_ERR_NONFINITE = 6     /* a normaliser was zero or not finite (device status word)        */
 } darkattn_status_t;
 
 typedef enum { DARKATTN_F32 = 0, DARKATTN_BF16 = 1 } darkattn_dtype_t;
@@ -108,8 +108,8 @@ darkattn_status_t darkattn_backward(darkattn_plan_t plan, const void *Q, const v
                                     float *dM, void *workspace, void *cuda_stream);
 
 /* Synchronise `cuda_stream`, then read the device status word kept at the start of `workspace`
- * (written by kernels whose bounded waits gave up). Returns DARKATTN_OK, DARKATTN_ERR_TIMEOUT or
- * DARKATTN_ERR_CUDA.                                                                             */
+ * (written by kernels whose bounded waits gave up, or that met a normaliser that is zero or not
+ * finite). Returns DARKATTN_OK, DARKATTN_ERR_TIMEOUT, DARKATTN_ERR_NONFINITE or DARKATTN_ERR_CUDA.  */
 darkattn_status_t darkattn_last_device_status(darkattn_plan_t plan, const void *workspace,
                                               void *cuda_stream);
 

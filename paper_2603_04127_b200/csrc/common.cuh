@@ -49,6 +49,21 @@ struct SimtLayout {
     size_t fwd_bytes, total_bytes;
 };
 
+// Offsets (bytes) into the workspace of the tensor-core forward path.
+struct TensorLayout {
+    size_t status;
+    size_t Om;      // folded projections log2(e) s W M, bf16 [H, m, d]
+    size_t cs;      // key-side shift per (bh, slab), fp32
+    size_t nK;      // key norms, fp32 [BH, N]
+    size_t pnum;    // partial numerators, bf16 [nslab, BH, N, dv]
+    size_t pdr;     // partial normaliser and scale exponent, fp32 [nslab, BH, N, 2]
+    size_t Sacc;    // non-causal state sums, fp32 [BH, m, dv]
+    size_t zacc;    // fp32 [BH, m]
+    size_t Sb;      // bf16 copy of the state, [BH, m, dv]
+    size_t total_bytes;
+    int nslab, T, nsplit;
+};
+
 }  // namespace darkattn
 
 struct darkattn_plan_s {
@@ -56,6 +71,7 @@ struct darkattn_plan_s {
     darkattn::Dims dims;
     int path;                      // resolved DARKATTN_PATH_*
     darkattn::SimtLayout simt;
+    darkattn::TensorLayout tensor;
     size_t workspace_bytes;
     size_t saved_bytes;
     int launches_fwd, launches_bwd;

@@ -125,7 +125,9 @@ darkattn_status_t darkattn_last_device_status(darkattn_plan_t plan, const void *
     int word = 0;
     DARKATTN_CUDA_TRY(cudaStreamSynchronize(st), "last_device_status: sync");
     DARKATTN_CUDA_TRY(cudaMemcpy(&word, workspace, sizeof(int), cudaMemcpyDeviceToHost), "last_device_status: read");
-    return word == 0 ? DARKATTN_OK : DARKATTN_ERR_TIMEOUT;
+    if (word == 0) return DARKATTN_OK;
+    if (word == DARKATTN_ERR_NONFINITE || word == DARKATTN_ERR_CUDA) return (darkattn_status_t)word;
+    return DARKATTN_ERR_TIMEOUT;
 }
 
 void darkattn_destroy(darkattn_plan_t plan) { delete plan; }

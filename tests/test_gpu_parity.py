@@ -118,3 +118,37 @@ def test_c5_training_step(binding):
             g = np.stack([got[k][b, h] for b in range(B)])[:, None]
             assert_close(g, want[k], TOL["bf16"], f"c5 head {h}: {k}")
         assert_close(got["dM"][h], want["dM"][0], TOL["bf16"], f"c5 head {h}: dM")
+
+
+TENSOR = [
+    # shapes the tcgen05 kernels cover: d, dv in {64,128}; m, N multiples of 128
+    ("nc_d64_m128", dict(B=1, H=2, N=256, d=64, m=128, causal=False)),
+    ("nc_d64_m256", dict(B=2, H=3, N=640, d=64, m=256, causal=False)),
+    ("nc_d128_m256", dict(B=1, H=2, N=384, d=128, m=256, causal=False)),
+    ("nc_d64_dv128_r32", dict(B=1, H=2, N=256, d=64, m=128, dv=128, r=32, causal=False)),
+    ("c_one_chunk", dict(B=1, H=1, N=128, d=64, m=128, causal=True)),
+    ("c_d64_m128", dict(B=1, H=2, N=512, d=64, m=128, causal=True)),
+    ("c_d64_m512", dict(B=2, H=2, N=384, d=64, m=512, causal=True)),
+    ("c_d128_m256", dict(B=1, H=3, N=640, d=128, m=256, causal=True)),
+    ("c_d128_dv64_r64", dict(B=1, H=2, N=256, d=128, m=128, dv=64, r=64, causal=True)),
+]
+
+
+@pytest.mark.parametrize("name,kw", TENSOR, ids=[s[0] for s in TENSOR])
+def test_tensor_path_forward(binding, name, kw):
+    wl = inputs.small(name=name, wid=50 + len(name), dtype="bf16", backward=False, **kw)
+    t = inputs.generate(wl)
+    got = run_gpu(binding, wl, t, path=binding.PATH_TENSOR)
+    _compare(got, _oracle(t, wl), TOL["bf16"], name)
+
+
+def test_tensor_path_rejects_uncovered_shapes(binding):
+    for kw in (dict(N=200), dict(d=48), dict(m=96)):
+        a = dict(B=1, H=1, N=256, d=64, m=128)
+        a.update(kw)
+        with pytest.raises(binding.DarkAttnError) as e:
+            binding.darkattn_plan(a["B"], a["H"], a["N"], a["d"], a["m"], dtype=binding.BF16, path=binding.PATH_TENSOR)
+        assert e.value.status == binding.ERR_UNSUPPORTED
+        p = binding.darkattn_plan(a["B"], a["H"], a["N"], a["d"], a["m"], dtype=binding.BF16)   # AUTO falls back
+        assert p.path == binding.PATH_SIMT
+        p.destroy()
