@@ -60,6 +60,16 @@ struct TensorLayout {
     size_t Sacc;    // non-causal state sums, fp32 [BH, m, dv]
     size_t zacc;    // fp32 [BH, m]
     size_t Sb;      // bf16 copy of the state, [BH, m, dv]
+    size_t sv;      // per-row normaliser and the exponent it is scaled by, float2 [BH, N] (forward -> backward)
+    // backward only
+    size_t Oscr;    // forward output when backward has to recompute it, bf16 [BH, N, dv]
+    size_t delta;   // dO_i . O_i, fp32 [BH, N]
+    size_t rhoc;    // per-chunk sums -sum_i A^_il delta_i, fp32 [BH, T, m]
+    size_t pdQ, pdK; // slab partials of dQ and dK, bf16 [nslab, BH, N, d]
+    size_t pdV;     // slab partials of dV, bf16 [nslab, BH, N, dv]
+    size_t espart;  // slab partials of rowsum(E_K), fp32 [nslab, BH, N]
+    size_t Tacc;    // sum_i E_i^T x_i over both sides and the batch, fp32 [H, m, d]
+    size_t dMn;     // gradient of M through the key norm term, fp32 [H, r, d]
     size_t total_bytes;
     int nslab, T, nsplit;
 };
@@ -94,10 +104,13 @@ darkattn_status_t simt_backward(const darkattn_plan_s *plan, const void *Q, cons
 bool tensor_supported(const darkattn_plan_s *plan);
 void tensor_make_layout(darkattn_plan_s *plan);
 darkattn_status_t tensor_forward(const darkattn_plan_s *plan, const void *Q, const void *K, const void *V,
-                                 const void *M, const void *W, void *O, char *ws, cudaStream_t st);
+                                 const void *M, const void *W, void *O, void *saved, char *ws, cudaStream_t st);
+// Folded projections, key-side shifts and key norms (written to the workspace); shared by forward and backward.
+cudaError_t tensor_prologue(const darkattn_plan_s *plan, const void *K, const void *M, const void *W, char *ws,
+                            cudaStream_t st);
 darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, const void *K, const void *V,
-                                  const void *M, const void *W, const void *dO, void *dQ, void *dK,
-                                  void *dV, float *dM, char *ws, cudaStream_t st);
+                                  const void *M, const void *W, const void *O, const void *dO, const void *saved,
+                                  void *dQ, void *dK, void *dV, float *dM, char *ws, cudaStream_t st);
 
 #define DARKATTN_CUDA_TRY(expr, where)                                   \
     do {                                                                 \

@@ -86,16 +86,15 @@ darkattn_status_t darkattn_forward(darkattn_plan_t plan, const void *Q, const vo
                                    const void *M, const void *W, void *O, void *saved, void *workspace,
                                    void *cuda_stream)
 {
-    (void)saved;
     if (!plan || !Q || !K || !V || !M || !W || !O) return DARKATTN_ERR_INVALID_ARG;
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(M) || !aligned16(W) || !aligned16(O))
         return DARKATTN_ERR_INVALID_ARG;
     if (plan->workspace_bytes && !workspace) return DARKATTN_ERR_WORKSPACE;
-    if (!aligned16(workspace)) return DARKATTN_ERR_INVALID_ARG;
+    if (!aligned16(workspace) || !aligned16(saved)) return DARKATTN_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     DARKATTN_CUDA_TRY(cudaMemsetAsync(workspace, 0, 256, st), "forward: clear status word");
     if (plan->path == DARKATTN_PATH_TENSOR)
-        return tensor_forward(plan, Q, K, V, M, W, O, static_cast<char *>(workspace), st);
+        return tensor_forward(plan, Q, K, V, M, W, O, saved, static_cast<char *>(workspace), st);
     return simt_forward(plan, Q, K, V, M, W, O, static_cast<char *>(workspace), st, false);
 }
 
@@ -104,17 +103,16 @@ darkattn_status_t darkattn_backward(darkattn_plan_t plan, const void *Q, const v
                                     const void *saved, void *dQ, void *dK, void *dV, float *dM,
                                     void *workspace, void *cuda_stream)
 {
-    (void)saved; (void)O;
     if (!plan || !Q || !K || !V || !M || !W || !dO || !dQ || !dK || !dV || !dM) return DARKATTN_ERR_INVALID_ARG;
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(M) || !aligned16(W) || !aligned16(dO) ||
         !aligned16(dQ) || !aligned16(dK) || !aligned16(dV) || !aligned16(dM))
         return DARKATTN_ERR_INVALID_ARG;
     if (plan->workspace_bytes && !workspace) return DARKATTN_ERR_WORKSPACE;
-    if (!aligned16(workspace)) return DARKATTN_ERR_INVALID_ARG;
+    if (!aligned16(workspace) || !aligned16(saved) || !aligned16(O)) return DARKATTN_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     DARKATTN_CUDA_TRY(cudaMemsetAsync(workspace, 0, 256, st), "backward: clear status word");
     if (plan->path == DARKATTN_PATH_TENSOR)
-        return tensor_backward(plan, Q, K, V, M, W, dO, dQ, dK, dV, dM, static_cast<char *>(workspace), st);
+        return tensor_backward(plan, Q, K, V, M, W, O, dO, saved, dQ, dK, dV, dM, static_cast<char *>(workspace), st);
     return simt_backward(plan, Q, K, V, M, W, dO, dQ, dK, dV, dM, static_cast<char *>(workspace), st);
 }
 

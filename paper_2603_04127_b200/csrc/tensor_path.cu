@@ -26,63 +26,8 @@ namespace {
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kMaxNsplit = 64;
 
-// ------------------------------------------------------------------ driver entry point for tensor maps
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn()
-{
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
-    return fn;
-}
-
-// 2-D bf16 tensor [rows, cols] (cols contiguous), box = 64 columns x box_rows rows, 128-byte swizzle.
-bool make_map(CUtensorMap *m, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows)
-{
-    EncodeTiledFn enc = encode_fn();
-    if (!enc) return false;
-    cuuint64_t dims[2] = {cols, rows};
-    cuuint64_t strides[1] = {cols * 2};
-    cuuint32_t box[2] = {64, box_rows};
-    cuuint32_t es[2] = {1, 1};
-    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, es,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 // ------------------------------------------------------------------ small helpers
-__device__ __forceinline__ float ex2f(float x)
-{
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
 __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-
-// mbarrier wait that also gives up when another thread of the CTA already did.
-__device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, int *status, volatile int *abort_flag)
-{
-    for (int i = 0; i < 128; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_timer_ns();
-    for (;;) {
-        for (int i = 0; i < 64; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (global_timer_ns() - t0 > kWaitLimitNs) break;
-    }
-    *abort_flag = 1;
-    atomicExch(status, (int)DARKATTN_ERR_TIMEOUT);
-    return false;
-}
 
 // ------------------------------------------------------------------ prologue kernels (SIMT, tiny)
 // Omega[h,l,c] = log2(e) * s * sum_a W[l,a] M[h,a,c]  (bf16);  one block per (h, l).
@@ -563,7 +508,9 @@ __global__ void state_to_bf16_kernel(const float *S, __nv_bfloat16 *Sb, long lon
 
 // O[row,:] = sum_s num_s[row,:] 2^(rho_s - rho) / sum_s den_s 2^(rho_s - rho), rho = max_s rho_s.
 // One thread per 8 output columns.
-__global__ void combine_kernel(const __nv_bfloat16 *pnum, const float *pdr, __nv_bfloat16 *O, long long rows, int dv, int nslab)
+// The combined normaliser and rho are also written to sv (and to sv2 when given) for the backward pass.
+__global__ void combine_kernel(const __nv_bfloat16 *pnum, const float *pdr, __nv_bfloat16 *O, float2 *sv, float2 *sv2,
+                               long long rows, int dv, int nslab)
 {
     const long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;
     const int per_row = dv / 8;
@@ -585,6 +532,10 @@ __global__ void combine_kernel(const __nv_bfloat16 *pnum, const float *pdr, __nv
             acc[2 * q] = fmaf(f.x, w, acc[2 * q]);
             acc[2 * q + 1] = fmaf(f.y, w, acc[2 * q + 1]);
         }
+    }
+    if (c0 == 0) {
+        sv[row] = make_float2(den, rho);
+        if (sv2) sv2[row] = make_float2(den, rho);
     }
     const float inv = 1.f / den;
     uint4 out;
@@ -663,33 +614,37 @@ void tensor_make_layout(darkattn_plan_s *plan)
     Y.Sacc = take(off, BH * m * dv * 4);
     Y.zacc = take(off, BH * m * 4);
     Y.Sb = take(off, BH * m * dv * 2);
+    Y.sv = take(off, BH * N * 8);
+    plan->launches_fwd = D.causal ? 5 : 7;
+    plan->saved_bytes = BH * N * 8;
+    if (D.causal) {       // tensor-core backward (the non-causal backward runs on the FP32 path)
+        Y.Oscr = take(off, BH * N * dv * 2);
+        Y.delta = take(off, BH * N * 4);
+        Y.rhoc = take(off, BH * (size_t)Y.T * m * 4);
+        Y.pdQ = take(off, (size_t)Y.nslab * BH * N * d * 2);
+        Y.pdK = take(off, (size_t)Y.nslab * BH * N * d * 2);
+        Y.pdV = take(off, (size_t)Y.nslab * BH * N * dv * 2);
+        Y.espart = take(off, (size_t)Y.nslab * BH * N * 4);
+        Y.Tacc = take(off, (size_t)D.H * m * d * 4);
+        Y.dMn = take(off, (size_t)D.H * D.r * d * 4);
+        plan->launches_bwd = 3 + 1 + 2 + 3 + 1;   // prologue, delta, two scan kernels, three combines, dM
+    }
     Y.total_bytes = off;
     if (Y.total_bytes > plan->workspace_bytes) plan->workspace_bytes = Y.total_bytes;
-    plan->launches_fwd = D.causal ? 5 : 7;
 }
 
-darkattn_status_t tensor_forward(const darkattn_plan_s *plan, const void *Q, const void *K, const void *V,
-                                 const void *M, const void *W, void *O, char *ws, cudaStream_t st)
+cudaError_t tensor_prologue(const darkattn_plan_s *plan, const void *K, const void *M, const void *W, char *ws,
+                            cudaStream_t st)
 {
     const Dims &D = plan->dims;
     const TensorLayout &Y = plan->tensor;
     const size_t BH = D.BH, N = D.N;
     auto bf = [&](size_t off) { return reinterpret_cast<__nv_bfloat16 *>(ws + off); };
     auto fl = [&](size_t off) { return reinterpret_cast<float *>(ws + off); };
-    if (!encode_fn()) { set_cuda_error(cudaErrorNotSupported, "tensor_forward: cuTensorMapEncodeTiled unavailable"); return DARKATTN_ERR_CUDA; }
-
-    MainParams P;
-    memset(&P, 0, sizeof(P));
     NormParams NP;
     memset(&NP, 0, sizeof(NP));
-    bool ok = make_map(&P.mapQ, Q, BH * N, D.d, 128) && make_map(&P.mapK, K, BH * N, D.d, 128) &&
-              make_map(&P.mapV, V, BH * N, D.dv, 128) && make_map(&P.mapOm, bf(Y.Om), (size_t)D.H * D.m, D.d, 128) &&
-              make_map(&P.mapSb, bf(Y.Sb), BH * D.m, D.dv, 128) &&
-              make_map(&P.mapPN, bf(Y.pnum), (size_t)Y.nslab * BH * N, D.dv, 128) &&
-              make_map(&NP.mapM, M, (size_t)D.H * D.r, D.d, 128);
-    if (!ok) { set_cuda_error(cudaErrorInvalidValue, "tensor_forward: tensor map encode"); return DARKATTN_ERR_CUDA; }
-    NP.mapK = P.mapK;
-
+    if (!make_map(&NP.mapK, K, BH * N, D.d, 128) || !make_map(&NP.mapM, M, (size_t)D.H * D.r, D.d, 128))
+        return cudaErrorInvalidValue;
     cudaError_t e = cudaSuccess;
     auto chk = [&]() { cudaError_t x = cudaGetLastError(); if (x != cudaSuccess && e == cudaSuccess) e = x; };
 
@@ -704,17 +659,38 @@ darkattn_status_t tensor_forward(const darkattn_plan_s *plan, const void *Q, con
     NP.nsplit = (int)((148 * 2 + BH - 1) / BH);
     if (NP.nsplit > Y.T) NP.nsplit = Y.T;
     NP.coef = kLog2e * 0.5f * D.s * D.s;
-    {
-        const int smem_bytes = 2 * 128 * D.d * 2 + 64;
-        if (D.d == 64) {
-            cudaFuncSetAttribute(tc_key_norms_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
-            tc_key_norms_kernel<64><<<(unsigned)(BH * NP.nsplit), 160, smem_bytes, st>>>(NP);
-        } else {
-            cudaFuncSetAttribute(tc_key_norms_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
-            tc_key_norms_kernel<128><<<(unsigned)(BH * NP.nsplit), 160, smem_bytes, st>>>(NP);
-        }
-        chk();
+    const int smem_bytes = 2 * 128 * D.d * 2 + 64;
+    if (D.d == 64) {
+        cudaFuncSetAttribute(tc_key_norms_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+        tc_key_norms_kernel<64><<<(unsigned)(BH * NP.nsplit), 160, smem_bytes, st>>>(NP);
+    } else {
+        cudaFuncSetAttribute(tc_key_norms_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+        tc_key_norms_kernel<128><<<(unsigned)(BH * NP.nsplit), 160, smem_bytes, st>>>(NP);
     }
+    chk();
+    return e;
+}
+
+darkattn_status_t tensor_forward(const darkattn_plan_s *plan, const void *Q, const void *K, const void *V,
+                                 const void *M, const void *W, void *O, void *saved, char *ws, cudaStream_t st)
+{
+    const Dims &D = plan->dims;
+    const TensorLayout &Y = plan->tensor;
+    const size_t BH = D.BH, N = D.N;
+    auto bf = [&](size_t off) { return reinterpret_cast<__nv_bfloat16 *>(ws + off); };
+    auto fl = [&](size_t off) { return reinterpret_cast<float *>(ws + off); };
+    if (!encode_fn()) { set_cuda_error(cudaErrorNotSupported, "tensor_forward: cuTensorMapEncodeTiled unavailable"); return DARKATTN_ERR_CUDA; }
+
+    MainParams P;
+    memset(&P, 0, sizeof(P));
+    bool ok = make_map(&P.mapQ, Q, BH * N, D.d, 128) && make_map(&P.mapK, K, BH * N, D.d, 128) &&
+              make_map(&P.mapV, V, BH * N, D.dv, 128) && make_map(&P.mapOm, bf(Y.Om), (size_t)D.H * D.m, D.d, 128) &&
+              make_map(&P.mapSb, bf(Y.Sb), BH * D.m, D.dv, 128) &&
+              make_map(&P.mapPN, bf(Y.pnum), (size_t)Y.nslab * BH * N, D.dv, 128);
+    if (!ok) { set_cuda_error(cudaErrorInvalidValue, "tensor_forward: tensor map encode"); return DARKATTN_ERR_CUDA; }
+
+    cudaError_t e = tensor_prologue(plan, K, M, W, ws, st);
+    auto chk = [&]() { cudaError_t x = cudaGetLastError(); if (x != cudaSuccess && e == cudaSuccess) e = x; };
 
     P.nK = fl(Y.nK); P.cs = fl(Y.cs); P.pdr = fl(Y.pdr); P.Sacc = fl(Y.Sacc); P.zacc = fl(Y.zacc);
     P.status = reinterpret_cast<int *>(ws + Y.status);
@@ -736,19 +712,13 @@ darkattn_status_t tensor_forward(const darkattn_plan_s *plan, const void *Q, con
     }
     {
         const long long rows = (long long)BH * N, threads = rows * (D.dv / 8);
-        combine_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(bf(Y.pnum), fl(Y.pdr), (__nv_bfloat16 *)O, rows, D.dv, Y.nslab);
+        combine_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(bf(Y.pnum), fl(Y.pdr), (__nv_bfloat16 *)O,
+                                                                          reinterpret_cast<float2 *>(ws + Y.sv),
+                                                                          reinterpret_cast<float2 *>(saved), rows, D.dv, Y.nslab);
         chk();
     }
     if (e != cudaSuccess) { set_cuda_error(e, "tensor_forward"); return DARKATTN_ERR_CUDA; }
     return DARKATTN_OK;
-}
-
-// The backward pass has no tensor-core kernels yet: it runs on the FP32 SIMT path (same workspace).
-darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, const void *K, const void *V,
-                                  const void *M, const void *W, const void *dO, void *dQ, void *dK, void *dV,
-                                  float *dM, char *ws, cudaStream_t st)
-{
-    return simt_backward(plan, Q, K, V, M, W, dO, dQ, dK, dV, dM, ws, st);
 }
 
 }  // namespace darkattn

@@ -142,6 +142,42 @@ def test_tensor_path_forward(binding, name, kw):
     _compare(got, _oracle(t, wl), TOL["bf16"], name)
 
 
+TENSOR_BWD = [
+    ("b_one_chunk", dict(B=1, H=1, N=128, d=64, m=128, causal=True)),
+    ("b_d64_m128", dict(B=1, H=2, N=512, d=64, m=128, causal=True)),
+    ("b_d64_m512", dict(B=2, H=2, N=384, d=64, m=512, causal=True)),
+    ("b_d128_m256", dict(B=2, H=3, N=640, d=128, m=256, causal=True)),
+    ("b_d128_dv64_r64", dict(B=1, H=2, N=256, d=128, m=128, dv=64, r=64, causal=True)),
+    ("b_d64_dv128_r32", dict(B=2, H=2, N=384, d=64, m=256, dv=128, r=32, causal=True)),
+]
+
+
+@pytest.mark.parametrize("use_saved", [False, True], ids=["recompute", "saved"])
+@pytest.mark.parametrize("name,kw", TENSOR_BWD, ids=[s[0] for s in TENSOR_BWD])
+def test_tensor_path_backward(binding, name, kw, use_saved):
+    wl = inputs.small(name=name, wid=70 + len(name), dtype="bf16", backward=True, **kw)
+    t = inputs.generate(wl)
+    got = run_gpu(binding, wl, t, path=binding.PATH_TENSOR, use_saved=use_saved)
+    _compare(got, _oracle(t, wl), TOL["bf16"], name)
+
+
+def test_headline_backward_sampled_heads(binding):
+    """Forward + backward at the benchmark's full size; dQ, dK, dV of sampled (batch, head) pairs and
+    the gradient of M of one head (summed over the whole batch) against the oracle."""
+    wl = inputs.WORKLOADS["headline"]
+    B, H = wl.B, wl.H
+    t = inputs.generate(wl)
+    got = run_gpu(binding, wl, t, use_saved=True)
+    h = 5
+    pairs = [(b, h) for b in range(B)]
+    sub = inputs.generate(wl, pairs=pairs, as_batch=True)
+    want = _oracle(sub, wl)
+    for k in ("O", "dQ", "dK", "dV"):
+        g = np.stack([got[k][b, h] for b in range(B)])[:, None]
+        assert_close(g, want[k], TOL["bf16"], f"headline head {h}: {k}")
+    assert_close(got["dM"][h], want["dM"][0], TOL["bf16"], f"headline head {h}: dM")
+
+
 def test_tensor_path_rejects_uncovered_shapes(binding):
     for kw in (dict(N=200), dict(d=48), dict(m=96)):
         a = dict(B=1, H=1, N=256, d=64, m=128)

@@ -18,8 +18,11 @@ def torch_dtype(name):
     return torch.float32 if name == "f32" else torch.bfloat16
 
 
-def run_gpu(binding, wl, t, path=0, chunk=0, scale=0.0, backward=None, w_per_head=False):
-    """Run forward (and backward) on the device for tensors ``t`` laid out [B', H', N, *]."""
+def run_gpu(binding, wl, t, path=0, chunk=0, scale=0.0, backward=None, w_per_head=False, use_saved=False):
+    """Run forward (and backward) on the device for tensors ``t`` laid out [B', H', N, *].
+
+    With ``use_saved`` the forward call fills the plan's forward->backward stash and the backward call
+    is given it (and O); otherwise backward gets neither and recomputes what it needs."""
     Bq, Hq, N, d = t.Q.shape
     dv = t.V.shape[-1]
     r = t.M.shape[-2]
@@ -30,14 +33,18 @@ def run_gpu(binding, wl, t, path=0, chunk=0, scale=0.0, backward=None, w_per_hea
     ws = plan.alloc_workspace()
     Q, K, V, M, W = (to_dev(x, dt) for x in (t.Q, t.K, t.V, t.M, t.W))
     O = torch.empty_like(V)
-    binding.darkattn_forward(plan, Q, K, V, M, W, O, ws)
+    saved = None
+    if use_saved and plan.saved_bytes:
+        saved = torch.empty(plan.saved_bytes, dtype=torch.uint8, device="cuda")
+    binding.darkattn_forward(plan, Q, K, V, M, W, O, ws, saved=saved)
     out = {"O": O.float().cpu().numpy().astype(np.float64)}
     do_bwd = wl.backward if backward is None else backward
     if do_bwd:
         dO = to_dev(t.dO, dt)
         dQ, dK, dV = torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V)
         dM = torch.empty(M.shape, dtype=torch.float32, device="cuda")
-        binding.darkattn_backward(plan, Q, K, V, M, W, O, dO, dQ, dK, dV, dM, ws)
+        binding.darkattn_backward(plan, Q, K, V, M, W, O if saved is not None else None, dO, dQ, dK, dV, dM, ws,
+                                  saved=saved)
         for k, v in (("dQ", dQ), ("dK", dK), ("dV", dV), ("dM", dM)):
             out[k] = v.float().cpu().numpy().astype(np.float64)
     assert binding.darkattn_last_device_status(plan, ws) == binding.OK
