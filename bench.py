@@ -208,12 +208,13 @@ def main():
     plan = binding.darkattn_plan(B, H, N, d, m, r=r, dv=dv, dtype=binding.BF16 if wl.dtype == "bf16" else binding.F32,
                                  causal=wl.causal, path=args.path)
     ws = plan.alloc_workspace()
+    saved = torch.empty(plan.saved_bytes, dtype=torch.uint8, device="cuda") if plan.saved_bytes else None
     stream = torch.cuda.current_stream()
 
     def step():
-        binding.darkattn_forward(plan, Q, K, V, M, W, O, ws, stream=stream)
+        binding.darkattn_forward(plan, Q, K, V, M, W, O, ws, saved=saved, stream=stream)
         if wl.backward:
-            binding.darkattn_backward(plan, Q, K, V, M, W, O, G, dQ, dK, dV, dM, ws, stream=stream)
+            binding.darkattn_backward(plan, Q, K, V, M, W, O, G, dQ, dK, dV, dM, ws, saved=saved, stream=stream)
             if world > 1:
                 dist.all_reduce(dM)
 

@@ -39,6 +39,12 @@ __device__ __forceinline__ void mbar_arrive(uint64_t *bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+// One arrival for the whole warp: every lane's earlier writes are ordered before it by the warp barrier.
+__device__ __forceinline__ void mbar_arrive_warp(uint64_t *bar)
+{
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) mbar_arrive(bar);
+}
 __device__ __forceinline__ uint32_t mbar_try_wait(uint64_t *bar, uint32_t parity)
 {
     uint32_t ok;

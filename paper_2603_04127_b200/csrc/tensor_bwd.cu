@@ -35,14 +35,14 @@ namespace {
 constexpr float kLn2 = 0.6931471805599453f;
 
 struct BwdParams {
-    CUtensorMap mapQ, mapK, mapV, mapG, mapOm;
+    CUtensorMap mapQ, mapK, mapV, mapG, mapOm, mapPQ, mapPK, mapPV;   // the last three: slab partials, for the stores
     const float2 *sv;     // [BH*N]  (normaliser, exponent it is scaled by) from the forward pass
     const float *delta;   // [BH*N]  dO_i . O_i
     const float *nK;      // [BH*N]  key norms, log2 units
     const float *cs;      // [BH*nslab] key-side shift per slab
     float *rhoc;          // [BH, T, m] per-chunk -sum_i A^_il delta_i (written by the query-side kernel)
     __nv_bfloat16 *pdQ, *pdK, *pdV;   // slab partials
-    float *espart;        // [nslab, BH*N] slab partials of rowsum(E^K)
+    float *espart;        // [4 nslab, BH*N] partials of rowsum(E^K): one per slab and 32-column group
     float *Tacc;          // [H, m, D]
     int *status;
     int N, H, BH, m, nslab, T;
@@ -57,10 +57,9 @@ struct BwdSmem {
     static constexpr int kV = kKB + 32768;                 // V tile                            [128, DV]
     static constexpr int kG = kV + 128 * DV * 2;           // dO tile; later the reloaded Q / K tile
     static constexpr int kSt = kG + 128 * kDmax * 2;       // bf16 copy of the scan state       [128 l, DV]
-    static constexpr int kB1 = kSt + 128 * DV * 2;         // 16 x 128 operand: a row of ones
-    static constexpr int kB2 = kB1 + 4096;                 // 16 x 128 operand: rows hi(-delta), lo(-delta)
-    static constexpr int kVec = kB2 + 4096;                // two float[128]
-    static constexpr int kBars = kVec + 1024;
+    static constexpr int kStg = kSt + 128 * DV * 2;        // staging tile of the TMA stores of the partials
+    static constexpr int kVec = kStg + 128 * kDmax * 2;    // three float[128]
+    static constexpr int kBars = kVec + 1536;
     static constexpr int kTotal = kBars + 256;
 };
 
@@ -89,59 +88,110 @@ __device__ __forceinline__ void unpack8(const uint4 &raw, float *f)
     }
 }
 
-// features 2^(U - offset) of one row: TMEM columns [col, col+128) -> bf16 tile row `row`
-__device__ __forceinline__ void features_to_tile(uint32_t taddr, float offset, unsigned char *tile, int row)
+// Epilogue thread layout: 16 warps. Warp w works on TMEM lanes (tile rows) 32 (w % 4) .. +31, the only
+// ones it may touch, and on the 32 columns starting at 32 (w / 4); four warps share each row.
+constexpr int kEpiWarps = 16, kEpiThreads = 512, kThreads = 544;
+
+// the four warps that share a lane quarter
+__device__ __forceinline__ void quarter_sync(int q) { asm volatile("bar.sync %0, 128;" ::"r"(q + 1) : "memory"); }
+// all epilogue threads
+__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 5, 512;" ::: "memory"); }
+
+// features 2^(U - offset): 32 TMEM columns at taddr -> bf16 tile row `row`, columns [col0, col0 + 32)
+__device__ __forceinline__ void features_to_tile(uint32_t taddr, float offset, unsigned char *tile, int row, int col0)
 {
-    for (int c0 = 0; c0 < 128; c0 += 32) {
-        uint32_t v[32], pk[16];
-        tmem_ld32(taddr + c0, v);
-        tmem_wait_ld();
+    uint32_t v[32], pk[16];
+    tmem_ld32(taddr, v);
+    tmem_wait_ld();
 #pragma unroll
-        for (int j = 0; j < 32; j += 2)
-            pk[j / 2] = pack_bf16(ex2f(__uint_as_float(v[j]) - offset), ex2f(__uint_as_float(v[j + 1]) - offset));
+    for (int j = 0; j < 32; j += 2)
+        pk[j / 2] = pack_bf16(ex2f(__uint_as_float(v[j]) - offset), ex2f(__uint_as_float(v[j + 1]) - offset));
 #pragma unroll
-        for (int q = 0; q < 4; ++q)
-            *reinterpret_cast<uint4 *>(tile_chunk(tile, row, c0 / 8 + q)) = make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
-    }
+    for (int q = 0; q < 4; ++q)
+        *reinterpret_cast<uint4 *>(tile_chunk(tile, row, col0 / 8 + q)) = make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
 }
 
-// fp32 TMEM columns [taddr, taddr + width) of one row -> bf16 tile row (swizzled smem)
-template <int WIDTH>
-__device__ __forceinline__ void tmem_row_to_tile(uint32_t taddr, unsigned char *tile, int row)
+// Sum over the 32 lanes of a warp of x[c], for every c: afterwards lane l holds the sum for c = l.
+// Butterfly reduce-scatter: 31 shuffles instead of 32 full reductions.
+__device__ __forceinline__ float warp_column_sums(float (&x)[32], int lane)
 {
-    for (int c0 = 0; c0 < WIDTH; c0 += 32) {
-        uint32_t v[32];
-        tmem_ld32(taddr + c0, v);
-        tmem_wait_ld();
 #pragma unroll
-        for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4 *>(tile_chunk(tile, row, c0 / 8 + q)) = pack8(v + 8 * q);
+    for (int s = 16; s >= 1; s >>= 1) {
+        const bool up = (lane & s) != 0;
+#pragma unroll
+        for (int i = 0; i < s; ++i) {
+            const float send = up ? x[i] : x[i + s];
+            const float keep = up ? x[i + s] : x[i];
+            x[i] = keep + __shfl_xor_sync(0xffffffffu, send, s);
+        }
     }
+    return x[0];
 }
 
-// fp32 TMEM columns of one row -> bf16 row in global memory (dst points at the row)
-template <int WIDTH>
+// features 2^(U - offset) as above; also adds, for every column, weight * feature summed over the
+// warp's 32 rows into colsum[col0 + column] (shared memory).
+__device__ __forceinline__ void features_to_tile_sums(uint32_t taddr, float offset, unsigned char *tile, int row, int col0,
+                                                      float weight, float *colsum, int lane)
+{
+    uint32_t v[32], pk[16];
+    float f[32];
+    tmem_ld32(taddr, v);
+    tmem_wait_ld();
+#pragma unroll
+    for (int j = 0; j < 32; ++j) f[j] = ex2f(__uint_as_float(v[j]) - offset);
+#pragma unroll
+    for (int j = 0; j < 32; j += 2) pk[j / 2] = pack_bf16(f[j], f[j + 1]);
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+        *reinterpret_cast<uint4 *>(tile_chunk(tile, row, col0 / 8 + q)) = make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+#pragma unroll
+    for (int j = 0; j < 32; ++j) f[j] *= weight;
+    atomicAdd(colsum + col0 + lane, warp_column_sums(f, lane));
+}
+
+// 32 fp32 TMEM columns at taddr -> bf16 tile row (swizzled smem), columns [col0, col0 + 32)
+__device__ __forceinline__ void tmem_row_to_tile(uint32_t taddr, unsigned char *tile, int row, int col0)
+{
+    uint32_t v[32];
+    tmem_ld32(taddr, v);
+    tmem_wait_ld();
+#pragma unroll
+    for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4 *>(tile_chunk(tile, row, col0 / 8 + q)) = pack8(v + 8 * q);
+}
+
+// 32 fp32 TMEM columns at taddr -> 32 bf16 at dst (global memory)
 __device__ __forceinline__ void tmem_row_to_global(uint32_t taddr, __nv_bfloat16 *dst)
 {
-    for (int c0 = 0; c0 < WIDTH; c0 += 32) {
-        uint32_t v[32];
-        tmem_ld32(taddr + c0, v);
-        tmem_wait_ld();
+    uint32_t v[32];
+    tmem_ld32(taddr, v);
+    tmem_wait_ld();
 #pragma unroll
-        for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4 *>(dst + c0 + 8 * q) = pack8(v + 8 * q);
-    }
+    for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4 *>(dst + 8 * q) = pack8(v + 8 * q);
 }
+
+// Matrix descriptors are built once per tile buffer; step k of an MMA loop only adds a constant to the
+// start-address field (units of 16 bytes), so that the issuing thread spends one add per instruction.
+struct TileDesc {
+    uint64_t kmaj, mnmaj;
+    __device__ __forceinline__ explicit TileDesc(const unsigned char *base)
+        : kmaj(make_sdesc(smem_u32(base), 16, 1024)), mnmaj(make_sdesc(smem_u32(base), 16384, 1024)) {}
+};
+// K-major operand, 64-element atoms 16 KB apart: step k covers 16 elements (32 bytes) of K
+__device__ __forceinline__ uint64_t kdesc(const TileDesc &t, int k) { return t.kmaj + (uint64_t)(((k / 4) * 16384 + (k % 4) * 32) >> 4); }
+// MN-major operand: step k covers 16 K-rows of 128 bytes
+__device__ __forceinline__ uint64_t mndesc(const TileDesc &t, int k) { return t.mnmaj + (uint64_t)((k * 2048) >> 4); }
 
 enum QBars { QB_OM, QB_Q, QB_K, QB_V, QB_G, QB_X2, QM1, QM2, QM3, QMS, QM4, QM5, QM6, QE1, QE2, QE3, QE4, QNBARS };
 
 // ------------------------------------------------------------------ query side (forward direction)
 template <int D, int DV>
-__global__ void __launch_bounds__(160, 1) tc_bwd_q_kernel(const __grid_constant__ BwdParams p)
+__global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_constant__ BwdParams p)
 {
     using L = BwdSmem<D, DV>;
     extern __shared__ __align__(1024) unsigned char smem[];
     unsigned char *sOm = smem + L::kOm, *sQA = smem + L::kQA, *sKB = smem + L::kKB, *sV = smem + L::kV;
-    unsigned char *sG = smem + L::kG, *sSt = smem + L::kSt, *sB1 = smem + L::kB1, *sB2 = smem + L::kB2;
-    float *sZ = reinterpret_cast<float *>(smem + L::kVec);
+    unsigned char *sG = smem + L::kG, *sSt = smem + L::kSt, *sStg = smem + L::kStg;
+    float *sZ = reinterpret_cast<float *>(smem + L::kVec), *sZc = sZ + 128, *sRc = sZ + 256;   // z_prev; chunk sums of Bf and of -delta A^
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::kBars);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + QNBARS);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + QNBARS + 1);
@@ -152,18 +202,12 @@ __global__ void __launch_bounds__(160, 1) tc_bwd_q_kernel(const __grid_constant_
 
     if (tid == 0) {
         for (int i = 0; i < QE1; ++i) mbar_init(bars + i, 1);
-        for (int i = QE1; i < QNBARS; ++i) mbar_init(bars + i, 128);
+        for (int i = QE1; i < QNBARS; ++i) mbar_init(bars + i, kEpiWarps);
         *abort_flag = (smem_u32(smem) & 1023u) ? 1 : 0;
         fence_mbar_init();
     }
-    if (tid < 128) {
-        for (int i = tid; i < 256; i += 128) {
-            *reinterpret_cast<uint4 *>(sB1 + i * 16) = make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
-            *reinterpret_cast<uint4 *>(sB2 + i * 16) = make_uint4(0, 0, 0, 0);
-        }
-        sZ[tid] = 0.f;
-    }
-    if (warp == 4) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+    if (tid < 384) sZ[tid] = 0.f;
+    if (warp == kEpiWarps) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -172,17 +216,14 @@ __global__ void __launch_bounds__(160, 1) tc_bwd_q_kernel(const __grid_constant_
 
     if (*abort_flag) {
         if (tid == 0) atomicExch(status, (int)DARKATTN_ERR_CUDA);
-    } else if (warp == 4) {
+    } else if (warp == kEpiWarps) {
         if ((tid & 31) == 0) {
             auto load_tile = [&](unsigned char *dst, const CUtensorMap *map, uint64_t *bar, int width, int t) {
                 mbar_expect_tx(bar, 128 * width * 2);
                 for (int a = 0; a < width / 64; ++a) tma_load_2d(dst + a * 16384, map, bar, a * 64, row0 + t * 128);
             };
-            auto kdesc = [](unsigned char *base, int k) { return make_sdesc(smem_u32(base) + (k / 4) * 16384 + (k % 4) * 32, 16, 1024); };
-            auto mndesc = [](unsigned char *base, int k) { return make_sdesc(smem_u32(base) + k * 2048, 16384, 1024); };
-            auto bdesc = [](unsigned char *base, int k) { return make_sdesc(smem_u32(base) + (k / 4) * 2048 + (k % 4) * 32, 16, 1024); };
+            const TileDesc tOm(sOm), tQA(sQA), tKB(sKB), tV(sV), tG(sG), tSt(sSt);
             const uint32_t id_kk = make_idesc(128, 128, 0, 0);
-            const uint32_t id_vec = make_idesc(128, 16, 1, 0);
             const uint32_t id_state = make_idesc(128, DV, 1, 1);
             const uint32_t id_tm = make_idesc(128, 128, 0, 1);
             const uint32_t id_dx = make_idesc(128, D, 0, 1);
@@ -203,28 +244,26 @@ __global__ void __launch_bounds__(160, 1) tc_bwd_q_kernel(const __grid_constant_
 #define QWAIT(b) do { ok = wait_or_abort(bars + (b), ph, status, abort_flag); } while (0)
                 QWAIT(QB_Q); if (!ok) break;
                 tc_fence_after();
-                for (int k = 0; k < D / 16; ++k) mma_ss(R1, kdesc(sQA, k), kdesc(sOm, k), id_kk, k > 0);       // U_Q
+                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R1, kdesc(tQA, k), kdesc(tOm, k), id_kk, k > 0);       // U_Q
                 mma_commit(bars + QM1);
                 QWAIT(QB_K); if (!ok) break;
                 tc_fence_after();
-                for (int k = 0; k < D / 16; ++k) mma_ss(R2, kdesc(sKB, k), kdesc(sOm, k), id_kk, k > 0);       // U_K
+                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R2, kdesc(tKB, k), kdesc(tOm, k), id_kk, k > 0);       // U_K
                 mma_commit(bars + QM2);
                 QWAIT(QE1); if (!ok) break;
                 tc_fence_after();
-                for (int k = 0; k < 8; ++k) mma_ss(R2, mndesc(sKB, k), bdesc(sB1, k), id_vec, k > 0);           // z_c = Bf^T 1
-                for (int k = 0; k < 8; ++k) mma_ss(R2 + 16, mndesc(sQA, k), bdesc(sB2, k), id_vec, k > 0);      // rho_c = -A^^T delta
                 QWAIT(QB_V); if (!ok) break;
                 QWAIT(QB_G); if (!ok) break;
                 tc_fence_after();
-                for (int k = 0; k < DV / 16; ++k) mma_ss(R1, kdesc(sG, k), kdesc(sV, k), id_kk, k > 0);         // dO V^T
+                _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R1, kdesc(tG, k), kdesc(tV, k), id_kk, k > 0);         // dO V^T
                 mma_commit(bars + QM3);
-                for (int k = 0; k < 8; ++k) mma_ss(tmem + kColState, mndesc(sKB, k), mndesc(sV, k), id_state, (!first) || k > 0);   // S += Bf^T V
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColState, mndesc(tKB, k), mndesc(tV, k), id_state, (!first) || k > 0);   // S += Bf^T V
                 mma_commit(bars + QMS);
                 QWAIT(QE2); if (!ok) break;
                 tc_fence_after();
-                for (int k = 0; k < 8; ++k) mma_ts(R2, R1 + k * 8, mndesc(sKB, k), id_tm, k > 0);               // dP Bf
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R2, R1 + k * 8, mndesc(tKB, k), id_tm, k > 0);               // dP Bf
                 if (!first)
-                    for (int k = 0; k < DV / 16; ++k) mma_ss(R2, kdesc(sG, k), kdesc(sSt, k), id_kk, 1);        // + dO S_prev^T
+                    _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R2, kdesc(tG, k), kdesc(tSt, k), id_kk, 1);        // + dO S_prev^T
                 mma_commit(bars + QM4);
                 QWAIT(QM4); if (!ok) break;
                 load_tile(sG, &p.mapQ, bars + QB_X2, D, t);                                                     // Q again, for T
@@ -232,9 +271,9 @@ __global__ void __launch_bounds__(160, 1) tc_bwd_q_kernel(const __grid_constant_
                 QWAIT(QE3); if (!ok) break;
                 QWAIT(QB_X2); if (!ok) break;
                 tc_fence_after();
-                for (int k = 0; k < 8; ++k) mma_ss(R1, kdesc(sQA, k), mndesc(sOm, k), id_dx, k > 0);            // E Omega
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R1, kdesc(tQA, k), mndesc(tOm, k), id_dx, k > 0);            // E Omega
                 mma_commit(bars + QM5);
-                for (int k = 0; k < 8; ++k) mma_ss(tmem + kColT, mndesc(sQA, k), mndesc(sG, k), id_t, (!first) || k > 0);   // T += E^T Q
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColT, mndesc(tQA, k), mndesc(tG, k), id_t, (!first) || k > 0);   // T += E^T Q
                 mma_commit(bars + QM6);
                 QWAIT(QM6); if (!ok) break;
                 if (!last) { load_tile(sQA, &p.mapQ, bars + QB_Q, D, t + 1); load_tile(sG, &p.mapG, bars + QB_G, DV, t + 1); }
@@ -243,8 +282,11 @@ __global__ void __launch_bounds__(160, 1) tc_bwd_q_kernel(const __grid_constant_
             }
         }
     } else {
-        // ============================== epilogue threads: thread = TMEM lane = tile row
-        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+        // ============================== epilogue threads (see kEpiWarps)
+        const int lane = tid & 31, q4 = warp & 3, col0 = (warp >> 2) * 32;
+        const int r = q4 * 32 + lane;                        // tile row = TMEM lane
+        const bool own = (q4 == 0);                          // these 128 threads each own one column's running sums
+        const uint32_t lane_addr = tmem + ((uint32_t)(q4 * 32) << 16);
         const uint32_t R1 = lane_addr + kColR1, R2 = lane_addr + kColR2;
         const float cshift = p.cs[bh * p.nslab + slab];
         float zrun = 0.f;
@@ -252,69 +294,61 @@ __global__ void __launch_bounds__(160, 1) tc_bwd_q_kernel(const __grid_constant_
         for (int t = 0; t < T && ok; ++t) {
             const uint32_t ph = t & 1;
             const bool last = (t + 1 == T);
-            const size_t row = (size_t)row0 + (size_t)t * 128 + tid;
-#define EWAIT(b) do { ok = wait_or_abort(bars + (b), ph, status, abort_flag); } while (0)
+            const size_t row = (size_t)row0 + (size_t)t * 128 + r;
+#define EWAIT(b) do { ok = __all_sync(0xffffffffu, wait_or_abort(bars + (b), ph, status, abort_flag)); } while (0)
             const float2 svv = p.sv[row];
             const float del = p.delta[row];
             const float nk = p.nK[row] + cshift;
             const float aq = svv.y - cshift + log2f(svv.x);
-            {   // rows 0 and 1 of the 16 x 128 operand: -delta split into two bf16 terms
-                const __nv_bfloat16 hi = __float2bfloat16_rn(-del);
-                const __nv_bfloat16 lo = __float2bfloat16_rn(-del - __bfloat162float(hi));
-                const int atom = tid >> 6, kk = tid & 63, ch = kk >> 3;
-                *reinterpret_cast<__nv_bfloat16 *>(sB2 + atom * 2048 + (ch << 4) + (kk & 7) * 2) = hi;
-                *reinterpret_cast<__nv_bfloat16 *>(sB2 + atom * 2048 + 128 + ((ch ^ 1) << 4) + (kk & 7) * 2) = lo;
-            }
             EWAIT(QM1); if (!ok) break;
             tc_fence_after();
-            features_to_tile(R1, aq, sQA, tid);
+            features_to_tile_sums(R1 + col0, aq, sQA, r, col0, -del, sRc, lane);      // A^ and rho_c = -sum_i delta_i A^_il
             EWAIT(QM2); if (!ok) break;
             tc_fence_after();
-            features_to_tile(R2, nk, sKB, tid);
+            features_to_tile_sums(R2 + col0, nk, sKB, r, col0, 1.f, sZc, lane);       // Bf and z_c = sum_j Bf_jl
             fence_async_smem();
             tc_fence_before();
-            mbar_arrive(bars + QE1);
+            mbar_arrive_warp(bars + QE1);
 
             EWAIT(QM3); if (!ok) break;
             tc_fence_after();
-            float znew;
-            {
-                uint32_t a[16], b[16];
-                tmem_ld16(R2, a);
-                tmem_ld16(R2 + 16, b);
-                tmem_wait_ld();
-                znew = zrun + __uint_as_float(a[0]);
-                p.rhoc[((size_t)bh * T + t) * p.m + slab * 128 + tid] = __uint_as_float(b[0]) + __uint_as_float(b[1]);
+            float znew = zrun;
+            if (own) {      // the column sums of all four lane quarters are in (every warp arrived at QE1)
+                znew = zrun + sZc[col0 + lane];
+                p.rhoc[((size_t)bh * T + t) * p.m + slab * 128 + col0 + lane] = sRc[col0 + lane];
+                sZc[col0 + lane] = 0.f;
+                sRc[col0 + lane] = 0.f;
             }
-            for (int c0 = 0; c0 < 128; c0 += 32) {       // dP = tril(dO V^T - delta) as a bf16 operand in TMEM
+            {   // dP = tril(dO V^T - delta) as a bf16 operand in TMEM (packed over the fp32 tile)
                 uint32_t v[32], pk[16];
-                tmem_ld32(R1 + c0, v);
+                tmem_ld32(R1 + col0, v);
                 tmem_wait_ld();
+                quarter_sync(q4);                         // every column group has read before anyone overwrites
 #pragma unroll
                 for (int j = 0; j < 32; j += 2) {
-                    const float x0 = (c0 + j <= tid) ? __uint_as_float(v[j]) - del : 0.f;
-                    const float x1 = (c0 + j + 1 <= tid) ? __uint_as_float(v[j + 1]) - del : 0.f;
+                    const float x0 = (col0 + j <= r) ? __uint_as_float(v[j]) - del : 0.f;
+                    const float x1 = (col0 + j + 1 <= r) ? __uint_as_float(v[j + 1]) - del : 0.f;
                     pk[j / 2] = pack_bf16(x0, x1);
                 }
-                tmem_st16(R1 + c0 / 2, pk);
+                tmem_st16(R1 + col0 / 2, pk);
             }
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(bars + QE2);
+            mbar_arrive_warp(bars + QE2);
 
             EWAIT(QM4); if (!ok) break;
             tc_fence_after();
-            for (int c0 = 0; c0 < 128; c0 += 32) {       // E = A^ .* (dP Bf + dO S^T - delta z^T), in place over A^
+            {   // E = A^ .* (dP Bf + dO S^T - delta z^T), in place over A^
                 uint32_t v[32];
-                tmem_ld32(R2 + c0, v);
+                tmem_ld32(R2 + col0, v);
                 tmem_wait_ld();
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
-                    uint4 *cell = reinterpret_cast<uint4 *>(tile_chunk(sQA, tid, c0 / 8 + q));
+                    uint4 *cell = reinterpret_cast<uint4 *>(tile_chunk(sQA, r, col0 / 8 + q));
                     float a[8];
                     unpack8(*cell, a);
-                    const float4 z0 = *reinterpret_cast<const float4 *>(sZ + c0 + 8 * q);
-                    const float4 z1 = *reinterpret_cast<const float4 *>(sZ + c0 + 8 * q + 4);
+                    const float4 z0 = *reinterpret_cast<const float4 *>(sZ + col0 + 8 * q);
+                    const float4 z1 = *reinterpret_cast<const float4 *>(sZ + col0 + 8 * q + 4);
                     const float zz[8] = {z0.x, z0.y, z0.z, z0.w, z1.x, z1.y, z1.z, z1.w};
                     float e[8];
 #pragma unroll
@@ -324,51 +358,58 @@ __global__ void __launch_bounds__(160, 1) tc_bwd_q_kernel(const __grid_constant_
             }
             fence_async_smem();
             tc_fence_before();
-            mbar_arrive(bars + QE3);
+            mbar_arrive_warp(bars + QE3);
 
             EWAIT(QM5); if (!ok) break;
             tc_fence_after();
-            tmem_row_to_global<D>(R1, p.pdQ + (((size_t)slab * p.BH + bh) * p.N + (size_t)t * 128 + tid) * D);
+            if (col0 < D) tmem_row_to_tile(R1 + col0, sStg, r, col0);       // slab partial of dQ -> staging -> TMA store
+            fence_async_smem();
+            epi_sync();
+            if (tid == 0) {
+                for (int a = 0; a < D / 64; ++a)
+                    tma_store_2d(&p.mapPQ, sStg + a * 16384, a * 64, (int)(((size_t)slab * p.BH + bh) * p.N + (size_t)t * 128));
+                tma_store_commit();
+            }
             EWAIT(QMS); if (!ok) break;
             zrun = znew;
             if (!last) {
-                tmem_row_to_tile<DV>(lane_addr + kColState, sSt, tid);
-                sZ[tid] = zrun;
+                if (col0 < DV) tmem_row_to_tile(lane_addr + kColState + col0, sSt, r, col0);
+                if (own) sZ[col0 + lane] = zrun;
                 fence_async_smem();
             }
+            if (tid == 0) tma_store_wait_read();      // the staging tile is free again before anyone passes QE4
             tc_fence_before();
-            mbar_arrive(bars + QE4);
+            mbar_arrive_warp(bars + QE4);
 #undef EWAIT
         }
+        if (tid == 0) tma_store_wait_all();
         if (ok) ok = wait_or_abort(bars + QM6, (T - 1) & 1, status, abort_flag);
-        if (ok) {
+        if (ok && col0 < D) {
             tc_fence_after();
-            float *dst = p.Tacc + ((size_t)h * p.m + slab * 128 + tid) * D;
-            for (int c0 = 0; c0 < D; c0 += 32) {
-                uint32_t v[32];
-                tmem_ld32(lane_addr + kColT + c0, v);
-                tmem_wait_ld();
+            float *dst = p.Tacc + ((size_t)h * p.m + slab * 128 + r) * D + col0;
+            uint32_t v[32];
+            tmem_ld32(lane_addr + kColT + col0, v);
+            tmem_wait_ld();
 #pragma unroll
-                for (int j = 0; j < 32; ++j) atomicAdd(dst + c0 + j, __uint_as_float(v[j]));
-            }
+            for (int j = 0; j < 32; ++j) atomicAdd(dst + j, __uint_as_float(v[j]));
         }
     }
     if (*abort_flag) __nanosleep(200000);   // error path only: let copies and MMAs in flight drain
     tc_fence_before();
     __syncthreads();
-    if (warp == 4) tmem_dealloc(tmem, 512);
+    if (warp == kEpiWarps) tmem_dealloc(tmem, 512);
 }
 
 enum KBars { KB_OM, KB_Q, KB_K, KB_V, KB_G, KB_X2, KM1, KM2, KM3, KM4, KM5, KM6, KM7, KM8, KM9, KE1, KE2, KE3, KE4, KE5, KNBARS };
 
 // ------------------------------------------------------------------ key side (reverse direction)
 template <int D, int DV>
-__global__ void __launch_bounds__(160, 1) tc_bwd_k_kernel(const __grid_constant__ BwdParams p)
+__global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_constant__ BwdParams p)
 {
     using L = BwdSmem<D, DV>;
     extern __shared__ __align__(1024) unsigned char smem[];
     unsigned char *sOm = smem + L::kOm, *sQA = smem + L::kQA, *sKB = smem + L::kKB, *sV = smem + L::kV;
-    unsigned char *sG = smem + L::kG, *sSt = smem + L::kSt;
+    unsigned char *sG = smem + L::kG, *sSt = smem + L::kSt, *sStg = smem + L::kStg;
     float *sRho = reinterpret_cast<float *>(smem + L::kVec), *sDel = sRho + 128;
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::kBars);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + KNBARS);
@@ -380,12 +421,12 @@ __global__ void __launch_bounds__(160, 1) tc_bwd_k_kernel(const __grid_constant_
 
     if (tid == 0) {
         for (int i = 0; i < KE1; ++i) mbar_init(bars + i, 1);
-        for (int i = KE1; i < KNBARS; ++i) mbar_init(bars + i, 128);
+        for (int i = KE1; i < KNBARS; ++i) mbar_init(bars + i, kEpiWarps);
         *abort_flag = (smem_u32(smem) & 1023u) ? 1 : 0;
         fence_mbar_init();
     }
     if (tid < 128) sRho[tid] = 0.f;
-    if (warp == 4) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+    if (warp == kEpiWarps) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -394,14 +435,13 @@ __global__ void __launch_bounds__(160, 1) tc_bwd_k_kernel(const __grid_constant_
 
     if (*abort_flag) {
         if (tid == 0) atomicExch(status, (int)DARKATTN_ERR_CUDA);
-    } else if (warp == 4) {
+    } else if (warp == kEpiWarps) {
         if ((tid & 31) == 0) {
             auto load_tile = [&](unsigned char *dst, const CUtensorMap *map, uint64_t *bar, int width, int t) {
                 mbar_expect_tx(bar, 128 * width * 2);
                 for (int a = 0; a < width / 64; ++a) tma_load_2d(dst + a * 16384, map, bar, a * 64, row0 + t * 128);
             };
-            auto kdesc = [](unsigned char *base, int k) { return make_sdesc(smem_u32(base) + (k / 4) * 16384 + (k % 4) * 32, 16, 1024); };
-            auto mndesc = [](unsigned char *base, int k) { return make_sdesc(smem_u32(base) + k * 2048, 16384, 1024); };
+            const TileDesc tOm(sOm), tQA(sQA), tKB(sKB), tV(sV), tG(sG), tSt(sSt);
             const uint32_t id_kk = make_idesc(128, 128, 0, 0);
             const uint32_t id_state = make_idesc(128, DV, 1, 1);
             const uint32_t id_dv_t = make_idesc(128, DV, 0, 1);
@@ -425,34 +465,34 @@ __global__ void __launch_bounds__(160, 1) tc_bwd_k_kernel(const __grid_constant_
 #define KWAIT(b) do { ok = wait_or_abort(bars + (b), ph, status, abort_flag); } while (0)
                 KWAIT(KB_Q); if (!ok) break;
                 tc_fence_after();
-                for (int k = 0; k < D / 16; ++k) mma_ss(R1, kdesc(sQA, k), kdesc(sOm, k), id_kk, k > 0);       // U_Q
+                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R1, kdesc(tQA, k), kdesc(tOm, k), id_kk, k > 0);       // U_Q
                 mma_commit(bars + KM1);
                 KWAIT(KB_K); if (!ok) break;
                 tc_fence_after();
-                for (int k = 0; k < D / 16; ++k) mma_ss(R2, kdesc(sKB, k), kdesc(sOm, k), id_kk, k > 0);       // U_K
+                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R2, kdesc(tKB, k), kdesc(tOm, k), id_kk, k > 0);       // U_K
                 mma_commit(bars + KM2);
                 KWAIT(KE1); if (!ok) break;
                 tc_fence_after();
-                for (int k = 0; k < 8; ++k) mma_ss(R1, kdesc(sKB, k), kdesc(sQA, k), id_kk, k > 0);             // P^^T = Bf A^^T
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R1, kdesc(tKB, k), kdesc(tQA, k), id_kk, k > 0);             // P^^T = Bf A^^T
                 mma_commit(bars + KM3);
                 KWAIT(KB_V); if (!ok) break;
                 KWAIT(KB_G); if (!ok) break;
                 tc_fence_after();
-                for (int k = 0; k < DV / 16; ++k) mma_ss(R2, kdesc(sV, k), kdesc(sG, k), id_kk, k > 0);         // V dO^T
+                _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R2, kdesc(tV, k), kdesc(tG, k), id_kk, k > 0);         // V dO^T
                 mma_commit(bars + KM4);
-                for (int k = 0; k < 8; ++k) mma_ss(tmem + kColState, mndesc(sQA, k), mndesc(sG, k), id_state, (!first) || k > 0);   // R += A^^T dO
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColState, mndesc(tQA, k), mndesc(tG, k), id_state, (!first) || k > 0);   // R += A^^T dO
                 mma_commit(bars + KM5);
                 KWAIT(KE2); if (!ok) break;
                 tc_fence_after();
-                for (int k = 0; k < 8; ++k) mma_ts(R2, R1 + k * 8, mndesc(sG, k), id_dv_t, k > 0);              // P^^T dO
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R2, R1 + k * 8, mndesc(tG, k), id_dv_t, k > 0);              // P^^T dO
                 if (!first)
-                    for (int k = 0; k < 8; ++k) mma_ss(R2, kdesc(sKB, k), mndesc(sSt, k), id_dv_t, 1);          // + Bf R_next
+                    _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R2, kdesc(tKB, k), mndesc(tSt, k), id_dv_t, 1);          // + Bf R_next
                 mma_commit(bars + KM6);
                 KWAIT(KE3); if (!ok) break;
                 tc_fence_after();
-                for (int k = 0; k < 8; ++k) mma_ts(R2, R1 + 64 + k * 8, mndesc(sQA, k), id_tm, k > 0);          // dP^T A^
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R2, R1 + 64 + k * 8, mndesc(tQA, k), id_tm, k > 0);          // dP^T A^
                 if (!first)
-                    for (int k = 0; k < DV / 16; ++k) mma_ss(R2, kdesc(sV, k), kdesc(sSt, k), id_kk, 1);        // + V R_next^T
+                    _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R2, kdesc(tV, k), kdesc(tSt, k), id_kk, 1);        // + V R_next^T
                 mma_commit(bars + KM7);
                 KWAIT(KM7); if (!ok) break;
                 load_tile(sG, &p.mapK, bars + KB_X2, D, t);                                                     // K again, for T
@@ -460,9 +500,9 @@ __global__ void __launch_bounds__(160, 1) tc_bwd_k_kernel(const __grid_constant_
                 KWAIT(KE4); if (!ok) break;
                 KWAIT(KB_X2); if (!ok) break;
                 tc_fence_after();
-                for (int k = 0; k < 8; ++k) mma_ss(R2, kdesc(sKB, k), mndesc(sOm, k), id_dx, k > 0);            // E Omega
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R2, kdesc(tKB, k), mndesc(tOm, k), id_dx, k > 0);            // E Omega
                 mma_commit(bars + KM8);
-                for (int k = 0; k < 8; ++k) mma_ss(tmem + kColT, mndesc(sKB, k), mndesc(sG, k), id_t, (!first) || k > 0);   // T += E^T K
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColT, mndesc(tKB, k), mndesc(tG, k), id_t, (!first) || k > 0);   // T += E^T K
                 mma_commit(bars + KM9);
                 KWAIT(KM9); if (!ok) break;
                 if (!last) { load_tile(sKB, &p.mapK, bars + KB_K, D, t - 1); load_tile(sG, &p.mapG, bars + KB_G, DV, t - 1); }
@@ -471,126 +511,147 @@ __global__ void __launch_bounds__(160, 1) tc_bwd_k_kernel(const __grid_constant_
             }
         }
     } else {
-        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+        const int lane = tid & 31, q4 = warp & 3, g = warp >> 2, col0 = g * 32;
+        const int r = q4 * 32 + lane;
+        const bool g0 = (col0 == 0);
+        const uint32_t lane_addr = tmem + ((uint32_t)(q4 * 32) << 16);
         const uint32_t R1 = lane_addr + kColR1, R2 = lane_addr + kColR2;
         const float cshift = p.cs[bh * p.nslab + slab];
+        const size_t rows = (size_t)p.BH * p.N;
         bool ok = true;
         for (int it = 0; it < T && ok; ++it) {
             const int t = T - 1 - it;
             const uint32_t ph = it & 1;
             const bool last = (it + 1 == T);
-            const size_t row = (size_t)row0 + (size_t)t * 128 + tid;
-            const size_t prow = ((size_t)slab * p.BH + bh) * p.N + (size_t)t * 128 + tid;
-#define EWAIT(b) do { ok = wait_or_abort(bars + (b), ph, status, abort_flag); } while (0)
+            const size_t row = (size_t)row0 + (size_t)t * 128 + r;
+            const size_t prow = ((size_t)slab * p.BH + bh) * p.N + (size_t)t * 128 + r;
+#define EWAIT(b) do { ok = __all_sync(0xffffffffu, wait_or_abort(bars + (b), ph, status, abort_flag)); } while (0)
             const float2 svv = p.sv[row];
             const float nk = p.nK[row] + cshift;
             const float aq = svv.y - cshift + log2f(svv.x);
-            const float rho_c = p.rhoc[((size_t)bh * T + t) * p.m + slab * 128 + tid];
-            sDel[tid] = p.delta[row];
+            float rho_c = 0.f;
+            if (g0) {
+                rho_c = p.rhoc[((size_t)bh * T + t) * p.m + slab * 128 + r];
+                sDel[r] = p.delta[row];
+            }
             EWAIT(KM1); if (!ok) break;
             tc_fence_after();
-            features_to_tile(R1, aq, sQA, tid);
+            features_to_tile(R1 + col0, aq, sQA, r, col0);
             EWAIT(KM2); if (!ok) break;
             tc_fence_after();
-            features_to_tile(R2, nk, sKB, tid);
+            features_to_tile(R2 + col0, nk, sKB, r, col0);
             fence_async_smem();
             tc_fence_before();
-            mbar_arrive(bars + KE1);
+            mbar_arrive_warp(bars + KE1);
 
             EWAIT(KM3); if (!ok) break;
             tc_fence_after();
-            for (int c0 = 0; c0 < 128; c0 += 32) {       // P^^T masked to queries i >= this key
+            {   // P^^T masked to queries i >= this key, packed over the fp32 tile
                 uint32_t v[32], pk[16];
-                tmem_ld32(R1 + c0, v);
+                tmem_ld32(R1 + col0, v);
                 tmem_wait_ld();
+                quarter_sync(q4);
 #pragma unroll
                 for (int j = 0; j < 32; j += 2) {
-                    const float x0 = (c0 + j >= tid) ? __uint_as_float(v[j]) : 0.f;
-                    const float x1 = (c0 + j + 1 >= tid) ? __uint_as_float(v[j + 1]) : 0.f;
+                    const float x0 = (col0 + j >= r) ? __uint_as_float(v[j]) : 0.f;
+                    const float x1 = (col0 + j + 1 >= r) ? __uint_as_float(v[j + 1]) : 0.f;
                     pk[j / 2] = pack_bf16(x0, x1);
                 }
-                tmem_st16(R1 + c0 / 2, pk);
+                tmem_st16(R1 + col0 / 2, pk);
             }
             EWAIT(KM4); if (!ok) break;
             tc_fence_after();
-            for (int c0 = 0; c0 < 128; c0 += 32) {       // dP^T = (V dO^T - delta_i) masked
+            {   // dP^T = (V dO^T - delta_i) masked, packed behind P^^T
                 uint32_t v[32], pk[16];
-                tmem_ld32(R2 + c0, v);
+                tmem_ld32(R2 + col0, v);
                 tmem_wait_ld();
 #pragma unroll
                 for (int j = 0; j < 32; j += 2) {
-                    const float2 dl = *reinterpret_cast<const float2 *>(sDel + c0 + j);
-                    const float x0 = (c0 + j >= tid) ? __uint_as_float(v[j]) - dl.x : 0.f;
-                    const float x1 = (c0 + j + 1 >= tid) ? __uint_as_float(v[j + 1]) - dl.y : 0.f;
+                    const float2 dl = *reinterpret_cast<const float2 *>(sDel + col0 + j);
+                    const float x0 = (col0 + j >= r) ? __uint_as_float(v[j]) - dl.x : 0.f;
+                    const float x1 = (col0 + j + 1 >= r) ? __uint_as_float(v[j + 1]) - dl.y : 0.f;
                     pk[j / 2] = pack_bf16(x0, x1);
                 }
-                tmem_st16(R1 + 64 + c0 / 2, pk);
+                tmem_st16(R1 + 64 + col0 / 2, pk);
             }
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(bars + KE2);
+            mbar_arrive_warp(bars + KE2);
 
             EWAIT(KM6); if (!ok) break;
             tc_fence_after();
-            tmem_row_to_global<DV>(R2, p.pdV + prow * DV);
+            if (col0 < DV) tmem_row_to_tile(R2 + col0, sStg, r, col0);      // slab partial of dV -> staging -> TMA store
+            fence_async_smem();
             tc_fence_before();
-            mbar_arrive(bars + KE3);
+            mbar_arrive_warp(bars + KE3);
+            epi_sync();
+            if (tid == 0) {
+                for (int a = 0; a < DV / 64; ++a) tma_store_2d(&p.mapPV, sStg + a * 16384, a * 64, (int)(prow - r));
+                tma_store_commit();
+            }
 
             EWAIT(KM7); if (!ok) break;
             tc_fence_after();
-            float es = 0.f;
-            for (int c0 = 0; c0 < 128; c0 += 32) {       // E = Bf .* (dP^T A^ + V R^T + rho^T), in place over Bf
+            {   // E = Bf .* (dP^T A^ + V R^T + rho^T), in place over Bf
+                float es = 0.f;
                 uint32_t v[32];
-                tmem_ld32(R2 + c0, v);
+                tmem_ld32(R2 + col0, v);
                 tmem_wait_ld();
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
-                    uint4 *cell = reinterpret_cast<uint4 *>(tile_chunk(sKB, tid, c0 / 8 + q));
+                    uint4 *cell = reinterpret_cast<uint4 *>(tile_chunk(sKB, r, col0 / 8 + q));
                     float b[8];
                     unpack8(*cell, b);
-                    const float4 r0 = *reinterpret_cast<const float4 *>(sRho + c0 + 8 * q);
-                    const float4 r1 = *reinterpret_cast<const float4 *>(sRho + c0 + 8 * q + 4);
+                    const float4 r0 = *reinterpret_cast<const float4 *>(sRho + col0 + 8 * q);
+                    const float4 r1 = *reinterpret_cast<const float4 *>(sRho + col0 + 8 * q + 4);
                     const float rr[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
                     float e[8];
 #pragma unroll
                     for (int j = 0; j < 8; ++j) { e[j] = b[j] * (__uint_as_float(v[8 * q + j]) + rr[j]); es += e[j]; }
                     *cell = make_uint4(pack_bf16(e[0], e[1]), pack_bf16(e[2], e[3]), pack_bf16(e[4], e[5]), pack_bf16(e[6], e[7]));
                 }
+                p.espart[((size_t)slab * 4 + g) * rows + row] = es;
             }
-            p.espart[prow] = es;
             fence_async_smem();
+            if (tid == 0) tma_store_wait_read();      // staging free again before anyone passes KE4
             tc_fence_before();
-            mbar_arrive(bars + KE4);
+            mbar_arrive_warp(bars + KE4);
 
             EWAIT(KM8); if (!ok) break;
             tc_fence_after();
-            tmem_row_to_global<D>(R2, p.pdK + prow * D);
-            if (!last) {     // R (updated before KM6 completed) -> bf16 copy; rho_next for the chunk below
-                tmem_row_to_tile<DV>(lane_addr + kColState, sSt, tid);
-                sRho[tid] += rho_c;
+            if (col0 < D) tmem_row_to_tile(R2 + col0, sStg, r, col0);       // slab partial of dK -> staging -> TMA store
+            fence_async_smem();
+            epi_sync();
+            if (tid == 0) {
+                for (int a = 0; a < D / 64; ++a) tma_store_2d(&p.mapPK, sStg + a * 16384, a * 64, (int)(prow - r));
+                tma_store_commit();
+            }
+            if (!last) {     // R (its update completed before KM6) -> bf16 copy; rho_next for the chunk below
+                if (col0 < DV) tmem_row_to_tile(lane_addr + kColState + col0, sSt, r, col0);
+                if (g0) sRho[r] += rho_c;
                 fence_async_smem();
             }
+            if (tid == 0) tma_store_wait_read();
             tc_fence_before();
-            mbar_arrive(bars + KE5);
+            mbar_arrive_warp(bars + KE5);
 #undef EWAIT
         }
+        if (tid == 0) tma_store_wait_all();
         if (ok) ok = wait_or_abort(bars + KM9, (T - 1) & 1, status, abort_flag);
-        if (ok) {
+        if (ok && col0 < D) {
             tc_fence_after();
-            float *dst = p.Tacc + ((size_t)h * p.m + slab * 128 + tid) * D;
-            for (int c0 = 0; c0 < D; c0 += 32) {
-                uint32_t v[32];
-                tmem_ld32(lane_addr + kColT + c0, v);
-                tmem_wait_ld();
+            float *dst = p.Tacc + ((size_t)h * p.m + slab * 128 + r) * D + col0;
+            uint32_t v[32];
+            tmem_ld32(lane_addr + kColT + col0, v);
+            tmem_wait_ld();
 #pragma unroll
-                for (int j = 0; j < 32; ++j) atomicAdd(dst + c0 + j, __uint_as_float(v[j]));
-            }
+            for (int j = 0; j < 32; ++j) atomicAdd(dst + j, __uint_as_float(v[j]));
         }
     }
     if (*abort_flag) __nanosleep(200000);
     tc_fence_before();
     __syncthreads();
-    if (warp == 4) tmem_dealloc(tmem, 512);
+    if (warp == kEpiWarps) tmem_dealloc(tmem, 512);
 }
 
 // ------------------------------------------------------------------ dK: slab sum + norm term (three MMAs per tile)
@@ -600,36 +661,36 @@ __global__ void __launch_bounds__(160, 1) tc_bwd_k_kernel(const __grid_constant_
 struct FinishParams {
     CUtensorMap mapK, mapM;
     const __nv_bfloat16 *pdK;
-    const float *espart;
+    const float *espart;  // [nes, BH*N]
     __nv_bfloat16 *dK;
     float *dMn;           // [H, r, D]
     int *status;
-    int N, H, BH, T, nsplit, r, nslab;
+    int N, H, BH, T, nsplit, r, nslab, nes;
     float s2;
 };
 
 template <int D>
-__global__ void __launch_bounds__(160, 1) tc_bwd_finish_k_kernel(const __grid_constant__ FinishParams p)
+__global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __grid_constant__ FinishParams p)
 {
     extern __shared__ __align__(1024) unsigned char smem[];
     constexpr int kTile = 128 * D * 2;
-    unsigned char *sM = smem, *sK = smem + kTile, *sW = smem + 2 * kTile;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + 2 * kTile + 32768);
-    uint64_t *bar_m = bars, *bar_k = bars + 1, *m1 = bars + 2, *m2 = bars + 3, *m3 = bars + 4, *e1 = bars + 5, *e2 = bars + 6;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 7);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 8);
+    unsigned char *sM = smem, *sK0 = smem + kTile, *sW = smem + 3 * kTile;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + 3 * kTile + 32768);
+    uint64_t *bar_m = bars, *bar_k = bars + 1 /* two */, *m1 = bars + 3, *m2 = bars + 4, *m3 = bars + 5, *e1 = bars + 6, *e2 = bars + 7;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 9);
     const int tid = threadIdx.x, warp = tid >> 5;
     const int bh = blockIdx.x / p.nsplit, split = blockIdx.x % p.nsplit, h = bh % p.H;
     const int t0 = (int)((long long)p.T * split / p.nsplit), t1 = (int)((long long)p.T * (split + 1) / p.nsplit);
     if (tid == 0) {
-        for (int i = 0; i < 5; ++i) mbar_init(bars + i, 1);
-        mbar_init(e1, 128); mbar_init(e2, 128);
+        for (int i = 0; i < 6; ++i) mbar_init(bars + i, 1);
+        mbar_init(e1, kEpiWarps); mbar_init(e2, kEpiWarps);
         *abort_flag = (smem_u32(smem) & 1023u) ? 1 : 0;
         fence_mbar_init();
     }
     if (tid < 128)      // columns >= r of the w tile stay zero
         for (int i = tid; i < 2048; i += 128) *reinterpret_cast<uint4 *>(sW + i * 16) = make_uint4(0, 0, 0, 0);
-    if (warp == 4) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+    if (warp == kEpiWarps) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -637,106 +698,120 @@ __global__ void __launch_bounds__(160, 1) tc_bwd_finish_k_kernel(const __grid_co
     constexpr uint32_t C1 = 0, C2 = 128, C3 = 256;
     if (*abort_flag) { if (tid == 0) atomicExch(p.status, (int)DARKATTN_ERR_CUDA); }
     else if (t1 <= t0) {}
-    else if (warp == 4) {
+    else if (warp == kEpiWarps) {
         if ((tid & 31) == 0) {
-            auto kdesc = [](unsigned char *base, int k) { return make_sdesc(smem_u32(base) + (k / 4) * 16384 + (k % 4) * 32, 16, 1024); };
-            auto mndesc = [](unsigned char *base, int k) { return make_sdesc(smem_u32(base) + k * 2048, 16384, 1024); };
+            const TileDesc tM(sM), tW(sW), tK0(sK0), tK1(sK0 + kTile);
+            auto load_k = [&](int t) {
+                const int b = (t - t0) & 1;
+                mbar_expect_tx(bar_k + b, kTile);
+                for (int a = 0; a < D / 64; ++a) tma_load_2d(sK0 + b * kTile + a * 16384, &p.mapK, bar_k + b, a * 64, bh * p.N + t * 128);
+            };
             mbar_expect_tx(bar_m, kTile);
             for (int a = 0; a < D / 64; ++a) tma_load_2d(sM + a * 16384, &p.mapM, bar_m, a * 64, h * p.r);
-            mbar_expect_tx(bar_k, kTile);
-            for (int a = 0; a < D / 64; ++a) tma_load_2d(sK + a * 16384, &p.mapK, bar_k, a * 64, bh * p.N + t0 * 128);
+            load_k(t0);
             const uint32_t id_x = make_idesc(128, p.r, 0, 0), id_d = make_idesc(128, D, 0, 1), id_t = make_idesc(128, D, 1, 1);
             bool ok = wait_or_abort(bar_m, 0, p.status, abort_flag);
             for (int t = t0; t < t1 && ok; ++t) {
-                const uint32_t ph = (t - t0) & 1;
-                ok = wait_or_abort(bar_k, ph, p.status, abort_flag);
+                const int i = t - t0, b = i & 1;
+                const uint32_t ph = i & 1, phk = (i >> 1) & 1;
+                const TileDesc &tK = b ? tK1 : tK0;
+                if (t + 1 < t1) load_k(t + 1);          // the other buffer: its last reader finished before m3 of tile t-1
+                ok = wait_or_abort(bar_k + b, phk, p.status, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                for (int k = 0; k < D / 16; ++k) mma_ss(tmem + C1, kdesc(sK, k), kdesc(sM, k), id_x, k > 0);
+                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(tmem + C1, kdesc(tK, k), kdesc(tM, k), id_x, k > 0);
                 mma_commit(m1);
                 ok = wait_or_abort(e1, ph, p.status, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                for (int k = 0; k < p.r / 16; ++k) mma_ss(tmem + C2, kdesc(sW, k), mndesc(sM, k), id_d, k > 0);
+                _Pragma("unroll") for (int k = 0; k < p.r / 16; ++k) mma_ss(tmem + C2, kdesc(tW, k), mndesc(tM, k), id_d, k > 0);
                 mma_commit(m2);
-                for (int k = 0; k < 8; ++k) mma_ss(tmem + C3, mndesc(sW, k), mndesc(sK, k), id_t, (t > t0) || k > 0);
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + C3, mndesc(tW, k), mndesc(tK, k), id_t, (t > t0) || k > 0);
                 mma_commit(m3);
                 ok = wait_or_abort(m3, ph, p.status, abort_flag);
                 if (!ok) break;
-                if (t + 1 < t1) {
-                    mbar_expect_tx(bar_k, kTile);
-                    for (int a = 0; a < D / 64; ++a) tma_load_2d(sK + a * 16384, &p.mapK, bar_k, a * 64, bh * p.N + (t + 1) * 128);
-                }
                 ok = wait_or_abort(e2, ph, p.status, abort_flag);
             }
         }
     } else {
-        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+        const int lane = tid & 31, q4 = warp & 3, col0 = (warp >> 2) * 32;
+        const int r = q4 * 32 + lane;
+        const uint32_t lane_addr = tmem + ((uint32_t)(q4 * 32) << 16);
         const size_t rows = (size_t)p.BH * p.N;
         bool ok = true;
         for (int t = t0; t < t1 && ok; ++t) {
             const uint32_t ph = (t - t0) & 1;
-            const size_t row = (size_t)bh * p.N + (size_t)t * 128 + tid;
+            const size_t row = (size_t)bh * p.N + (size_t)t * 128 + r;
             float es = 0.f;
-            for (int s = 0; s < p.nslab; ++s) es += p.espart[(size_t)s * rows + row];
+            for (int s = 0; s < p.nes; ++s) es += p.espart[(size_t)s * rows + row];
             const float coef = -p.s2 * es;
-            ok = wait_or_abort(m1, ph, p.status, abort_flag);
+            float acc[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) acc[j] = 0.f;
+            if (col0 < D) {
+                for (int s = 0; s < p.nslab; ++s) {
+                    const uint4 *src = reinterpret_cast<const uint4 *>(p.pdK + ((size_t)s * rows + row) * D + col0);
+                    uint4 raw[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) raw[q] = src[q];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        float f[8];
+                        unpack8(raw[q], f);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) acc[8 * q + j] += f[j];
+                    }
+                }
+            }
+            ok = __all_sync(0xffffffffu, wait_or_abort(m1, ph, p.status, abort_flag));
             if (!ok) break;
             tc_fence_after();
-            for (int c0 = 0; c0 < p.r; c0 += 16) {
-                uint32_t v[16];
-                tmem_ld16(lane_addr + C1 + c0, v);
-                tmem_wait_ld();
 #pragma unroll
-                for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(coef * __uint_as_float(v[j]));
-                *reinterpret_cast<uint4 *>(tile_chunk(sW, tid, c0 / 8)) = pack8(v);
-                *reinterpret_cast<uint4 *>(tile_chunk(sW, tid, c0 / 8 + 1)) = pack8(v + 8);
+            for (int hh = 0; hh < 2; ++hh) {
+                const int c = col0 + 16 * hh;
+                if (c < p.r) {
+                    uint32_t v[16];
+                    tmem_ld16(lane_addr + C1 + c, v);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(coef * __uint_as_float(v[j]));
+                    *reinterpret_cast<uint4 *>(tile_chunk(sW, r, c / 8)) = pack8(v);
+                    *reinterpret_cast<uint4 *>(tile_chunk(sW, r, c / 8 + 1)) = pack8(v + 8);
+                }
             }
             fence_async_smem();
             tc_fence_before();
-            mbar_arrive(e1);
-            ok = wait_or_abort(m2, ph, p.status, abort_flag);
+            mbar_arrive_warp(e1);
+            ok = __all_sync(0xffffffffu, wait_or_abort(m2, ph, p.status, abort_flag));
             if (!ok) break;
             tc_fence_after();
-            for (int c0 = 0; c0 < D; c0 += 32) {
+            if (col0 < D) {
                 uint32_t v[32];
-                tmem_ld32(lane_addr + C2 + c0, v);
+                tmem_ld32(lane_addr + C2 + col0, v);
                 tmem_wait_ld();
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-                    for (int s = 0; s < p.nslab; ++s) {
-                        float f[8];
-                        unpack8(*reinterpret_cast<const uint4 *>(p.pdK + ((size_t)s * rows + row) * D + c0 + 8 * q), f);
+                for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(fmaf(kLn2, acc[j], __uint_as_float(v[j])));
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) acc[j] += f[j];
-                    }
-                    uint32_t o[8];
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) o[j] = __float_as_uint(fmaf(kLn2, acc[j], __uint_as_float(v[8 * q + j])));
-                    *reinterpret_cast<uint4 *>(p.dK + row * D + c0 + 8 * q) = pack8(o);
-                }
+                for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4 *>(p.dK + row * D + col0 + 8 * q) = pack8(v + 8 * q);
             }
             tc_fence_before();
-            mbar_arrive(e2);
+            mbar_arrive_warp(e2);
         }
         if (ok) ok = wait_or_abort(m3, (t1 - 1 - t0) & 1, p.status, abort_flag);
-        if (ok && tid < p.r) {
+        if (ok && r < p.r && col0 < D) {
             tc_fence_after();
-            float *dst = p.dMn + ((size_t)h * p.r + tid) * D;
-            for (int c0 = 0; c0 < D; c0 += 32) {
-                uint32_t v[32];
-                tmem_ld32(lane_addr + C3 + c0, v);
-                tmem_wait_ld();
+            float *dst = p.dMn + ((size_t)h * p.r + r) * D + col0;
+            uint32_t v[32];
+            tmem_ld32(lane_addr + C3 + col0, v);
+            tmem_wait_ld();
 #pragma unroll
-                for (int j = 0; j < 32; ++j) atomicAdd(dst + c0 + j, __uint_as_float(v[j]));
-            }
+            for (int j = 0; j < 32; ++j) atomicAdd(dst + j, __uint_as_float(v[j]));
         }
     }
     if (*abort_flag) __nanosleep(200000);
     tc_fence_before();
     __syncthreads();
-    if (warp == 4) tmem_dealloc(tmem, 512);
+    if (warp == kEpiWarps) tmem_dealloc(tmem, 512);
 }
 
 // ------------------------------------------------------------------ small SIMT kernels
@@ -796,20 +871,20 @@ cudaError_t launch_scan(const BwdParams &P, int grid, cudaStream_t st)
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(tc_bwd_k_kernel<D, DV>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
     if (e != cudaSuccess) return e;
-    tc_bwd_q_kernel<D, DV><<<grid, 160, L::kTotal, st>>>(P);
+    tc_bwd_q_kernel<D, DV><<<grid, kThreads, L::kTotal, st>>>(P);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    tc_bwd_k_kernel<D, DV><<<grid, 160, L::kTotal, st>>>(P);
+    tc_bwd_k_kernel<D, DV><<<grid, kThreads, L::kTotal, st>>>(P);
     return cudaGetLastError();
 }
 
 template <int D>
 cudaError_t launch_finish(const FinishParams &P, int grid, cudaStream_t st)
 {
-    constexpr int smem_bytes = 2 * 128 * D * 2 + 32768 + 128;
+    constexpr int smem_bytes = 3 * 128 * D * 2 + 32768 + 128;
     cudaError_t e = cudaFuncSetAttribute(tc_bwd_finish_k_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
     if (e != cudaSuccess) return e;
-    tc_bwd_finish_k_kernel<D><<<grid, 160, smem_bytes, st>>>(P);
+    tc_bwd_finish_k_kernel<D><<<grid, kThreads, smem_bytes, st>>>(P);
     return cudaGetLastError();
 }
 
@@ -854,7 +929,10 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
     memset(&P, 0, sizeof(P));
     bool ok = make_map(&P.mapQ, Q, BH * N, D.d, 128) && make_map(&P.mapK, K, BH * N, D.d, 128) &&
               make_map(&P.mapV, V, BH * N, D.dv, 128) && make_map(&P.mapG, dO, BH * N, D.dv, 128) &&
-              make_map(&P.mapOm, bf(Y.Om), (size_t)D.H * D.m, D.d, 128);
+              make_map(&P.mapOm, bf(Y.Om), (size_t)D.H * D.m, D.d, 128) &&
+              make_map(&P.mapPQ, bf(Y.pdQ), (size_t)Y.nslab * BH * N, D.d, 128) &&
+              make_map(&P.mapPK, bf(Y.pdK), (size_t)Y.nslab * BH * N, D.d, 128) &&
+              make_map(&P.mapPV, bf(Y.pdV), (size_t)Y.nslab * BH * N, D.dv, 128);
     FinishParams F;
     memset(&F, 0, sizeof(F));
     ok = ok && make_map(&F.mapM, M, (size_t)D.H * D.r, D.d, 128);
@@ -879,7 +957,7 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
     }
     F.pdK = bf(Y.pdK); F.espart = fl(Y.espart); F.dK = (__nv_bfloat16 *)dK; F.dMn = fl(Y.dMn);
     F.status = P.status;
-    F.N = D.N; F.H = D.H; F.BH = D.BH; F.T = Y.T; F.r = D.r; F.nslab = Y.nslab; F.s2 = D.s * D.s;
+    F.N = D.N; F.H = D.H; F.BH = D.BH; F.T = Y.T; F.r = D.r; F.nslab = Y.nslab; F.nes = 4 * Y.nslab; F.s2 = D.s * D.s;
     F.nsplit = (int)((148 * 2 + BH - 1) / BH);
     if (F.nsplit > Y.T) F.nsplit = Y.T;
     if (D.d == 64) keep(launch_finish<64>(F, (int)(BH * F.nsplit), st));

@@ -624,7 +624,7 @@ void tensor_make_layout(darkattn_plan_s *plan)
         Y.pdQ = take(off, (size_t)Y.nslab * BH * N * d * 2);
         Y.pdK = take(off, (size_t)Y.nslab * BH * N * d * 2);
         Y.pdV = take(off, (size_t)Y.nslab * BH * N * dv * 2);
-        Y.espart = take(off, (size_t)Y.nslab * BH * N * 4);
+        Y.espart = take(off, (size_t)4 * Y.nslab * BH * N * 4);
         Y.Tacc = take(off, (size_t)D.H * m * d * 4);
         Y.dMn = take(off, (size_t)D.H * D.r * d * 4);
         plan->launches_bwd = 3 + 1 + 2 + 3 + 1;   // prologue, delta, two scan kernels, three combines, dM
