@@ -181,7 +181,7 @@ __device__ __forceinline__ uint64_t kdesc(const TileDesc &t, int k) { return t.k
 // MN-major operand: step k covers 16 K-rows of 128 bytes
 __device__ __forceinline__ uint64_t mndesc(const TileDesc &t, int k) { return t.mnmaj + (uint64_t)((k * 2048) >> 4); }
 
-enum QBars { QB_OM, QB_Q, QB_K, QB_V, QB_G, QB_X2, QM1, QM2, QM3, QMS, QM4, QM5, QM6, QE1, QE2, QE3, QE4, QNBARS };
+enum QBars { QB_OM, QB_Q, QB_K, QB_V, QB_G, QB_X2, QM1, QM2, QM3, QMS, QM4, QM5, QM6, QE0, QE1, QE2, QE3, QE4, QNBARS };
 
 // ------------------------------------------------------------------ query side (forward direction)
 template <int D, int DV>
@@ -201,8 +201,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
     const int row0 = bh * p.N, T = p.T;
 
     if (tid == 0) {
-        for (int i = 0; i < QE1; ++i) mbar_init(bars + i, 1);
-        for (int i = QE1; i < QNBARS; ++i) mbar_init(bars + i, kEpiWarps);
+        for (int i = 0; i < QE0; ++i) mbar_init(bars + i, 1);
+        for (int i = QE0; i < QNBARS; ++i) mbar_init(bars + i, kEpiWarps);
         *abort_flag = (smem_u32(smem) & 1023u) ? 1 : 0;
         fence_mbar_init();
     }
@@ -237,7 +237,17 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
             load_tile(sV, &p.mapV, bars + QB_V, DV, 0);
             load_tile(sG, &p.mapG, bars + QB_G, DV, 0);
 
+            // Schedule of one chunk (R1, R2: the two scratch regions of TMEM). U_K of the next chunk is issued in
+            // the tail of the current one, and dO V^T runs while the epilogue is still busy with A^.
+            //   R2: U_K -> (Bf read) -> dO V^T -> packed dP (A operand of dP Bf) -> U_K of the next chunk
+            //   R1: U_Q -> (A^ read) -> dP Bf + dO S^T -> (E read) -> E Omega -> (dQ read)
             bool ok = wait_or_abort(bars + QB_OM, 0, status, abort_flag);
+            if (ok) ok = wait_or_abort(bars + QB_K, 0, status, abort_flag);
+            if (ok) {
+                tc_fence_after();
+                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R2, kdesc(tKB, k), kdesc(tOm, k), id_kk, k > 0);       // U_K of chunk 0
+                mma_commit(bars + QM2);
+            }
             for (int t = 0; t < T && ok; ++t) {
                 const uint32_t ph = t & 1;
                 const bool first = (t == 0), last = (t + 1 == T);
@@ -246,24 +256,20 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                 tc_fence_after();
                 _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R1, kdesc(tQA, k), kdesc(tOm, k), id_kk, k > 0);       // U_Q
                 mma_commit(bars + QM1);
-                QWAIT(QB_K); if (!ok) break;
-                tc_fence_after();
-                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R2, kdesc(tKB, k), kdesc(tOm, k), id_kk, k > 0);       // U_K
-                mma_commit(bars + QM2);
-                QWAIT(QE1); if (!ok) break;
-                tc_fence_after();
+                QWAIT(QE0); if (!ok) break;                                                                      // Bf in smem, R2 read
                 QWAIT(QB_V); if (!ok) break;
                 QWAIT(QB_G); if (!ok) break;
                 tc_fence_after();
-                _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R1, kdesc(tG, k), kdesc(tV, k), id_kk, k > 0);         // dO V^T
+                _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R2, kdesc(tG, k), kdesc(tV, k), id_kk, k > 0);         // dO V^T
                 mma_commit(bars + QM3);
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColState, mndesc(tKB, k), mndesc(tV, k), id_state, (!first) || k > 0);   // S += Bf^T V
                 mma_commit(bars + QMS);
-                QWAIT(QE2); if (!ok) break;
+                QWAIT(QE1); if (!ok) break;                                                                      // A^ in smem, R1 read
+                QWAIT(QE2); if (!ok) break;                                                                      // dP packed in R2
                 tc_fence_after();
-                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R2, R1 + k * 8, mndesc(tKB, k), id_tm, k > 0);               // dP Bf
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R1, R2 + k * 8, mndesc(tKB, k), id_tm, k > 0);               // dP Bf
                 if (!first)
-                    _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R2, kdesc(tG, k), kdesc(tSt, k), id_kk, 1);        // + dO S_prev^T
+                    _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R1, kdesc(tG, k), kdesc(tSt, k), id_kk, 1);        // + dO S_prev^T
                 mma_commit(bars + QM4);
                 QWAIT(QM4); if (!ok) break;
                 load_tile(sG, &p.mapQ, bars + QB_X2, D, t);                                                     // Q again, for T
@@ -275,6 +281,13 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                 mma_commit(bars + QM5);
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColT, mndesc(tQA, k), mndesc(tG, k), id_t, (!first) || k > 0);   // T += E^T Q
                 mma_commit(bars + QM6);
+                if (!last) {
+                    ok = wait_or_abort(bars + QB_K, ph ^ 1, status, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R2, kdesc(tKB, k), kdesc(tOm, k), id_kk, k > 0);   // U_K of the next chunk
+                    mma_commit(bars + QM2);
+                }
                 QWAIT(QM6); if (!ok) break;
                 if (!last) { load_tile(sQA, &p.mapQ, bars + QB_Q, D, t + 1); load_tile(sG, &p.mapG, bars + QB_G, DV, t + 1); }
                 QWAIT(QE4); if (!ok) break;
@@ -300,28 +313,24 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
             const float del = p.delta[row];
             const float nk = p.nK[row] + cshift;
             const float aq = svv.y - cshift + log2f(svv.x);
-            EWAIT(QM1); if (!ok) break;
-            tc_fence_after();
-            features_to_tile_sums(R1 + col0, aq, sQA, r, col0, -del, sRc, lane);      // A^ and rho_c = -sum_i delta_i A^_il
             EWAIT(QM2); if (!ok) break;
             tc_fence_after();
             features_to_tile_sums(R2 + col0, nk, sKB, r, col0, 1.f, sZc, lane);       // Bf and z_c = sum_j Bf_jl
+            fence_async_smem();
+            tc_fence_before();
+            mbar_arrive_warp(bars + QE0);
+            EWAIT(QM1); if (!ok) break;
+            tc_fence_after();
+            features_to_tile_sums(R1 + col0, aq, sQA, r, col0, -del, sRc, lane);      // A^ and rho_c = -sum_i delta_i A^_il
             fence_async_smem();
             tc_fence_before();
             mbar_arrive_warp(bars + QE1);
 
             EWAIT(QM3); if (!ok) break;
             tc_fence_after();
-            float znew = zrun;
-            if (own) {      // the column sums of all four lane quarters are in (every warp arrived at QE1)
-                znew = zrun + sZc[col0 + lane];
-                p.rhoc[((size_t)bh * T + t) * p.m + slab * 128 + col0 + lane] = sRc[col0 + lane];
-                sZc[col0 + lane] = 0.f;
-                sRc[col0 + lane] = 0.f;
-            }
             {   // dP = tril(dO V^T - delta) as a bf16 operand in TMEM (packed over the fp32 tile)
                 uint32_t v[32], pk[16];
-                tmem_ld32(R1 + col0, v);
+                tmem_ld32(R2 + col0, v);
                 tmem_wait_ld();
                 quarter_sync(q4);                         // every column group has read before anyone overwrites
 #pragma unroll
@@ -330,7 +339,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                     const float x1 = (col0 + j + 1 <= r) ? __uint_as_float(v[j + 1]) - del : 0.f;
                     pk[j / 2] = pack_bf16(x0, x1);
                 }
-                tmem_st16(R1 + col0 / 2, pk);
+                tmem_st16(R2 + col0 / 2, pk);
             }
             tmem_wait_st();
             tc_fence_before();
@@ -338,9 +347,16 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
 
             EWAIT(QM4); if (!ok) break;
             tc_fence_after();
+            float znew = zrun;
+            if (own) {      // the column sums of all four lane quarters are in (every warp arrived at QE0 and QE1)
+                znew = zrun + sZc[col0 + lane];
+                p.rhoc[((size_t)bh * T + t) * p.m + slab * 128 + col0 + lane] = sRc[col0 + lane];
+                sZc[col0 + lane] = 0.f;
+                sRc[col0 + lane] = 0.f;
+            }
             {   // E = A^ .* (dP Bf + dO S^T - delta z^T), in place over A^
                 uint32_t v[32];
-                tmem_ld32(R2 + col0, v);
+                tmem_ld32(R1 + col0, v);
                 tmem_wait_ld();
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
@@ -400,7 +416,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
     if (warp == kEpiWarps) tmem_dealloc(tmem, 512);
 }
 
-enum KBars { KB_OM, KB_Q, KB_K, KB_V, KB_G, KB_X2, KM1, KM2, KM3, KM4, KM5, KM6, KM7, KM8, KM9, KE1, KE2, KE3, KE4, KE5, KNBARS };
+enum KBars { KB_OM, KB_Q, KB_K, KB_V, KB_G, KB_X2, KM1, KM2, KM3, KM4, KM5, KM6, KM7, KM8, KM9, KE0, KE1, KE2, KE3, KE4, KE5, KNBARS };
 
 // ------------------------------------------------------------------ key side (reverse direction)
 template <int D, int DV>
@@ -420,8 +436,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
     const int row0 = bh * p.N, T = p.T;
 
     if (tid == 0) {
-        for (int i = 0; i < KE1; ++i) mbar_init(bars + i, 1);
-        for (int i = KE1; i < KNBARS; ++i) mbar_init(bars + i, kEpiWarps);
+        for (int i = 0; i < KE0; ++i) mbar_init(bars + i, 1);
+        for (int i = KE0; i < KNBARS; ++i) mbar_init(bars + i, kEpiWarps);
         *abort_flag = (smem_u32(smem) & 1023u) ? 1 : 0;
         fence_mbar_init();
     }
@@ -457,40 +473,47 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
             load_tile(sV, &p.mapV, bars + KB_V, DV, T - 1);
             load_tile(sG, &p.mapG, bars + KB_G, DV, T - 1);
 
+            // Schedule of one chunk. U_Q of the next chunk is issued in the tail of the current one, and V dO^T
+            // runs while the epilogue is still busy with Bf.
+            //   R1: U_Q -> (A^ read) -> V dO^T -> packed dP^T [0,64) and P^^T [64,128) (A operands) -> U_Q of the next chunk
+            //   R2: U_K -> (Bf read) -> Bf A^^T -> dV -> dBf -> dK partial
             bool ok = wait_or_abort(bars + KB_OM, 0, status, abort_flag);
+            if (ok) ok = wait_or_abort(bars + KB_Q, 0, status, abort_flag);
+            if (ok) {
+                tc_fence_after();
+                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R1, kdesc(tQA, k), kdesc(tOm, k), id_kk, k > 0);       // U_Q of the last chunk
+                mma_commit(bars + KM1);
+            }
             for (int it = 0; it < T && ok; ++it) {
                 const int t = T - 1 - it;
                 const uint32_t ph = it & 1;
                 const bool first = (it == 0), last = (it + 1 == T);
 #define KWAIT(b) do { ok = wait_or_abort(bars + (b), ph, status, abort_flag); } while (0)
-                KWAIT(KB_Q); if (!ok) break;
-                tc_fence_after();
-                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R1, kdesc(tQA, k), kdesc(tOm, k), id_kk, k > 0);       // U_Q
-                mma_commit(bars + KM1);
                 KWAIT(KB_K); if (!ok) break;
                 tc_fence_after();
                 _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R2, kdesc(tKB, k), kdesc(tOm, k), id_kk, k > 0);       // U_K
                 mma_commit(bars + KM2);
-                KWAIT(KE1); if (!ok) break;
-                tc_fence_after();
-                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R1, kdesc(tKB, k), kdesc(tQA, k), id_kk, k > 0);             // P^^T = Bf A^^T
-                mma_commit(bars + KM3);
+                KWAIT(KE0); if (!ok) break;                                                                      // A^ in smem, R1 read
                 KWAIT(KB_V); if (!ok) break;
                 KWAIT(KB_G); if (!ok) break;
                 tc_fence_after();
-                _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R2, kdesc(tV, k), kdesc(tG, k), id_kk, k > 0);         // V dO^T
-                mma_commit(bars + KM4);
+                _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R1, kdesc(tV, k), kdesc(tG, k), id_kk, k > 0);         // V dO^T
+                mma_commit(bars + KM3);
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColState, mndesc(tQA, k), mndesc(tG, k), id_state, (!first) || k > 0);   // R += A^^T dO
                 mma_commit(bars + KM5);
+                KWAIT(KE1); if (!ok) break;                                                                      // Bf in smem, R2 read
+                tc_fence_after();
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R2, kdesc(tKB, k), kdesc(tQA, k), id_kk, k > 0);             // P^^T = Bf A^^T
+                mma_commit(bars + KM4);
                 KWAIT(KE2); if (!ok) break;
                 tc_fence_after();
-                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R2, R1 + k * 8, mndesc(tG, k), id_dv_t, k > 0);              // P^^T dO
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R2, R1 + 64 + k * 8, mndesc(tG, k), id_dv_t, k > 0);         // P^^T dO
                 if (!first)
                     _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R2, kdesc(tKB, k), mndesc(tSt, k), id_dv_t, 1);          // + Bf R_next
                 mma_commit(bars + KM6);
                 KWAIT(KE3); if (!ok) break;
                 tc_fence_after();
-                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R2, R1 + 64 + k * 8, mndesc(tQA, k), id_tm, k > 0);          // dP^T A^
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R2, R1 + k * 8, mndesc(tQA, k), id_tm, k > 0);               // dP^T A^
                 if (!first)
                     _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R2, kdesc(tV, k), kdesc(tSt, k), id_kk, 1);        // + V R_next^T
                 mma_commit(bars + KM7);
@@ -504,6 +527,13 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
                 mma_commit(bars + KM8);
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColT, mndesc(tKB, k), mndesc(tG, k), id_t, (!first) || k > 0);   // T += E^T K
                 mma_commit(bars + KM9);
+                if (!last) {
+                    ok = wait_or_abort(bars + KB_Q, ph ^ 1, status, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R1, kdesc(tQA, k), kdesc(tOm, k), id_kk, k > 0);   // U_Q of the next chunk
+                    mma_commit(bars + KM1);
+                }
                 KWAIT(KM9); if (!ok) break;
                 if (!last) { load_tile(sKB, &p.mapK, bars + KB_K, D, t - 1); load_tile(sG, &p.mapG, bars + KB_G, DV, t - 1); }
                 KWAIT(KE5); if (!ok) break;
@@ -537,6 +567,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
             EWAIT(KM1); if (!ok) break;
             tc_fence_after();
             features_to_tile(R1 + col0, aq, sQA, r, col0);
+            fence_async_smem();
+            tc_fence_before();
+            mbar_arrive_warp(bars + KE0);
             EWAIT(KM2); if (!ok) break;
             tc_fence_after();
             features_to_tile(R2 + col0, nk, sKB, r, col0);
@@ -546,30 +579,30 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
 
             EWAIT(KM3); if (!ok) break;
             tc_fence_after();
-            {   // P^^T masked to queries i >= this key, packed over the fp32 tile
+            {   // dP^T = (V dO^T - delta_i) masked to queries i >= this key, packed over the fp32 tile
                 uint32_t v[32], pk[16];
                 tmem_ld32(R1 + col0, v);
                 tmem_wait_ld();
                 quarter_sync(q4);
 #pragma unroll
                 for (int j = 0; j < 32; j += 2) {
-                    const float x0 = (col0 + j >= r) ? __uint_as_float(v[j]) : 0.f;
-                    const float x1 = (col0 + j + 1 >= r) ? __uint_as_float(v[j + 1]) : 0.f;
+                    const float2 dl = *reinterpret_cast<const float2 *>(sDel + col0 + j);
+                    const float x0 = (col0 + j >= r) ? __uint_as_float(v[j]) - dl.x : 0.f;
+                    const float x1 = (col0 + j + 1 >= r) ? __uint_as_float(v[j + 1]) - dl.y : 0.f;
                     pk[j / 2] = pack_bf16(x0, x1);
                 }
                 tmem_st16(R1 + col0 / 2, pk);
             }
             EWAIT(KM4); if (!ok) break;
             tc_fence_after();
-            {   // dP^T = (V dO^T - delta_i) masked, packed behind P^^T
+            {   // P^^T masked the same way, packed behind dP^T
                 uint32_t v[32], pk[16];
                 tmem_ld32(R2 + col0, v);
                 tmem_wait_ld();
 #pragma unroll
                 for (int j = 0; j < 32; j += 2) {
-                    const float2 dl = *reinterpret_cast<const float2 *>(sDel + col0 + j);
-                    const float x0 = (col0 + j >= r) ? __uint_as_float(v[j]) - dl.x : 0.f;
-                    const float x1 = (col0 + j + 1 >= r) ? __uint_as_float(v[j + 1]) - dl.y : 0.f;
+                    const float x0 = (col0 + j >= r) ? __uint_as_float(v[j]) : 0.f;
+                    const float x1 = (col0 + j + 1 >= r) ? __uint_as_float(v[j + 1]) : 0.f;
                     pk[j / 2] = pack_bf16(x0, x1);
                 }
                 tmem_st16(R1 + 64 + col0 / 2, pk);
@@ -659,32 +692,34 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
 //   w_j  = -s^2 rowsum(E^K)_j x~'_j   (bf16 operand)
 //   dK_j = ln2 sum_slabs part_j + w_j M          dMn += w^T K
 struct FinishParams {
-    CUtensorMap mapK, mapM;
-    const __nv_bfloat16 *pdK;
+    CUtensorMap mapK, mapM, mapP, mapOut;   // K, M, the slab partials of dK [nslab BH N, D], dK
     const float *espart;  // [nes, BH*N]
-    __nv_bfloat16 *dK;
     float *dMn;           // [H, r, D]
     int *status;
-    int N, H, BH, T, nsplit, r, nslab, nes;
+    int N, H, BH, T, nsplit, r, nslab, nes, pbufs;   // pbufs: partial tiles resident at a time
     float s2;
 };
 
+// Shared memory: M tile, two K tiles, the w tile (32 KB), the output staging tile, pbufs partial tiles, barriers.
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __grid_constant__ FinishParams p)
 {
     extern __shared__ __align__(1024) unsigned char smem[];
     constexpr int kTile = 128 * D * 2;
-    unsigned char *sM = smem, *sK0 = smem + kTile, *sW = smem + 3 * kTile;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + 3 * kTile + 32768);
-    uint64_t *bar_m = bars, *bar_k = bars + 1 /* two */, *m1 = bars + 3, *m2 = bars + 4, *m3 = bars + 5, *e1 = bars + 6, *e2 = bars + 7;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 8);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 9);
+    unsigned char *sM = smem, *sK0 = smem + kTile, *sW = smem + 3 * kTile, *sOut = sW + 32768, *sP = sOut + kTile;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(sP + (size_t)p.pbufs * kTile);
+    uint64_t *bar_m = bars, *bar_k = bars + 1 /* two */, *bar_p = bars + 3, *m1 = bars + 4, *m2 = bars + 5, *m3 = bars + 6;
+    uint64_t *e1 = bars + 7, *e2 = bars + 8, *e_p = bars + 9;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 10);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 11);
     const int tid = threadIdx.x, warp = tid >> 5;
     const int bh = blockIdx.x / p.nsplit, split = blockIdx.x % p.nsplit, h = bh % p.H;
     const int t0 = (int)((long long)p.T * split / p.nsplit), t1 = (int)((long long)p.T * (split + 1) / p.nsplit);
+    const int nrounds = (p.nslab + p.pbufs - 1) / p.pbufs;
+    const size_t rows = (size_t)p.BH * p.N;
     if (tid == 0) {
-        for (int i = 0; i < 6; ++i) mbar_init(bars + i, 1);
-        mbar_init(e1, kEpiWarps); mbar_init(e2, kEpiWarps);
+        for (int i = 0; i < 7; ++i) mbar_init(bars + i, 1);
+        mbar_init(e1, kEpiWarps); mbar_init(e2, kEpiWarps); mbar_init(e_p, kEpiWarps);
         *abort_flag = (smem_u32(smem) & 1023u) ? 1 : 0;
         fence_mbar_init();
     }
@@ -706,15 +741,26 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __gr
                 mbar_expect_tx(bar_k + b, kTile);
                 for (int a = 0; a < D / 64; ++a) tma_load_2d(sK0 + b * kTile + a * 16384, &p.mapK, bar_k + b, a * 64, bh * p.N + t * 128);
             };
+            auto load_partials = [&](int t, int round) {
+                const int s0 = round * p.pbufs, n = min(p.pbufs, p.nslab - s0);
+                mbar_expect_tx(bar_p, n * kTile);
+                for (int j = 0; j < n; ++j)
+                    for (int a = 0; a < D / 64; ++a)
+                        tma_load_2d(sP + (size_t)j * kTile + a * 16384, &p.mapP, bar_p, a * 64, (int)((size_t)(s0 + j) * rows + (size_t)bh * p.N + (size_t)t * 128));
+            };
             mbar_expect_tx(bar_m, kTile);
             for (int a = 0; a < D / 64; ++a) tma_load_2d(sM + a * 16384, &p.mapM, bar_m, a * 64, h * p.r);
             load_k(t0);
             const uint32_t id_x = make_idesc(128, p.r, 0, 0), id_d = make_idesc(128, D, 0, 1), id_t = make_idesc(128, D, 1, 1);
             bool ok = wait_or_abort(bar_m, 0, p.status, abort_flag);
+            uint32_t np = 0;                             // rounds of partial loads issued so far
             for (int t = t0; t < t1 && ok; ++t) {
                 const int i = t - t0, b = i & 1;
                 const uint32_t ph = i & 1, phk = (i >> 1) & 1;
                 const TileDesc &tK = b ? tK1 : tK0;
+                if (np > 0) ok = wait_or_abort(e_p, (np - 1) & 1, p.status, abort_flag);   // partial tiles consumed
+                if (!ok) break;
+                load_partials(t, 0); ++np;
                 if (t + 1 < t1) load_k(t + 1);          // the other buffer: its last reader finished before m3 of tile t-1
                 ok = wait_or_abort(bar_k + b, phk, p.status, abort_flag);
                 if (!ok) break;
@@ -724,10 +770,15 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __gr
                 ok = wait_or_abort(e1, ph, p.status, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                _Pragma("unroll") for (int k = 0; k < p.r / 16; ++k) mma_ss(tmem + C2, kdesc(tW, k), mndesc(tM, k), id_d, k > 0);
+                for (int k = 0; k < p.r / 16; ++k) mma_ss(tmem + C2, kdesc(tW, k), mndesc(tM, k), id_d, k > 0);
                 mma_commit(m2);
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + C3, mndesc(tW, k), mndesc(tK, k), id_t, (t > t0) || k > 0);
                 mma_commit(m3);
+                for (int round = 1; round < nrounds && ok; ++round) {
+                    ok = wait_or_abort(e_p, (np - 1) & 1, p.status, abort_flag);
+                    if (ok) { load_partials(t, round); ++np; }
+                }
+                if (!ok) break;
                 ok = wait_or_abort(m3, ph, p.status, abort_flag);
                 if (!ok) break;
                 ok = wait_or_abort(e2, ph, p.status, abort_flag);
@@ -737,32 +788,14 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __gr
         const int lane = tid & 31, q4 = warp & 3, col0 = (warp >> 2) * 32;
         const int r = q4 * 32 + lane;
         const uint32_t lane_addr = tmem + ((uint32_t)(q4 * 32) << 16);
-        const size_t rows = (size_t)p.BH * p.N;
         bool ok = true;
+        uint32_t np = 0;
         for (int t = t0; t < t1 && ok; ++t) {
             const uint32_t ph = (t - t0) & 1;
             const size_t row = (size_t)bh * p.N + (size_t)t * 128 + r;
             float es = 0.f;
             for (int s = 0; s < p.nes; ++s) es += p.espart[(size_t)s * rows + row];
             const float coef = -p.s2 * es;
-            float acc[32];
-#pragma unroll
-            for (int j = 0; j < 32; ++j) acc[j] = 0.f;
-            if (col0 < D) {
-                for (int s = 0; s < p.nslab; ++s) {
-                    const uint4 *src = reinterpret_cast<const uint4 *>(p.pdK + ((size_t)s * rows + row) * D + col0);
-                    uint4 raw[4];
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) raw[q] = src[q];
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        float f[8];
-                        unpack8(raw[q], f);
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) acc[8 * q + j] += f[j];
-                    }
-                }
-            }
             ok = __all_sync(0xffffffffu, wait_or_abort(m1, ph, p.status, abort_flag));
             if (!ok) break;
             tc_fence_after();
@@ -780,8 +813,30 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __gr
                 }
             }
             fence_async_smem();
+            if (tid == 0) tma_store_wait_read();          // the staging tile of the previous store is free again
             tc_fence_before();
             mbar_arrive_warp(e1);
+
+            float acc[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) acc[j] = 0.f;
+            for (int round = 0; round < nrounds && ok; ++round, ++np) {
+                ok = __all_sync(0xffffffffu, wait_or_abort(bar_p, np & 1, p.status, abort_flag));
+                if (!ok) break;
+                const int n = min(p.pbufs, p.nslab - round * p.pbufs);
+                if (col0 < D)
+                    for (int j = 0; j < n; ++j) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            float f[8];
+                            unpack8(*reinterpret_cast<const uint4 *>(tile_chunk(sP + (size_t)j * kTile, r, col0 / 8 + q)), f);
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) acc[8 * q + e] += f[e];
+                        }
+                    }
+                mbar_arrive_warp(e_p);
+            }
+            if (!ok) break;
             ok = __all_sync(0xffffffffu, wait_or_abort(m2, ph, p.status, abort_flag));
             if (!ok) break;
             tc_fence_after();
@@ -792,11 +847,18 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __gr
 #pragma unroll
                 for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(fmaf(kLn2, acc[j], __uint_as_float(v[j])));
 #pragma unroll
-                for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4 *>(p.dK + row * D + col0 + 8 * q) = pack8(v + 8 * q);
+                for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4 *>(tile_chunk(sOut, r, col0 / 8 + q)) = pack8(v + 8 * q);
+            }
+            fence_async_smem();
+            epi_sync();
+            if (tid == 0) {
+                for (int a = 0; a < D / 64; ++a) tma_store_2d(&p.mapOut, sOut + a * 16384, a * 64, (int)(row - r));
+                tma_store_commit();
             }
             tc_fence_before();
             mbar_arrive_warp(e2);
         }
+        if (tid == 0) tma_store_wait_all();
         if (ok) ok = wait_or_abort(m3, (t1 - 1 - t0) & 1, p.status, abort_flag);
         if (ok && r < p.r && col0 < D) {
             tc_fence_after();
@@ -879,9 +941,12 @@ cudaError_t launch_scan(const BwdParams &P, int grid, cudaStream_t st)
 }
 
 template <int D>
-cudaError_t launch_finish(const FinishParams &P, int grid, cudaStream_t st)
+cudaError_t launch_finish(FinishParams &P, int grid, cudaStream_t st)
 {
-    constexpr int smem_bytes = 3 * 128 * D * 2 + 32768 + 128;
+    constexpr int kTile = 128 * D * 2, kFixed = 4 * kTile + 32768 + 128;
+    P.pbufs = (232448 - kFixed) / kTile;
+    if (P.pbufs > P.nslab) P.pbufs = P.nslab;
+    const int smem_bytes = kFixed + P.pbufs * kTile;
     cudaError_t e = cudaFuncSetAttribute(tc_bwd_finish_k_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
     if (e != cudaSuccess) return e;
     tc_bwd_finish_k_kernel<D><<<grid, kThreads, smem_bytes, st>>>(P);
@@ -955,7 +1020,9 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
         sum_slabs_kernel<<<(unsigned)((tv + 255) / 256), 256, 0, st>>>(bf(Y.pdV), (__nv_bfloat16 *)dV, rows, D.dv, Y.nslab, 1.f);
         chk();
     }
-    F.pdK = bf(Y.pdK); F.espart = fl(Y.espart); F.dK = (__nv_bfloat16 *)dK; F.dMn = fl(Y.dMn);
+    F.mapP = P.mapPK;
+    if (!make_map(&F.mapOut, dK, BH * N, D.d, 128)) { set_cuda_error(cudaErrorInvalidValue, "tensor_backward: tensor map encode"); return DARKATTN_ERR_CUDA; }
+    F.espart = fl(Y.espart); F.dMn = fl(Y.dMn);
     F.status = P.status;
     F.N = D.N; F.H = D.H; F.BH = D.BH; F.T = Y.T; F.r = D.r; F.nslab = Y.nslab; F.nes = 4 * Y.nslab; F.s2 = D.s * D.s;
     F.nsplit = (int)((148 * 2 + BH - 1) / BH);
