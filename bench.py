@@ -26,6 +26,10 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# DRAM bytes (read + write) per launch of the dominant kernel from its ncu capture (profiles/), keyed by
+# kernel; a kernel that changed since its capture has no entry.
+NCU_TRAFFIC = {}
+
 METRIC = "DARK-attention fwd+bwd tokens/s"
 UNIT = "tokens/s"
 
@@ -48,6 +52,29 @@ def bytes_per_token_head(d, dv, backward, e=2):
 
 def exps_per_token_head(m, backward):
     return 2 * m * (2 if backward else 1)
+
+
+def kernel_work(d, r, m, dv, C, nslab, causal):
+    """Algorithmic work per (token, head) of each kernel of the tensor-core path: (flops, exps, bytes,
+    bound). The scan kernels split the step's total of flops_per_token_head() between them (each is
+    charged half of the backward feature recompute and of the feature-map backward); the helper kernels
+    are HBM-bound and are charged the tensors they read and write once."""
+    feat = 2 * (2 * d * r + 2 * r * m)
+    tri = C + 1
+    e = 2
+    k = {
+        "tc_attn_kernel<causal>": (feat + 4 * m * dv + tri * (m + dv), 2 * m, (2 * d + 2 * dv) * e, "tensor"),
+        "tc_attn_kernel<keys>": (feat // 2 + 2 * m * dv, m, (d + dv) * e, "tensor"),
+        "tc_attn_kernel<queries>": (feat // 2 + 2 * m * dv, m, (d + dv) * e, "tensor"),
+        "tc_bwd_q_kernel": (feat // 2 + 4 * m * dv + tri * (m + dv) + 2 * m * r + 4 * r * d, m, (3 * d + 2 * dv) * e, "tensor"),
+        "tc_bwd_k_kernel": (feat // 2 + 6 * m * dv + tri * (2 * m + dv) + 2 * m * r + 4 * r * d, m, (3 * d + 3 * dv) * e, "tensor"),
+        "tc_bwd_finish_k_kernel": (6 * r * d, 0, (nslab * d + 2 * d) * e, "hbm"),
+        "tc_key_norms_kernel": (2 * r * d, 0, d * e + 4, "hbm"),
+        "combine_kernel": (0, 0, (nslab * dv + dv) * e + nslab * 8, "hbm"),
+        "sum_slabs_kernel": (0, 0, (nslab * d + d) * e, "hbm"),
+        "delta_kernel": (0, 0, 2 * dv * e + 4, "hbm"),
+    }
+    return k
 
 
 class ClockSampler:
@@ -166,6 +193,7 @@ def main():
     ap.add_argument("--workload", default="headline")
     ap.add_argument("--path", type=int, default=0, help="0 auto, 1 SIMT, 2 tensor")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-kernel-times", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -259,6 +287,15 @@ def main():
     e2e_ms = timed(e2e_step, e2e_steps) / e2e_steps
     assert binding.darkattn_last_device_status(plan, ws) == binding.OK
 
+    # per-kernel device times: a second pass over the same steps with an event in front of every kernel
+    ktimes = {}
+    if plan.path == binding.PATH_TENSOR and not args.no_kernel_times:
+        binding.darkattn_kernel_timing(plan, True)
+        for _ in range(args.steps):
+            step()
+            ktimes = binding.darkattn_kernel_times(plan)
+        binding.darkattn_kernel_timing(plan, False)
+
     ms_step = ms / args.steps
     tokens = B * N
     value = world * tokens / (ms_step * 1e-3)
@@ -275,11 +312,40 @@ def main():
     legs = {"tensor_us": flops / (peaks["bf16_tflops_sustained"] * 1e12) * 1e6,
             "exp_us": nexp / ex2_peak * 1e6, "hbm_us": nbytes / (peaks["hbm_gbs"] * 1e9) * 1e6}
     achieved_tf = flops / (ms_step * 1e-3) / 1e12
-    roofline = {"bound": "tensor", "achieved": achieved_tf, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                "frac": achieved_tf / peaks["bf16_tflops_sustained"], "traffic": None,
-                "kernel": "whole step (forward + backward call)", "peak_source": peaks["source"] + " (sustained)",
-                "legs_us": legs, "ex2_per_s_measured": ex2_peak, "fma_per_s_measured": fma_peak,
-                "forward_ms": fwd_ms, "forward_tokens_per_s": world * tokens / (fwd_ms * 1e-3)}
+    whole = {"bound": "tensor", "achieved": achieved_tf, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+             "frac": achieved_tf / peaks["bf16_tflops_sustained"], "legs_us": legs}
+    # each kernel against the slowest of its three legs (tensor at the sustained measured peak, ex2 at the
+    # measured MUFU rate, bytes at the measured copy bandwidth)
+    nslab = max(1, m // 128)
+    work = kernel_work(d, r, m, dv, 128, nslab, wl.causal)
+    kernels = []
+    for name, (tot_ms, cnt) in sorted(ktimes.items(), key=lambda kv: -kv[1][0]):
+        entry = {"kernel": name, "launches_per_step": cnt / args.steps, "us_per_launch": 1e3 * tot_ms / max(cnt, 1),
+                 "us_per_step": 1e3 * tot_ms / args.steps}
+        if name in work:
+            f, x, b, bound = work[name]
+            us = entry["us_per_launch"]
+            t_tensor = f * th / (peaks["bf16_tflops_sustained"] * 1e12) * 1e6
+            t_exp = x * th / ex2_peak * 1e6
+            t_hbm = b * th / (peaks["hbm_gbs"] * 1e9) * 1e6
+            entry.update(bound=bound, legs_us={"tensor_us": t_tensor, "exp_us": t_exp, "hbm_us": t_hbm},
+                         frac_of_slowest_leg=max(t_tensor, t_exp, t_hbm) / us)
+            if bound == "tensor":
+                entry.update(achieved=f * th / (us * 1e-6) / 1e12, unit="TFLOP/s", peak=peaks["bf16_tflops_sustained"])
+            else:
+                entry.update(achieved=b * th / (us * 1e-6) / 1e9, unit="GB/s", peak=peaks["hbm_gbs"])
+            entry["frac"] = entry["achieved"] / entry["peak"]
+        kernels.append(entry)
+    top = next((k for k in kernels if "frac" in k), None)
+    if top is not None:
+        roofline = {"bound": top["bound"], "achieved": top["achieved"], "peak": top["peak"], "unit": top["unit"],
+                    "frac": top["frac"], "traffic": NCU_TRAFFIC.get(top["kernel"]), "kernel": top["kernel"],
+                    "us_per_launch": top["us_per_launch"], "legs_us": top["legs_us"]}
+    else:
+        roofline = dict(whole, traffic=None, kernel="whole step")
+    roofline.update(peak_source=peaks["source"] + " (sustained bf16 GEMM / copy bandwidth)", whole_step=whole, kernels=kernels,
+                    ex2_per_s_measured=ex2_peak, fma_per_s_measured=fma_peak, forward_ms=fwd_ms,
+                    forward_tokens_per_s=world * tokens / (fwd_ms * 1e-3))
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,

@@ -126,6 +126,20 @@ const char *darkattn_last_cuda_error(void);
 darkattn_status_t darkattn_measure_alu_peak(int32_t which, int32_t iters, double *ops_per_second,
                                             void *cuda_stream);
 
+/* Per-kernel device times, for benchmarks. While enabled, forward and backward record a CUDA event on
+ * the call's stream in front of every kernel they launch and one behind the last (events are host
+ * objects created by the first enabling call; no device memory is involved). Enabling also clears the
+ * accumulated times. Leave it off when measuring whole-call throughput.                           */
+darkattn_status_t darkattn_kernel_timing(darkattn_plan_t plan, int32_t enable);
+
+/* Wait for the events recorded since the last harvest, add the elapsed time between consecutive events
+ * to the kernel in front of which the first was recorded, and report the totals since timing was
+ * enabled: names (HOST buffer of 64 * max_entries bytes, one NUL-terminated name per 64 bytes),
+ * total_ms and launches (HOST arrays of max_entries), *count = entries written. Call it at least once
+ * per 96 kernels, since only that many events are kept.                                            */
+darkattn_status_t darkattn_kernel_times(darkattn_plan_t plan, int32_t max_entries, char *names, float *total_ms,
+                                        int32_t *launches, int32_t *count);
+
 /* Forward pass that needs no workspace from the caller and allocates nothing.
  *
  * (The paper has no counterpart to this entry point; it exists for deployment reasons only.)

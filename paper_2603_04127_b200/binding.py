@@ -23,7 +23,7 @@ EXPORTS = [
     "darkattn_plan", "darkattn_workspace_bytes", "darkattn_saved_bytes", "darkattn_plan_path",
     "darkattn_plan_launches", "darkattn_forward", "darkattn_backward", "darkattn_last_device_status",
     "darkattn_destroy", "darkattn_status_string", "darkattn_last_cuda_error", "darkattn_measure_alu_peak",
-    "darkattn_static_scratch_needed", "darkattn_forward_static",
+    "darkattn_static_scratch_needed", "darkattn_forward_static", "darkattn_kernel_timing", "darkattn_kernel_times",
 ]
 STATIC_SCRATCH_BYTES = 16 << 20
 
@@ -65,6 +65,11 @@ lib.darkattn_last_cuda_error.argtypes = []
 lib.darkattn_last_cuda_error.restype = ctypes.c_char_p
 lib.darkattn_measure_alu_peak.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(ctypes.c_double), _vp]
 lib.darkattn_measure_alu_peak.restype = ctypes.c_int
+lib.darkattn_kernel_timing.argtypes = [_vp, ctypes.c_int32]
+lib.darkattn_kernel_timing.restype = ctypes.c_int
+lib.darkattn_kernel_times.argtypes = [_vp, ctypes.c_int32, ctypes.c_char_p, ctypes.POINTER(ctypes.c_float),
+                                      ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]
+lib.darkattn_kernel_times.restype = ctypes.c_int
 lib.darkattn_static_scratch_needed.argtypes = [_vp]
 lib.darkattn_static_scratch_needed.restype = ctypes.c_size_t
 lib.darkattn_forward_static.argtypes = [_vp] * 8
@@ -164,6 +169,23 @@ def darkattn_measure_alu_peak(which: int, iters: int = 20, stream=None) -> float
     _check(lib.darkattn_measure_alu_peak(which, iters, ctypes.byref(out), _stream(stream)),
            "darkattn_measure_alu_peak")
     return out.value
+
+
+def darkattn_kernel_timing(plan: Plan, enable: bool):
+    _check(lib.darkattn_kernel_timing(plan.handle, int(bool(enable))), "darkattn_kernel_timing")
+
+
+def darkattn_kernel_times(plan: Plan, max_entries: int = 32) -> dict:
+    """{kernel name: (total milliseconds, launches)} since timing was enabled."""
+    names = ctypes.create_string_buffer(64 * max_entries)
+    ms = (ctypes.c_float * max_entries)()
+    cnt = (ctypes.c_int32 * max_entries)()
+    n = ctypes.c_int32(0)
+    _check(lib.darkattn_kernel_times(plan.handle, max_entries, names, ms, cnt, ctypes.byref(n)), "darkattn_kernel_times")
+    out = {}
+    for i in range(n.value):
+        out[names.raw[64 * i:64 * (i + 1)].split(b"\0", 1)[0].decode()] = (float(ms[i]), int(cnt[i]))
+    return out
 
 
 def darkattn_static_scratch_needed(plan: Plan) -> int:

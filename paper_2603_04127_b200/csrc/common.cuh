@@ -76,6 +76,21 @@ struct TensorLayout {
 
 }  // namespace darkattn
 
+namespace darkattn {
+// Optional per-kernel timing: an event before every kernel of a call and one after the last.
+struct KernelTimer {
+    static constexpr int kMaxMarks = 96, kMaxKernels = 32;
+    bool on = false, created = false;
+    int n = 0;                               // marks since the last harvest
+    cudaEvent_t ev[kMaxMarks];
+    const char *name[kMaxMarks];             // nullptr: closing mark of a call
+    int nk = 0;                              // accumulated per kernel name
+    const char *kname[kMaxKernels];
+    double kms[kMaxKernels];
+    int kcount[kMaxKernels];
+};
+}  // namespace darkattn
+
 struct darkattn_plan_s {
     darkattn_desc_t desc;
     darkattn::Dims dims;
@@ -85,11 +100,14 @@ struct darkattn_plan_s {
     size_t workspace_bytes;
     size_t saved_bytes;
     int launches_fwd, launches_bwd;
+    mutable darkattn::KernelTimer timer;
 };
 
 namespace darkattn {
 
 void set_cuda_error(cudaError_t e, const char *where);
+// Records an event in front of the kernel `name` (nullptr: after the last kernel of a call) when timing is on.
+void timer_mark(const darkattn_plan_s *plan, cudaStream_t st, const char *name);
 
 // SIMT (FP32 FFMA) path
 void simt_make_layout(darkattn_plan_s *plan);

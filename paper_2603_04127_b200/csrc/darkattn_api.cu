@@ -15,6 +15,15 @@ void set_cuda_error(cudaError_t e, const char *where)
     snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s (%s)", where, cudaGetErrorName(e), cudaGetErrorString(e));
 }
 
+void timer_mark(const darkattn_plan_s *plan, cudaStream_t st, const char *name)
+{
+    KernelTimer &t = plan->timer;
+    if (!t.on || t.n >= KernelTimer::kMaxMarks) return;
+    t.name[t.n] = name;
+    cudaEventRecord(t.ev[t.n], st);
+    ++t.n;
+}
+
 static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 }  // namespace darkattn
@@ -93,9 +102,15 @@ darkattn_status_t darkattn_forward(darkattn_plan_t plan, const void *Q, const vo
     if (!aligned16(workspace) || !aligned16(saved)) return DARKATTN_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     DARKATTN_CUDA_TRY(cudaMemsetAsync(workspace, 0, 256, st), "forward: clear status word");
-    if (plan->path == DARKATTN_PATH_TENSOR)
-        return tensor_forward(plan, Q, K, V, M, W, O, saved, static_cast<char *>(workspace), st);
-    return simt_forward(plan, Q, K, V, M, W, O, static_cast<char *>(workspace), st, false);
+    darkattn_status_t rc;
+    if (plan->path == DARKATTN_PATH_TENSOR) {
+        rc = tensor_forward(plan, Q, K, V, M, W, O, saved, static_cast<char *>(workspace), st);
+    } else {
+        timer_mark(plan, st, "simt_forward (all kernels)");
+        rc = simt_forward(plan, Q, K, V, M, W, O, static_cast<char *>(workspace), st, false);
+    }
+    timer_mark(plan, st, nullptr);
+    return rc;
 }
 
 darkattn_status_t darkattn_backward(darkattn_plan_t plan, const void *Q, const void *K, const void *V,
@@ -111,9 +126,15 @@ darkattn_status_t darkattn_backward(darkattn_plan_t plan, const void *Q, const v
     if (!aligned16(workspace) || !aligned16(saved) || !aligned16(O)) return DARKATTN_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     DARKATTN_CUDA_TRY(cudaMemsetAsync(workspace, 0, 256, st), "backward: clear status word");
-    if (plan->path == DARKATTN_PATH_TENSOR)
-        return tensor_backward(plan, Q, K, V, M, W, O, dO, saved, dQ, dK, dV, dM, static_cast<char *>(workspace), st);
-    return simt_backward(plan, Q, K, V, M, W, dO, dQ, dK, dV, dM, static_cast<char *>(workspace), st);
+    darkattn_status_t rc;
+    if (plan->path == DARKATTN_PATH_TENSOR) {
+        rc = tensor_backward(plan, Q, K, V, M, W, O, dO, saved, dQ, dK, dV, dM, static_cast<char *>(workspace), st);
+    } else {
+        timer_mark(plan, st, "simt_backward (all kernels)");
+        rc = simt_backward(plan, Q, K, V, M, W, dO, dQ, dK, dV, dM, static_cast<char *>(workspace), st);
+    }
+    timer_mark(plan, st, nullptr);
+    return rc;
 }
 
 darkattn_status_t darkattn_last_device_status(darkattn_plan_t plan, const void *workspace, void *cuda_stream)
@@ -128,7 +149,59 @@ darkattn_status_t darkattn_last_device_status(darkattn_plan_t plan, const void *
     return DARKATTN_ERR_TIMEOUT;
 }
 
-void darkattn_destroy(darkattn_plan_t plan) { delete plan; }
+darkattn_status_t darkattn_kernel_timing(darkattn_plan_t plan, int32_t enable)
+{
+    if (!plan) return DARKATTN_ERR_INVALID_ARG;
+    KernelTimer &t = plan->timer;
+    if (enable && !t.created) {
+        for (int i = 0; i < KernelTimer::kMaxMarks; ++i)
+            DARKATTN_CUDA_TRY(cudaEventCreate(&t.ev[i]), "kernel_timing: cudaEventCreate");
+        t.created = true;
+    }
+    t.on = enable != 0;
+    t.n = 0;
+    if (enable) t.nk = 0;
+    return DARKATTN_OK;
+}
+
+darkattn_status_t darkattn_kernel_times(darkattn_plan_t plan, int32_t max_entries, char *names, float *total_ms,
+                                        int32_t *launches, int32_t *count)
+{
+    if (!plan || !names || !total_ms || !launches || !count || max_entries < 0) return DARKATTN_ERR_INVALID_ARG;
+    KernelTimer &t = plan->timer;
+    if (t.n > 0) {
+        DARKATTN_CUDA_TRY(cudaEventSynchronize(t.ev[t.n - 1]), "kernel_times: cudaEventSynchronize");
+        for (int i = 0; i + 1 < t.n; ++i) {
+            if (!t.name[i]) continue;
+            float ms = 0.f;
+            DARKATTN_CUDA_TRY(cudaEventElapsedTime(&ms, t.ev[i], t.ev[i + 1]), "kernel_times: cudaEventElapsedTime");
+            int k = 0;
+            while (k < t.nk && strcmp(t.kname[k], t.name[i]) != 0) ++k;
+            if (k == t.nk) {
+                if (t.nk == KernelTimer::kMaxKernels) continue;
+                t.kname[k] = t.name[i]; t.kms[k] = 0.0; t.kcount[k] = 0; ++t.nk;
+            }
+            t.kms[k] += ms;
+            ++t.kcount[k];
+        }
+        t.n = 0;
+    }
+    const int n = t.nk < max_entries ? t.nk : max_entries;
+    for (int k = 0; k < n; ++k) {
+        snprintf(names + 64 * k, 64, "%s", t.kname[k]);
+        total_ms[k] = (float)t.kms[k];
+        launches[k] = t.kcount[k];
+    }
+    *count = n;
+    return DARKATTN_OK;
+}
+
+void darkattn_destroy(darkattn_plan_t plan)
+{
+    if (plan && plan->timer.created)
+        for (int i = 0; i < KernelTimer::kMaxMarks; ++i) cudaEventDestroy(plan->timer.ev[i]);
+    delete plan;
+}
 
 const char *darkattn_status_string(darkattn_status_t s)
 {

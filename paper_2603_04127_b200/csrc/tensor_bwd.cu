@@ -925,7 +925,7 @@ __global__ void dm_kernel(const __nv_bfloat16 *W, const float *Tacc, const float
 }
 
 template <int D, int DV>
-cudaError_t launch_scan(const BwdParams &P, int grid, cudaStream_t st)
+cudaError_t launch_scan(const darkattn_plan_s *plan, const BwdParams &P, int grid, cudaStream_t st)
 {
     using L = BwdSmem<D, DV>;
     static_assert(L::kTotal <= 232448, "shared memory budget of one CTA exceeded");
@@ -933,9 +933,11 @@ cudaError_t launch_scan(const BwdParams &P, int grid, cudaStream_t st)
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(tc_bwd_k_kernel<D, DV>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
     if (e != cudaSuccess) return e;
+    timer_mark(plan, st, "tc_bwd_q_kernel");
     tc_bwd_q_kernel<D, DV><<<grid, kThreads, L::kTotal, st>>>(P);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
+    timer_mark(plan, st, "tc_bwd_k_kernel");
     tc_bwd_k_kernel<D, DV><<<grid, kThreads, L::kTotal, st>>>(P);
     return cudaGetLastError();
 }
@@ -961,8 +963,10 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
 {
     const Dims &D = plan->dims;
     const TensorLayout &Y = plan->tensor;
-    if (!D.causal)   // the non-causal backward has no tensor-core kernels: FP32 path, same workspace
+    if (!D.causal) {   // the non-causal backward has no tensor-core kernels: FP32 path, same workspace
+        timer_mark(plan, st, "simt_backward (all kernels)");
         return simt_backward(plan, Q, K, V, M, W, dO, dQ, dK, dV, dM, ws, st);
+    }
     const size_t BH = D.BH, N = D.N;
     auto bf = [&](size_t off) { return reinterpret_cast<__nv_bfloat16 *>(ws + off); };
     auto fl = [&](size_t off) { return reinterpret_cast<float *>(ws + off); };
@@ -985,6 +989,7 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
     }
 
     const long long rows = (long long)BH * N;
+    timer_mark(plan, st, "delta_kernel");
     delta_kernel<<<(unsigned)((rows * 32 + 255) / 256), 256, 0, st>>>((const __nv_bfloat16 *)dO, (const __nv_bfloat16 *)O, fl(Y.delta), rows, D.dv);
     chk();
     keep(cudaMemsetAsync(ws + Y.Tacc, 0, (size_t)D.H * D.m * D.d * 4, st));
@@ -1008,15 +1013,17 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
     P.status = reinterpret_cast<int *>(ws + Y.status);
     P.N = D.N; P.H = D.H; P.BH = D.BH; P.m = D.m; P.nslab = Y.nslab; P.T = Y.T;
     const int units = (int)(BH * Y.nslab);
-    if (D.d == 64 && D.dv == 64) keep(launch_scan<64, 64>(P, units, st));
-    else if (D.d == 128 && D.dv == 128) keep(launch_scan<128, 128>(P, units, st));
-    else if (D.d == 64 && D.dv == 128) keep(launch_scan<64, 128>(P, units, st));
-    else keep(launch_scan<128, 64>(P, units, st));
+    if (D.d == 64 && D.dv == 64) keep(launch_scan<64, 64>(plan, P, units, st));
+    else if (D.d == 128 && D.dv == 128) keep(launch_scan<128, 128>(plan, P, units, st));
+    else if (D.d == 64 && D.dv == 128) keep(launch_scan<64, 128>(plan, P, units, st));
+    else keep(launch_scan<128, 64>(plan, P, units, st));
 
     {
         const long long tq = rows * (D.d / 8), tv = rows * (D.dv / 8);
+        timer_mark(plan, st, "sum_slabs_kernel");
         sum_slabs_kernel<<<(unsigned)((tq + 255) / 256), 256, 0, st>>>(bf(Y.pdQ), (__nv_bfloat16 *)dQ, rows, D.d, Y.nslab, kLn2);
         chk();
+        timer_mark(plan, st, "sum_slabs_kernel");
         sum_slabs_kernel<<<(unsigned)((tv + 255) / 256), 256, 0, st>>>(bf(Y.pdV), (__nv_bfloat16 *)dV, rows, D.dv, Y.nslab, 1.f);
         chk();
     }
@@ -1027,9 +1034,11 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
     F.N = D.N; F.H = D.H; F.BH = D.BH; F.T = Y.T; F.r = D.r; F.nslab = Y.nslab; F.nes = 4 * Y.nslab; F.s2 = D.s * D.s;
     F.nsplit = (int)((148 * 2 + BH - 1) / BH);
     if (F.nsplit > Y.T) F.nsplit = Y.T;
+    timer_mark(plan, st, "tc_bwd_finish_k_kernel");
     if (D.d == 64) keep(launch_finish<64>(F, (int)(BH * F.nsplit), st));
     else keep(launch_finish<128>(F, (int)(BH * F.nsplit), st));
 
+    timer_mark(plan, st, "dm_kernel");
     dm_kernel<<<dim3(D.r, D.H), 128, 0, st>>>((const __nv_bfloat16 *)W, fl(Y.Tacc), fl(Y.dMn), dM, D.m, D.r, D.d, D.w_per_head, D.s);
     chk();
     if (e != cudaSuccess) { set_cuda_error(e, "tensor_backward"); return DARKATTN_ERR_CUDA; }

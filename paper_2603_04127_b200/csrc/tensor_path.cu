@@ -648,9 +648,11 @@ cudaError_t tensor_prologue(const darkattn_plan_s *plan, const void *K, const vo
     cudaError_t e = cudaSuccess;
     auto chk = [&]() { cudaError_t x = cudaGetLastError(); if (x != cudaSuccess && e == cudaSuccess) e = x; };
 
+    timer_mark(plan, st, "fold_omega_kernel");
     fold_omega_kernel<<<dim3(D.m, D.H), 128, 0, st>>>((const __nv_bfloat16 *)W, (const __nv_bfloat16 *)M, bf(Y.Om), D.m, D.r, D.d,
                                                       D.w_per_head, kLog2e * D.s);
     chk();
+    timer_mark(plan, st, "slab_shift_kernel");
     slab_shift_kernel<<<(unsigned)(BH * Y.nslab), 128, 0, st>>>((const __nv_bfloat16 *)W, fl(Y.cs), D.H, D.m, D.r, Y.nslab, D.w_per_head);
     chk();
 
@@ -660,6 +662,7 @@ cudaError_t tensor_prologue(const darkattn_plan_s *plan, const void *K, const vo
     if (NP.nsplit > Y.T) NP.nsplit = Y.T;
     NP.coef = kLog2e * 0.5f * D.s * D.s;
     const int smem_bytes = 2 * 128 * D.d * 2 + 64;
+    timer_mark(plan, st, "tc_key_norms_kernel");
     if (D.d == 64) {
         cudaFuncSetAttribute(tc_key_norms_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
         tc_key_norms_kernel<64><<<(unsigned)(BH * NP.nsplit), 160, smem_bytes, st>>>(NP);
@@ -698,20 +701,25 @@ darkattn_status_t tensor_forward(const darkattn_plan_s *plan, const void *Q, con
     const int units = (int)(BH * Y.nslab);
     if (D.causal) {
         P.nsplit = 1;
+        timer_mark(plan, st, "tc_attn_kernel<causal>");
         cudaError_t x = launch_main_shape<MODE_CAUSAL>(D.d, D.dv, P, units, st);
         if (x != cudaSuccess && e == cudaSuccess) e = x;
     } else {
         e = (e == cudaSuccess) ? cudaMemsetAsync(ws + Y.Sacc, 0, (Y.Sb - Y.Sacc), st) : e;   // S and z sums
+        timer_mark(plan, st, "tc_attn_kernel<keys>");
         cudaError_t x = launch_main_shape<MODE_KEYS>(D.d, D.dv, P, units * Y.nsplit, st);
         if (x != cudaSuccess && e == cudaSuccess) e = x;
         const long long n = (long long)BH * D.m * D.dv;
+        timer_mark(plan, st, "state_to_bf16_kernel");
         state_to_bf16_kernel<<<(unsigned)((n + 1023) / 1024), 256, 0, st>>>(fl(Y.Sacc), bf(Y.Sb), n);
         chk();
+        timer_mark(plan, st, "tc_attn_kernel<queries>");
         x = launch_main_shape<MODE_QUERIES>(D.d, D.dv, P, units * Y.nsplit, st);
         if (x != cudaSuccess && e == cudaSuccess) e = x;
     }
     {
         const long long rows = (long long)BH * N, threads = rows * (D.dv / 8);
+        timer_mark(plan, st, "combine_kernel");
         combine_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(bf(Y.pnum), fl(Y.pdr), (__nv_bfloat16 *)O,
                                                                           reinterpret_cast<float2 *>(ws + Y.sv),
                                                                           reinterpret_cast<float2 *>(saved), rows, D.dv, Y.nslab);
