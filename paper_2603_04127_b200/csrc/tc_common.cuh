@@ -252,6 +252,74 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, in
     return false;
 }
 
+// ---------------------------------------------------------------- tiles, epilogue layout, descriptors
+__device__ __forceinline__ unsigned char *tile_chunk(unsigned char *base, int row, int chunk16)
+{
+    return base + (chunk16 >> 3) * 16384 + swz128((uint32_t)row, (uint32_t)(chunk16 & 7));
+}
+
+__device__ __forceinline__ uint4 pack8(const uint32_t *v)
+{
+    return make_uint4(pack_bf16(__uint_as_float(v[0]), __uint_as_float(v[1])), pack_bf16(__uint_as_float(v[2]), __uint_as_float(v[3])),
+                      pack_bf16(__uint_as_float(v[4]), __uint_as_float(v[5])), pack_bf16(__uint_as_float(v[6]), __uint_as_float(v[7])));
+}
+
+__device__ __forceinline__ void unpack8(const uint4 &raw, float *f)
+{
+    const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const float2 x = __bfloat1622float2(h2[q]);
+        f[2 * q] = x.x;
+        f[2 * q + 1] = x.y;
+    }
+}
+
+// Epilogue thread layout: 16 warps. Warp w works on TMEM lanes (tile rows) 32 (w % 4) .. +31, the only
+// ones it may touch, and on the 32 columns starting at 32 (w / 4); four warps share each row.
+constexpr int kEpiWarps = 16, kEpiThreads = 512, kThreads = 544;
+
+// the four warps that share a lane quarter
+__device__ __forceinline__ void quarter_sync(int q) { asm volatile("bar.sync %0, 128;" ::"r"(q + 1) : "memory"); }
+// all epilogue threads
+__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 5, 512;" ::: "memory"); }
+
+// features 2^(U - offset): 32 TMEM columns at taddr -> bf16 tile row `row`, columns [col0, col0 + 32)
+__device__ __forceinline__ void features_to_tile(uint32_t taddr, float offset, unsigned char *tile, int row, int col0)
+{
+    uint32_t v[32], pk[16];
+    tmem_ld32(taddr, v);
+    tmem_wait_ld();
+#pragma unroll
+    for (int j = 0; j < 32; j += 2)
+        pk[j / 2] = pack_bf16(ex2f(__uint_as_float(v[j]) - offset), ex2f(__uint_as_float(v[j + 1]) - offset));
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+        *reinterpret_cast<uint4 *>(tile_chunk(tile, row, col0 / 8 + q)) = make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+}
+
+// 32 fp32 TMEM columns at taddr -> bf16 tile row (swizzled smem), columns [col0, col0 + 32)
+__device__ __forceinline__ void tmem_row_to_tile(uint32_t taddr, unsigned char *tile, int row, int col0)
+{
+    uint32_t v[32];
+    tmem_ld32(taddr, v);
+    tmem_wait_ld();
+#pragma unroll
+    for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4 *>(tile_chunk(tile, row, col0 / 8 + q)) = pack8(v + 8 * q);
+}
+
+// Matrix descriptors are built once per tile buffer; step k of an MMA loop only adds a constant to the
+// start-address field (units of 16 bytes), so that the issuing thread spends one add per instruction.
+struct TileDesc {
+    uint64_t kmaj, mnmaj;
+    __device__ __forceinline__ explicit TileDesc(const unsigned char *base)
+        : kmaj(make_sdesc(smem_u32(base), 16, 1024)), mnmaj(make_sdesc(smem_u32(base), 16384, 1024)) {}
+};
+// K-major operand, 64-element atoms 16 KB apart: step k covers 16 elements (32 bytes) of K
+__device__ __forceinline__ uint64_t kdesc(const TileDesc &t, int k) { return t.kmaj + (uint64_t)(((k / 4) * 16384 + (k % 4) * 32) >> 4); }
+// MN-major operand: step k covers 16 K-rows of 128 bytes
+__device__ __forceinline__ uint64_t mndesc(const TileDesc &t, int k) { return t.mnmaj + (uint64_t)((k * 2048) >> 4); }
+
 // ---------------------------------------------------------------- host side: tensor maps
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
