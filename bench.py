@@ -63,9 +63,9 @@ def kernel_work(d, r, m, dv, C, nslab, causal):
     tri = C + 1
     e = 2
     k = {
-        "tc_attn_kernel<causal>": (feat + 4 * m * dv + tri * (m + dv), 2 * m, (2 * d + 2 * dv) * e, "tensor"),
-        "tc_attn_kernel<keys>": (feat // 2 + 2 * m * dv, m, (d + dv) * e, "tensor"),
-        "tc_attn_kernel<queries>": (feat // 2 + 2 * m * dv, m, (d + dv) * e, "tensor"),
+        "tc_fwd_causal_kernel": (feat + 4 * m * dv + tri * (m + dv), 2 * m, (2 * d + 2 * dv) * e, "tensor"),
+        "tc_fwd_keys_kernel": (feat // 2 + 2 * m * dv, m, (d + dv) * e, "tensor"),
+        "tc_fwd_queries_kernel": (feat // 2 + 2 * m * dv, m, (d + dv) * e, "tensor"),
         "tc_bwd_q_kernel": (feat // 2 + 4 * m * dv + tri * (m + dv) + 2 * m * r + 4 * r * d, m, (3 * d + 2 * dv) * e, "tensor"),
         "tc_bwd_k_kernel": (feat // 2 + 6 * m * dv + tri * (2 * m + dv) + 2 * m * r + 4 * r * d, m, (3 * d + 3 * dv) * e, "tensor"),
         "tc_bwd_finish_k_kernel": (6 * r * d, 0, (nslab * d + 2 * d) * e, "hbm"),

@@ -27,7 +27,6 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kMaxNsplit = 64;
 
 // ------------------------------------------------------------------ small helpers
-__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 // ------------------------------------------------------------------ prologue kernels (SIMT, tiny)
 // Omega[h,l,c] = log2(e) * s * sum_a W[l,a] M[h,a,c]  (bf16);  one block per (h, l).
@@ -159,58 +158,94 @@ struct MainParams {
 
 enum { MODE_CAUSAL = 0, MODE_KEYS = 1, MODE_QUERIES = 2 };
 
-template <int D, int DV, int MODE>
-struct SmemLayout {
+// ------------------------------------------------------------------ forward scan kernels
+// All three use 16 epilogue warps (warp w: TMEM lanes 32 (w % 4) .. +31, columns 32 (w / 4) .. +31) and one
+// control warp whose first lane issues the TMA loads and the MMAs. phi(Q) and the masked kernel tile P are only
+// ever the A operand of an MMA whose rows are tokens, so they are packed to bf16 in tensor memory and read
+// by the MMA from there; phi(K) also serves transposed and as a B operand and goes to shared memory.
+
+__device__ __forceinline__ void store_row_f32x32_bf16(const uint32_t (&v)[32], unsigned char *tile, int row, int col0)
+{
+#pragma unroll
+    for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4 *>(tile_chunk(tile, row, col0 / 8 + q)) = pack8(v + 8 * q);
+}
+
+// phi(Q) of one row segment: row maximum over the slab's 128 features (exchanged with the three other warps
+// of the lane quarter through red[4][128]), 2^(u - max) packed to bf16 into TMEM columns fq + col0/2,
+// returns sum_l phi(Q)_l z_l over the segment. rmax receives the row maximum.
+__device__ __forceinline__ float query_features_to_tmem(uint32_t u_addr, uint32_t fq_addr, float *red, const float *z, int q4,
+                                                        int g, int r, int col0, float &rmax)
+{
+    uint32_t v[32], pk[16];
+    tmem_ld32(u_addr + col0, v);
+    tmem_wait_ld();
+    float mx = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(v[j]));
+    red[g * 128 + r] = mx;
+    quarter_sync(q4);
+    rmax = fmaxf(fmaxf(red[r], red[128 + r]), fmaxf(red[256 + r], red[384 + r]));
+    float dz = 0.f;
+#pragma unroll
+    for (int j = 0; j < 32; j += 2) {
+        const float f0 = ex2f(__uint_as_float(v[j]) - rmax), f1 = ex2f(__uint_as_float(v[j + 1]) - rmax);
+        const float2 zz = *reinterpret_cast<const float2 *>(z + col0 + j);
+        dz = fmaf(f0, zz.x, dz);
+        dz = fmaf(f1, zz.y, dz);
+        pk[j / 2] = pack_bf16(f0, f1);
+    }
+    tmem_st16(fq_addr + col0 / 2, pk);
+    tmem_wait_st();
+    return dz;
+}
+
+template <int D, int DV>
+struct FwdCausalSmem {
     static constexpr int kOm = 0;
     static constexpr int kQ = kOm + 128 * D * 2;
-    static constexpr int kK = kQ + 128 * D * 2;                                  // also the masked P tile (causal)
-    static constexpr int kKBytes = (MODE == MODE_CAUSAL && D < 128) ? 32768 : 128 * D * 2;
-    static constexpr int kV = kK + kKBytes;
-    static constexpr int kFQ = kV + 128 * DV * 2;                                // also the output staging tile
-    static constexpr int kFK = kFQ + 32768;
-    static constexpr int kSb = kFK + 32768;
-    static constexpr int kOnes = kSb + 128 * DV * 2;
-    static constexpr int kZ = kOnes + 2048;
-    static constexpr int kBars = kZ + 512;
-    static constexpr int kTotal = kBars + 192;
+    static constexpr int kK = kQ + 128 * D * 2;
+    static constexpr int kV = kK + 128 * D * 2;
+    static constexpr int kFK = kV + 128 * DV * 2;          // phi(K)                              [128, 128]
+    static constexpr int kSb = kFK + 32768;                // bf16 copy of the state              [128 l, DV]
+    static constexpr int kStg = kSb + 128 * DV * 2;        // output staging; its first 2 KB hold the ones operand mid-chunk
+    static constexpr int kZ = kStg + 128 * DV * 2;         // z_prev, float[128]
+    static constexpr int kRed = kZ + 512;                  // float[4][128] exchange between the warps of a row
+    static constexpr int kBars = kRed + 2048;
+    static constexpr int kTotal = kBars + 256;
 };
 
-// TMEM columns (512 allocated): state S at 0 (DV columns), z at DV (16), R1 at 256, R2 at 384 (128 each).
-constexpr uint32_t kColS = 0, kColR1 = 256, kColR2 = 384;
+// TMEM columns of the causal kernel: state S at 0 (DV), z at 128 (16), packed phi(Q) at 160 (64), R1 at 256, R2 at 384.
+constexpr uint32_t kColS = 0, kColZ = 128, kColFQ = 160, kColR1 = 256, kColR2 = 384;
 
-template <int D, int DV, int MODE>
-__global__ void __launch_bounds__(160, 1) tc_attn_kernel(const __grid_constant__ MainParams p)
+enum CBars { CB_OM, CB_Q, CB_K, CB_V, CM1, CM2, CM3, CMS, CM4, CE0, CE1, CE2, CE3, CE4, CNBARS };
+
+// Causal: one CTA per (b, h, slab) walks the chunks of the sequence.
+//   R1: U_Q -> (phi(Q) read) -> P = phi(Q) phi(K)^T -> packed tril(P) (A operand of P V) -> U_Q of the next chunk
+//   R2: U_K -> (phi(K) read) -> O = phi(Q) S_prev + P V -> (O read)
+template <int D, int DV>
+__global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid_constant__ MainParams p)
 {
-    using L = SmemLayout<D, DV, MODE>;
+    using L = FwdCausalSmem<D, DV>;
     extern __shared__ __align__(1024) unsigned char smem[];
     unsigned char *sOm = smem + L::kOm, *sQ = smem + L::kQ, *sK = smem + L::kK, *sV = smem + L::kV;
-    unsigned char *sFQ = smem + L::kFQ, *sFK = smem + L::kFK, *sSb = smem + L::kSb, *sOnes = smem + L::kOnes;
-    unsigned char *sP = sK, *sStage = sFQ;
-    float *sZ = reinterpret_cast<float *>(smem + L::kZ);
+    unsigned char *sFK = smem + L::kFK, *sSb = smem + L::kSb, *sStg = smem + L::kStg;
+    float *sZ = reinterpret_cast<float *>(smem + L::kZ), *sRed = reinterpret_cast<float *>(smem + L::kRed);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::kBars);
-    uint64_t *bar_om = bars + 0, *bar_q = bars + 1, *bar_k = bars + 2, *bar_v = bars + 3, *bar_uq = bars + 4,
-             *bar_uk = bars + 5, *bar_p = bars + 6, *bar_o = bars + 7, *bar_s = bars + 8, *bar_eq = bars + 9,
-             *bar_ek = bars + 10, *bar_ep = bars + 11, *bar_eo = bars + 12, *bar_es = bars + 13;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 14);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 15);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + CNBARS);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + CNBARS + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5;
-    const int unit = blockIdx.x / p.nsplit, split = blockIdx.x % p.nsplit;
-    const int bh = unit / p.nslab, slab = unit % p.nslab, h = bh % p.H;
-    const int t0 = (int)((long long)p.T * split / p.nsplit), t1 = (int)((long long)p.T * (split + 1) / p.nsplit);
-    const int row0 = bh * p.N;                    // first row of this (b,h) in the [BH*N, *] views
+    const int bh = blockIdx.x / p.nslab, slab = blockIdx.x % p.nslab, h = bh % p.H;
+    const int row0 = bh * p.N, T = p.T;
 
     if (tid == 0) {
-        for (int i = 0; i < 9; ++i) mbar_init(bars + i, 1);
-        for (int i = 9; i < 14; ++i) mbar_init(bars + i, 128);
+        for (int i = 0; i < CE0; ++i) mbar_init(bars + i, 1);
+        for (int i = CE0; i < CNBARS; ++i) mbar_init(bars + i, kEpiWarps);
         *abort_flag = (smem_u32(smem) & 1023u) ? 1 : 0;
         fence_mbar_init();
     }
-    if (tid < 128) {   // 2 KB of bf16 ones: B operand of the z += phi(K)^T 1 MMAs
-        *reinterpret_cast<uint4 *>(sOnes + tid * 16) = make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
-        fence_async_smem();
-    }
-    if (warp == 4) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+    if (tid < 128) sZ[tid] = 0.f;
+    if (warp == kEpiWarps) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -219,284 +254,464 @@ __global__ void __launch_bounds__(160, 1) tc_attn_kernel(const __grid_constant__
 
     if (*abort_flag) {
         if (tid == 0) atomicExch(status, (int)DARKATTN_ERR_CUDA);
-    } else if (t1 <= t0) {
-        // nothing to do for this split
-    } else if (warp == 4) {
-        // ============================== control thread: TMA loads and MMA issue
+    } else if (warp == kEpiWarps) {
         if ((tid & 31) == 0) {
-            constexpr uint32_t kXBytes = 128 * D * 2, kVBytes = 128 * DV * 2;
-            auto load_x = [&](unsigned char *dst, const CUtensorMap *map, uint64_t *bar, int t) {
-                mbar_expect_tx(bar, kXBytes);
-                for (int a = 0; a < D / 64; ++a) tma_load_2d(dst + a * 16384, map, bar, a * 64, row0 + t * 128);
+            auto load_tile = [&](unsigned char *dst, const CUtensorMap *map, uint64_t *bar, int width, int t) {
+                mbar_expect_tx(bar, 128 * width * 2);
+                for (int a = 0; a < width / 64; ++a) tma_load_2d(dst + a * 16384, map, bar, a * 64, row0 + t * 128);
             };
-            auto load_v = [&](int t) {
-                mbar_expect_tx(bar_v, kVBytes);
-                for (int a = 0; a < DV / 64; ++a) tma_load_2d(sV + a * 16384, &p.mapV, bar_v, a * 64, row0 + t * 128);
-            };
-            // K-major operand with K split over 64-element atoms: step k of 16 elements
-            auto kdesc = [](unsigned char *base, int k) { return make_sdesc(smem_u32(base) + (k / 4) * 16384 + (k % 4) * 32, 16, 1024); };
-            // MN-major operand: 16 K-rows per step, 64-element blocks along M/N are 16 KB apart
-            auto mndesc = [](unsigned char *base, int k) { return make_sdesc(smem_u32(base) + k * 2048, 16384, 1024); };
-            const uint32_t id_u = make_idesc(128, 128, 0, 0);     // U = X Omega^T, P = phi(Q) phi(K)^T
-            const uint32_t id_o = make_idesc(128, DV, 0, 1);      // O += A[K-major] B[MN-major]
-            const uint32_t id_s = make_idesc(128, DV, 1, 1);      // S += phi(K)^T V
-            const uint32_t id_z = make_idesc(128, 16, 1, 1);      // z += phi(K)^T 1
+            const TileDesc tOm(sOm), tQ(sQ), tK(sK), tV(sV), tFK(sFK), tSb(sSb);
+            const uint64_t ones_desc = make_sdesc(smem_u32(sStg), 16384, 1024);
+            const uint32_t id_kk = make_idesc(128, 128, 0, 0);
+            const uint32_t id_o = make_idesc(128, DV, 0, 1);
+            const uint32_t id_s = make_idesc(128, DV, 1, 1);
+            const uint32_t id_z = make_idesc(128, 16, 1, 1);
+            const uint32_t R1 = tmem + kColR1, R2 = tmem + kColR2, FQ = tmem + kColFQ;
 
-            mbar_expect_tx(bar_om, 128 * D * 2 + (MODE == MODE_QUERIES ? 128 * DV * 2 : 0));
-            for (int a = 0; a < D / 64; ++a) tma_load_2d(sOm + a * 16384, &p.mapOm, bar_om, a * 64, h * p.m + slab * 128);
-            if (MODE == MODE_QUERIES)
-                for (int a = 0; a < DV / 64; ++a) tma_load_2d(sSb + a * 16384, &p.mapSb, bar_om, a * 64, bh * p.m + slab * 128);
-            if (MODE != MODE_KEYS) load_x(sQ, &p.mapQ, bar_q, t0);
-            if (MODE != MODE_QUERIES) { load_x(sK, &p.mapK, bar_k, t0); load_v(t0); }
+            mbar_expect_tx(bars + CB_OM, 128 * D * 2);
+            for (int a = 0; a < D / 64; ++a) tma_load_2d(sOm + a * 16384, &p.mapOm, bars + CB_OM, a * 64, h * p.m + slab * 128);
+            load_tile(sQ, &p.mapQ, bars + CB_Q, D, 0);
+            load_tile(sK, &p.mapK, bars + CB_K, D, 0);
+            load_tile(sV, &p.mapV, bars + CB_V, DV, 0);
 
-            bool ok = wait_or_abort(bar_om, 0, status, abort_flag);
-            for (int t = t0; t < t1 && ok; ++t) {
-                const uint32_t ph = (t - t0) & 1;
-                const bool first = (t == t0), last = (t + 1 == t1);
-                if (MODE != MODE_KEYS) {            // U_Q -> R1
-                    ok = wait_or_abort(bar_q, ph, status, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after();
-                    for (int k = 0; k < D / 16; ++k) mma_ss(tmem + kColR1, kdesc(sQ, k), kdesc(sOm, k), id_u, k > 0);
-                    mma_commit(bar_uq);
-                }
-                if (MODE != MODE_QUERIES) {         // U_K -> R2
-                    if (MODE == MODE_CAUSAL && !first) ok = wait_or_abort(bar_eo, ph ^ 1, status, abort_flag);
-                    if (ok) ok = wait_or_abort(bar_k, ph, status, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after();
-                    for (int k = 0; k < D / 16; ++k) mma_ss(tmem + kColR2, kdesc(sK, k), kdesc(sOm, k), id_u, k > 0);
-                    mma_commit(bar_uk);
-                }
-                if (MODE != MODE_KEYS) {            // the query tile is free once U_Q has run: prefetch the next
-                    ok = wait_or_abort(bar_uq, ph, status, abort_flag);
-                    if (!ok) break;
-                    if (!last) load_x(sQ, &p.mapQ, bar_q, t + 1);
-                }
-                if (MODE == MODE_KEYS) {            // the key tile is free once U_K has run
-                    ok = wait_or_abort(bar_uk, ph, status, abort_flag);
-                    if (!ok) break;
-                    if (!last) load_x(sK, &p.mapK, bar_k, t + 1);
-                }
-                if (MODE != MODE_KEYS) { ok = wait_or_abort(bar_eq, ph, status, abort_flag); if (!ok) break; }
-                if (MODE != MODE_QUERIES) { ok = wait_or_abort(bar_ek, ph, status, abort_flag); if (!ok) break; }
+            bool ok = wait_or_abort(bars + CB_OM, 0, status, abort_flag);
+            if (ok) ok = wait_or_abort(bars + CB_Q, 0, status, abort_flag);
+            if (ok) {
                 tc_fence_after();
-                if (MODE == MODE_CAUSAL) {          // P = phi(Q) phi(K)^T -> R1
-                    for (int k = 0; k < 8; ++k) mma_ss(tmem + kColR1, kdesc(sFQ, k), kdesc(sFK, k), id_u, k > 0);
-                    mma_commit(bar_p);
-                }
-                bool o_started = false;
-                if (MODE == MODE_QUERIES || (MODE == MODE_CAUSAL && !first)) {   // O = phi(Q) S_prev -> R2
-                    if (MODE == MODE_CAUSAL) ok = wait_or_abort(bar_es, ph ^ 1, status, abort_flag);
-                    if (MODE == MODE_QUERIES && !first) ok = wait_or_abort(bar_eo, ph ^ 1, status, abort_flag);
+                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R1, kdesc(tQ, k), kdesc(tOm, k), id_kk, k > 0);         // U_Q of chunk 0
+                mma_commit(bars + CM1);
+            }
+            for (int t = 0; t < T && ok; ++t) {
+                const uint32_t ph = t & 1;
+                const bool first = (t == 0), last = (t + 1 == T);
+#define CWAIT(b) do { ok = wait_or_abort(bars + (b), ph, status, abort_flag); } while (0)
+                CWAIT(CB_K); if (!ok) break;
+                tc_fence_after();
+                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R2, kdesc(tK, k), kdesc(tOm, k), id_kk, k > 0);         // U_K
+                mma_commit(bars + CM2);
+                CWAIT(CE0); if (!ok) break;                                     // phi(Q) packed in TMEM, R1 read, Q tile consumed
+                if (!last) load_tile(sQ, &p.mapQ, bars + CB_Q, D, t + 1);
+                CWAIT(CE1); if (!ok) break;                                     // phi(K) in smem, R2 read, K tile consumed
+                if (!last) load_tile(sK, &p.mapK, bars + CB_K, D, t + 1);
+                tc_fence_after();
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R1, FQ + k * 8, kdesc(tFK, k), id_kk, k > 0);                // P = phi(Q) phi(K)^T
+                mma_commit(bars + CM3);
+                if (!first)
+                    _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R2, FQ + k * 8, mndesc(tSb, k), id_o, k > 0);            // O = phi(Q) S_prev
+                CWAIT(CB_V); if (!ok) break;
+                tc_fence_after();
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColS, mndesc(tFK, k), mndesc(tV, k), id_s, (!first) || k > 0);   // S += phi(K)^T V
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColZ, mndesc(tFK, k), ones_desc, id_z, (!first) || k > 0);       // z += phi(K)^T 1
+                mma_commit(bars + CMS);
+                CWAIT(CE2); if (!ok) break;                                     // tril(P) packed in R1
+                tc_fence_after();
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R2, R1 + k * 8, mndesc(tV, k), id_o, (!first) || k > 0);     // O += P V
+                mma_commit(bars + CM4);
+                if (!last) {
+                    ok = wait_or_abort(bars + CB_Q, ph ^ 1, status, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    for (int k = 0; k < 8; ++k) mma_ss(tmem + kColR2, kdesc(sFQ, k), mndesc(sSb, k), id_o, k > 0);
-                    o_started = true;
+                    _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R1, kdesc(tQ, k), kdesc(tOm, k), id_kk, k > 0);     // U_Q of the next chunk
+                    mma_commit(bars + CM1);
                 }
-                if (MODE == MODE_QUERIES) mma_commit(bar_o);
-                if (MODE != MODE_QUERIES) {         // S += phi(K)^T V ; z += phi(K)^T 1
-                    ok = wait_or_abort(bar_v, ph, status, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after();
-                    for (int k = 0; k < 8; ++k) mma_ss(tmem + kColS, mndesc(sFK, k), mndesc(sV, k), id_s, (!first) || k > 0);
-                    for (int k = 0; k < 8; ++k)
-                        mma_ss(tmem + kColS + DV, mndesc(sFK, k), make_sdesc(smem_u32(sOnes), 16384, 1024), id_z, (!first) || k > 0);
-                    mma_commit(bar_s);
-                }
-                if (MODE == MODE_CAUSAL) {          // O += P V
-                    ok = wait_or_abort(bar_ep, ph, status, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after();
-                    for (int k = 0; k < 8; ++k) mma_ss(tmem + kColR2, kdesc(sP, k), mndesc(sV, k), id_o, o_started || k > 0);
-                    mma_commit(bar_o);
-                }
-                if (MODE != MODE_QUERIES && !last) { // key (causal) and value tiles are free: load the next
-                    if (MODE == MODE_CAUSAL) ok = wait_or_abort(bar_o, ph, status, abort_flag);
-                    if (ok) ok = wait_or_abort(bar_s, ph, status, abort_flag);
-                    if (!ok) break;
-                    if (MODE == MODE_CAUSAL) load_x(sK, &p.mapK, bar_k, t + 1);
-                    load_v(t + 1);
-                }
+                CWAIT(CM4); if (!ok) break;
+                if (!last) load_tile(sV, &p.mapV, bars + CB_V, DV, t + 1);
+                CWAIT(CE3); if (!ok) break;
+                CWAIT(CE4); if (!ok) break;
+#undef CWAIT
             }
         }
     } else {
-        // ============================== epilogue threads: thread = TMEM lane = tile row
-        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+        const int lane = tid & 31, q4 = warp & 3, g = warp >> 2, col0 = g * 32;
+        const int r = q4 * 32 + lane;
+        const uint32_t lane_addr = tmem + ((uint32_t)(q4 * 32) << 16);
+        const uint32_t R1 = lane_addr + kColR1, R2 = lane_addr + kColR2;
         const float cshift = p.cs[bh * p.nslab + slab];
-        const size_t prow0 = ((size_t)slab * p.BH + bh) * p.N;       // first row of this CTA's partial
+        const size_t prow0 = ((size_t)slab * p.BH + bh) * p.N;
         bool ok = true;
-        if (MODE == MODE_QUERIES) sZ[tid] = p.zacc[(size_t)bh * p.m + slab * 128 + tid];
-        if (MODE == MODE_CAUSAL) sZ[tid] = 0.f;
-        for (int t = t0; t < t1 && ok; ++t) {
-            const uint32_t ph = (t - t0) & 1;
-            const bool first = (t == t0), last = (t + 1 == t1);
-            float rmax = -INFINITY, dz = 0.f, rowsum = 0.f;
-            // ---------------- phi(Q)
-            if (MODE != MODE_KEYS) {
-                ok = wait_or_abort(bar_uq, ph, status, abort_flag);
-                if (!ok) break;
-                tc_fence_after();
-                for (int c0 = 0; c0 < 128; c0 += 32) {
-                    uint32_t v[32];
-                    tmem_ld32(lane_addr + kColR1 + c0, v);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) rmax = fmaxf(rmax, __uint_as_float(v[j]));
-                }
-                if (tid == 0) tma_store_wait_read();      // the staging tile (same memory) has been read out
-                epi_bar_sync();                            // also: z of the previous chunk is visible
-                for (int c0 = 0; c0 < 128; c0 += 32) {
-                    uint32_t v[32], pk[16];
-                    tmem_ld32(lane_addr + kColR1 + c0, v);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int j = 0; j < 32; j += 2) {
-                        const float f0 = ex2f(__uint_as_float(v[j]) - rmax), f1 = ex2f(__uint_as_float(v[j + 1]) - rmax);
-                        dz = fmaf(f0, sZ[c0 + j], dz);
-                        dz = fmaf(f1, sZ[c0 + j + 1], dz);
-                        pk[j / 2] = pack_bf16(f0, f1);
-                    }
-                    unsigned char *atom = sFQ + (c0 / 64) * 16384;
-#pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        *reinterpret_cast<uint4 *>(atom + swz128(tid, (c0 % 64) / 8 + q)) = make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
-                }
-                fence_async_smem();
-                tc_fence_before();
-                mbar_arrive(bar_eq);
-            }
-            // ---------------- phi(K)
-            if (MODE != MODE_QUERIES) {
-                const float nk = p.nK[(size_t)bh * p.N + (size_t)t * 128 + tid] + cshift;
-                if (MODE == MODE_KEYS && !first) ok = wait_or_abort(bar_s, ph ^ 1, status, abort_flag);
-                if (ok) ok = wait_or_abort(bar_uk, ph, status, abort_flag);
-                if (!ok) break;
-                tc_fence_after();
-                for (int c0 = 0; c0 < 128; c0 += 32) {
-                    uint32_t v[32], pk[16];
-                    tmem_ld32(lane_addr + kColR2 + c0, v);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int j = 0; j < 32; j += 2)
-                        pk[j / 2] = pack_bf16(ex2f(__uint_as_float(v[j]) - nk), ex2f(__uint_as_float(v[j + 1]) - nk));
-                    unsigned char *atom = sFK + (c0 / 64) * 16384;
-#pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        *reinterpret_cast<uint4 *>(atom + swz128(tid, (c0 % 64) / 8 + q)) = make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
-                }
-                fence_async_smem();
-                tc_fence_before();
-                mbar_arrive(bar_ek);
-            }
-            // ---------------- P = tril(phi(Q) phi(K)^T) as bf16 operand, and its row sums
-            if (MODE == MODE_CAUSAL) {
-                ok = wait_or_abort(bar_p, ph, status, abort_flag);
-                if (!ok) break;
-                tc_fence_after();
-                for (int c0 = 0; c0 < 128; c0 += 32) {
-                    uint32_t v[32], pk[16];
-                    tmem_ld32(lane_addr + kColR1 + c0, v);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int j = 0; j < 32; j += 2) {
-                        const float x0 = (c0 + j <= tid) ? __uint_as_float(v[j]) : 0.f;
-                        const float x1 = (c0 + j + 1 <= tid) ? __uint_as_float(v[j + 1]) : 0.f;
-                        rowsum += x0 + x1;
-                        pk[j / 2] = pack_bf16(x0, x1);
-                    }
-                    unsigned char *atom = sP + (c0 / 64) * 16384;
-#pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        *reinterpret_cast<uint4 *>(atom + swz128(tid, (c0 % 64) / 8 + q)) = make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
-                }
-                fence_async_smem();
-                tc_fence_before();
-                mbar_arrive(bar_ep);
-            }
-            // ---------------- partial output rows
-            if (MODE != MODE_KEYS) {
-                ok = wait_or_abort(bar_o, ph, status, abort_flag);
-                if (!ok) break;
-                tc_fence_after();
-                for (int c0 = 0; c0 < DV; c0 += 32) {
-                    uint32_t v[32];
-                    tmem_ld32(lane_addr + kColR2 + c0, v);
-                    tmem_wait_ld();
-                    unsigned char *atom = sStage + (c0 / 64) * 16384;
-#pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        *reinterpret_cast<uint4 *>(atom + swz128(tid, (c0 % 64) / 8 + q)) =
-                            make_uint4(pack_bf16(__uint_as_float(v[8 * q]), __uint_as_float(v[8 * q + 1])),
-                                       pack_bf16(__uint_as_float(v[8 * q + 2]), __uint_as_float(v[8 * q + 3])),
-                                       pack_bf16(__uint_as_float(v[8 * q + 4]), __uint_as_float(v[8 * q + 5])),
-                                       pack_bf16(__uint_as_float(v[8 * q + 6]), __uint_as_float(v[8 * q + 7])));
-                }
-                fence_async_smem();
-                tc_fence_before();
-                mbar_arrive(bar_eo);
-                epi_bar_sync();
-                if (tid == 0) {
-                    for (int a = 0; a < DV / 64; ++a) tma_store_2d(&p.mapPN, sStage + a * 16384, a * 64, (int)(prow0 + (size_t)t * 128));
-                    tma_store_commit();
-                }
-                const float den = rowsum + dz;
-                if (!(den > 0.f) || !isfinite(den)) atomicCAS(status, 0, (int)DARKATTN_ERR_NONFINITE);
-                *reinterpret_cast<float2 *>(p.pdr + 2 * (prow0 + (size_t)t * 128 + tid)) = make_float2(den, rmax + cshift);
-            }
-            // ---------------- bf16 copy of the state for the next chunk's phi(Q) S_prev
-            if (MODE == MODE_CAUSAL && !last) {
-                ok = wait_or_abort(bar_s, ph, status, abort_flag);
-                if (!ok) break;
-                tc_fence_after();
-                for (int c0 = 0; c0 < DV; c0 += 32) {
-                    uint32_t v[32];
-                    tmem_ld32(lane_addr + kColS + c0, v);
-                    tmem_wait_ld();
-                    unsigned char *atom = sSb + (c0 / 64) * 16384;
-#pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        *reinterpret_cast<uint4 *>(atom + swz128(tid, (c0 % 64) / 8 + q)) =
-                            make_uint4(pack_bf16(__uint_as_float(v[8 * q]), __uint_as_float(v[8 * q + 1])),
-                                       pack_bf16(__uint_as_float(v[8 * q + 2]), __uint_as_float(v[8 * q + 3])),
-                                       pack_bf16(__uint_as_float(v[8 * q + 4]), __uint_as_float(v[8 * q + 5])),
-                                       pack_bf16(__uint_as_float(v[8 * q + 6]), __uint_as_float(v[8 * q + 7])));
-                }
-                {
-                    uint32_t v[16];
-                    tmem_ld16(lane_addr + kColS + DV, v);
-                    tmem_wait_ld();
-                    sZ[tid] = __uint_as_float(v[0]);
-                }
-                fence_async_smem();
-                tc_fence_before();
-                mbar_arrive(bar_es);
-            }
-        }
-        if (MODE == MODE_KEYS && ok) {        // add this CTA's state to the global sums
-            ok = wait_or_abort(bar_s, (t1 - 1 - t0) & 1, status, abort_flag);
-            if (ok) {
-                tc_fence_after();
-                float *dst = p.Sacc + ((size_t)bh * p.m + slab * 128 + tid) * DV;
-                for (int c0 = 0; c0 < DV; c0 += 32) {
-                    uint32_t v[32];
-                    tmem_ld32(lane_addr + kColS + c0, v);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) atomicAdd(dst + c0 + j, __uint_as_float(v[j]));
-                }
-                uint32_t v[16];
-                tmem_ld16(lane_addr + kColS + DV, v);
+        for (int t = 0; t < T && ok; ++t) {
+            const uint32_t ph = t & 1;
+            const bool last = (t + 1 == T);
+#define EWAIT(b) do { ok = __all_sync(0xffffffffu, wait_or_abort(bars + (b), ph, status, abort_flag)); } while (0)
+            const float nk = p.nK[(size_t)row0 + (size_t)t * 128 + r] + cshift;
+            float rmax;
+            EWAIT(CM1); if (!ok) break;
+            tc_fence_after();
+            const float dz = query_features_to_tmem(R1, lane_addr + kColFQ, sRed, sZ, q4, g, r, col0, rmax);
+            tc_fence_before();
+            mbar_arrive_warp(bars + CE0);
+
+            EWAIT(CM2); if (!ok) break;
+            tc_fence_after();
+            features_to_tile(R2 + col0, nk, sFK, r, col0);
+            if (warp < 4)    // 2 KB of bf16 ones at the start of the staging tile: B operand of z += phi(K)^T 1
+                *reinterpret_cast<uint4 *>(sStg + tid * 16) = make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
+            fence_async_smem();
+            tc_fence_before();
+            mbar_arrive_warp(bars + CE1);
+
+            EWAIT(CM3); if (!ok) break;
+            tc_fence_after();
+            float rowsum = 0.f;
+            {
+                uint32_t v[32], pk[16];
+                tmem_ld32(R1 + col0, v);
                 tmem_wait_ld();
-                atomicAdd(p.zacc + (size_t)bh * p.m + slab * 128 + tid, __uint_as_float(v[0]));
+                quarter_sync(q4);
+#pragma unroll
+                for (int j = 0; j < 32; j += 2) {
+                    const float x0 = (col0 + j <= r) ? __uint_as_float(v[j]) : 0.f;
+                    const float x1 = (col0 + j + 1 <= r) ? __uint_as_float(v[j + 1]) : 0.f;
+                    rowsum += x0 + x1;
+                    pk[j / 2] = pack_bf16(x0, x1);
+                }
+                tmem_st16(R1 + col0 / 2, pk);
+                tmem_wait_st();
             }
+            tc_fence_before();
+            mbar_arrive_warp(bars + CE2);
+
+            EWAIT(CM4); if (!ok) break;
+            tc_fence_after();
+            if (col0 < DV) {
+                uint32_t v[32];
+                tmem_ld32(R2 + col0, v);
+                tmem_wait_ld();
+                store_row_f32x32_bf16(v, sStg, r, col0);
+            }
+            sRed[g * 128 + r] = rowsum + dz;
+            fence_async_smem();
+            tc_fence_before();
+            mbar_arrive_warp(bars + CE3);
+            epi_sync();
+            if (tid == 0) {
+                for (int a = 0; a < DV / 64; ++a) tma_store_2d(&p.mapPN, sStg + a * 16384, a * 64, (int)(prow0 + (size_t)t * 128));
+                tma_store_commit();
+            }
+            if (g == 0) {
+                const float den = sRed[r] + sRed[128 + r] + sRed[256 + r] + sRed[384 + r];
+                if (!(den > 0.f) || !isfinite(den)) atomicCAS(status, 0, (int)DARKATTN_ERR_NONFINITE);
+                *reinterpret_cast<float2 *>(p.pdr + 2 * (prow0 + (size_t)t * 128 + r)) = make_float2(den, rmax + cshift);
+            }
+            quarter_sync(q4);                      // the exchange array is free for the next chunk's maxima
+            EWAIT(CMS); if (!ok) break;
+            tc_fence_after();
+            if (!last) {
+                if (col0 < DV) tmem_row_to_tile(lane_addr + kColS + col0, sSb, r, col0);
+                if (g == 0) {
+                    uint32_t v[16];
+                    tmem_ld16(lane_addr + kColZ, v);
+                    tmem_wait_ld();
+                    sZ[r] = __uint_as_float(v[0]);
+                }
+                fence_async_smem();
+            }
+            if (tid == 0) tma_store_wait_read();   // staging (and the ones in it) may be rewritten after CE4
+            tc_fence_before();
+            mbar_arrive_warp(bars + CE4);
+#undef EWAIT
         }
-        if (MODE != MODE_KEYS && tid == 0) tma_store_wait_all();
+        if (tid == 0) tma_store_wait_all();
     }
     if (*abort_flag) __nanosleep(200000);   // error path only: let copies and MMAs in flight drain
     tc_fence_before();
     __syncthreads();
-    if (warp == 4) tmem_dealloc(tmem, 512);
+    if (warp == kEpiWarps) tmem_dealloc(tmem, 512);
+}
+
+// ------------------------------------------------------------------ non-causal, key pass: S = phi(K)^T V, z = phi(K)^T 1
+template <int D, int DV>
+struct FwdKeysSmem {
+    static constexpr int kOm = 0;
+    static constexpr int kK = kOm + 128 * D * 2;           // two K tiles
+    static constexpr int kV = kK + 2 * 128 * D * 2;        // two V tiles
+    static constexpr int kFK = kV + 2 * 128 * DV * 2;      // two phi(K) tiles
+    static constexpr int kOnes = kFK + 2 * 32768;
+    static constexpr int kBars = kOnes + 2048;
+    static constexpr int kTotal = kBars + 256;
+};
+
+enum KyBars { YB_OM, YB_K0, YB_K1, YB_V0, YB_V1, YM2_0, YM2_1, YMS_0, YMS_1, YE1_0, YE1_1, YNBARS };
+
+// One CTA per (b, h, slab, token split); tiles alternate between two sets of buffers and two TMEM regions so that
+// the projection of tile i+1 runs while the epilogue warps exponentiate tile i.
+template <int D, int DV>
+__global__ void __launch_bounds__(kThreads, 1) tc_fwd_keys_kernel(const __grid_constant__ MainParams p)
+{
+    using L = FwdKeysSmem<D, DV>;
+    extern __shared__ __align__(1024) unsigned char smem[];
+    constexpr int kXT = 128 * D * 2, kVT = 128 * DV * 2;
+    unsigned char *sOm = smem + L::kOm, *sK = smem + L::kK, *sV = smem + L::kV, *sFK = smem + L::kFK, *sOnes = smem + L::kOnes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::kBars);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + YNBARS);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + YNBARS + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int unit = blockIdx.x / p.nsplit, split = blockIdx.x % p.nsplit;
+    const int bh = unit / p.nslab, slab = unit % p.nslab, h = bh % p.H;
+    const int t0 = (int)((long long)p.T * split / p.nsplit), t1 = (int)((long long)p.T * (split + 1) / p.nsplit);
+    const int n = t1 - t0, row0 = bh * p.N;
+
+    if (tid == 0) {
+        for (int i = 0; i < YE1_0; ++i) mbar_init(bars + i, 1);
+        mbar_init(bars + YE1_0, kEpiWarps); mbar_init(bars + YE1_1, kEpiWarps);
+        *abort_flag = (smem_u32(smem) & 1023u) ? 1 : 0;
+        fence_mbar_init();
+    }
+    if (tid < 128) {
+        *reinterpret_cast<uint4 *>(sOnes + tid * 16) = make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
+        fence_async_smem();
+    }
+    if (warp == kEpiWarps) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    int *status = p.status;
+
+    if (*abort_flag) {
+        if (tid == 0) atomicExch(status, (int)DARKATTN_ERR_CUDA);
+    } else if (n <= 0) {
+    } else if (warp == kEpiWarps) {
+        if ((tid & 31) == 0) {
+            auto load_k = [&](int i) {
+                const int b = i & 1;
+                mbar_expect_tx(bars + YB_K0 + b, kXT);
+                for (int a = 0; a < D / 64; ++a) tma_load_2d(sK + b * kXT + a * 16384, &p.mapK, bars + YB_K0 + b, a * 64, row0 + (t0 + i) * 128);
+            };
+            auto load_v = [&](int i) {
+                const int b = i & 1;
+                mbar_expect_tx(bars + YB_V0 + b, kVT);
+                for (int a = 0; a < DV / 64; ++a) tma_load_2d(sV + b * kVT + a * 16384, &p.mapV, bars + YB_V0 + b, a * 64, row0 + (t0 + i) * 128);
+            };
+            const TileDesc tOm(sOm), tK0(sK), tK1(sK + kXT), tV0(sV), tV1(sV + kVT), tF0(sFK), tF1(sFK + 32768);
+            const uint64_t ones_desc = make_sdesc(smem_u32(sOnes), 16384, 1024);
+            const uint32_t id_kk = make_idesc(128, 128, 0, 0), id_s = make_idesc(128, DV, 1, 1), id_z = make_idesc(128, 16, 1, 1);
+
+            mbar_expect_tx(bars + YB_OM, 128 * D * 2);
+            for (int a = 0; a < D / 64; ++a) tma_load_2d(sOm + a * 16384, &p.mapOm, bars + YB_OM, a * 64, h * p.m + slab * 128);
+            load_k(0); load_v(0);
+            if (n > 1) { load_k(1); load_v(1); }
+            bool ok = wait_or_abort(bars + YB_OM, 0, status, abort_flag);
+            if (ok) ok = wait_or_abort(bars + YB_K0, 0, status, abort_flag);
+            if (ok) {
+                tc_fence_after();
+                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(tmem + kColR1, kdesc(tK0, k), kdesc(tOm, k), id_kk, k > 0);
+                mma_commit(bars + YM2_0);
+            }
+            for (int i = 0; i < n && ok; ++i) {
+                const int b = i & 1;
+                const uint32_t phb = (i >> 1) & 1;
+                if (i + 1 < n) {       // projection of the next tile into the other region (read out two tiles ago)
+                    ok = wait_or_abort(bars + YB_K0 + (b ^ 1), ((i + 1) >> 1) & 1, status, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const TileDesc &tKn = b ? tK0 : tK1;
+                    _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(tmem + (b ? kColR1 : kColR2), kdesc(tKn, k), kdesc(tOm, k), id_kk, k > 0);
+                    mma_commit(bars + YM2_0 + (b ^ 1));
+                }
+                ok = wait_or_abort(bars + YE1_0 + b, phb, status, abort_flag);      // phi(K) of tile i in smem; its K tile is consumed
+                if (!ok) break;
+                if (i + 2 < n) load_k(i + 2);
+                ok = wait_or_abort(bars + YB_V0 + b, phb, status, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                const TileDesc &tF = b ? tF1 : tF0, &tVb = b ? tV1 : tV0;
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColS, mndesc(tF, k), mndesc(tVb, k), id_s, i > 0 || k > 0);
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColZ, mndesc(tF, k), ones_desc, id_z, i > 0 || k > 0);
+                mma_commit(bars + YMS_0 + b);
+                ok = wait_or_abort(bars + YMS_0 + b, phb, status, abort_flag);
+                if (!ok) break;
+                if (i + 2 < n) load_v(i + 2);
+            }
+        }
+    } else {
+        const int lane = tid & 31, q4 = warp & 3, g = warp >> 2, col0 = g * 32;
+        const int r = q4 * 32 + lane;
+        const uint32_t lane_addr = tmem + ((uint32_t)(q4 * 32) << 16);
+        const float cshift = p.cs[bh * p.nslab + slab];
+        bool ok = true;
+        for (int i = 0; i < n && ok; ++i) {
+            const int b = i & 1;
+            const uint32_t phb = (i >> 1) & 1;
+            const float nk = p.nK[(size_t)row0 + (size_t)(t0 + i) * 128 + r] + cshift;
+            ok = __all_sync(0xffffffffu, wait_or_abort(bars + YM2_0 + b, phb, status, abort_flag));
+            if (!ok) break;
+            tc_fence_after();
+            features_to_tile(lane_addr + (b ? kColR2 : kColR1) + col0, nk, sFK + b * 32768, r, col0);
+            fence_async_smem();
+            tc_fence_before();
+            mbar_arrive_warp(bars + YE1_0 + b);
+        }
+        if (ok) ok = __all_sync(0xffffffffu, wait_or_abort(bars + YMS_0 + ((n - 1) & 1), ((n - 1) >> 1) & 1, status, abort_flag));
+        if (ok) {        // add this CTA's state to the global sums
+            tc_fence_after();
+            if (col0 < DV) {
+                float *dst = p.Sacc + ((size_t)bh * p.m + slab * 128 + r) * DV + col0;
+                uint32_t v[32];
+                tmem_ld32(lane_addr + kColS + col0, v);
+                tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 32; ++j) atomicAdd(dst + j, __uint_as_float(v[j]));
+            }
+            if (g == 0) {
+                uint32_t v[16];
+                tmem_ld16(lane_addr + kColZ, v);
+                tmem_wait_ld();
+                atomicAdd(p.zacc + (size_t)bh * p.m + slab * 128 + r, __uint_as_float(v[0]));
+            }
+        }
+    }
+    if (*abort_flag) __nanosleep(200000);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kEpiWarps) tmem_dealloc(tmem, 512);
+}
+
+// ------------------------------------------------------------------ non-causal, query pass: partial O = phi(Q) S, den = phi(Q) z
+template <int D, int DV>
+struct FwdQueriesSmem {
+    static constexpr int kOm = 0;
+    static constexpr int kQ = kOm + 128 * D * 2;           // two Q tiles
+    static constexpr int kSb = kQ + 2 * 128 * D * 2;       // bf16 state of the slab [128 l, DV]
+    static constexpr int kStg = kSb + 128 * DV * 2;
+    static constexpr int kZ = kStg + 128 * DV * 2;
+    static constexpr int kRed = kZ + 512;
+    static constexpr int kBars = kRed + 2048;
+    static constexpr int kTotal = kBars + 256;
+};
+
+enum QyBars { UB_OM, UB_Q0, UB_Q1, UM1_0, UM1_1, UM4_0, UM4_1, UE0_0, UE0_1, UE3_0, UE3_1, UNBARS };
+
+// TMEM: packed phi(Q) of the two tiles in flight at 0 and 64; R1, R2 hold U_Q and then the output tile.
+template <int D, int DV>
+__global__ void __launch_bounds__(kThreads, 1) tc_fwd_queries_kernel(const __grid_constant__ MainParams p)
+{
+    using L = FwdQueriesSmem<D, DV>;
+    extern __shared__ __align__(1024) unsigned char smem[];
+    constexpr int kXT = 128 * D * 2;
+    unsigned char *sOm = smem + L::kOm, *sQ = smem + L::kQ, *sSb = smem + L::kSb, *sStg = smem + L::kStg;
+    float *sZ = reinterpret_cast<float *>(smem + L::kZ), *sRed = reinterpret_cast<float *>(smem + L::kRed);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::kBars);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + UNBARS);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + UNBARS + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int unit = blockIdx.x / p.nsplit, split = blockIdx.x % p.nsplit;
+    const int bh = unit / p.nslab, slab = unit % p.nslab, h = bh % p.H;
+    const int t0 = (int)((long long)p.T * split / p.nsplit), t1 = (int)((long long)p.T * (split + 1) / p.nsplit);
+    const int n = t1 - t0, row0 = bh * p.N;
+
+    if (tid == 0) {
+        for (int i = 0; i < UE0_0; ++i) mbar_init(bars + i, 1);
+        for (int i = UE0_0; i < UNBARS; ++i) mbar_init(bars + i, kEpiWarps);
+        *abort_flag = (smem_u32(smem) & 1023u) ? 1 : 0;
+        fence_mbar_init();
+    }
+    if (tid < 128) sZ[tid] = p.zacc[(size_t)bh * p.m + slab * 128 + tid];
+    if (warp == kEpiWarps) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    int *status = p.status;
+
+    if (*abort_flag) {
+        if (tid == 0) atomicExch(status, (int)DARKATTN_ERR_CUDA);
+    } else if (n <= 0) {
+    } else if (warp == kEpiWarps) {
+        if ((tid & 31) == 0) {
+            auto load_q = [&](int i) {
+                const int b = i & 1;
+                mbar_expect_tx(bars + UB_Q0 + b, kXT);
+                for (int a = 0; a < D / 64; ++a) tma_load_2d(sQ + b * kXT + a * 16384, &p.mapQ, bars + UB_Q0 + b, a * 64, row0 + (t0 + i) * 128);
+            };
+            const TileDesc tOm(sOm), tQ0(sQ), tQ1(sQ + kXT), tSb(sSb);
+            const uint32_t id_kk = make_idesc(128, 128, 0, 0), id_o = make_idesc(128, DV, 0, 1);
+            mbar_expect_tx(bars + UB_OM, 128 * D * 2 + 128 * DV * 2);
+            for (int a = 0; a < D / 64; ++a) tma_load_2d(sOm + a * 16384, &p.mapOm, bars + UB_OM, a * 64, h * p.m + slab * 128);
+            for (int a = 0; a < DV / 64; ++a) tma_load_2d(sSb + a * 16384, &p.mapSb, bars + UB_OM, a * 64, bh * p.m + slab * 128);
+            load_q(0);
+            if (n > 1) load_q(1);
+            bool ok = wait_or_abort(bars + UB_OM, 0, status, abort_flag);
+            if (ok) ok = wait_or_abort(bars + UB_Q0, 0, status, abort_flag);
+            if (ok) {
+                tc_fence_after();
+                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(tmem + kColR1, kdesc(tQ0, k), kdesc(tOm, k), id_kk, k > 0);
+                mma_commit(bars + UM1_0);
+            }
+            for (int i = 0; i < n && ok; ++i) {
+                const int b = i & 1;
+                const uint32_t phb = (i >> 1) & 1;
+                if (i + 1 < n) {       // projection of the next tile into the other region, once its last output tile was read
+                    ok = wait_or_abort(bars + UB_Q0 + (b ^ 1), ((i + 1) >> 1) & 1, status, abort_flag);
+                    if (ok && i >= 1) ok = wait_or_abort(bars + UE3_0 + (b ^ 1), ((i - 1) >> 1) & 1, status, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const TileDesc &tQn = b ? tQ0 : tQ1;
+                    _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(tmem + (b ? kColR1 : kColR2), kdesc(tQn, k), kdesc(tOm, k), id_kk, k > 0);
+                    mma_commit(bars + UM1_0 + (b ^ 1));
+                }
+                ok = wait_or_abort(bars + UE0_0 + b, phb, status, abort_flag);      // phi(Q) packed; U read; Q tile consumed
+                if (!ok) break;
+                if (i + 2 < n) load_q(i + 2);
+                tc_fence_after();
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(tmem + (b ? kColR2 : kColR1), tmem + b * 64 + k * 8, mndesc(tSb, k), id_o, k > 0);
+                mma_commit(bars + UM4_0 + b);
+            }
+        }
+    } else {
+        const int lane = tid & 31, q4 = warp & 3, g = warp >> 2, col0 = g * 32;
+        const int r = q4 * 32 + lane;
+        const uint32_t lane_addr = tmem + ((uint32_t)(q4 * 32) << 16);
+        const float cshift = p.cs[bh * p.nslab + slab];
+        const size_t prow0 = ((size_t)slab * p.BH + bh) * p.N;
+        bool ok = true;
+        for (int i = 0; i < n && ok; ++i) {
+            const int b = i & 1;
+            const uint32_t phb = (i >> 1) & 1;
+            const uint32_t R = lane_addr + (b ? kColR2 : kColR1);
+            float rmax;
+            ok = __all_sync(0xffffffffu, wait_or_abort(bars + UM1_0 + b, phb, status, abort_flag));
+            if (!ok) break;
+            tc_fence_after();
+            const float dz = query_features_to_tmem(R, lane_addr + b * 64, sRed, sZ, q4, g, r, col0, rmax);
+            tc_fence_before();
+            mbar_arrive_warp(bars + UE0_0 + b);
+
+            ok = __all_sync(0xffffffffu, wait_or_abort(bars + UM4_0 + b, phb, status, abort_flag));
+            if (!ok) break;
+            tc_fence_after();
+            uint32_t v[32];
+            if (col0 < DV) {
+                tmem_ld32(R + col0, v);
+                tmem_wait_ld();
+            }
+            tc_fence_before();
+            mbar_arrive_warp(bars + UE3_0 + b);
+            if (tid == 0) tma_store_wait_read();       // the previous tile's store has left the staging tile
+            epi_sync();
+            if (col0 < DV) store_row_f32x32_bf16(v, sStg, r, col0);
+            sRed[g * 128 + r] = dz;
+            fence_async_smem();
+            epi_sync();
+            if (tid == 0) {
+                for (int a = 0; a < DV / 64; ++a) tma_store_2d(&p.mapPN, sStg + a * 16384, a * 64, (int)(prow0 + (size_t)(t0 + i) * 128));
+                tma_store_commit();
+            }
+            if (g == 0) {
+                const float den = sRed[r] + sRed[128 + r] + sRed[256 + r] + sRed[384 + r];
+                if (!(den > 0.f) || !isfinite(den)) atomicCAS(status, 0, (int)DARKATTN_ERR_NONFINITE);
+                *reinterpret_cast<float2 *>(p.pdr + 2 * (prow0 + (size_t)(t0 + i) * 128 + r)) = make_float2(den, rmax + cshift);
+            }
+            quarter_sync(q4);
+        }
+        if (tid == 0) tma_store_wait_all();
+    }
+    if (*abort_flag) __nanosleep(200000);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kEpiWarps) tmem_dealloc(tmem, 512);
 }
 
 // Sb[bh,l,:] = bf16(Sacc[bh,l,:])  (operand of the query pass)
@@ -554,11 +769,25 @@ size_t take(size_t &off, size_t bytes)
 template <int D, int DV, int MODE>
 cudaError_t launch_main(const MainParams &P, int grid, cudaStream_t st)
 {
-    using L = SmemLayout<D, DV, MODE>;
-    static_assert(L::kTotal <= 232448, "shared memory budget of one CTA exceeded");
-    cudaError_t e = cudaFuncSetAttribute(tc_attn_kernel<D, DV, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
-    if (e != cudaSuccess) return e;
-    tc_attn_kernel<D, DV, MODE><<<grid, 160, L::kTotal, st>>>(P);
+    if constexpr (MODE == MODE_CAUSAL) {
+        using L = FwdCausalSmem<D, DV>;
+        static_assert(L::kTotal <= 232448, "shared memory budget of one CTA exceeded");
+        cudaError_t e = cudaFuncSetAttribute(tc_fwd_causal_kernel<D, DV>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
+        if (e != cudaSuccess) return e;
+        tc_fwd_causal_kernel<D, DV><<<grid, kThreads, L::kTotal, st>>>(P);
+    } else if constexpr (MODE == MODE_KEYS) {
+        using L = FwdKeysSmem<D, DV>;
+        static_assert(L::kTotal <= 232448, "shared memory budget of one CTA exceeded");
+        cudaError_t e = cudaFuncSetAttribute(tc_fwd_keys_kernel<D, DV>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
+        if (e != cudaSuccess) return e;
+        tc_fwd_keys_kernel<D, DV><<<grid, kThreads, L::kTotal, st>>>(P);
+    } else {
+        using L = FwdQueriesSmem<D, DV>;
+        static_assert(L::kTotal <= 232448, "shared memory budget of one CTA exceeded");
+        cudaError_t e = cudaFuncSetAttribute(tc_fwd_queries_kernel<D, DV>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
+        if (e != cudaSuccess) return e;
+        tc_fwd_queries_kernel<D, DV><<<grid, kThreads, L::kTotal, st>>>(P);
+    }
     return cudaGetLastError();
 }
 
@@ -701,19 +930,19 @@ darkattn_status_t tensor_forward(const darkattn_plan_s *plan, const void *Q, con
     const int units = (int)(BH * Y.nslab);
     if (D.causal) {
         P.nsplit = 1;
-        timer_mark(plan, st, "tc_attn_kernel<causal>");
+        timer_mark(plan, st, "tc_fwd_causal_kernel");
         cudaError_t x = launch_main_shape<MODE_CAUSAL>(D.d, D.dv, P, units, st);
         if (x != cudaSuccess && e == cudaSuccess) e = x;
     } else {
         e = (e == cudaSuccess) ? cudaMemsetAsync(ws + Y.Sacc, 0, (Y.Sb - Y.Sacc), st) : e;   // S and z sums
-        timer_mark(plan, st, "tc_attn_kernel<keys>");
+        timer_mark(plan, st, "tc_fwd_keys_kernel");
         cudaError_t x = launch_main_shape<MODE_KEYS>(D.d, D.dv, P, units * Y.nsplit, st);
         if (x != cudaSuccess && e == cudaSuccess) e = x;
         const long long n = (long long)BH * D.m * D.dv;
         timer_mark(plan, st, "state_to_bf16_kernel");
         state_to_bf16_kernel<<<(unsigned)((n + 1023) / 1024), 256, 0, st>>>(fl(Y.Sacc), bf(Y.Sb), n);
         chk();
-        timer_mark(plan, st, "tc_attn_kernel<queries>");
+        timer_mark(plan, st, "tc_fwd_queries_kernel");
         x = launch_main_shape<MODE_QUERIES>(D.d, D.dv, P, units * Y.nsplit, st);
         if (x != cudaSuccess && e == cudaSuccess) e = x;
     }
