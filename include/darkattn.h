@@ -83,8 +83,10 @@ darkattn_status_t darkattn_plan(const darkattn_desc_t *desc, darkattn_plan_t *ou
  * the two needs). Contents need not be preserved between calls.                                  */
 size_t darkattn_workspace_bytes(darkattn_plan_t plan);
 
-/* Bytes of the forward->backward stash (`saved`). 0 means backward recomputes what it needs and
- * `saved` may be NULL in both calls.                                                             */
+/* Bytes of the forward->backward stash (`saved`): what the forward pass computed and the backward
+ * pass needs again (on the tensor-core path the per-row normalisers, the key norms, the folded
+ * projections and the key-side shifts). 0 means there is none. `saved` may always be NULL in both
+ * calls: backward then recomputes what it needs, at the cost of running the forward kernels again. */
 size_t darkattn_saved_bytes(darkattn_plan_t plan);
 
 /* The path (DARKATTN_PATH_SIMT or DARKATTN_PATH_TENSOR) the plan resolved to.                   */

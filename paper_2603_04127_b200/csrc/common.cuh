@@ -71,8 +71,30 @@ struct TensorLayout {
     size_t Tacc;    // sum_i E_i^T x_i over both sides and the batch, fp32 [H, m, d]
     size_t dMn;     // gradient of M through the key norm term, fp32 [H, r, d]
     size_t total_bytes;
+    // the forward -> backward stash (`saved`): per-row normalisers, key norms, folded projections, key shifts
+    size_t sv_sv, sv_nK, sv_Om, sv_cs, sv_bytes;
     int nslab, T, nsplit;
 };
+
+// Where one call keeps what the prologue and the forward pass leave for the backward pass: in the
+// caller's `saved` buffer when there is one, else in the workspace.
+struct Stash {
+    float2 *sv;
+    float *nK;
+    __nv_bfloat16 *Om;
+    float *cs;
+};
+inline Stash stash_in_workspace(const TensorLayout &Y, char *ws)
+{
+    return Stash{reinterpret_cast<float2 *>(ws + Y.sv), reinterpret_cast<float *>(ws + Y.nK),
+                 reinterpret_cast<__nv_bfloat16 *>(ws + Y.Om), reinterpret_cast<float *>(ws + Y.cs)};
+}
+inline Stash stash_in_saved(const TensorLayout &Y, void *saved)
+{
+    char *b = static_cast<char *>(saved);
+    return Stash{reinterpret_cast<float2 *>(b + Y.sv_sv), reinterpret_cast<float *>(b + Y.sv_nK),
+                 reinterpret_cast<__nv_bfloat16 *>(b + Y.sv_Om), reinterpret_cast<float *>(b + Y.sv_cs)};
+}
 
 }  // namespace darkattn
 
@@ -123,9 +145,9 @@ bool tensor_supported(const darkattn_plan_s *plan);
 void tensor_make_layout(darkattn_plan_s *plan);
 darkattn_status_t tensor_forward(const darkattn_plan_s *plan, const void *Q, const void *K, const void *V,
                                  const void *M, const void *W, void *O, void *saved, char *ws, cudaStream_t st);
-// Folded projections, key-side shifts and key norms (written to the workspace); shared by forward and backward.
+// Folded projections, key-side shifts and key norms (written to `out`).
 cudaError_t tensor_prologue(const darkattn_plan_s *plan, const void *K, const void *M, const void *W, char *ws,
-                            cudaStream_t st);
+                            const Stash &out, cudaStream_t st);
 darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, const void *K, const void *V,
                                   const void *M, const void *W, const void *O, const void *dO, const void *saved,
                                   void *dQ, void *dK, void *dV, float *dM, char *ws, cudaStream_t st);

@@ -104,16 +104,6 @@ __device__ __forceinline__ void features_to_tile_sums(uint32_t taddr, float offs
     atomicAdd(colsum + col0 + lane, warp_column_sums(f, lane));
 }
 
-// 32 fp32 TMEM columns at taddr -> 32 bf16 at dst (global memory)
-__device__ __forceinline__ void tmem_row_to_global(uint32_t taddr, __nv_bfloat16 *dst)
-{
-    uint32_t v[32];
-    tmem_ld32(taddr, v);
-    tmem_wait_ld();
-#pragma unroll
-    for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4 *>(dst + 8 * q) = pack8(v + 8 * q);
-}
-
 enum QBars { QB_OM, QB_Q, QB_K, QB_V, QB_G, QB_X2, QM1, QM2, QM3, QMS, QM4, QM5, QM6, QE0, QE1, QE2, QE3, QE4, QNBARS };
 
 // ------------------------------------------------------------------ query side (forward direction)
@@ -810,20 +800,22 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __gr
 }
 
 // ------------------------------------------------------------------ small SIMT kernels
-// delta[row] = dO[row,:] . O[row,:]; one warp per row.
+// delta[row] = dO[row,:] . O[row,:]; dv/8 threads per row, 16 bytes of each tensor per thread.
 __global__ void delta_kernel(const __nv_bfloat16 *G, const __nv_bfloat16 *O, float *delta, long long rows, int dv)
 {
-    const long long row = (blockIdx.x * (long long)blockDim.x + threadIdx.x) / 32;
-    const int lane = threadIdx.x % 32;
-    if (row >= rows) return;
+    const int per_row = dv / 8;                       // 8 or 16: a power of two that divides the warp
+    const long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+    const long long row = i / per_row;
     float acc = 0.f;
-    for (int c = lane * 2; c < dv; c += 64) {
-        const float2 g = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(G + row * dv + c));
-        const float2 o = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(O + row * dv + c));
-        acc = fmaf(g.x, o.x, fmaf(g.y, o.y, acc));
+    if (row < rows) {
+        float g[8], o[8];
+        unpack8(*reinterpret_cast<const uint4 *>(G + i * 8), g);
+        unpack8(*reinterpret_cast<const uint4 *>(O + i * 8), o);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc = fmaf(g[j], o[j], acc);
     }
-    for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) delta[row] = acc;
+    for (int o = per_row / 2; o; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (row < rows && (i % per_row) == 0) delta[row] = acc;
 }
 
 // out[row, c] = scale * sum_s part[s, row, c]; one thread per 8 columns.
@@ -909,21 +901,22 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
     auto keep = [&](cudaError_t x) { if (x != cudaSuccess && e == cudaSuccess) e = x; };
     auto chk = [&]() { keep(cudaGetLastError()); };
 
-    // The forward result and its per-row normalisers: taken from the caller when both are given,
-    // otherwise recomputed into the workspace (that run also leaves the prologue's results there).
-    const float2 *sv = reinterpret_cast<const float2 *>(saved);
+    // The forward result and what the forward pass stashed (per-row normalisers, key norms, folded
+    // projections, key shifts): taken from the caller when both are given, otherwise recomputed into the
+    // workspace by running the forward kernels again.
+    Stash stash;
     if (!O || !saved) {
         darkattn_status_t s = tensor_forward(plan, Q, K, V, M, W, bf(Y.Oscr), nullptr, ws, st);
         if (s != DARKATTN_OK) return s;
         O = bf(Y.Oscr);
-        sv = reinterpret_cast<const float2 *>(ws + Y.sv);
+        stash = stash_in_workspace(Y, ws);
     } else {
-        keep(tensor_prologue(plan, K, M, W, ws, st));
+        stash = stash_in_saved(Y, const_cast<void *>(saved));
     }
 
     const long long rows = (long long)BH * N;
     timer_mark(plan, st, "delta_kernel");
-    delta_kernel<<<(unsigned)((rows * 32 + 255) / 256), 256, 0, st>>>((const __nv_bfloat16 *)dO, (const __nv_bfloat16 *)O, fl(Y.delta), rows, D.dv);
+    delta_kernel<<<(unsigned)((rows * (D.dv / 8) + 255) / 256), 256, 0, st>>>((const __nv_bfloat16 *)dO, (const __nv_bfloat16 *)O, fl(Y.delta), rows, D.dv);
     chk();
     keep(cudaMemsetAsync(ws + Y.Tacc, 0, (size_t)D.H * D.m * D.d * 4, st));
     keep(cudaMemsetAsync(ws + Y.dMn, 0, (size_t)D.H * D.r * D.d * 4, st));
@@ -932,7 +925,7 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
     memset(&P, 0, sizeof(P));
     bool ok = make_map(&P.mapQ, Q, BH * N, D.d, 128) && make_map(&P.mapK, K, BH * N, D.d, 128) &&
               make_map(&P.mapV, V, BH * N, D.dv, 128) && make_map(&P.mapG, dO, BH * N, D.dv, 128) &&
-              make_map(&P.mapOm, bf(Y.Om), (size_t)D.H * D.m, D.d, 128) &&
+              make_map(&P.mapOm, stash.Om, (size_t)D.H * D.m, D.d, 128) &&
               make_map(&P.mapPQ, bf(Y.pdQ), (size_t)Y.nslab * BH * N, D.d, 128) &&
               make_map(&P.mapPK, bf(Y.pdK), (size_t)Y.nslab * BH * N, D.d, 128) &&
               make_map(&P.mapPV, bf(Y.pdV), (size_t)Y.nslab * BH * N, D.dv, 128);
@@ -941,7 +934,7 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
     ok = ok && make_map(&F.mapM, M, (size_t)D.H * D.r, D.d, 128);
     if (!ok) { set_cuda_error(cudaErrorInvalidValue, "tensor_backward: tensor map encode"); return DARKATTN_ERR_CUDA; }
     F.mapK = P.mapK;
-    P.sv = sv; P.delta = fl(Y.delta); P.nK = fl(Y.nK); P.cs = fl(Y.cs); P.rhoc = fl(Y.rhoc);
+    P.sv = stash.sv; P.delta = fl(Y.delta); P.nK = stash.nK; P.cs = stash.cs; P.rhoc = fl(Y.rhoc);
     P.pdQ = bf(Y.pdQ); P.pdK = bf(Y.pdK); P.pdV = bf(Y.pdV); P.espart = fl(Y.espart); P.Tacc = fl(Y.Tacc);
     P.status = reinterpret_cast<int *>(ws + Y.status);
     P.N = D.N; P.H = D.H; P.BH = D.BH; P.m = D.m; P.nslab = Y.nslab; P.T = Y.T;

@@ -722,36 +722,57 @@ __global__ void state_to_bf16_kernel(const float *S, __nv_bfloat16 *Sb, long lon
 }
 
 // O[row,:] = sum_s num_s[row,:] 2^(rho_s - rho) / sum_s den_s 2^(rho_s - rho), rho = max_s rho_s.
-// One thread per 8 output columns.
-// The combined normaliser and rho are also written to sv (and to sv2 when given) for the backward pass.
-__global__ void combine_kernel(const __nv_bfloat16 *pnum, const float *pdr, __nv_bfloat16 *O, float2 *sv, float2 *sv2,
-                               long long rows, int dv, int nslab)
+// One thread per 8 output columns. The combined normaliser and rho are also written to sv for the backward pass.
+// NS > 0: the number of slabs at compile time (all loads of a thread are issued before the first use).
+template <int NS>
+__global__ void combine_kernel(const __nv_bfloat16 *pnum, const float *pdr, __nv_bfloat16 *O, float2 *sv,
+                               long long rows, int dv, int nslab_rt)
 {
     const long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;
     const int per_row = dv / 8;
     if (i >= rows * per_row) return;
     const long long row = i / per_row;
     const int c0 = (int)(i % per_row) * 8;
-    float rho = -INFINITY;
-    for (int s = 0; s < nslab; ++s) rho = fmaxf(rho, pdr[2 * ((size_t)s * rows + row) + 1]);
-    float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}, den = 0.f;
-    for (int s = 0; s < nslab; ++s) {
-        const float2 dr = *reinterpret_cast<const float2 *>(pdr + 2 * ((size_t)s * rows + row));
-        const float w = exp2f(dr.y - rho);
-        den = fmaf(dr.x, w, den);
-        const uint4 raw = *reinterpret_cast<const uint4 *>(pnum + ((size_t)s * rows + row) * dv + c0);
-        const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
+    float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}, den = 0.f, rho = -INFINITY;
+    if constexpr (NS > 0) {
+        float2 dr[NS];
+        uint4 raw[NS];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const float2 f = __bfloat1622float2(h2[q]);
-            acc[2 * q] = fmaf(f.x, w, acc[2 * q]);
-            acc[2 * q + 1] = fmaf(f.y, w, acc[2 * q + 1]);
+        for (int s = 0; s < NS; ++s) {
+            dr[s] = *reinterpret_cast<const float2 *>(pdr + 2 * ((size_t)s * rows + row));
+            raw[s] = *reinterpret_cast<const uint4 *>(pnum + ((size_t)s * rows + row) * dv + c0);
+        }
+#pragma unroll
+        for (int s = 0; s < NS; ++s) rho = fmaxf(rho, dr[s].y);
+#pragma unroll
+        for (int s = 0; s < NS; ++s) {
+            const float w = exp2f(dr[s].y - rho);
+            den = fmaf(dr[s].x, w, den);
+            const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&raw[s]);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const float2 f = __bfloat1622float2(h2[q]);
+                acc[2 * q] = fmaf(f.x, w, acc[2 * q]);
+                acc[2 * q + 1] = fmaf(f.y, w, acc[2 * q + 1]);
+            }
+        }
+    } else {
+        for (int s = 0; s < nslab_rt; ++s) rho = fmaxf(rho, pdr[2 * ((size_t)s * rows + row) + 1]);
+        for (int s = 0; s < nslab_rt; ++s) {
+            const float2 dr = *reinterpret_cast<const float2 *>(pdr + 2 * ((size_t)s * rows + row));
+            const float w = exp2f(dr.y - rho);
+            den = fmaf(dr.x, w, den);
+            const uint4 raw = *reinterpret_cast<const uint4 *>(pnum + ((size_t)s * rows + row) * dv + c0);
+            const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const float2 f = __bfloat1622float2(h2[q]);
+                acc[2 * q] = fmaf(f.x, w, acc[2 * q]);
+                acc[2 * q + 1] = fmaf(f.y, w, acc[2 * q + 1]);
+            }
         }
     }
-    if (c0 == 0) {
-        sv[row] = make_float2(den, rho);
-        if (sv2) sv2[row] = make_float2(den, rho);
-    }
+    if (c0 == 0) sv[row] = make_float2(den, rho);
     const float inv = 1.f / den;
     uint4 out;
     out.x = pack_bf16(acc[0] * inv, acc[1] * inv); out.y = pack_bf16(acc[2] * inv, acc[3] * inv);
@@ -845,7 +866,15 @@ void tensor_make_layout(darkattn_plan_s *plan)
     Y.Sb = take(off, BH * m * dv * 2);
     Y.sv = take(off, BH * N * 8);
     plan->launches_fwd = D.causal ? 5 : 7;
-    plan->saved_bytes = BH * N * 8;
+    {
+        size_t so = 0;
+        Y.sv_sv = take(so, BH * N * 8);
+        Y.sv_nK = take(so, BH * N * 4);
+        Y.sv_Om = take(so, (size_t)D.H * m * d * 2);
+        Y.sv_cs = take(so, BH * Y.nslab * 4);
+        Y.sv_bytes = so;
+        plan->saved_bytes = so;
+    }
     if (D.causal) {       // tensor-core backward (the non-causal backward runs on the FP32 path)
         Y.Oscr = take(off, BH * N * dv * 2);
         Y.delta = take(off, BH * N * 4);
@@ -863,13 +892,11 @@ void tensor_make_layout(darkattn_plan_s *plan)
 }
 
 cudaError_t tensor_prologue(const darkattn_plan_s *plan, const void *K, const void *M, const void *W, char *ws,
-                            cudaStream_t st)
+                            const Stash &out, cudaStream_t st)
 {
     const Dims &D = plan->dims;
     const TensorLayout &Y = plan->tensor;
     const size_t BH = D.BH, N = D.N;
-    auto bf = [&](size_t off) { return reinterpret_cast<__nv_bfloat16 *>(ws + off); };
-    auto fl = [&](size_t off) { return reinterpret_cast<float *>(ws + off); };
     NormParams NP;
     memset(&NP, 0, sizeof(NP));
     if (!make_map(&NP.mapK, K, BH * N, D.d, 128) || !make_map(&NP.mapM, M, (size_t)D.H * D.r, D.d, 128))
@@ -878,14 +905,14 @@ cudaError_t tensor_prologue(const darkattn_plan_s *plan, const void *K, const vo
     auto chk = [&]() { cudaError_t x = cudaGetLastError(); if (x != cudaSuccess && e == cudaSuccess) e = x; };
 
     timer_mark(plan, st, "fold_omega_kernel");
-    fold_omega_kernel<<<dim3(D.m, D.H), 128, 0, st>>>((const __nv_bfloat16 *)W, (const __nv_bfloat16 *)M, bf(Y.Om), D.m, D.r, D.d,
+    fold_omega_kernel<<<dim3(D.m, D.H), 128, 0, st>>>((const __nv_bfloat16 *)W, (const __nv_bfloat16 *)M, out.Om, D.m, D.r, D.d,
                                                       D.w_per_head, kLog2e * D.s);
     chk();
     timer_mark(plan, st, "slab_shift_kernel");
-    slab_shift_kernel<<<(unsigned)(BH * Y.nslab), 128, 0, st>>>((const __nv_bfloat16 *)W, fl(Y.cs), D.H, D.m, D.r, Y.nslab, D.w_per_head);
+    slab_shift_kernel<<<(unsigned)(BH * Y.nslab), 128, 0, st>>>((const __nv_bfloat16 *)W, out.cs, D.H, D.m, D.r, Y.nslab, D.w_per_head);
     chk();
 
-    NP.nK = fl(Y.nK); NP.status = reinterpret_cast<int *>(ws + Y.status);
+    NP.nK = out.nK; NP.status = reinterpret_cast<int *>(ws + Y.status);
     NP.N = D.N; NP.H = D.H; NP.T = Y.T; NP.r = D.r;
     NP.nsplit = (int)((148 * 2 + BH - 1) / BH);
     if (NP.nsplit > Y.T) NP.nsplit = Y.T;
@@ -913,18 +940,19 @@ darkattn_status_t tensor_forward(const darkattn_plan_s *plan, const void *Q, con
     auto fl = [&](size_t off) { return reinterpret_cast<float *>(ws + off); };
     if (!encode_fn()) { set_cuda_error(cudaErrorNotSupported, "tensor_forward: cuTensorMapEncodeTiled unavailable"); return DARKATTN_ERR_CUDA; }
 
+    const Stash stash = saved ? stash_in_saved(Y, saved) : stash_in_workspace(Y, ws);
     MainParams P;
     memset(&P, 0, sizeof(P));
     bool ok = make_map(&P.mapQ, Q, BH * N, D.d, 128) && make_map(&P.mapK, K, BH * N, D.d, 128) &&
-              make_map(&P.mapV, V, BH * N, D.dv, 128) && make_map(&P.mapOm, bf(Y.Om), (size_t)D.H * D.m, D.d, 128) &&
+              make_map(&P.mapV, V, BH * N, D.dv, 128) && make_map(&P.mapOm, stash.Om, (size_t)D.H * D.m, D.d, 128) &&
               make_map(&P.mapSb, bf(Y.Sb), BH * D.m, D.dv, 128) &&
               make_map(&P.mapPN, bf(Y.pnum), (size_t)Y.nslab * BH * N, D.dv, 128);
     if (!ok) { set_cuda_error(cudaErrorInvalidValue, "tensor_forward: tensor map encode"); return DARKATTN_ERR_CUDA; }
 
-    cudaError_t e = tensor_prologue(plan, K, M, W, ws, st);
+    cudaError_t e = tensor_prologue(plan, K, M, W, ws, stash, st);
     auto chk = [&]() { cudaError_t x = cudaGetLastError(); if (x != cudaSuccess && e == cudaSuccess) e = x; };
 
-    P.nK = fl(Y.nK); P.cs = fl(Y.cs); P.pdr = fl(Y.pdr); P.Sacc = fl(Y.Sacc); P.zacc = fl(Y.zacc);
+    P.nK = stash.nK; P.cs = stash.cs; P.pdr = fl(Y.pdr); P.Sacc = fl(Y.Sacc); P.zacc = fl(Y.zacc);
     P.status = reinterpret_cast<int *>(ws + Y.status);
     P.N = D.N; P.H = D.H; P.BH = D.BH; P.m = D.m; P.nslab = Y.nslab; P.T = Y.T; P.nsplit = Y.nsplit;
     const int units = (int)(BH * Y.nslab);
@@ -949,9 +977,12 @@ darkattn_status_t tensor_forward(const darkattn_plan_s *plan, const void *Q, con
     {
         const long long rows = (long long)BH * N, threads = rows * (D.dv / 8);
         timer_mark(plan, st, "combine_kernel");
-        combine_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(bf(Y.pnum), fl(Y.pdr), (__nv_bfloat16 *)O,
-                                                                          reinterpret_cast<float2 *>(ws + Y.sv),
-                                                                          reinterpret_cast<float2 *>(saved), rows, D.dv, Y.nslab);
+        const unsigned grid = (unsigned)((threads + 255) / 256);
+        __nv_bfloat16 *Ob = (__nv_bfloat16 *)O;
+        if (Y.nslab == 1) combine_kernel<1><<<grid, 256, 0, st>>>(bf(Y.pnum), fl(Y.pdr), Ob, stash.sv, rows, D.dv, 1);
+        else if (Y.nslab == 2) combine_kernel<2><<<grid, 256, 0, st>>>(bf(Y.pnum), fl(Y.pdr), Ob, stash.sv, rows, D.dv, 2);
+        else if (Y.nslab == 4) combine_kernel<4><<<grid, 256, 0, st>>>(bf(Y.pnum), fl(Y.pdr), Ob, stash.sv, rows, D.dv, 4);
+        else combine_kernel<0><<<grid, 256, 0, st>>>(bf(Y.pnum), fl(Y.pdr), Ob, stash.sv, rows, D.dv, Y.nslab);
         chk();
     }
     if (e != cudaSuccess) { set_cuda_error(e, "tensor_forward"); return DARKATTN_ERR_CUDA; }
