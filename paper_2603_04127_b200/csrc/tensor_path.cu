@@ -29,18 +29,33 @@ constexpr int kMaxNsplit = 64;
 // ------------------------------------------------------------------ small helpers
 
 // ------------------------------------------------------------------ prologue kernels (SIMT, tiny)
-// Omega[h,l,c] = log2(e) * s * sum_a W[l,a] M[h,a,c]  (bf16);  one block per (h, l).
+// Omega[h,l,c] = log2(e) * s * sum_a W[l,a] M[h,a,c]  (bf16). One block per (head, 16 rows l); thread = column c
+// (d <= 128 threads... the block has d threads). The 16 rows of W sit in shared memory as floats.
 __global__ void fold_omega_kernel(const __nv_bfloat16 *W, const __nv_bfloat16 *M, __nv_bfloat16 *Om, int m, int r, int d,
                                   int w_per_head, float coef)
 {
-    const int h = blockIdx.y, l = blockIdx.x;
-    const __nv_bfloat16 *w = W + ((size_t)(w_per_head ? h : 0) * m + l) * r;
+    __shared__ float sw[16][129];
+    const int h = blockIdx.y, l0 = blockIdx.x * 16, c = threadIdx.x;
+    const __nv_bfloat16 *w = W + ((size_t)(w_per_head ? h : 0) * m + l0) * r;
+    for (int i = threadIdx.x; i < 16 * r; i += blockDim.x) sw[i / r][i % r] = __bfloat162float(w[i]);
+    __syncthreads();
     const __nv_bfloat16 *Mh = M + (size_t)h * r * d;
-    for (int c = threadIdx.x; c < d; c += blockDim.x) {
-        float acc = 0.f;
-        for (int a = 0; a < r; ++a) acc = fmaf(__bfloat162float(w[a]), __bfloat162float(Mh[(size_t)a * d + c]), acc);
-        Om[((size_t)h * m + l) * d + c] = __float2bfloat16_rn(coef * acc);
+    float acc[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) acc[i] = 0.f;
+    for (int a0 = 0; a0 < r; a0 += 16) {            // r is a multiple of 16; 16 independent loads in flight
+        __nv_bfloat16 mv[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) mv[j] = Mh[(size_t)(a0 + j) * d + c];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const float x = __bfloat162float(mv[j]);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) acc[i] = fmaf(sw[i][a0 + j], x, acc[i]);
+        }
     }
+#pragma unroll
+    for (int i = 0; i < 16; ++i) Om[((size_t)h * m + l0 + i) * d + c] = __float2bfloat16_rn(coef * acc[i]);
 }
 
 // Key-side shift of a slab, in log2 units: c = log2(e) * max(0, max_l |w_l|^2/2 - 40).
@@ -905,7 +920,7 @@ cudaError_t tensor_prologue(const darkattn_plan_s *plan, const void *K, const vo
     auto chk = [&]() { cudaError_t x = cudaGetLastError(); if (x != cudaSuccess && e == cudaSuccess) e = x; };
 
     timer_mark(plan, st, "fold_omega_kernel");
-    fold_omega_kernel<<<dim3(D.m, D.H), 128, 0, st>>>((const __nv_bfloat16 *)W, (const __nv_bfloat16 *)M, out.Om, D.m, D.r, D.d,
+    fold_omega_kernel<<<dim3(D.m / 16, D.H), D.d, 0, st>>>((const __nv_bfloat16 *)W, (const __nv_bfloat16 *)M, out.Om, D.m, D.r, D.d,
                                                       D.w_per_head, kLog2e * D.s);
     chk();
     timer_mark(plan, st, "slab_shift_kernel");
