@@ -65,8 +65,6 @@ struct TensorLayout {
     size_t Oscr;    // forward output when backward has to recompute it, bf16 [BH, N, dv]
     size_t delta;   // dO_i . O_i, fp32 [BH, N]
     size_t rhoc;    // per-chunk sums -sum_i A^_il delta_i, fp32 [BH, T, m]
-    size_t pdQ, pdK; // slab partials of dQ and dK, bf16 [nslab, BH, N, d]
-    size_t pdV;     // slab partials of dV, bf16 [nslab, BH, N, dv]
     size_t espart;  // partials of rowsum(E_K) per slab and 32-column group, fp32 [4 nslab, BH, N]
     size_t Tacc;    // sum_i E_i^T x_i over both sides and the batch, fp32 [H, m, d]
     size_t dMn;     // gradient of M through the key norm term, fp32 [H, r, d]

@@ -92,6 +92,14 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, const void 
                  ::"l"(map), "r"(smem_u32(smem_src)), "r"(x), "r"(y)
                  : "memory");
 }
+// Element-wise add of a shared-memory tile into global memory (the additions are done in the tensor's type, bf16
+// here, by the memory system): several CTAs may add into the same tile.
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap *map, const void *smem_src, int x, int y)
+{
+    asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(map), "r"(smem_u32(smem_src)), "r"(x), "r"(y)
+                 : "memory");
+}
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
@@ -298,12 +306,16 @@ __device__ __forceinline__ void features_to_tile(uint32_t taddr, float offset, u
         *reinterpret_cast<uint4 *>(tile_chunk(tile, row, col0 / 8 + q)) = make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
 }
 
-// 32 fp32 TMEM columns at taddr -> bf16 tile row (swizzled smem), columns [col0, col0 + 32)
-__device__ __forceinline__ void tmem_row_to_tile(uint32_t taddr, unsigned char *tile, int row, int col0)
+// 32 fp32 TMEM columns at taddr, times scale -> bf16 tile row (swizzled smem), columns [col0, col0 + 32)
+__device__ __forceinline__ void tmem_row_to_tile(uint32_t taddr, unsigned char *tile, int row, int col0, float scale = 1.f)
 {
     uint32_t v[32];
     tmem_ld32(taddr, v);
     tmem_wait_ld();
+    if (scale != 1.f) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(scale * __uint_as_float(v[j]));
+    }
 #pragma unroll
     for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4 *>(tile_chunk(tile, row, col0 / 8 + q)) = pack8(v + 8 * q);
 }

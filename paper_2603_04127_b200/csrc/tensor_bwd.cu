@@ -35,13 +35,12 @@ namespace {
 constexpr float kLn2 = 0.6931471805599453f;
 
 struct BwdParams {
-    CUtensorMap mapQ, mapK, mapV, mapG, mapOm, mapPQ, mapPK, mapPV;   // the last three: slab partials, for the stores
+    CUtensorMap mapQ, mapK, mapV, mapG, mapOm, mapDQ, mapDK, mapDV;   // the last three: the gradients, for the (adding) stores
     const float2 *sv;     // [BH*N]  (normaliser, exponent it is scaled by) from the forward pass
     const float *delta;   // [BH*N]  dO_i . O_i
     const float *nK;      // [BH*N]  key norms, log2 units
     const float *cs;      // [BH*nslab] key-side shift per slab
     float *rhoc;          // [BH, T, m] per-chunk -sum_i A^_il delta_i (written by the query-side kernel)
-    __nv_bfloat16 *pdQ, *pdK, *pdV;   // slab partials
     float *espart;        // [4 nslab, BH*N] partials of rowsum(E^K): one per slab and 32-column group
     float *Tacc;          // [H, m, D]
     int *status;
@@ -301,12 +300,14 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
 
             EWAIT(QM5); if (!ok) break;
             tc_fence_after();
-            if (col0 < D) tmem_row_to_tile(R1 + col0, sStg, r, col0);       // slab partial of dQ -> staging -> TMA store
+            if (col0 < D) tmem_row_to_tile(R1 + col0, sStg, r, col0, kLn2);  // this slab's part of dQ -> staging -> added into dQ
             fence_async_smem();
             epi_sync();
             if (tid == 0) {
-                for (int a = 0; a < D / 64; ++a)
-                    tma_store_2d(&p.mapPQ, sStg + a * 16384, a * 64, (int)(((size_t)slab * p.BH + bh) * p.N + (size_t)t * 128));
+                for (int a = 0; a < D / 64; ++a) {
+                    if (p.nslab > 1) tma_reduce_add_2d(&p.mapDQ, sStg + a * 16384, a * 64, row0 + t * 128);
+                    else tma_store_2d(&p.mapDQ, sStg + a * 16384, a * 64, row0 + t * 128);
+                }
                 tma_store_commit();
             }
             EWAIT(QMS); if (!ok) break;
@@ -477,7 +478,6 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
             const uint32_t ph = it & 1;
             const bool last = (it + 1 == T);
             const size_t row = (size_t)row0 + (size_t)t * 128 + r;
-            const size_t prow = ((size_t)slab * p.BH + bh) * p.N + (size_t)t * 128 + r;
 #define EWAIT(b) do { ok = __all_sync(0xffffffffu, wait_or_abort(bars + (b), ph, status, abort_flag)); } while (0)
             const float2 svv = p.sv[row];
             const float nk = p.nK[row] + cshift;
@@ -536,13 +536,16 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
 
             EWAIT(KM6); if (!ok) break;
             tc_fence_after();
-            if (col0 < DV) tmem_row_to_tile(R2 + col0, sStg, r, col0);      // slab partial of dV -> staging -> TMA store
+            if (col0 < DV) tmem_row_to_tile(R2 + col0, sStg, r, col0);      // this slab's part of dV -> staging -> added into dV
             fence_async_smem();
             tc_fence_before();
             mbar_arrive_warp(bars + KE3);
             epi_sync();
             if (tid == 0) {
-                for (int a = 0; a < DV / 64; ++a) tma_store_2d(&p.mapPV, sStg + a * 16384, a * 64, (int)(prow - r));
+                for (int a = 0; a < DV / 64; ++a) {
+                    if (p.nslab > 1) tma_reduce_add_2d(&p.mapDV, sStg + a * 16384, a * 64, row0 + t * 128);
+                    else tma_store_2d(&p.mapDV, sStg + a * 16384, a * 64, row0 + t * 128);
+                }
                 tma_store_commit();
             }
 
@@ -575,11 +578,14 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
 
             EWAIT(KM8); if (!ok) break;
             tc_fence_after();
-            if (col0 < D) tmem_row_to_tile(R2 + col0, sStg, r, col0);       // slab partial of dK -> staging -> TMA store
+            if (col0 < D) tmem_row_to_tile(R2 + col0, sStg, r, col0, kLn2); // this slab's part of dK (without the norm term) -> added into dK
             fence_async_smem();
             epi_sync();
             if (tid == 0) {
-                for (int a = 0; a < D / 64; ++a) tma_store_2d(&p.mapPK, sStg + a * 16384, a * 64, (int)(prow - r));
+                for (int a = 0; a < D / 64; ++a) {
+                    if (p.nslab > 1) tma_reduce_add_2d(&p.mapDK, sStg + a * 16384, a * 64, row0 + t * 128);
+                    else tma_store_2d(&p.mapDK, sStg + a * 16384, a * 64, row0 + t * 128);
+                }
                 tma_store_commit();
             }
             if (!last) {     // R (its update completed before KM6) -> bf16 copy; rho_next for the chunk below
@@ -613,9 +619,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
 // ------------------------------------------------------------------ dK: slab sum + norm term (three MMAs per tile)
 //   x~'  = K M^T                      (128 x r)
 //   w_j  = -s^2 rowsum(E^K)_j x~'_j   (bf16 operand)
-//   dK_j = ln2 sum_slabs part_j + w_j M          dMn += w^T K
+//   dK_j = (dK_j as the scan kernel left it) + w_j M          dMn += w^T K
 struct FinishParams {
-    CUtensorMap mapK, mapM, mapP, mapOut;   // K, M, the slab partials of dK [nslab BH N, D], dK
+    CUtensorMap mapK, mapM, mapP, mapOut;   // K, M, dK without the norm term (nslab tensors stacked; here one: dK itself), dK
     const float *espart;  // [nes, BH*N]
     float *dMn;           // [H, r, D]
     int *status;
@@ -768,7 +774,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __gr
                 tmem_ld32(lane_addr + C2 + col0, v);
                 tmem_wait_ld();
 #pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(fmaf(kLn2, acc[j], __uint_as_float(v[j])));
+                for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(acc[j] + __uint_as_float(v[j]));
 #pragma unroll
                 for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4 *>(tile_chunk(sOut, r, col0 / 8 + q)) = pack8(v + 8 * q);
             }
@@ -816,25 +822,6 @@ __global__ void delta_kernel(const __nv_bfloat16 *G, const __nv_bfloat16 *O, flo
     }
     for (int o = per_row / 2; o; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
     if (row < rows && (i % per_row) == 0) delta[row] = acc;
-}
-
-// out[row, c] = scale * sum_s part[s, row, c]; one thread per 8 columns.
-__global__ void sum_slabs_kernel(const __nv_bfloat16 *part, __nv_bfloat16 *out, long long rows, int width, int nslab, float scale)
-{
-    const long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;
-    const int per_row = width / 8;
-    if (i >= rows * per_row) return;
-    float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    for (int s = 0; s < nslab; ++s) {
-        float f[8];
-        unpack8(*reinterpret_cast<const uint4 *>(part + ((size_t)s * rows * per_row + i) * 8), f);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) acc[j] += f[j];
-    }
-    uint32_t o[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) o[j] = __float_as_uint(scale * acc[j]);
-    *reinterpret_cast<uint4 *>(out + i * 8) = pack8(o);
 }
 
 // dM[h,a,c] = s * sum_l W[l,a] T[h,l,c] + dMn[h,a,c]. One block per (8 rows a, head), one thread per column c;
@@ -940,22 +927,26 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
     chk();
     keep(cudaMemsetAsync(ws + Y.Tacc, 0, (size_t)D.H * D.m * D.d * 4, st));
     keep(cudaMemsetAsync(ws + Y.dMn, 0, (size_t)D.H * D.r * D.d * 4, st));
+    if (Y.nslab > 1) {      // the slabs of a head add their parts into the gradients
+        keep(cudaMemsetAsync(dQ, 0, BH * N * D.d * 2, st));
+        keep(cudaMemsetAsync(dK, 0, BH * N * D.d * 2, st));
+        keep(cudaMemsetAsync(dV, 0, BH * N * D.dv * 2, st));
+    }
 
     BwdParams P;
     memset(&P, 0, sizeof(P));
     bool ok = make_map(&P.mapQ, Q, BH * N, D.d, 128) && make_map(&P.mapK, K, BH * N, D.d, 128) &&
               make_map(&P.mapV, V, BH * N, D.dv, 128) && make_map(&P.mapG, dO, BH * N, D.dv, 128) &&
               make_map(&P.mapOm, stash.Om, (size_t)D.H * D.m, D.d, 128) &&
-              make_map(&P.mapPQ, bf(Y.pdQ), (size_t)Y.nslab * BH * N, D.d, 128) &&
-              make_map(&P.mapPK, bf(Y.pdK), (size_t)Y.nslab * BH * N, D.d, 128) &&
-              make_map(&P.mapPV, bf(Y.pdV), (size_t)Y.nslab * BH * N, D.dv, 128);
+              make_map(&P.mapDQ, dQ, BH * N, D.d, 128) && make_map(&P.mapDK, dK, BH * N, D.d, 128) &&
+              make_map(&P.mapDV, dV, BH * N, D.dv, 128);
     FinishParams F;
     memset(&F, 0, sizeof(F));
     ok = ok && make_map(&F.mapM, M, (size_t)D.H * D.r, D.d, 128);
     if (!ok) { set_cuda_error(cudaErrorInvalidValue, "tensor_backward: tensor map encode"); return DARKATTN_ERR_CUDA; }
     F.mapK = P.mapK;
     P.sv = stash.sv; P.delta = fl(Y.delta); P.nK = stash.nK; P.cs = stash.cs; P.rhoc = fl(Y.rhoc);
-    P.pdQ = bf(Y.pdQ); P.pdK = bf(Y.pdK); P.pdV = bf(Y.pdV); P.espart = fl(Y.espart); P.Tacc = fl(Y.Tacc);
+    P.espart = fl(Y.espart); P.Tacc = fl(Y.Tacc);
     P.status = reinterpret_cast<int *>(ws + Y.status);
     P.N = D.N; P.H = D.H; P.BH = D.BH; P.m = D.m; P.nslab = Y.nslab; P.T = Y.T;
     const int units = (int)(BH * Y.nslab);
@@ -964,20 +955,11 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
     else if (D.d == 64 && D.dv == 128) keep(launch_scan<64, 128>(plan, P, units, st));
     else keep(launch_scan<128, 64>(plan, P, units, st));
 
-    {
-        const long long tq = rows * (D.d / 8), tv = rows * (D.dv / 8);
-        timer_mark(plan, st, "sum_slabs_kernel");
-        sum_slabs_kernel<<<(unsigned)((tq + 255) / 256), 256, 0, st>>>(bf(Y.pdQ), (__nv_bfloat16 *)dQ, rows, D.d, Y.nslab, kLn2);
-        chk();
-        timer_mark(plan, st, "sum_slabs_kernel");
-        sum_slabs_kernel<<<(unsigned)((tv + 255) / 256), 256, 0, st>>>(bf(Y.pdV), (__nv_bfloat16 *)dV, rows, D.dv, Y.nslab, 1.f);
-        chk();
-    }
-    F.mapP = P.mapPK;
+    F.mapP = P.mapDK;
     if (!make_map(&F.mapOut, dK, BH * N, D.d, 128)) { set_cuda_error(cudaErrorInvalidValue, "tensor_backward: tensor map encode"); return DARKATTN_ERR_CUDA; }
     F.espart = fl(Y.espart); F.dMn = fl(Y.dMn);
     F.status = P.status;
-    F.N = D.N; F.H = D.H; F.BH = D.BH; F.T = Y.T; F.r = D.r; F.nslab = Y.nslab; F.nes = 4 * Y.nslab; F.s2 = D.s * D.s;
+    F.N = D.N; F.H = D.H; F.BH = D.BH; F.T = Y.T; F.r = D.r; F.nslab = 1; F.nes = 4 * Y.nslab; F.s2 = D.s * D.s;
     F.nsplit = (int)((148 * 2 + BH - 1) / BH);
     if (F.nsplit > Y.T) F.nsplit = Y.T;
     timer_mark(plan, st, "tc_bwd_finish_k_kernel");

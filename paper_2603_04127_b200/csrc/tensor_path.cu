@@ -894,13 +894,10 @@ void tensor_make_layout(darkattn_plan_s *plan)
         Y.Oscr = take(off, BH * N * dv * 2);
         Y.delta = take(off, BH * N * 4);
         Y.rhoc = take(off, BH * (size_t)Y.T * m * 4);
-        Y.pdQ = take(off, (size_t)Y.nslab * BH * N * d * 2);
-        Y.pdK = take(off, (size_t)Y.nslab * BH * N * d * 2);
-        Y.pdV = take(off, (size_t)Y.nslab * BH * N * dv * 2);
         Y.espart = take(off, (size_t)4 * Y.nslab * BH * N * 4);
         Y.Tacc = take(off, (size_t)D.H * m * d * 4);
         Y.dMn = take(off, (size_t)D.H * D.r * d * 4);
-        plan->launches_bwd = 3 + 1 + 2 + 3 + 1;   // prologue, delta, two scan kernels, three combines, dM
+        plan->launches_bwd = 1 + 2 + 1 + 1;   // delta, two scan kernels, dK finishing, dM (with `saved`; without it the forward launches come on top)
     }
     Y.total_bytes = off;
     if (Y.total_bytes > plan->workspace_bytes) plan->workspace_bytes = Y.total_bytes;
