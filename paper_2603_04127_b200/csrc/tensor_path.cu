@@ -167,6 +167,10 @@ struct MainParams {
     float *pdr;          // [nslab, BH*N, 2]  partial normaliser and the exponent the partial is scaled by
     float *Sacc;         // [BH, m, DV]  fp32 state sums (non-causal key pass, atomics)
     float *zacc;         // [BH, m]
+    // causal scan cut into nsplit segments of the sequence: the key pass stores one state per segment
+    // (Sseg [BH, nsplit, m, DV], zseg [BH, nsplit, m]) instead of adding into Sacc; after an exclusive prefix over the
+    // segments the causal kernel of segment s > 0 starts from Sseg[bh, s] (its bf16 copy comes through mapSb).
+    float *Sseg, *zseg;
     int *status;
     int N, H, BH, m, nslab, T, nsplit;
 };
@@ -250,8 +254,11 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + CNBARS + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5;
-    const int bh = blockIdx.x / p.nslab, slab = blockIdx.x % p.nslab, h = bh % p.H;
-    const int row0 = bh * p.N, T = p.T;
+    const int unit = blockIdx.x / p.nsplit, seg = blockIdx.x % p.nsplit;
+    const int bh = unit / p.nslab, slab = unit % p.nslab, h = bh % p.H;
+    const int row0 = bh * p.N;
+    const int tbeg = (int)((long long)p.T * seg / p.nsplit), tend = (int)((long long)p.T * (seg + 1) / p.nsplit);
+    const bool fresh = (seg == 0);                 // the scan state starts at zero (else at the segment's prefix state)
 
     if (tid == 0) {
         for (int i = 0; i < CE0; ++i) mbar_init(bars + i, 1);
@@ -259,16 +266,43 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
         *abort_flag = (smem_u32(smem) & 1023u) ? 1 : 0;
         fence_mbar_init();
     }
-    if (tid < 128) sZ[tid] = 0.f;
+    if (tid < 128) sZ[tid] = fresh ? 0.f : p.zseg[((size_t)bh * p.nsplit + seg) * p.m + slab * 128 + tid];
     if (warp == kEpiWarps) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
     int *status = p.status;
+    if (!fresh && warp < kEpiWarps) {      // the segment's prefix state into the fp32 accumulators in TMEM
+        const int lane = tid & 31, q4 = warp & 3, col0 = (warp >> 2) * 32, r = q4 * 32 + lane;
+        const uint32_t lane_addr = tmem + ((uint32_t)(q4 * 32) << 16);
+        const size_t srow = ((size_t)bh * p.nsplit + seg) * p.m + slab * 128 + r;
+        if (col0 < DV) {
+            uint32_t v[32];
+            const float4 *src = reinterpret_cast<const float4 *>(p.Sseg + srow * DV + col0);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const float4 x = src[j];
+                v[4 * j] = __float_as_uint(x.x); v[4 * j + 1] = __float_as_uint(x.y);
+                v[4 * j + 2] = __float_as_uint(x.z); v[4 * j + 3] = __float_as_uint(x.w);
+            }
+            tmem_st32(lane_addr + kColS + col0, v);
+        }
+        if (col0 == 0) {
+            uint32_t v[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(sZ[r]);
+            tmem_st16(lane_addr + kColZ, v);
+        }
+        tmem_wait_st();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
 
     if (*abort_flag) {
         if (tid == 0) atomicExch(status, (int)DARKATTN_ERR_CUDA);
+    } else if (tend <= tbeg) {
     } else if (warp == kEpiWarps) {
         if ((tid & 31) == 0) {
             auto load_tile = [&](unsigned char *dst, const CUtensorMap *map, uint64_t *bar, int width, int t) {
@@ -283,11 +317,14 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
             const uint32_t id_z = make_idesc(128, 16, 1, 1);
             const uint32_t R1 = tmem + kColR1, R2 = tmem + kColR2, FQ = tmem + kColFQ;
 
-            mbar_expect_tx(bars + CB_OM, 128 * D * 2);
+            mbar_expect_tx(bars + CB_OM, 128 * D * 2 + (fresh ? 0 : 128 * DV * 2));
             for (int a = 0; a < D / 64; ++a) tma_load_2d(sOm + a * 16384, &p.mapOm, bars + CB_OM, a * 64, h * p.m + slab * 128);
-            load_tile(sQ, &p.mapQ, bars + CB_Q, D, 0);
-            load_tile(sK, &p.mapK, bars + CB_K, D, 0);
-            load_tile(sV, &p.mapV, bars + CB_V, DV, 0);
+            if (!fresh)     // bf16 copy of the segment's prefix state
+                for (int a = 0; a < DV / 64; ++a)
+                    tma_load_2d(sSb + a * 16384, &p.mapSb, bars + CB_OM, a * 64, (bh * p.nsplit + seg) * p.m + slab * 128);
+            load_tile(sQ, &p.mapQ, bars + CB_Q, D, tbeg);
+            load_tile(sK, &p.mapK, bars + CB_K, D, tbeg);
+            load_tile(sV, &p.mapV, bars + CB_V, DV, tbeg);
 
             bool ok = wait_or_abort(bars + CB_OM, 0, status, abort_flag);
             if (ok) ok = wait_or_abort(bars + CB_Q, 0, status, abort_flag);
@@ -296,9 +333,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
                 _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R1, kdesc(tQ, k), kdesc(tOm, k), id_kk, k > 0);         // U_Q of chunk 0
                 mma_commit(bars + CM1);
             }
-            for (int t = 0; t < T && ok; ++t) {
-                const uint32_t ph = t & 1;
-                const bool first = (t == 0), last = (t + 1 == T);
+            for (int t = tbeg; t < tend && ok; ++t) {
+                const uint32_t ph = (t - tbeg) & 1;
+                const bool first = (t == tbeg) && fresh, last = (t + 1 == tend);
 #define CWAIT(b) do { ok = wait_or_abort(bars + (b), ph, status, abort_flag); } while (0)
                 CWAIT(CB_K); if (!ok) break;
                 tc_fence_after();
@@ -344,9 +381,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
         const float cshift = p.cs[bh * p.nslab + slab];
         const size_t prow0 = ((size_t)slab * p.BH + bh) * p.N;
         bool ok = true;
-        for (int t = 0; t < T && ok; ++t) {
-            const uint32_t ph = t & 1;
-            const bool last = (t + 1 == T);
+        for (int t = tbeg; t < tend && ok; ++t) {
+            const uint32_t ph = (t - tbeg) & 1;
+            const bool last = (t + 1 == tend);
 #define EWAIT(b) do { ok = __all_sync(0xffffffffu, wait_or_abort(bars + (b), ph, status, abort_flag)); } while (0)
             const float nk = p.nK[(size_t)row0 + (size_t)t * 128 + r] + cshift;
             float rmax;
@@ -395,6 +432,14 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
                 store_row_f32x32_bf16(v, sStg, r, col0);
             }
             sRed[g * 128 + r] = rowsum + dz;
+            // z through this chunk for the next chunk's normaliser (its update completed before the output MMAs did).
+            // Written ahead of the barrier below: a warp that runs ahead into the next chunk reads it right away.
+            if (g == 0 && !last) {
+                uint32_t v[16];
+                tmem_ld16(lane_addr + kColZ, v);
+                tmem_wait_ld();
+                sZ[r] = __uint_as_float(v[0]);
+            }
             fence_async_smem();
             tc_fence_before();
             mbar_arrive_warp(bars + CE3);
@@ -413,12 +458,6 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
             tc_fence_after();
             if (!last) {
                 if (col0 < DV) tmem_row_to_tile(lane_addr + kColS + col0, sSb, r, col0);
-                if (g == 0) {
-                    uint32_t v[16];
-                    tmem_ld16(lane_addr + kColZ, v);
-                    tmem_wait_ld();
-                    sZ[r] = __uint_as_float(v[0]);
-                }
                 fence_async_smem();
             }
             if (tid == 0) tma_store_wait_read();   // staging (and the ones in it) may be rewritten after CE4
@@ -559,21 +598,30 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_keys_kernel(const __grid_c
             mbar_arrive_warp(bars + YE1_0 + b);
         }
         if (ok) ok = __all_sync(0xffffffffu, wait_or_abort(bars + YMS_0 + ((n - 1) & 1), ((n - 1) >> 1) & 1, status, abort_flag));
-        if (ok) {        // add this CTA's state to the global sums
+        if (ok) {        // add this CTA's state to the global sums, or store it as its segment's state
             tc_fence_after();
+            const size_t srow = ((size_t)bh * p.nsplit + split) * p.m + slab * 128 + r;
             if (col0 < DV) {
-                float *dst = p.Sacc + ((size_t)bh * p.m + slab * 128 + r) * DV + col0;
                 uint32_t v[32];
                 tmem_ld32(lane_addr + kColS + col0, v);
                 tmem_wait_ld();
+                if (p.Sseg) {
+                    float4 *dst = reinterpret_cast<float4 *>(p.Sseg + srow * DV + col0);
 #pragma unroll
-                for (int j = 0; j < 32; ++j) atomicAdd(dst + j, __uint_as_float(v[j]));
+                    for (int j = 0; j < 8; ++j)
+                        dst[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]), __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+                } else {
+                    float *dst = p.Sacc + ((size_t)bh * p.m + slab * 128 + r) * DV + col0;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) atomicAdd(dst + j, __uint_as_float(v[j]));
+                }
             }
             if (g == 0) {
                 uint32_t v[16];
                 tmem_ld16(lane_addr + kColZ, v);
                 tmem_wait_ld();
-                atomicAdd(p.zacc + (size_t)bh * p.m + slab * 128 + r, __uint_as_float(v[0]));
+                if (p.Sseg) p.zseg[srow] = __uint_as_float(v[0]);
+                else atomicAdd(p.zacc + (size_t)bh * p.m + slab * 128 + r, __uint_as_float(v[0]));
             }
         }
     }
@@ -736,6 +784,32 @@ __global__ void state_to_bf16_kernel(const float *S, __nv_bfloat16 *Sb, long lon
         Sb[i] = __float2bfloat16_rn(S[i]);
 }
 
+// In-place exclusive prefix over the segments of S[bh, seg, e] (e over m*dv) and z[bh, seg, l]; Sb receives the bf16
+// copy of the prefixed S. One thread per (bh, e).
+__global__ void segment_prefix_kernel(float *S, __nv_bfloat16 *Sb, float *z, int nseg, long long E, int m, long long total)
+{
+    const long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+    if (i >= total) return;
+    const long long bh = i / E, e = i % E;
+    float run = 0.f;
+    for (int s = 0; s < nseg; ++s) {
+        const long long at = (bh * nseg + s) * E + e;
+        const float v = S[at];
+        S[at] = run;
+        Sb[at] = __float2bfloat16_rn(run);
+        run += v;
+    }
+    if (e < m) {
+        float zr = 0.f;
+        for (int s = 0; s < nseg; ++s) {
+            const long long at = (bh * nseg + s) * m + e;
+            const float v = z[at];
+            z[at] = zr;
+            zr += v;
+        }
+    }
+}
+
 // O[row,:] = sum_s num_s[row,:] 2^(rho_s - rho) / sum_s den_s 2^(rho_s - rho), rho = max_s rho_s.
 // One thread per 8 output columns. The combined normaliser and rho are also written to sv for the backward pass.
 // NS > 0: the number of slabs at compile time (all loads of a thread are issued before the first use).
@@ -861,14 +935,22 @@ void tensor_make_layout(darkattn_plan_s *plan)
     Y.nslab = D.m / 128;
     Y.T = D.N / 128;
     int nsplit = 1;
+    const long long units = (long long)BH * Y.nslab;
     if (!D.causal) {
-        const long long units = (long long)BH * Y.nslab;
         nsplit = (int)((148ll * 4 + units - 1) / units);
         if (nsplit > Y.T) nsplit = Y.T;
         if (nsplit > kMaxNsplit) nsplit = kMaxNsplit;
         if (nsplit < 1) nsplit = 1;
+    } else if (units * 2 <= 148) {
+        // few long sequences: cut each into segments (a key pass computes the segment states, the causal
+        // kernels of all segments then run side by side), as many as fill the SMs, at least 4 chunks each
+        nsplit = (int)(148 / units);
+        if (nsplit > Y.T / 4) nsplit = Y.T / 4;
+        if (nsplit > 16) nsplit = 16;
+        if (nsplit < 1) nsplit = 1;
     }
     Y.nsplit = nsplit;
+    const size_t nstate = D.causal ? (size_t)nsplit : 1;
     size_t off = 0;
     Y.status = take(off, 256);
     Y.Om = take(off, (size_t)D.H * m * d * 2);
@@ -876,11 +958,11 @@ void tensor_make_layout(darkattn_plan_s *plan)
     Y.nK = take(off, BH * N * 4);
     Y.pnum = take(off, (size_t)Y.nslab * BH * N * dv * 2);
     Y.pdr = take(off, (size_t)Y.nslab * BH * N * 8);
-    Y.Sacc = take(off, BH * m * dv * 4);
-    Y.zacc = take(off, BH * m * 4);
-    Y.Sb = take(off, BH * m * dv * 2);
+    Y.Sacc = take(off, BH * nstate * m * dv * 4);
+    Y.zacc = take(off, BH * nstate * m * 4);
+    Y.Sb = take(off, BH * nstate * m * dv * 2);
     Y.sv = take(off, BH * N * 8);
-    plan->launches_fwd = D.causal ? 5 : 7;
+    plan->launches_fwd = D.causal ? (nsplit > 1 ? 7 : 5) : 7;
     {
         size_t so = 0;
         Y.sv_sv = take(so, BH * N * 8);
@@ -957,7 +1039,7 @@ darkattn_status_t tensor_forward(const darkattn_plan_s *plan, const void *Q, con
     memset(&P, 0, sizeof(P));
     bool ok = make_map(&P.mapQ, Q, BH * N, D.d, 128) && make_map(&P.mapK, K, BH * N, D.d, 128) &&
               make_map(&P.mapV, V, BH * N, D.dv, 128) && make_map(&P.mapOm, stash.Om, (size_t)D.H * D.m, D.d, 128) &&
-              make_map(&P.mapSb, bf(Y.Sb), BH * D.m, D.dv, 128) &&
+              make_map(&P.mapSb, bf(Y.Sb), BH * (D.causal ? Y.nsplit : 1) * D.m, D.dv, 128) &&
               make_map(&P.mapPN, bf(Y.pnum), (size_t)Y.nslab * BH * N, D.dv, 128);
     if (!ok) { set_cuda_error(cudaErrorInvalidValue, "tensor_forward: tensor map encode"); return DARKATTN_ERR_CUDA; }
 
@@ -969,9 +1051,18 @@ darkattn_status_t tensor_forward(const darkattn_plan_s *plan, const void *Q, con
     P.N = D.N; P.H = D.H; P.BH = D.BH; P.m = D.m; P.nslab = Y.nslab; P.T = Y.T; P.nsplit = Y.nsplit;
     const int units = (int)(BH * Y.nslab);
     if (D.causal) {
-        P.nsplit = 1;
+        if (Y.nsplit > 1) {      // segment states, then their exclusive prefix
+            P.Sseg = fl(Y.Sacc); P.zseg = fl(Y.zacc);
+            timer_mark(plan, st, "tc_fwd_keys_kernel");
+            cudaError_t x = launch_main_shape<MODE_KEYS>(D.d, D.dv, P, units * Y.nsplit, st);
+            if (x != cudaSuccess && e == cudaSuccess) e = x;
+            const long long E = (long long)D.m * D.dv, total = (long long)BH * E;
+            timer_mark(plan, st, "segment_prefix_kernel");
+            segment_prefix_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(fl(Y.Sacc), bf(Y.Sb), fl(Y.zacc), Y.nsplit, E, D.m, total);
+            chk();
+        }
         timer_mark(plan, st, "tc_fwd_causal_kernel");
-        cudaError_t x = launch_main_shape<MODE_CAUSAL>(D.d, D.dv, P, units, st);
+        cudaError_t x = launch_main_shape<MODE_CAUSAL>(D.d, D.dv, P, units * Y.nsplit, st);
         if (x != cudaSuccess && e == cudaSuccess) e = x;
     } else {
         e = (e == cudaSuccess) ? cudaMemsetAsync(ws + Y.Sacc, 0, (Y.Sb - Y.Sacc), st) : e;   // S and z sums
