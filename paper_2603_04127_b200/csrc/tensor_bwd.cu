@@ -239,6 +239,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
             tc_fence_after();
             features_to_tile_sums(R2 + col0, nk, sKB, r, col0, 1.f, sZc, lane);       // Bf and z_c = sum_j Bf_jl
             fence_async_smem();
+            if (tid == 0) tma_store_wait_read();      // the previous chunk's store has left the staging tile (every later
+                                                      // writer of it first passes a barrier that needs this arrival)
             tc_fence_before();
             mbar_arrive_warp(bars + QE0);
             EWAIT(QM1); if (!ok) break;
@@ -317,7 +319,6 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                 if (own) sZ[col0 + lane] = zrun;
                 fence_async_smem();
             }
-            if (tid == 0) tma_store_wait_read();      // the staging tile is free again before anyone passes QE4
             tc_fence_before();
             mbar_arrive_warp(bars + QE4);
 #undef EWAIT
@@ -491,6 +492,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
             tc_fence_after();
             features_to_tile(R1 + col0, aq, sQA, r, col0);
             fence_async_smem();
+            if (tid == 0) tma_store_wait_read();      // the previous chunk's dK store has left the staging tile
             tc_fence_before();
             mbar_arrive_warp(bars + KE0);
             EWAIT(KM2); if (!ok) break;
@@ -593,7 +595,6 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
                 if (g0) sRho[r] += rho_c;
                 fence_async_smem();
             }
-            if (tid == 0) tma_store_wait_read();
             tc_fence_before();
             mbar_arrive_warp(bars + KE5);
 #undef EWAIT

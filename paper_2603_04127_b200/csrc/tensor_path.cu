@@ -396,8 +396,13 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
             EWAIT(CM2); if (!ok) break;
             tc_fence_after();
             features_to_tile(R2 + col0, nk, sFK, r, col0);
-            if (warp < 4)    // 2 KB of bf16 ones at the start of the staging tile: B operand of z += phi(K)^T 1
-                *reinterpret_cast<uint4 *>(sStg + tid * 16) = make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
+            if (warp == 0) {  // 2 KB of bf16 ones at the start of the staging tile: B operand of z += phi(K)^T 1
+                if (tid == 0) tma_store_wait_read();       // once the previous chunk's store has left the tile
+                __syncwarp();
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    *reinterpret_cast<uint4 *>(sStg + (i * 32 + tid) * 16) = make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
+            }
             fence_async_smem();
             tc_fence_before();
             mbar_arrive_warp(bars + CE1);
@@ -460,7 +465,6 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
                 if (col0 < DV) tmem_row_to_tile(lane_addr + kColS + col0, sSb, r, col0);
                 fence_async_smem();
             }
-            if (tid == 0) tma_store_wait_read();   // staging (and the ones in it) may be rewritten after CE4
             tc_fence_before();
             mbar_arrive_warp(bars + CE4);
 #undef EWAIT
