@@ -480,16 +480,20 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
 // ------------------------------------------------------------------ non-causal, key pass: S = phi(K)^T V, z = phi(K)^T 1
 template <int D, int DV>
 struct FwdKeysSmem {
+    // K and V tiles sit in rings of kStages buffers (4 where they are small enough), so that a tile's load is issued
+    // several tiles before its use; phi(K) tiles and TMEM regions alternate between two.
+    static constexpr int kStages = (3 * 128 * (D + DV) * 2 + 128 * D * 2 + 2 * 32768 + 4096 <= 232448) ? 4 : 2;
     static constexpr int kOm = 0;
-    static constexpr int kK = kOm + 128 * D * 2;           // two K tiles
-    static constexpr int kV = kK + 2 * 128 * D * 2;        // two V tiles
-    static constexpr int kFK = kV + 2 * 128 * DV * 2;      // two phi(K) tiles
+    static constexpr int kK = kOm + 128 * D * 2;
+    static constexpr int kV = kK + kStages * 128 * D * 2;
+    static constexpr int kFK = kV + kStages * 128 * DV * 2;   // two phi(K) tiles
     static constexpr int kOnes = kFK + 2 * 32768;
     static constexpr int kBars = kOnes + 2048;
     static constexpr int kTotal = kBars + 256;
 };
 
-enum KyBars { YB_OM, YB_K0, YB_K1, YB_V0, YB_V1, YM2_0, YM2_1, YMS_0, YMS_1, YE1_0, YE1_1, YNBARS };
+// barriers of the key pass: Omega, K ring, V ring, then pairs (projection done, state update done, phi(K) written)
+enum KyBars { YB_OM = 0, YB_K0 = 1, YB_V0 = 5, YM2_0 = 9, YM2_1, YMS_0, YMS_1, YE1_0, YE1_1, YNBARS };
 
 // One CTA per (b, h, slab, token split); tiles alternate between two sets of buffers and two TMEM regions so that
 // the projection of tile i+1 runs while the epilogue warps exponentiate tile i.
@@ -532,28 +536,29 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_keys_kernel(const __grid_c
     } else if (n <= 0) {
     } else if (warp == kEpiWarps) {
         if ((tid & 31) == 0) {
+            constexpr int NST = L::kStages;
             auto load_k = [&](int i) {
-                const int b = i & 1;
+                const int b = i % NST;
                 mbar_expect_tx(bars + YB_K0 + b, kXT);
                 for (int a = 0; a < D / 64; ++a) tma_load_2d(sK + b * kXT + a * 16384, &p.mapK, bars + YB_K0 + b, a * 64, row0 + (t0 + i) * 128);
             };
             auto load_v = [&](int i) {
-                const int b = i & 1;
+                const int b = i % NST;
                 mbar_expect_tx(bars + YB_V0 + b, kVT);
                 for (int a = 0; a < DV / 64; ++a) tma_load_2d(sV + b * kVT + a * 16384, &p.mapV, bars + YB_V0 + b, a * 64, row0 + (t0 + i) * 128);
             };
-            const TileDesc tOm(sOm), tK0(sK), tK1(sK + kXT), tV0(sV), tV1(sV + kVT), tF0(sFK), tF1(sFK + 32768);
+            const TileDesc tOm(sOm), tF0(sFK), tF1(sFK + 32768);
             const uint64_t ones_desc = make_sdesc(smem_u32(sOnes), 16384, 1024);
             const uint32_t id_kk = make_idesc(128, 128, 0, 0), id_s = make_idesc(128, DV, 1, 1), id_z = make_idesc(128, 16, 1, 1);
 
             mbar_expect_tx(bars + YB_OM, 128 * D * 2);
             for (int a = 0; a < D / 64; ++a) tma_load_2d(sOm + a * 16384, &p.mapOm, bars + YB_OM, a * 64, h * p.m + slab * 128);
-            load_k(0); load_v(0);
-            if (n > 1) { load_k(1); load_v(1); }
+            for (int i = 0; i < NST && i < n; ++i) { load_k(i); load_v(i); }
             bool ok = wait_or_abort(bars + YB_OM, 0, status, abort_flag);
             if (ok) ok = wait_or_abort(bars + YB_K0, 0, status, abort_flag);
             if (ok) {
                 tc_fence_after();
+                const TileDesc tK0(sK);
                 _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(tmem + kColR1, kdesc(tK0, k), kdesc(tOm, k), id_kk, k > 0);
                 mma_commit(bars + YM2_0);
             }
@@ -561,26 +566,28 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_keys_kernel(const __grid_c
                 const int b = i & 1;
                 const uint32_t phb = (i >> 1) & 1;
                 if (i + 1 < n) {       // projection of the next tile into the other region (read out two tiles ago)
-                    ok = wait_or_abort(bars + YB_K0 + (b ^ 1), ((i + 1) >> 1) & 1, status, abort_flag);
+                    const int sn = (i + 1) % NST;
+                    ok = wait_or_abort(bars + YB_K0 + sn, ((i + 1) / NST) & 1, status, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    const TileDesc &tKn = b ? tK0 : tK1;
+                    const TileDesc tKn(sK + sn * kXT);
                     _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(tmem + (b ? kColR1 : kColR2), kdesc(tKn, k), kdesc(tOm, k), id_kk, k > 0);
                     mma_commit(bars + YM2_0 + (b ^ 1));
                 }
                 ok = wait_or_abort(bars + YE1_0 + b, phb, status, abort_flag);      // phi(K) of tile i in smem; its K tile is consumed
                 if (!ok) break;
-                if (i + 2 < n) load_k(i + 2);
-                ok = wait_or_abort(bars + YB_V0 + b, phb, status, abort_flag);
+                if (i + NST < n) load_k(i + NST);
+                ok = wait_or_abort(bars + YB_V0 + i % NST, (i / NST) & 1, status, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                const TileDesc &tF = b ? tF1 : tF0, &tVb = b ? tV1 : tV0;
+                const TileDesc &tF = b ? tF1 : tF0;
+                const TileDesc tVb(sV + (i % NST) * kVT);
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColS, mndesc(tF, k), mndesc(tVb, k), id_s, i > 0 || k > 0);
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColZ, mndesc(tF, k), ones_desc, id_z, i > 0 || k > 0);
                 mma_commit(bars + YMS_0 + b);
                 ok = wait_or_abort(bars + YMS_0 + b, phb, status, abort_flag);
                 if (!ok) break;
-                if (i + 2 < n) load_v(i + 2);
+                if (i + NST < n) load_v(i + NST);
             }
         }
     } else {
@@ -638,9 +645,10 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_keys_kernel(const __grid_c
 // ------------------------------------------------------------------ non-causal, query pass: partial O = phi(Q) S, den = phi(Q) z
 template <int D, int DV>
 struct FwdQueriesSmem {
+    static constexpr int kStages = 4;                      // ring of Q tiles
     static constexpr int kOm = 0;
-    static constexpr int kQ = kOm + 128 * D * 2;           // two Q tiles
-    static constexpr int kSb = kQ + 2 * 128 * D * 2;       // bf16 state of the slab [128 l, DV]
+    static constexpr int kQ = kOm + 128 * D * 2;
+    static constexpr int kSb = kQ + kStages * 128 * D * 2; // bf16 state of the slab [128 l, DV]
     static constexpr int kStg = kSb + 128 * DV * 2;
     static constexpr int kZ = kStg + 128 * DV * 2;
     static constexpr int kRed = kZ + 512;
@@ -648,7 +656,7 @@ struct FwdQueriesSmem {
     static constexpr int kTotal = kBars + 256;
 };
 
-enum QyBars { UB_OM, UB_Q0, UB_Q1, UM1_0, UM1_1, UM4_0, UM4_1, UE0_0, UE0_1, UE3_0, UE3_1, UNBARS };
+enum QyBars { UB_OM = 0, UB_Q0 = 1, UM1_0 = 5, UM1_1, UM4_0, UM4_1, UE0_0, UE0_1, UE3_0, UE3_1, UNBARS };
 
 // TMEM: packed phi(Q) of the two tiles in flight at 0 and 64; R1, R2 hold U_Q and then the output tile.
 template <int D, int DV>
@@ -688,18 +696,18 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_queries_kernel(const __gri
     } else if (n <= 0) {
     } else if (warp == kEpiWarps) {
         if ((tid & 31) == 0) {
+            constexpr int NST = L::kStages;
             auto load_q = [&](int i) {
-                const int b = i & 1;
+                const int b = i % NST;
                 mbar_expect_tx(bars + UB_Q0 + b, kXT);
                 for (int a = 0; a < D / 64; ++a) tma_load_2d(sQ + b * kXT + a * 16384, &p.mapQ, bars + UB_Q0 + b, a * 64, row0 + (t0 + i) * 128);
             };
-            const TileDesc tOm(sOm), tQ0(sQ), tQ1(sQ + kXT), tSb(sSb);
+            const TileDesc tOm(sOm), tQ0(sQ), tSb(sSb);
             const uint32_t id_kk = make_idesc(128, 128, 0, 0), id_o = make_idesc(128, DV, 0, 1);
             mbar_expect_tx(bars + UB_OM, 128 * D * 2 + 128 * DV * 2);
             for (int a = 0; a < D / 64; ++a) tma_load_2d(sOm + a * 16384, &p.mapOm, bars + UB_OM, a * 64, h * p.m + slab * 128);
             for (int a = 0; a < DV / 64; ++a) tma_load_2d(sSb + a * 16384, &p.mapSb, bars + UB_OM, a * 64, bh * p.m + slab * 128);
-            load_q(0);
-            if (n > 1) load_q(1);
+            for (int i = 0; i < NST && i < n; ++i) load_q(i);
             bool ok = wait_or_abort(bars + UB_OM, 0, status, abort_flag);
             if (ok) ok = wait_or_abort(bars + UB_Q0, 0, status, abort_flag);
             if (ok) {
@@ -711,17 +719,17 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_queries_kernel(const __gri
                 const int b = i & 1;
                 const uint32_t phb = (i >> 1) & 1;
                 if (i + 1 < n) {       // projection of the next tile into the other region, once its last output tile was read
-                    ok = wait_or_abort(bars + UB_Q0 + (b ^ 1), ((i + 1) >> 1) & 1, status, abort_flag);
+                    ok = wait_or_abort(bars + UB_Q0 + (i + 1) % NST, ((i + 1) / NST) & 1, status, abort_flag);
                     if (ok && i >= 1) ok = wait_or_abort(bars + UE3_0 + (b ^ 1), ((i - 1) >> 1) & 1, status, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    const TileDesc &tQn = b ? tQ0 : tQ1;
+                    const TileDesc tQn(sQ + ((i + 1) % NST) * kXT);
                     _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(tmem + (b ? kColR1 : kColR2), kdesc(tQn, k), kdesc(tOm, k), id_kk, k > 0);
                     mma_commit(bars + UM1_0 + (b ^ 1));
                 }
                 ok = wait_or_abort(bars + UE0_0 + b, phb, status, abort_flag);      // phi(Q) packed; U read; Q tile consumed
                 if (!ok) break;
-                if (i + 2 < n) load_q(i + 2);
+                if (i + NST < n) load_q(i + NST);
                 tc_fence_after();
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(tmem + (b ? kColR2 : kColR1), tmem + b * 64 + k * 8, mndesc(tSb, k), id_o, k > 0);
                 mma_commit(bars + UM4_0 + b);
@@ -941,10 +949,14 @@ void tensor_make_layout(darkattn_plan_s *plan)
     int nsplit = 1;
     const long long units = (long long)BH * Y.nslab;
     if (!D.causal) {
-        nsplit = (int)((148ll * 4 + units - 1) / units);
-        if (nsplit > Y.T) nsplit = Y.T;
-        if (nsplit > kMaxNsplit) nsplit = kMaxNsplit;
-        if (nsplit < 1) nsplit = 1;
+        // token splits per (b, h, slab): the count that minimises (waves of CTAs over the 148 SMs) x (time of one CTA),
+        // one CTA costing about 1.4 us per tile plus 5 us to start and to add its state to the sums
+        double best = 1e30;
+        for (int c = 1; c <= kMaxNsplit && c <= Y.T; ++c) {
+            const long long waves = (units * c + 147) / 148;
+            const double cost = (double)waves * (1.4 * ((Y.T + c - 1) / c) + 5.0);
+            if (cost < best) { best = cost; nsplit = c; }
+        }
     } else if (units * 2 <= 148) {
         // few long sequences: cut each into segments (a key pass computes the segment states, the causal
         // kernels of all segments then run side by side), as many as fill the SMs, at least 4 chunks each
