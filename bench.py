@@ -26,9 +26,10 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-# DRAM bytes (read + write) per launch of the dominant kernel from its ncu capture (profiles/), keyed by
-# kernel; a kernel that changed since its capture has no entry.
-NCU_TRAFFIC = {}
+# DRAM bytes (read + write) per (token, head) of the scan kernels at d = dv = 128, m = 256 from their ncu capture on the
+# small profiling workload (profiles/scan_kernels_d128_small.md); traffic is proportional to the (token, head) count.
+# A kernel that changed since its capture has no entry.
+NCU_TRAFFIC_PER_TOKEN_HEAD = {"tc_fwd_causal_kernel": 1073.0, "tc_bwd_q_kernel": 1503.0, "tc_bwd_k_kernel": 1965.0}
 
 METRIC = "DARK-attention fwd+bwd tokens/s"
 UNIT = "tokens/s"
@@ -336,9 +337,12 @@ def main():
             entry["frac"] = entry["achieved"] / entry["peak"]
         kernels.append(entry)
     top = next((k for k in kernels if "frac" in k), None)
+    traffic = None
+    if top is not None and (d, dv, m) == (128, 128, 256) and top["kernel"] in NCU_TRAFFIC_PER_TOKEN_HEAD:
+        traffic = NCU_TRAFFIC_PER_TOKEN_HEAD[top["kernel"]] * th
     if top is not None:
         roofline = {"bound": top["bound"], "achieved": top["achieved"], "peak": top["peak"], "unit": top["unit"],
-                    "frac": top["frac"], "traffic": NCU_TRAFFIC.get(top["kernel"]), "kernel": top["kernel"],
+                    "frac": top["frac"], "traffic": traffic, "kernel": top["kernel"],
                     "us_per_launch": top["us_per_launch"], "legs_us": top["legs_us"]}
     else:
         roofline = dict(whole, traffic=None, kernel="whole step")
