@@ -825,36 +825,37 @@ __global__ void delta_kernel(const __nv_bfloat16 *G, const __nv_bfloat16 *O, flo
     if (row < rows && (i % per_row) == 0) delta[row] = acc;
 }
 
-// dM[h,a,c] = s * sum_l W[l,a] T[h,l,c] + dMn[h,a,c]. One block per (8 rows a, head), one thread per column c;
-// the block's 8 columns of W sit in shared memory as floats.
+// dM[h,a,c] += s * sum_{l in this block's 64 rows} W[l,a] T[h,l,c]  (+ dMn[h,a,c] from the first block of rows);
+// dM is zeroed before the launch. One block per (8 rows a, head, 64 rows l), one thread per column c: many small
+// blocks, because the kernel is bound by the latency of its loads.
 __global__ void dm_kernel(const __nv_bfloat16 *W, const float *Tacc, const float *dMn, float *dM, int m, int r, int d, int w_per_head, float s)
 {
-    __shared__ float sw[256 * 8];                     // 256 rows l at a time, [l][8]
-    const int a0 = blockIdx.x * 8, h = blockIdx.y, c = threadIdx.x;
+    __shared__ float sw[64 * 8];
+    const int a0 = blockIdx.x * 8, h = blockIdx.y, lb = blockIdx.z * 64, c = threadIdx.x;
     const __nv_bfloat16 *w = W + (size_t)(w_per_head ? h : 0) * m * r;
+    for (int i = threadIdx.x; i < 64 * 8; i += blockDim.x) {
+        const int l = i / 8, j = i % 8;
+        sw[i] = (a0 + j < r) ? __bfloat162float(w[(size_t)(lb + l) * r + a0 + j]) : 0.f;
+    }
+    __syncthreads();
     float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    for (int lb = 0; lb < m; lb += 256) {
-        const int nl = min(256, m - lb);
-        __syncthreads();
-        for (int i = threadIdx.x; i < nl * 8; i += blockDim.x) {
-            const int l = i / 8, j = i % 8;
-            sw[i] = (a0 + j < r) ? __bfloat162float(w[(size_t)(lb + l) * r + a0 + j]) : 0.f;
-        }
-        __syncthreads();
-        const float *Th = Tacc + ((size_t)h * m + lb) * d + c;
-        for (int l0 = 0; l0 < nl; l0 += 16) {       // m is a multiple of 128; 16 independent loads in flight
-            float tv[16];
+    const float *Th = Tacc + ((size_t)h * m + lb) * d + c;
+    for (int l0 = 0; l0 < 64; l0 += 16) {
+        float tv[16];
 #pragma unroll
-            for (int i = 0; i < 16; ++i) tv[i] = Th[(size_t)(l0 + i) * d];
+        for (int i = 0; i < 16; ++i) tv[i] = Th[(size_t)(l0 + i) * d];
 #pragma unroll
-            for (int i = 0; i < 16; ++i)
+        for (int i = 0; i < 16; ++i)
 #pragma unroll
-                for (int j = 0; j < 8; ++j) acc[j] = fmaf(sw[(l0 + i) * 8 + j], tv[i], acc[j]);
-        }
+            for (int j = 0; j < 8; ++j) acc[j] = fmaf(sw[(l0 + i) * 8 + j], tv[i], acc[j]);
     }
 #pragma unroll
     for (int j = 0; j < 8; ++j)
-        if (a0 + j < r) dM[((size_t)h * r + a0 + j) * d + c] = fmaf(s, acc[j], dMn[((size_t)h * r + a0 + j) * d + c]);
+        if (a0 + j < r) {
+            float v = s * acc[j];
+            if (lb == 0) v += dMn[((size_t)h * r + a0 + j) * d + c];
+            atomicAdd(dM + ((size_t)h * r + a0 + j) * d + c, v);
+        }
 }
 
 template <int D, int DV>
@@ -968,7 +969,8 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
     else keep(launch_finish<128>(F, (int)(BH * F.nsplit), st));
 
     timer_mark(plan, st, "dm_kernel");
-    dm_kernel<<<dim3((D.r + 7) / 8, D.H), D.d, 0, st>>>((const __nv_bfloat16 *)W, fl(Y.Tacc), fl(Y.dMn), dM, D.m, D.r, D.d, D.w_per_head, D.s);
+    keep(cudaMemsetAsync(dM, 0, (size_t)D.H * D.r * D.d * 4, st));
+    dm_kernel<<<dim3((D.r + 7) / 8, D.H, D.m / 64), D.d, 0, st>>>((const __nv_bfloat16 *)W, fl(Y.Tacc), fl(Y.dMn), dM, D.m, D.r, D.d, D.w_per_head, D.s);
     chk();
     if (e != cudaSuccess) { set_cuda_error(e, "tensor_backward"); return DARKATTN_ERR_CUDA; }
     return DARKATTN_OK;

@@ -29,33 +29,35 @@ constexpr int kMaxNsplit = 64;
 // ------------------------------------------------------------------ small helpers
 
 // ------------------------------------------------------------------ prologue kernels (SIMT, tiny)
-// Omega[h,l,c] = log2(e) * s * sum_a W[l,a] M[h,a,c]  (bf16). One block per (head, 16 rows l); thread = column c
-// (d <= 128 threads... the block has d threads). The 16 rows of W sit in shared memory as floats.
+// Omega[h,l,c] = log2(e) * s * sum_a W[l,a] M[h,a,c]  (bf16). One block per (head, 4 rows l), one thread per column c
+// (the block has d threads); many small blocks, because the kernel is bound by the latency of its loads.
 __global__ void fold_omega_kernel(const __nv_bfloat16 *W, const __nv_bfloat16 *M, __nv_bfloat16 *Om, int m, int r, int d,
                                   int w_per_head, float coef)
 {
-    __shared__ float sw[16][129];
-    const int h = blockIdx.y, l0 = blockIdx.x * 16, c = threadIdx.x;
+    __shared__ __align__(16) float sw[4][128];
+    const int h = blockIdx.y, l0 = blockIdx.x * 4, c = threadIdx.x;
     const __nv_bfloat16 *w = W + ((size_t)(w_per_head ? h : 0) * m + l0) * r;
-    for (int i = threadIdx.x; i < 16 * r; i += blockDim.x) sw[i / r][i % r] = __bfloat162float(w[i]);
+    for (int i = threadIdx.x; i < 4 * r; i += blockDim.x) sw[i / r][i % r] = __bfloat162float(w[i]);
     __syncthreads();
     const __nv_bfloat16 *Mh = M + (size_t)h * r * d;
-    float acc[16];
-#pragma unroll
-    for (int i = 0; i < 16; ++i) acc[i] = 0.f;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
     for (int a0 = 0; a0 < r; a0 += 16) {            // r is a multiple of 16; 16 independent loads in flight
         __nv_bfloat16 mv[16];
 #pragma unroll
         for (int j = 0; j < 16; ++j) mv[j] = Mh[(size_t)(a0 + j) * d + c];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-            const float x = __bfloat162float(mv[j]);
+        for (int j = 0; j < 16; j += 4) {
+            const float x0 = __bfloat162float(mv[j]), x1 = __bfloat162float(mv[j + 1]);
+            const float x2 = __bfloat162float(mv[j + 2]), x3 = __bfloat162float(mv[j + 3]);
 #pragma unroll
-            for (int i = 0; i < 16; ++i) acc[i] = fmaf(sw[i][a0 + j], x, acc[i]);
+            for (int i = 0; i < 4; ++i) {
+                const float4 wv = *reinterpret_cast<const float4 *>(&sw[i][a0 + j]);   // one broadcast load per four products
+                acc[i] = fmaf(wv.x, x0, fmaf(wv.y, x1, fmaf(wv.z, x2, fmaf(wv.w, x3, acc[i]))));
+            }
         }
     }
 #pragma unroll
-    for (int i = 0; i < 16; ++i) Om[((size_t)h * m + l0 + i) * d + c] = __float2bfloat16_rn(coef * acc[i]);
+    for (int i = 0; i < 4; ++i) Om[((size_t)h * m + l0 + i) * d + c] = __float2bfloat16_rn(coef * acc[i]);
 }
 
 // Key-side shift of a slab, in log2 units: c = log2(e) * max(0, max_l |w_l|^2/2 - 40).
@@ -66,7 +68,12 @@ __global__ void slab_shift_kernel(const __nv_bfloat16 *W, float *cs, int H, int 
     const int bh = blockIdx.x / nslab, slab = blockIdx.x % nslab, h = bh % H;
     const __nv_bfloat16 *w = W + ((size_t)(w_per_head ? h : 0) * m + (size_t)slab * 128 + threadIdx.x) * r;
     float acc = 0.f;
-    for (int a = 0; a < r; ++a) { const float v = __bfloat162float(w[a]); acc = fmaf(v, v, acc); }
+    for (int a = 0; a < r; a += 8) {                // r is a multiple of 16 and the rows are 16-byte aligned
+        const uint4 raw = *reinterpret_cast<const uint4 *>(w + a);
+        const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) { const float2 f = __bfloat1622float2(h2[q]); acc = fmaf(f.x, f.x, fmaf(f.y, f.y, acc)); }
+    }
     acc *= 0.5f;
     __shared__ float red[128];
     red[threadIdx.x] = acc;
@@ -1015,7 +1022,7 @@ cudaError_t tensor_prologue(const darkattn_plan_s *plan, const void *K, const vo
     auto chk = [&]() { cudaError_t x = cudaGetLastError(); if (x != cudaSuccess && e == cudaSuccess) e = x; };
 
     timer_mark(plan, st, "fold_omega_kernel");
-    fold_omega_kernel<<<dim3(D.m / 16, D.H), D.d, 0, st>>>((const __nv_bfloat16 *)W, (const __nv_bfloat16 *)M, out.Om, D.m, D.r, D.d,
+    fold_omega_kernel<<<dim3(D.m / 4, D.H), D.d, 0, st>>>((const __nv_bfloat16 *)W, (const __nv_bfloat16 *)M, out.Om, D.m, D.r, D.d,
                                                       D.w_per_head, kLog2e * D.s);
     chk();
     timer_mark(plan, st, "slab_shift_kernel");
