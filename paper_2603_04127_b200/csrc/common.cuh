@@ -150,6 +150,21 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
                                   const void *M, const void *W, const void *O, const void *dO, const void *saved,
                                   void *dQ, void *dK, void *dV, float *dM, char *ws, cudaStream_t st);
 
+// Number of pieces (1..max_splits, at most T) to cut each of `units` sequences of T tiles into, for kernels that run one CTA
+// per piece and SM: the count that minimises (waves of CTAs over the 148 SMs) x (time of one CTA), one CTA costing
+// us_per_tile per tile plus us_fixed to start and to flush its accumulators.
+inline int pick_splits(long long units, int T, double us_per_tile, double us_fixed, int max_splits, int slots = 148)
+{
+    int best_c = 1;
+    double best = 1e30;
+    for (int c = 1; c <= max_splits && c <= T; ++c) {
+        const long long waves = (units * c + slots - 1) / slots;
+        const double cost = (double)waves * (us_per_tile * ((T + c - 1) / c) + us_fixed);
+        if (cost < best) { best = cost; best_c = c; }
+    }
+    return best_c;
+}
+
 #define DARKATTN_CUDA_TRY(expr, where)                                   \
     do {                                                                 \
         cudaError_t e__ = (expr);                                        \

@@ -682,21 +682,24 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __gr
             for (int a = 0; a < D / 64; ++a) tma_load_2d(sM + a * 16384, &p.mapM, bar_m, a * 64, h * p.r);
             load_k(t0);
             const uint32_t id_x = make_idesc(128, p.r, 0, 0), id_d = make_idesc(128, D, 0, 1), id_t = make_idesc(128, D, 1, 1);
+            // K M^T of tile i+1 is issued right behind the two products of tile i, so that it runs while the epilogue
+            // warps still write tile i out.
             bool ok = wait_or_abort(bar_m, 0, p.status, abort_flag);
             uint32_t np = 0;                             // rounds of partial loads issued so far
+            if (t0 + 1 < t1) load_k(t0 + 1);
+            if (ok) ok = wait_or_abort(bar_k, 0, p.status, abort_flag);
+            if (ok) {
+                tc_fence_after();
+                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(tmem + C1, kdesc(tK0, k), kdesc(tM, k), id_x, k > 0);
+                mma_commit(m1);
+            }
             for (int t = t0; t < t1 && ok; ++t) {
                 const int i = t - t0, b = i & 1;
-                const uint32_t ph = i & 1, phk = (i >> 1) & 1;
+                const uint32_t ph = i & 1;
                 const TileDesc &tK = b ? tK1 : tK0;
                 if (np > 0) ok = wait_or_abort(e_p, (np - 1) & 1, p.status, abort_flag);   // partial tiles consumed
                 if (!ok) break;
                 load_partials(t, 0); ++np;
-                if (t + 1 < t1) load_k(t + 1);          // the other buffer: its last reader finished before m3 of tile t-1
-                ok = wait_or_abort(bar_k + b, phk, p.status, abort_flag);
-                if (!ok) break;
-                tc_fence_after();
-                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(tmem + C1, kdesc(tK, k), kdesc(tM, k), id_x, k > 0);
-                mma_commit(m1);
                 ok = wait_or_abort(e1, ph, p.status, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
@@ -704,6 +707,14 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __gr
                 mma_commit(m2);
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + C3, mndesc(tW, k), mndesc(tK, k), id_t, (t > t0) || k > 0);
                 mma_commit(m3);
+                if (t + 1 < t1) {
+                    ok = wait_or_abort(bar_k + (b ^ 1), ((i + 1) >> 1) & 1, p.status, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const TileDesc &tKn = b ? tK0 : tK1;
+                    _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(tmem + C1, kdesc(tKn, k), kdesc(tM, k), id_x, k > 0);
+                    mma_commit(m1);
+                }
                 for (int round = 1; round < nrounds && ok; ++round) {
                     ok = wait_or_abort(e_p, (np - 1) & 1, p.status, abort_flag);
                     if (ok) { load_partials(t, round); ++np; }
@@ -711,6 +722,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __gr
                 if (!ok) break;
                 ok = wait_or_abort(m3, ph, p.status, abort_flag);
                 if (!ok) break;
+                if (t + 2 < t1) load_k(t + 2);          // this tile's K buffer has been read by both of its products
                 ok = wait_or_abort(e2, ph, p.status, abort_flag);
             }
         }
@@ -720,12 +732,18 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __gr
         const uint32_t lane_addr = tmem + ((uint32_t)(q4 * 32) << 16);
         bool ok = true;
         uint32_t np = 0;
+        // rowsum(E) of a tile's row: its partials are loaded one tile ahead (their latency is hidden behind a tile's work)
+        auto row_sum = [&](int t) {
+            const size_t rw = (size_t)bh * p.N + (size_t)t * 128 + r;
+            float e = 0.f;
+            for (int s = 0; s < p.nes; ++s) e += __ldg(p.espart + (size_t)s * rows + rw);
+            return e;
+        };
+        float es_next = row_sum(t0);
         for (int t = t0; t < t1 && ok; ++t) {
             const uint32_t ph = (t - t0) & 1;
             const size_t row = (size_t)bh * p.N + (size_t)t * 128 + r;
-            float es = 0.f;
-            for (int s = 0; s < p.nes; ++s) es += p.espart[(size_t)s * rows + row];
-            const float coef = -p.s2 * es;
+            const float coef = -p.s2 * es_next;
             ok = __all_sync(0xffffffffu, wait_or_abort(m1, ph, p.status, abort_flag));
             if (!ok) break;
             tc_fence_after();
@@ -746,6 +764,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __gr
             if (tid == 0) tma_store_wait_read();          // the staging tile of the previous store is free again
             tc_fence_before();
             mbar_arrive_warp(e1);
+            if (t + 1 < t1) es_next = row_sum(t + 1);
 
             float acc[32];
 #pragma unroll
@@ -962,8 +981,7 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
     F.espart = fl(Y.espart); F.dMn = fl(Y.dMn);
     F.status = P.status;
     F.N = D.N; F.H = D.H; F.BH = D.BH; F.T = Y.T; F.r = D.r; F.nslab = 1; F.nes = 4 * Y.nslab; F.s2 = D.s * D.s;
-    F.nsplit = (int)((148 * 2 + BH - 1) / BH);
-    if (F.nsplit > Y.T) F.nsplit = Y.T;
+    F.nsplit = pick_splits((long long)BH, Y.T, 3.5, 5.0, 64);
     timer_mark(plan, st, "tc_bwd_finish_k_kernel");
     if (D.d == 64) keep(launch_finish<64>(F, (int)(BH * F.nsplit), st));
     else keep(launch_finish<128>(F, (int)(BH * F.nsplit), st));

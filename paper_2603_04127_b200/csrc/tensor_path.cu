@@ -956,14 +956,7 @@ void tensor_make_layout(darkattn_plan_s *plan)
     int nsplit = 1;
     const long long units = (long long)BH * Y.nslab;
     if (!D.causal) {
-        // token splits per (b, h, slab): the count that minimises (waves of CTAs over the 148 SMs) x (time of one CTA),
-        // one CTA costing about 1.4 us per tile plus 5 us to start and to add its state to the sums
-        double best = 1e30;
-        for (int c = 1; c <= kMaxNsplit && c <= Y.T; ++c) {
-            const long long waves = (units * c + 147) / 148;
-            const double cost = (double)waves * (1.4 * ((Y.T + c - 1) / c) + 5.0);
-            if (cost < best) { best = cost; nsplit = c; }
-        }
+        nsplit = pick_splits(units, Y.T, 1.4, 5.0, kMaxNsplit);
     } else if (units * 2 <= 148) {
         // few long sequences: cut each into segments (a key pass computes the segment states, the causal
         // kernels of all segments then run side by side), as many as fill the SMs, at least 4 chunks each
@@ -1031,8 +1024,7 @@ cudaError_t tensor_prologue(const darkattn_plan_s *plan, const void *K, const vo
 
     NP.nK = out.nK; NP.status = reinterpret_cast<int *>(ws + Y.status);
     NP.N = D.N; NP.H = D.H; NP.T = Y.T; NP.r = D.r;
-    NP.nsplit = (int)((148 * 2 + BH - 1) / BH);
-    if (NP.nsplit > Y.T) NP.nsplit = Y.T;
+    NP.nsplit = pick_splits((long long)BH, Y.T, 2.5, 3.0, 64, 3 * 148);      // three CTAs of this kernel fit one SM
     NP.coef = kLog2e * 0.5f * D.s * D.s;
     const int smem_bytes = 2 * 128 * D.d * 2 + 64;
     timer_mark(plan, st, "tc_key_norms_kernel");
