@@ -198,6 +198,31 @@ def test_tensor_path_is_deterministic(binding):
             assert worst < 2.0 ** -7, f"{k} differs between runs by {worst:.2e} of its largest value"
 
 
+def test_kernel_timing_reports_every_kernel_of_a_step(binding):
+    import torch
+    wl = inputs.small(name="timing", wid=91, B=1, H=2, N=512, d=64, m=256, causal=True, dtype="bf16", backward=True)
+    t = inputs.generate(wl)
+    from tests.util import to_dev
+    Q, K, V, M, W, dO = (to_dev(x, torch.bfloat16) for x in (t.Q, t.K, t.V, t.M, t.W, t.dO))
+    plan = binding.darkattn_plan(1, 2, 512, 64, 256, causal=True)
+    ws = plan.alloc_workspace()
+    saved = torch.empty(plan.saved_bytes, dtype=torch.uint8, device="cuda")
+    O, dQ, dK, dV = torch.empty_like(V), torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V)
+    dM = torch.empty(M.shape, dtype=torch.float32, device="cuda")
+    binding.darkattn_kernel_timing(plan, True)
+    for _ in range(2):
+        binding.darkattn_forward(plan, Q, K, V, M, W, O, ws, saved=saved)
+        binding.darkattn_backward(plan, Q, K, V, M, W, O, dO, dQ, dK, dV, dM, ws, saved=saved)
+        times = binding.darkattn_kernel_times(plan)
+    binding.darkattn_kernel_timing(plan, False)
+    assert binding.darkattn_last_device_status(plan, ws) == binding.OK
+    for name in ("tc_fwd_causal_kernel", "combine_kernel", "tc_bwd_q_kernel", "tc_bwd_k_kernel", "tc_bwd_finish_k_kernel"):
+        ms, launches = times[name]
+        assert launches == 2 and 0.0 < ms < 1e3, (name, ms, launches)
+    assert sum(c for _, c in times.values()) == 2 * (plan.launches(False) + plan.launches(True))
+    plan.destroy()
+
+
 def test_tensor_path_rejects_uncovered_shapes(binding):
     for kw in (dict(N=200), dict(d=48), dict(m=96)):
         a = dict(B=1, H=1, N=256, d=64, m=128)
