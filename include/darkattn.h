@@ -103,7 +103,10 @@ darkattn_status_t darkattn_forward(darkattn_plan_t plan, const void *Q, const vo
 /* Gradients of L = sum(dO .* O) with respect to Q, K, V and M (the paper learns M by
  * back-propagation, Section 4; the formulas follow from the chain rule through the definitions at
  * the top of this file, with every stabilising shift held constant, which is exact because O does
- * not depend on them). `O` is the forward result for the same inputs (may be NULL: recomputed).  */
+ * not depend on them). `O` is the forward result for the same inputs (may be NULL: recomputed).
+ * On the tensor-core path part of the zeroing of dK and dV runs on a stream of the plan's own (created by the
+ * first such call, non-blocking), forked from `cuda_stream` and joined back into it with events before the
+ * call's later kernels: to the caller everything still happens in stream order on `cuda_stream`.           */
 darkattn_status_t darkattn_backward(darkattn_plan_t plan, const void *Q, const void *K, const void *V,
                                     const void *M, const void *W, const void *O, const void *dO,
                                     const void *saved /* nullable */, void *dQ, void *dK, void *dV,

@@ -121,6 +121,10 @@ struct darkattn_plan_s {
     size_t saved_bytes;
     int launches_fwd, launches_bwd;
     mutable darkattn::KernelTimer timer;
+    // side stream of the tensor-core backward (created by its first call on the device current then) and the two
+    // events that fork it from and join it back into the caller's stream
+    mutable cudaStream_t aux_stream = nullptr;
+    mutable cudaEvent_t aux_fork = nullptr, aux_join = nullptr;
 };
 
 namespace darkattn {

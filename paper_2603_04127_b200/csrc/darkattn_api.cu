@@ -200,6 +200,11 @@ void darkattn_destroy(darkattn_plan_t plan)
 {
     if (plan && plan->timer.created)
         for (int i = 0; i < KernelTimer::kMaxMarks; ++i) cudaEventDestroy(plan->timer.ev[i]);
+    if (plan && plan->aux_stream) {
+        cudaEventDestroy(plan->aux_fork);
+        cudaEventDestroy(plan->aux_join);
+        cudaStreamDestroy(plan->aux_stream);
+    }
     delete plan;
 }
 

@@ -890,6 +890,10 @@ cudaError_t launch_scan(const darkattn_plan_s *plan, const BwdParams &P, int gri
     tc_bwd_q_kernel<D, DV><<<grid, kThreads, L::kTotal, st>>>(P);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
+    if (P.nslab > 1) {
+        e = cudaStreamWaitEvent(st, plan->aux_join, 0);      // dK and dV have been zeroed
+        if (e != cudaSuccess) return e;
+    }
     timer_mark(plan, st, "tc_bwd_k_kernel");
     tc_bwd_k_kernel<D, DV><<<grid, kThreads, L::kTotal, st>>>(P);
     return cudaGetLastError();
@@ -948,10 +952,21 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
     chk();
     keep(cudaMemsetAsync(ws + Y.Tacc, 0, (size_t)D.H * D.m * D.d * 4, st));
     keep(cudaMemsetAsync(ws + Y.dMn, 0, (size_t)D.H * D.r * D.d * 4, st));
-    if (Y.nslab > 1) {      // the slabs of a head add their parts into the gradients
+    if (Y.nslab > 1) {
+        // The slabs of a head add their parts into the gradients, which therefore start at zero. dQ is needed first;
+        // dK and dV are zeroed on a side stream while the query-side scan runs (it leaves SMs and bandwidth free).
+        if (!plan->aux_stream) {
+            keep(cudaStreamCreateWithFlags(&plan->aux_stream, cudaStreamNonBlocking));
+            keep(cudaEventCreateWithFlags(&plan->aux_fork, cudaEventDisableTiming));
+            keep(cudaEventCreateWithFlags(&plan->aux_join, cudaEventDisableTiming));
+            if (e != cudaSuccess) { set_cuda_error(e, "tensor_backward: side stream"); return DARKATTN_ERR_CUDA; }
+        }
+        keep(cudaEventRecord(plan->aux_fork, st));
+        keep(cudaStreamWaitEvent(plan->aux_stream, plan->aux_fork, 0));
+        keep(cudaMemsetAsync(dK, 0, BH * N * D.d * 2, plan->aux_stream));
+        keep(cudaMemsetAsync(dV, 0, BH * N * D.dv * 2, plan->aux_stream));
+        keep(cudaEventRecord(plan->aux_join, plan->aux_stream));
         keep(cudaMemsetAsync(dQ, 0, BH * N * D.d * 2, st));
-        keep(cudaMemsetAsync(dK, 0, BH * N * D.d * 2, st));
-        keep(cudaMemsetAsync(dV, 0, BH * N * D.dv * 2, st));
     }
 
     BwdParams P;
