@@ -70,7 +70,8 @@ struct TensorLayout {
     size_t dMn;     // gradient of M through the key norm term, fp32 [H, r, d]
     size_t total_bytes;
     // the forward -> backward stash (`saved`): per-row normalisers, key norms, folded projections, key shifts
-    size_t sv_sv, sv_nK, sv_Om, sv_cs, sv_bytes;
+    size_t sv_sv, sv_nK, sv_Om, sv_cs, sv_zc, sv_bytes;
+    size_t zc;      // workspace copy of the stash's per-chunk z (causal): sum_j phi(K)_jl over the chunks before t, fp32 [BH, T, m]
     int nslab, T, nsplit;
 };
 
@@ -81,17 +82,20 @@ struct Stash {
     float *nK;
     __nv_bfloat16 *Om;
     float *cs;
+    float *zc;      // causal: z before chunk t, [BH, T, m] (row t = 0 is not written: it is zero)
 };
 inline Stash stash_in_workspace(const TensorLayout &Y, char *ws)
 {
     return Stash{reinterpret_cast<float2 *>(ws + Y.sv), reinterpret_cast<float *>(ws + Y.nK),
-                 reinterpret_cast<__nv_bfloat16 *>(ws + Y.Om), reinterpret_cast<float *>(ws + Y.cs)};
+                 reinterpret_cast<__nv_bfloat16 *>(ws + Y.Om), reinterpret_cast<float *>(ws + Y.cs),
+                 reinterpret_cast<float *>(ws + Y.zc)};
 }
 inline Stash stash_in_saved(const TensorLayout &Y, void *saved)
 {
     char *b = static_cast<char *>(saved);
     return Stash{reinterpret_cast<float2 *>(b + Y.sv_sv), reinterpret_cast<float *>(b + Y.sv_nK),
-                 reinterpret_cast<__nv_bfloat16 *>(b + Y.sv_Om), reinterpret_cast<float *>(b + Y.sv_cs)};
+                 reinterpret_cast<__nv_bfloat16 *>(b + Y.sv_Om), reinterpret_cast<float *>(b + Y.sv_cs),
+                 reinterpret_cast<float *>(b + Y.sv_zc)};
 }
 
 }  // namespace darkattn

@@ -40,6 +40,7 @@ struct BwdParams {
     const float *delta;   // [BH*N]  dO_i . O_i
     const float *nK;      // [BH*N]  key norms, log2 units
     const float *cs;      // [BH*nslab] key-side shift per slab
+    const float *zc;      // [BH, T, m] z before chunk t, from the forward pass (row 0 is not read)
     float *rhoc;          // [BH, T, m] per-chunk -sum_i A^_il delta_i (written by the query-side kernel)
     float *espart;        // [4 nslab, BH*N] partials of rowsum(E^K): one per slab and 32-column group
     float *Tacc;          // [H, m, D]
@@ -65,45 +66,10 @@ struct BwdSmem {
 // TMEM columns (512 allocated): scan state at 0, T at 128, scratch R1 at 256 and R2 at 384.
 constexpr uint32_t kColState = 0, kColT = 128, kColR1 = 256, kColR2 = 384;
 
-// Sum over the 32 lanes of a warp of x[c], for every c: afterwards lane l holds the sum for c = l.
-// Butterfly reduce-scatter: 31 shuffles instead of 32 full reductions.
-__device__ __forceinline__ float warp_column_sums(float (&x)[32], int lane)
-{
-#pragma unroll
-    for (int s = 16; s >= 1; s >>= 1) {
-        const bool up = (lane & s) != 0;
-#pragma unroll
-        for (int i = 0; i < s; ++i) {
-            const float send = up ? x[i] : x[i + s];
-            const float keep = up ? x[i + s] : x[i];
-            x[i] = keep + __shfl_xor_sync(0xffffffffu, send, s);
-        }
-    }
-    return x[0];
-}
+// K-major 16 x 128 bf16 operand (two atoms of 2 KB): step k covers 16 elements of K
+__device__ __forceinline__ uint64_t vecdesc(const TileDesc &t, int k) { return t.kmaj + (uint64_t)(((k / 4) * 2048 + (k % 4) * 32) >> 4); }
 
-// features 2^(U - offset) as above; also adds, for every column, weight * feature summed over the
-// warp's 32 rows into colsum[col0 + column] (shared memory).
-__device__ __forceinline__ void features_to_tile_sums(uint32_t taddr, float offset, unsigned char *tile, int row, int col0,
-                                                      float weight, float *colsum, int lane)
-{
-    uint32_t v[32], pk[16];
-    float f[32];
-    tmem_ld32(taddr, v);
-    tmem_wait_ld();
-#pragma unroll
-    for (int j = 0; j < 32; ++j) f[j] = ex2f(__uint_as_float(v[j]) - offset);
-#pragma unroll
-    for (int j = 0; j < 32; j += 2) pk[j / 2] = pack_bf16(f[j], f[j + 1]);
-#pragma unroll
-    for (int q = 0; q < 4; ++q)
-        *reinterpret_cast<uint4 *>(tile_chunk(tile, row, col0 / 8 + q)) = make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
-#pragma unroll
-    for (int j = 0; j < 32; ++j) f[j] *= weight;
-    atomicAdd(colsum + col0 + lane, warp_column_sums(f, lane));
-}
-
-enum QBars { QB_OM, QB_Q, QB_K, QB_V, QB_G, QB_X2, QM1, QM2, QM3, QMS, QM4, QM5, QM6, QE0, QE1, QE2, QE3, QE4, QNBARS };
+enum QBars { QB_OM, QB_Q, QB_K, QB_V, QB_G, QB_X2, QM1, QM2, QM3, QMR, QMS, QM4, QM5, QM6, QE0, QE1, QE2, QE3, QE4, QNBARS };
 
 // ------------------------------------------------------------------ query side (forward direction)
 template <int D, int DV>
@@ -113,7 +79,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
     extern __shared__ __align__(1024) unsigned char smem[];
     unsigned char *sOm = smem + L::kOm, *sQA = smem + L::kQA, *sKB = smem + L::kKB, *sV = smem + L::kV;
     unsigned char *sG = smem + L::kG, *sSt = smem + L::kSt, *sStg = smem + L::kStg;
-    float *sZ = reinterpret_cast<float *>(smem + L::kVec), *sZc = sZ + 128, *sRc = sZ + 256;   // z_prev; chunk sums of Bf and of -delta A^
+    float *sZ = reinterpret_cast<float *>(smem + L::kVec);      // z before this chunk
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::kBars);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + QNBARS);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + QNBARS + 1);
@@ -128,7 +94,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
         *abort_flag = (smem_u32(smem) & 1023u) ? 1 : 0;
         fence_mbar_init();
     }
-    if (tid < 384) sZ[tid] = 0.f;
+    if (tid < 128) sZ[tid] = 0.f;
     if (warp == kEpiWarps) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
@@ -144,8 +110,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                 mbar_expect_tx(bar, 128 * width * 2);
                 for (int a = 0; a < width / 64; ++a) tma_load_2d(dst + a * 16384, map, bar, a * 64, row0 + t * 128);
             };
-            const TileDesc tOm(sOm), tQA(sQA), tKB(sKB), tV(sV), tG(sG), tSt(sSt);
+            const TileDesc tOm(sOm), tQA(sQA), tKB(sKB), tV(sV), tG(sG), tSt(sSt), tDel(sStg);
             const uint32_t id_kk = make_idesc(128, 128, 0, 0);
+            const uint32_t id_vec = make_idesc(128, 16, 1, 0);
             const uint32_t id_state = make_idesc(128, DV, 1, 1);
             const uint32_t id_tm = make_idesc(128, 128, 0, 1);
             const uint32_t id_dx = make_idesc(128, D, 0, 1);
@@ -162,7 +129,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
             // Schedule of one chunk (R1, R2: the two scratch regions of TMEM). U_K of the next chunk is issued in
             // the tail of the current one, and dO V^T runs while the epilogue is still busy with A^.
             //   R2: U_K -> (Bf read) -> dO V^T -> packed dP (A operand of dP Bf) -> U_K of the next chunk
-            //   R1: U_Q -> (A^ read) -> dP Bf + dO S^T -> (E read) -> E Omega -> (dQ read)
+            //   R1: U_Q -> (A^ read) -> rho_c (16 columns) -> dP Bf + dO S^T -> (E read) -> E Omega -> (dQ read)
             bool ok = wait_or_abort(bars + QB_OM, 0, status, abort_flag);
             if (ok) ok = wait_or_abort(bars + QB_K, 0, status, abort_flag);
             if (ok) {
@@ -187,7 +154,10 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColState, mndesc(tKB, k), mndesc(tV, k), id_state, (!first) || k > 0);   // S += Bf^T V
                 mma_commit(bars + QMS);
                 QWAIT(QE1); if (!ok) break;                                                                      // A^ in smem, R1 read
-                QWAIT(QE2); if (!ok) break;                                                                      // dP packed in R2
+                tc_fence_after();
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R1, mndesc(tQA, k), vecdesc(tDel, k), id_vec, k > 0);       // rho_c = -A^^T delta (columns 0, 1)
+                mma_commit(bars + QMR);
+                QWAIT(QE2); if (!ok) break;                                                                      // dP packed in R2, rho_c read
                 tc_fence_after();
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R1, R2 + k * 8, mndesc(tKB, k), id_tm, k > 0);               // dP Bf
                 if (!first)
@@ -220,11 +190,10 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
         // ============================== epilogue threads (see kEpiWarps)
         const int lane = tid & 31, q4 = warp & 3, col0 = (warp >> 2) * 32;
         const int r = q4 * 32 + lane;                        // tile row = TMEM lane
-        const bool own = (q4 == 0);                          // these 128 threads each own one column's running sums
+        const bool g0 = (col0 == 0);                         // these 128 threads: row r also stands for feature r of the slab
         const uint32_t lane_addr = tmem + ((uint32_t)(q4 * 32) << 16);
         const uint32_t R1 = lane_addr + kColR1, R2 = lane_addr + kColR2;
         const float cshift = p.cs[bh * p.nslab + slab];
-        float zrun = 0.f;
         bool ok = true;
         for (int t = 0; t < T && ok; ++t) {
             const uint32_t ph = t & 1;
@@ -235,17 +204,34 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
             const float del = p.delta[row];
             const float nk = p.nK[row] + cshift;
             const float aq = svv.y - cshift + log2f(svv.x);
+            // z before the next chunk, from the forward pass (loaded early, used at the end of the chunk)
+            const float znext = (g0 && !last) ? __ldg(p.zc + ((size_t)bh * T + t + 1) * p.m + slab * 128 + r) : 0.f;
             EWAIT(QM2); if (!ok) break;
             tc_fence_after();
-            features_to_tile_sums(R2 + col0, nk, sKB, r, col0, 1.f, sZc, lane);       // Bf and z_c = sum_j Bf_jl
+            features_to_tile(R2 + col0, nk, sKB, r, col0);                             // Bf
+            if (warp == 0) {
+                // 16 x 128 K-major operand of rho_c = -A^^T delta at the start of the staging tile: row 0 = -delta rounded
+                // to bf16, row 1 = the rounding's remainder. Written by the warp whose first lane has just seen the
+                // previous chunk's store leave the tile.
+                if (tid == 0) tma_store_wait_read();
+                __syncwarp();
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int k = i * 32 + lane;
+                    const float dk = -__ldg(p.delta + (size_t)row0 + (size_t)t * 128 + k);
+                    const __nv_bfloat16 hi = __float2bfloat16_rn(dk);
+                    const __nv_bfloat16 lo = __float2bfloat16_rn(dk - __bfloat162float(hi));
+                    const int atom = k >> 6, kk = k & 63, ch = kk >> 3;
+                    *reinterpret_cast<__nv_bfloat16 *>(sStg + atom * 2048 + (ch << 4) + (kk & 7) * 2) = hi;
+                    *reinterpret_cast<__nv_bfloat16 *>(sStg + atom * 2048 + 128 + ((ch ^ 1) << 4) + (kk & 7) * 2) = lo;
+                }
+            }
             fence_async_smem();
-            if (tid == 0) tma_store_wait_read();      // the previous chunk's store has left the staging tile (every later
-                                                      // writer of it first passes a barrier that needs this arrival)
             tc_fence_before();
             mbar_arrive_warp(bars + QE0);
             EWAIT(QM1); if (!ok) break;
             tc_fence_after();
-            features_to_tile_sums(R1 + col0, aq, sQA, r, col0, -del, sRc, lane);      // A^ and rho_c = -sum_i delta_i A^_il
+            features_to_tile(R1 + col0, aq, sQA, r, col0);                             // A^
             fence_async_smem();
             tc_fence_before();
             mbar_arrive_warp(bars + QE1);
@@ -266,18 +252,19 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                 tmem_st16(R2 + col0 / 2, pk);
             }
             tmem_wait_st();
+            if (g0) {       // rho_c of feature r (TMEM lane r), for the key-side kernel
+                EWAIT(QMR); if (!ok) break;
+                tc_fence_after();
+                uint32_t v[16];
+                tmem_ld16(R1, v);
+                tmem_wait_ld();
+                p.rhoc[((size_t)bh * T + t) * p.m + slab * 128 + r] = __uint_as_float(v[0]) + __uint_as_float(v[1]);
+            }
             tc_fence_before();
             mbar_arrive_warp(bars + QE2);
 
             EWAIT(QM4); if (!ok) break;
             tc_fence_after();
-            float znew = zrun;
-            if (own) {      // the column sums of all four lane quarters are in (every warp arrived at QE0 and QE1)
-                znew = zrun + sZc[col0 + lane];
-                p.rhoc[((size_t)bh * T + t) * p.m + slab * 128 + col0 + lane] = sRc[col0 + lane];
-                sZc[col0 + lane] = 0.f;
-                sRc[col0 + lane] = 0.f;
-            }
             {   // E = A^ .* (dP Bf + dO S^T - delta z^T), in place over A^
                 uint32_t v[32];
                 tmem_ld32(R1 + col0, v);
@@ -313,10 +300,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                 tma_store_commit();
             }
             EWAIT(QMS); if (!ok) break;
-            zrun = znew;
             if (!last) {
                 if (col0 < DV) tmem_row_to_tile(lane_addr + kColState + col0, sSt, r, col0);
-                if (own) sZ[col0 + lane] = zrun;
+                if (g0) sZ[r] = znext;
                 fence_async_smem();
             }
             tc_fence_before();
@@ -981,7 +967,7 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
     ok = ok && make_map(&F.mapM, M, (size_t)D.H * D.r, D.d, 128);
     if (!ok) { set_cuda_error(cudaErrorInvalidValue, "tensor_backward: tensor map encode"); return DARKATTN_ERR_CUDA; }
     F.mapK = P.mapK;
-    P.sv = stash.sv; P.delta = fl(Y.delta); P.nK = stash.nK; P.cs = stash.cs; P.rhoc = fl(Y.rhoc);
+    P.sv = stash.sv; P.delta = fl(Y.delta); P.nK = stash.nK; P.cs = stash.cs; P.zc = stash.zc; P.rhoc = fl(Y.rhoc);
     P.espart = fl(Y.espart); P.Tacc = fl(Y.Tacc);
     P.status = reinterpret_cast<int *>(ws + Y.status);
     P.N = D.N; P.H = D.H; P.BH = D.BH; P.m = D.m; P.nslab = Y.nslab; P.T = Y.T;

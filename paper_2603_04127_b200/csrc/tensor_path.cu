@@ -178,6 +178,7 @@ struct MainParams {
     // (Sseg [BH, nsplit, m, DV], zseg [BH, nsplit, m]) instead of adding into Sacc; after an exclusive prefix over the
     // segments the causal kernel of segment s > 0 starts from Sseg[bh, s] (its bf16 copy comes through mapSb).
     float *Sseg, *zseg;
+    float *zc;           // causal: z before chunk t for the backward pass, [BH, T, m] (row 0 not written)
     int *status;
     int N, H, BH, m, nslab, T, nsplit;
 };
@@ -446,11 +447,12 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
             sRed[g * 128 + r] = rowsum + dz;
             // z through this chunk for the next chunk's normaliser (its update completed before the output MMAs did).
             // Written ahead of the barrier below: a warp that runs ahead into the next chunk reads it right away.
-            if (g == 0 && !last) {
+            if (g == 0 && t + 1 < p.T) {        // (also after a segment's last chunk: the next segment's backward needs it)
                 uint32_t v[16];
                 tmem_ld16(lane_addr + kColZ, v);
                 tmem_wait_ld();
                 sZ[r] = __uint_as_float(v[0]);
+                p.zc[((size_t)bh * p.T + t + 1) * p.m + slab * 128 + r] = __uint_as_float(v[0]);
             }
             fence_async_smem();
             tc_fence_before();
@@ -978,6 +980,7 @@ void tensor_make_layout(darkattn_plan_s *plan)
     Y.zacc = take(off, BH * nstate * m * 4);
     Y.Sb = take(off, BH * nstate * m * dv * 2);
     Y.sv = take(off, BH * N * 8);
+    Y.zc = take(off, D.causal ? BH * (size_t)Y.T * m * 4 : 0);
     plan->launches_fwd = D.causal ? (nsplit > 1 ? 7 : 5) : 7;
     {
         size_t so = 0;
@@ -985,6 +988,7 @@ void tensor_make_layout(darkattn_plan_s *plan)
         Y.sv_nK = take(so, BH * N * 4);
         Y.sv_Om = take(so, (size_t)D.H * m * d * 2);
         Y.sv_cs = take(so, BH * Y.nslab * 4);
+        Y.sv_zc = take(so, D.causal ? BH * (size_t)Y.T * m * 4 : 0);
         Y.sv_bytes = so;
         plan->saved_bytes = so;
     }
@@ -1061,7 +1065,7 @@ darkattn_status_t tensor_forward(const darkattn_plan_s *plan, const void *Q, con
     cudaError_t e = tensor_prologue(plan, K, M, W, ws, stash, st);
     auto chk = [&]() { cudaError_t x = cudaGetLastError(); if (x != cudaSuccess && e == cudaSuccess) e = x; };
 
-    P.nK = stash.nK; P.cs = stash.cs; P.pdr = fl(Y.pdr); P.Sacc = fl(Y.Sacc); P.zacc = fl(Y.zacc);
+    P.nK = stash.nK; P.cs = stash.cs; P.zc = stash.zc; P.pdr = fl(Y.pdr); P.Sacc = fl(Y.Sacc); P.zacc = fl(Y.zacc);
     P.status = reinterpret_cast<int *>(ws + Y.status);
     P.N = D.N; P.H = D.H; P.BH = D.BH; P.m = D.m; P.nslab = Y.nslab; P.T = Y.T; P.nsplit = Y.nsplit;
     const int units = (int)(BH * Y.nslab);
