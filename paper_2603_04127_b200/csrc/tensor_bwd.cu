@@ -69,7 +69,7 @@ constexpr uint32_t kColState = 0, kColT = 128, kColR1 = 256, kColR2 = 384;
 // K-major 16 x 128 bf16 operand (two atoms of 2 KB): step k covers 16 elements of K
 __device__ __forceinline__ uint64_t vecdesc(const TileDesc &t, int k) { return t.kmaj + (uint64_t)(((k / 4) * 2048 + (k % 4) * 32) >> 4); }
 
-enum QBars { QB_OM, QB_Q, QB_K, QB_V, QB_G, QB_X2, QM1, QM2, QM3, QMR, QMS, QM4, QM5, QM6, QE0, QE1, QE2, QE3, QE4, QNBARS };
+enum QBars { QB_OM, QB_Q, QB_K, QB_V, QB_G, QB_X2, QM1, QM2, QM3, QMS, QM4, QM5, QM6, QE0, QE1, QE2A, QE2, QE3, QE4, QNBARS };
 
 // ------------------------------------------------------------------ query side (forward direction)
 template <int D, int DV>
@@ -128,8 +128,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
 
             // Schedule of one chunk (R1, R2: the two scratch regions of TMEM). U_K of the next chunk is issued in
             // the tail of the current one, and dO V^T runs while the epilogue is still busy with A^.
-            //   R2: U_K -> (Bf read) -> dO V^T -> packed dP (A operand of dP Bf) -> U_K of the next chunk
-            //   R1: U_Q -> (A^ read) -> rho_c (16 columns) -> dP Bf + dO S^T -> (E read) -> E Omega -> (dQ read)
+            //   R2: U_K -> (Bf read) -> dO V^T -> packed dP in [0,64) (A operand of dP Bf), rho_c in [64,80) -> U_K of the next chunk
+            //   R1: U_Q -> (A^ read) -> dP Bf + dO S^T -> (E read) -> E Omega -> (dQ read)
             bool ok = wait_or_abort(bars + QB_OM, 0, status, abort_flag);
             if (ok) ok = wait_or_abort(bars + QB_K, 0, status, abort_flag);
             if (ok) {
@@ -154,10 +154,10 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColState, mndesc(tKB, k), mndesc(tV, k), id_state, (!first) || k > 0);   // S += Bf^T V
                 mma_commit(bars + QMS);
                 QWAIT(QE1); if (!ok) break;                                                                      // A^ in smem, R1 read
+                QWAIT(QE2A); if (!ok) break;                                                                     // dO V^T read out of R2
                 tc_fence_after();
-                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R1, mndesc(tQA, k), vecdesc(tDel, k), id_vec, k > 0);       // rho_c = -A^^T delta (columns 0, 1)
-                mma_commit(bars + QMR);
-                QWAIT(QE2); if (!ok) break;                                                                      // dP packed in R2, rho_c read
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R2 + 64, mndesc(tQA, k), vecdesc(tDel, k), id_vec, k > 0);  // rho_c = -A^^T delta (columns 0, 1)
+                QWAIT(QE2); if (!ok) break;                                                                      // dP packed in R2
                 tc_fence_after();
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R1, R2 + k * 8, mndesc(tKB, k), id_tm, k > 0);               // dP Bf
                 if (!first)
@@ -206,6 +206,11 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
             const float aq = svv.y - cshift + log2f(svv.x);
             // z before the next chunk, from the forward pass (loaded early, used at the end of the chunk)
             const float znext = (g0 && !last) ? __ldg(p.zc + ((size_t)bh * T + t + 1) * p.m + slab * 128 + r) : 0.f;
+            float dtile[4] = {0.f, 0.f, 0.f, 0.f};       // warp 0: -delta of rows lane, lane + 32, ... for the operand of rho_c
+            if (warp == 0) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) dtile[i] = -__ldg(p.delta + (size_t)row0 + (size_t)t * 128 + i * 32 + lane);
+            }
             EWAIT(QM2); if (!ok) break;
             tc_fence_after();
             features_to_tile(R2 + col0, nk, sKB, r, col0);                             // Bf
@@ -218,7 +223,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const int k = i * 32 + lane;
-                    const float dk = -__ldg(p.delta + (size_t)row0 + (size_t)t * 128 + k);
+                    const float dk = dtile[i];
                     const __nv_bfloat16 hi = __float2bfloat16_rn(dk);
                     const __nv_bfloat16 lo = __float2bfloat16_rn(dk - __bfloat162float(hi));
                     const int atom = k >> 6, kk = k & 63, ch = kk >> 3;
@@ -242,6 +247,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                 uint32_t v[32], pk[16];
                 tmem_ld32(R2 + col0, v);
                 tmem_wait_ld();
+                tc_fence_before();
+                mbar_arrive_warp(bars + QE2A);
                 quarter_sync(q4);                         // every column group has read before anyone overwrites
 #pragma unroll
                 for (int j = 0; j < 32; j += 2) {
@@ -252,19 +259,17 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                 tmem_st16(R2 + col0 / 2, pk);
             }
             tmem_wait_st();
-            if (g0) {       // rho_c of feature r (TMEM lane r), for the key-side kernel
-                EWAIT(QMR); if (!ok) break;
-                tc_fence_after();
-                uint32_t v[16];
-                tmem_ld16(R1, v);
-                tmem_wait_ld();
-                p.rhoc[((size_t)bh * T + t) * p.m + slab * 128 + r] = __uint_as_float(v[0]) + __uint_as_float(v[1]);
-            }
             tc_fence_before();
             mbar_arrive_warp(bars + QE2);
 
             EWAIT(QM4); if (!ok) break;
             tc_fence_after();
+            if (g0) {       // rho_c of feature r (TMEM lane r; its MMAs ran ahead of dP Bf), for the key-side kernel
+                uint32_t v[16];
+                tmem_ld16(R2 + 64, v);
+                tmem_wait_ld();
+                p.rhoc[((size_t)bh * T + t) * p.m + slab * 128 + r] = __uint_as_float(v[0]) + __uint_as_float(v[1]);
+            }
             {   // E = A^ .* (dP Bf + dO S^T - delta z^T), in place over A^
                 uint32_t v[32];
                 tmem_ld32(R1 + col0, v);

@@ -165,6 +165,15 @@ def test_tensor_path_backward(binding, name, kw, use_saved):
     _compare(got, _oracle(t, wl), TOL["bf16"], name)
 
 
+def test_tensor_path_per_head_projections_and_scale(binding):
+    wl = inputs.small(name="t_wph", wid=77, B=2, H=3, N=384, d=64, m=256, causal=True, dtype="bf16", backward=True)
+    t = inputs.generate(wl)
+    rng = np.random.default_rng(11)
+    t.W = inputs.round_to_bf16(rng.standard_normal((3, 256, 64))).astype(np.float64)
+    got = run_gpu(binding, wl, t, path=binding.PATH_TENSOR, scale=0.2, w_per_head=True, use_saved=True)
+    _compare(got, _oracle(t, wl, scale=0.2), TOL["bf16"], "t_wph")
+
+
 def test_headline_backward_sampled_heads(binding):
     """Forward + backward at the benchmark's full size; dQ, dK, dV of sampled (batch, head) pairs and
     the gradient of M of one head (summed over the whole batch) against the oracle."""
