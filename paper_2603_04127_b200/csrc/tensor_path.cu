@@ -1002,7 +1002,9 @@ void tensor_make_layout(darkattn_plan_s *plan)
         plan->launches_bwd = 1 + 2 + 1 + 1;   // delta, two scan kernels, dK finishing, dM (with `saved`; without it the forward launches come on top)
     }
     Y.total_bytes = off;
-    if (Y.total_bytes > plan->workspace_bytes) plan->workspace_bytes = Y.total_bytes;
+    // causal plans run entirely on the tensor kernels; the non-causal backward still needs the FP32 path's layout
+    if (D.causal) plan->workspace_bytes = Y.total_bytes;
+    else if (Y.total_bytes > plan->workspace_bytes) plan->workspace_bytes = Y.total_bytes;
 }
 
 cudaError_t tensor_prologue(const darkattn_plan_s *plan, const void *K, const void *M, const void *W, char *ws,
