@@ -151,8 +151,6 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                 tc_fence_after();
                 _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R2, kdesc(tG, k), kdesc(tV, k), id_kk, k > 0);         // dO V^T
                 mma_commit(bars + QM3);
-                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColState, mndesc(tKB, k), mndesc(tV, k), id_state, (!first) || k > 0);   // S += Bf^T V
-                mma_commit(bars + QMS);
                 QWAIT(QE1); if (!ok) break;                                                                      // A^ in smem, R1 read
                 QWAIT(QE2A); if (!ok) break;                                                                     // dO V^T read out of R2
                 tc_fence_after();
@@ -163,7 +161,10 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                 if (!first)
                     _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R1, kdesc(tG, k), kdesc(tSt, k), id_kk, 1);        // + dO S_prev^T
                 mma_commit(bars + QM4);
-                QWAIT(QM4); if (!ok) break;
+                // the state update is not on the chunk's critical path: it runs while the epilogue forms E
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColState, mndesc(tKB, k), mndesc(tV, k), id_state, (!first) || k > 0);   // S += Bf^T V
+                mma_commit(bars + QMS);
+                QWAIT(QMS); if (!ok) break;                                                                      // (also: dP Bf before it is done)
                 load_tile(sG, &p.mapQ, bars + QB_X2, D, t);                                                     // Q again, for T
                 if (!last) { load_tile(sV, &p.mapV, bars + QB_V, DV, t + 1); load_tile(sKB, &p.mapK, bars + QB_K, D, t + 1); }
                 QWAIT(QE3); if (!ok) break;
@@ -415,8 +416,6 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
                 tc_fence_after();
                 _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R1, kdesc(tV, k), kdesc(tG, k), id_kk, k > 0);         // V dO^T
                 mma_commit(bars + KM3);
-                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColState, mndesc(tQA, k), mndesc(tG, k), id_state, (!first) || k > 0);   // R += A^^T dO
-                mma_commit(bars + KM5);
                 KWAIT(KE1); if (!ok) break;                                                                      // Bf in smem, R2 read
                 tc_fence_after();
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R2, kdesc(tKB, k), kdesc(tQA, k), id_kk, k > 0);             // P^^T = Bf A^^T
@@ -427,6 +426,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
                 if (!first)
                     _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R2, kdesc(tKB, k), mndesc(tSt, k), id_dv_t, 1);          // + Bf R_next
                 mma_commit(bars + KM6);
+                // the state update is not on the chunk's critical path: it runs while dV is read out
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColState, mndesc(tQA, k), mndesc(tG, k), id_state, (!first) || k > 0);   // R += A^^T dO
+                mma_commit(bars + KM5);
                 KWAIT(KE3); if (!ok) break;
                 tc_fence_after();
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R2, R1 + k * 8, mndesc(tQA, k), id_tm, k > 0);               // dP^T A^
@@ -581,7 +583,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
                 }
                 tma_store_commit();
             }
-            if (!last) {     // R (its update completed before KM6) -> bf16 copy; rho_next for the chunk below
+            if (!last) {     // R (updated behind the dV MMAs, before KM7) -> bf16 copy; rho_next for the chunk below
                 if (col0 < DV) tmem_row_to_tile(lane_addr + kColState + col0, sSt, r, col0);
                 if (g0) sRho[r] += rho_c;
                 fence_async_smem();

@@ -358,15 +358,16 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
                 mma_commit(bars + CM3);
                 if (!first)
                     _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R2, FQ + k * 8, mndesc(tSb, k), id_o, k > 0);            // O = phi(Q) S_prev
+                // z += phi(K)^T 1 now: its operand of ones lies in the staging tile, which the output read-out overwrites
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColZ, mndesc(tFK, k), ones_desc, id_z, (!first) || k > 0);
                 CWAIT(CB_V); if (!ok) break;
-                tc_fence_after();
-                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColS, mndesc(tFK, k), mndesc(tV, k), id_s, (!first) || k > 0);   // S += phi(K)^T V
-                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColZ, mndesc(tFK, k), ones_desc, id_z, (!first) || k > 0);       // z += phi(K)^T 1
-                mma_commit(bars + CMS);
                 CWAIT(CE2); if (!ok) break;                                     // tril(P) packed in R1
                 tc_fence_after();
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R2, R1 + k * 8, mndesc(tV, k), id_o, (!first) || k > 0);     // O += P V
                 mma_commit(bars + CM4);
+                // the state update is not on the chunk's critical path: it runs while the output tile is read out
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColS, mndesc(tFK, k), mndesc(tV, k), id_s, (!first) || k > 0);   // S += phi(K)^T V
+                mma_commit(bars + CMS);
                 if (!last) {
                     ok = wait_or_abort(bars + CB_Q, ph ^ 1, status, abort_flag);
                     if (!ok) break;
@@ -374,7 +375,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
                     _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R1, kdesc(tQ, k), kdesc(tOm, k), id_kk, k > 0);     // U_Q of the next chunk
                     mma_commit(bars + CM1);
                 }
-                CWAIT(CM4); if (!ok) break;
+                CWAIT(CMS); if (!ok) break;                                     // (also: the output MMAs before it are done)
                 if (!last) load_tile(sV, &p.mapV, bars + CB_V, DV, t + 1);
                 CWAIT(CE3); if (!ok) break;
                 CWAIT(CE4); if (!ok) break;
@@ -445,15 +446,6 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
                 store_row_f32x32_bf16(v, sStg, r, col0);
             }
             sRed[g * 128 + r] = rowsum + dz;
-            // z through this chunk for the next chunk's normaliser (its update completed before the output MMAs did).
-            // Written ahead of the barrier below: a warp that runs ahead into the next chunk reads it right away.
-            if (g == 0 && t + 1 < p.T) {        // (also after a segment's last chunk: the next segment's backward needs it)
-                uint32_t v[16];
-                tmem_ld16(lane_addr + kColZ, v);
-                tmem_wait_ld();
-                sZ[r] = __uint_as_float(v[0]);
-                p.zc[((size_t)bh * p.T + t + 1) * p.m + slab * 128 + r] = __uint_as_float(v[0]);
-            }
             fence_async_smem();
             tc_fence_before();
             mbar_arrive_warp(bars + CE3);
@@ -474,6 +466,14 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
                 if (col0 < DV) tmem_row_to_tile(lane_addr + kColS + col0, sSb, r, col0);
                 fence_async_smem();
             }
+            if (g == 0 && t + 1 < p.T) {        // z through this chunk: the next chunk's normaliser term, and the backward pass's
+                uint32_t v[16];                 // (also after a segment's last chunk: the next segment's backward needs it)
+                tmem_ld16(lane_addr + kColZ, v);
+                tmem_wait_ld();
+                sZ[r] = __uint_as_float(v[0]);
+                p.zc[((size_t)bh * p.T + t + 1) * p.m + slab * 128 + r] = __uint_as_float(v[0]);
+            }
+            epi_sync();       // a warp that runs ahead into the next chunk reads every z right away
             tc_fence_before();
             mbar_arrive_warp(bars + CE4);
 #undef EWAIT
