@@ -207,17 +207,15 @@ def main():
     import torch.distributed as dist
     from paper_2603_04127_b200 import binding
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2603_04127_b200 import sharding
+    rank, world, local = sharding.env_rank_world()
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     B, H, N, d, r, m, dv = wl.dims()
     # every rank draws its own batch (weak scaling): shift the workload id by the rank
-    wl_rank = inputs.Workload(**{**wl.__dict__, "wid": wl.wid + 100 * rank})
-    t = inputs.generate(wl_rank)
+    t = inputs.generate(sharding.rank_workload(wl, rank))
     dt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
 
     def host(a):
@@ -243,8 +241,7 @@ def main():
         binding.darkattn_forward(plan, Q, K, V, M, W, O, ws, saved=saved, stream=stream)
         if wl.backward:
             binding.darkattn_backward(plan, Q, K, V, M, W, O, G, dQ, dK, dV, dM, ws, saved=saved, stream=stream)
-            if world > 1:
-                dist.all_reduce(dM)
+            sharding.all_reduce_dm(dM)
 
     # End to end: every step copies its inputs from pinned host memory, runs, and copies its results back. Two sets
     # of device buffers and three streams (upload, compute, download) let the upload of step i+1 and the download of
@@ -280,8 +277,7 @@ def main():
             g = st["in"][5]
             dq, dk, dv_, dm_ = st["out"][1:]
             binding.darkattn_backward(plan, q, k, v, mm, ww, o, g, dq, dk, dv_, dm_, ws, saved=saved, stream=stream)
-            if world > 1:
-                dist.all_reduce(dm_)
+            sharding.all_reduce_dm(dm_)
         st["computed"].record(stream)
         with torch.cuda.stream(s_out):
             s_out.wait_event(st["computed"])
@@ -305,10 +301,7 @@ def main():
         torch.cuda.synchronize()
         if world > 1:
             dist.barrier()
-        ms = torch.tensor([e0.elapsed_time(e1)], device="cuda")
-        if world > 1:
-            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-        return float(ms.item())
+        return sharding.max_over_ranks(e0.elapsed_time(e1), device="cuda")
 
     for _ in range(args.warmup):
         step()
@@ -340,7 +333,7 @@ def main():
 
     ms_step = ms / args.steps
     tokens = B * N
-    value = world * tokens / (ms_step * 1e-3)
+    value = sharding.job_throughput(tokens, world, ms_step * 1e-3)
     h2d = sum(x.numel() * x.element_size() for x in (hQ, hK, hV, hM, hW) + ((hG,) if wl.backward else ()))
     d2h = hO.numel() * hO.element_size() + (sum(x.numel() * x.element_size() for x in (hdQ, hdK, hdV, hdM)) if wl.backward else 0)
 
