@@ -112,6 +112,16 @@ darkattn_status_t darkattn_backward(darkattn_plan_t plan, const void *Q, const v
                                     const void *saved /* nullable */, void *dQ, void *dK, void *dV,
                                     float *dM, void *workspace, void *cuda_stream);
 
+/* Gradient of L with respect to the projection rows W, for the variant of the model that trains them (the
+ * learned-feature kernel the paper compares against, Section 5: the random projections are replaced by
+ * trainable vectors). Chain rule through u_l = w_l . x~: dW_l = sum_i (dphi .* phi)_il x~_i over queries and keys,
+ * batches (and heads, when W is shared by the heads).
+ * Call it after darkattn_backward, with the same plan, M and `workspace` and nothing else run on that workspace in
+ * between: it is computed from accumulators that call left there. dW is float32, laid out like W ([m, r], or
+ * [H, m, r] when desc.w_per_head != 0), OVERWRITTEN. Asynchronous on `cuda_stream`.                           */
+darkattn_status_t darkattn_backward_dw(darkattn_plan_t plan, const void *M, float *dW, void *workspace,
+                                       void *cuda_stream);
+
 /* Synchronise `cuda_stream`, then read the device status word kept at the start of `workspace`
  * (written by kernels whose bounded waits gave up, or that met a normaliser that is zero or not
  * finite). Returns DARKATTN_OK, DARKATTN_ERR_TIMEOUT, DARKATTN_ERR_NONFINITE or DARKATTN_ERR_CUDA.  */

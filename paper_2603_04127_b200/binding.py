@@ -24,6 +24,7 @@ EXPORTS = [
     "darkattn_plan_launches", "darkattn_forward", "darkattn_backward", "darkattn_last_device_status",
     "darkattn_destroy", "darkattn_status_string", "darkattn_last_cuda_error", "darkattn_measure_alu_peak",
     "darkattn_static_scratch_needed", "darkattn_forward_static", "darkattn_kernel_timing", "darkattn_kernel_times",
+    "darkattn_backward_dw",
 ]
 STATIC_SCRATCH_BYTES = 16 << 20
 
@@ -55,6 +56,8 @@ lib.darkattn_forward.argtypes = [_vp] * 10
 lib.darkattn_forward.restype = ctypes.c_int
 lib.darkattn_backward.argtypes = [_vp] * 15
 lib.darkattn_backward.restype = ctypes.c_int
+lib.darkattn_backward_dw.argtypes = [_vp] * 5
+lib.darkattn_backward_dw.restype = ctypes.c_int
 lib.darkattn_last_device_status.argtypes = [_vp, _vp, _vp]
 lib.darkattn_last_device_status.restype = ctypes.c_int
 lib.darkattn_destroy.argtypes = [_vp]
@@ -158,6 +161,14 @@ def darkattn_backward(plan: Plan, Q, K, V, M, W, O, dO, dQ, dK, dV, dM, workspac
                                  _ptr(saved), _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(dM), _ptr(workspace),
                                  _stream(stream)), "darkattn_backward")
     return dQ, dK, dV, dM
+
+
+def darkattn_backward_dw(plan: Plan, M, dW, workspace, stream=None):
+    """Gradient of the projection rows W, from what the preceding darkattn_backward left in ``workspace``."""
+    assert dW.dtype == torch.float32
+    _check(lib.darkattn_backward_dw(plan.handle, _ptr(M), _ptr(dW), _ptr(workspace), _stream(stream)),
+           "darkattn_backward_dw")
+    return dW
 
 
 def darkattn_last_device_status(plan: Plan, workspace, stream=None) -> int:

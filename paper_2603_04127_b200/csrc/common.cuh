@@ -46,6 +46,7 @@ struct SimtLayout {
     size_t dxtQ, dxtK;             // dx~                        [BH, N, r]
     size_t dXf;                    // fp32 dX before the cast    [BH, N, d]
     size_t dMp;                    // per-(b,h) dM               [BH, r, d]
+    size_t dWp;                    // per-(b,h) dW               [BH, m, r]
     size_t fwd_bytes, total_bytes;
 };
 
@@ -154,6 +155,9 @@ darkattn_status_t tensor_forward(const darkattn_plan_s *plan, const void *Q, con
 // Folded projections, key-side shifts and key norms (written to `out`).
 cudaError_t tensor_prologue(const darkattn_plan_s *plan, const void *K, const void *M, const void *W, char *ws,
                             const Stash &out, cudaStream_t st);
+// dW from what the last backward call left in the workspace
+darkattn_status_t simt_backward_dw(const darkattn_plan_s *plan, float *dW, char *ws, cudaStream_t st);
+darkattn_status_t tensor_backward_dw(const darkattn_plan_s *plan, const void *M, float *dW, char *ws, cudaStream_t st);
 darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, const void *K, const void *V,
                                   const void *M, const void *W, const void *O, const void *dO, const void *saved,
                                   void *dQ, void *dK, void *dV, float *dM, char *ws, cudaStream_t st);

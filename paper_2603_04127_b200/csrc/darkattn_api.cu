@@ -137,6 +137,18 @@ darkattn_status_t darkattn_backward(darkattn_plan_t plan, const void *Q, const v
     return rc;
 }
 
+darkattn_status_t darkattn_backward_dw(darkattn_plan_t plan, const void *M, float *dW, void *workspace, void *cuda_stream)
+{
+    if (!plan || !M || !dW || !workspace) return DARKATTN_ERR_INVALID_ARG;
+    if (!aligned16(M) || !aligned16(dW) || !aligned16(workspace)) return DARKATTN_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    darkattn_status_t rc = plan->path == DARKATTN_PATH_TENSOR
+                               ? tensor_backward_dw(plan, M, dW, static_cast<char *>(workspace), st)
+                               : simt_backward_dw(plan, dW, static_cast<char *>(workspace), st);
+    timer_mark(plan, st, nullptr);
+    return rc;
+}
+
 darkattn_status_t darkattn_last_device_status(darkattn_plan_t plan, const void *workspace, void *cuda_stream)
 {
     if (!plan || !workspace) return DARKATTN_ERR_INVALID_ARG;

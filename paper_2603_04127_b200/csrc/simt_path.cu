@@ -412,6 +412,7 @@ void simt_make_layout(darkattn_plan_s *plan)
     Y.dxtQ = take(off, BH * N * r); Y.dxtK = take(off, BH * N * r);
     Y.dXf = take(off, BH * N * d);
     Y.dMp = take(off, BH * r * d);
+    Y.dWp = take(off, BH * m * r);
     Y.total_bytes = off;
 }
 
@@ -487,6 +488,41 @@ darkattn_status_t simt_backward(const darkattn_plan_s *plan, const void *Q, cons
     }
     reduce_batch_kernel<<<(unsigned)(((long long)D.H * r * d + 255) / 256), 256, 0, st>>>(F(Y.dMp), dM, D.B, (long long)D.H * r * d, (long long)D.H * r * d); L.check();
     if (L.err != cudaSuccess) { set_cuda_error(L.err, "simt_backward"); return DARKATTN_ERR_CUDA; }
+    return DARKATTN_OK;
+}
+
+// dW_l = sum_i E_il x~_i over queries and keys: E (in the buffers dA, dBf) and x~ are still in the workspace after
+// simt_backward. Per (b,h) products, then the sum over the batch (and over the heads when W is shared).
+__global__ void reduce_dw_kernel(const float *dWp, float *dW, int B, int H, long long per_head, int w_per_head, long long total)
+{
+    const long long t = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+    if (t >= total) return;
+    float acc = 0.f;
+    if (w_per_head) {
+        const long long h = t / per_head, e = t % per_head;
+        for (int b = 0; b < B; ++b) acc += dWp[((long long)b * H + h) * per_head + e];
+    } else {
+        for (int bh = 0; bh < B * H; ++bh) acc += dWp[(long long)bh * per_head + t];
+    }
+    dW[t] = acc;
+}
+
+darkattn_status_t simt_backward_dw(const darkattn_plan_s *plan, float *dW, char *ws, cudaStream_t st)
+{
+    const Dims &D = plan->dims;
+    const SimtLayout &Y = plan->simt;
+    const long long BH = D.BH, N = D.N, Np = D.Npad, r = D.r, m = D.m;
+    auto F = [&](size_t off) { return reinterpret_cast<float *>(ws + off); };
+    Launcher L{st};
+    for (int side = 0; side < 2; ++side) {
+        const float *E = F(side ? Y.dBf : Y.dA), *xt = F(side ? Y.xtK : Y.xtQ);
+        // dWp_(b,h) (+)= E^T x~   [m x r], contraction over the N tokens (padding rows of E are zero, but x~ has only N rows)
+        L.gemm(E, xt, F(Y.dWp), (int)m, (int)r, (int)N, 1, m, r, 1, r, 1, BH, 1, Np * m, 0, N * r, 0, m * r, 0, 1.f, side, 0);
+    }
+    const long long per_head = m * r, total = (D.w_per_head ? D.H : 1) * per_head;
+    reduce_dw_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(F(Y.dWp), dW, D.B, D.H, per_head, D.w_per_head, total);
+    L.check();
+    if (L.err != cudaSuccess) { set_cuda_error(L.err, "simt_backward_dw"); return DARKATTN_ERR_CUDA; }
     return DARKATTN_OK;
 }
 

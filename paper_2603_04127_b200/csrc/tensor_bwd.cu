@@ -870,6 +870,26 @@ __global__ void dm_kernel(const __nv_bfloat16 *W, const float *Tacc, const float
         }
 }
 
+// dW[(h,) l, a] = s * sum_c T[h,l,c] M[h,a,c], summed over the heads when W is shared: through the folded projection
+// u_l = s w_l . (M x) the gradient of w_l is s M (sum_i E_il x_i). One block per row l (and head), one thread per a.
+__global__ void dw_kernel(const float *Tacc, const __nv_bfloat16 *M, float *dW, int H, int m, int r, int d, int w_per_head, float s)
+{
+    const int l = blockIdx.x, a = threadIdx.x;
+    const int h0 = w_per_head ? blockIdx.y : 0, h1 = w_per_head ? blockIdx.y + 1 : H;
+    float acc = 0.f;
+    for (int h = h0; h < h1; ++h) {
+        const float *T = Tacc + ((size_t)h * m + l) * d;
+        const __nv_bfloat16 *Ma = M + ((size_t)h * r + a) * d;
+        for (int c = 0; c < d; c += 8) {
+            float f[8];
+            unpack8(*reinterpret_cast<const uint4 *>(Ma + c), f);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc = fmaf(T[c + j], f[j], acc);
+        }
+    }
+    dW[((size_t)(w_per_head ? blockIdx.y : 0) * m + l) * r + a] = s * acc;
+}
+
 template <int D, int DV>
 cudaError_t launch_scan(const darkattn_plan_s *plan, const BwdParams &P, int grid, cudaStream_t st)
 {
@@ -999,6 +1019,19 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
     dm_kernel<<<dim3((D.r + 7) / 8, D.H, D.m / 64), D.d, 0, st>>>((const __nv_bfloat16 *)W, fl(Y.Tacc), fl(Y.dMn), dM, D.m, D.r, D.d, D.w_per_head, D.s);
     chk();
     if (e != cudaSuccess) { set_cuda_error(e, "tensor_backward"); return DARKATTN_ERR_CUDA; }
+    return DARKATTN_OK;
+}
+
+darkattn_status_t tensor_backward_dw(const darkattn_plan_s *plan, const void *M, float *dW, char *ws, cudaStream_t st)
+{
+    const Dims &D = plan->dims;
+    const TensorLayout &Y = plan->tensor;
+    if (!D.causal) return simt_backward_dw(plan, dW, ws, st);     // that backward ran on the FP32 path
+    timer_mark(plan, st, "dw_kernel");
+    dw_kernel<<<dim3(D.m, D.w_per_head ? D.H : 1), D.r, 0, st>>>(reinterpret_cast<const float *>(ws + Y.Tacc), (const __nv_bfloat16 *)M, dW,
+                                                                D.H, D.m, D.r, D.d, D.w_per_head, D.s);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { set_cuda_error(e, "tensor_backward_dw"); return DARKATTN_ERR_CUDA; }
     return DARKATTN_OK;
 }
 

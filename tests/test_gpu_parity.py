@@ -174,6 +174,22 @@ def test_tensor_path_per_head_projections_and_scale(binding):
     _compare(got, _oracle(t, wl, scale=0.2), TOL["bf16"], "t_wph")
 
 
+@pytest.mark.parametrize("case", ["simt_f32", "simt_f32_noncausal_wph", "tensor", "tensor_wph"])
+def test_gradient_of_the_projection_rows(binding, case):
+    wph = case.endswith("wph")
+    tensor = case.startswith("tensor")
+    kw = dict(B=2, H=3, N=384, d=64, m=256, causal=True) if tensor else dict(B=2, H=2, N=150, d=24, m=40, r=16, causal="noncausal" not in case)
+    wl = inputs.small(name=case, wid=81, dtype="bf16" if tensor else "f32", backward=True, **kw)
+    t = inputs.generate(wl)
+    if wph:
+        rng = np.random.default_rng(12)
+        W = rng.standard_normal((wl.H,) + t.W.shape)
+        t.W = inputs.round_to_bf16(W).astype(np.float64) if tensor else W.astype(np.float32).astype(np.float64)
+    got = run_gpu(binding, wl, t, path=binding.PATH_TENSOR if tensor else binding.PATH_SIMT, w_per_head=wph, want_dw=True)
+    want = ref.backward(t.Q, t.K, t.V, t.M, t.W, t.dO, causal=wl.causal)[4]
+    assert_close(got["dW"], want, TOL[wl.dtype], f"{case}: dW")
+
+
 def test_headline_backward_sampled_heads(binding):
     """Forward + backward at the benchmark's full size; dQ, dK, dV of sampled (batch, head) pairs and
     the gradient of M of one head (summed over the whole batch) against the oracle."""

@@ -18,7 +18,7 @@ def torch_dtype(name):
     return torch.float32 if name == "f32" else torch.bfloat16
 
 
-def run_gpu(binding, wl, t, path=0, chunk=0, scale=0.0, backward=None, w_per_head=False, use_saved=False):
+def run_gpu(binding, wl, t, path=0, chunk=0, scale=0.0, backward=None, w_per_head=False, use_saved=False, want_dw=False):
     """Run forward (and backward) on the device for tensors ``t`` laid out [B', H', N, *].
 
     With ``use_saved`` the forward call fills the plan's forward->backward stash and the backward call
@@ -47,6 +47,10 @@ def run_gpu(binding, wl, t, path=0, chunk=0, scale=0.0, backward=None, w_per_hea
                                   saved=saved)
         for k, v in (("dQ", dQ), ("dK", dK), ("dV", dV), ("dM", dM)):
             out[k] = v.float().cpu().numpy().astype(np.float64)
+        if want_dw:
+            dW = torch.empty(W.shape, dtype=torch.float32, device="cuda")
+            binding.darkattn_backward_dw(plan, M, dW, ws)
+            out["dW"] = dW.cpu().numpy().astype(np.float64)
     assert binding.darkattn_last_device_status(plan, ws) == binding.OK
     torch.cuda.synchronize()
     plan.destroy()
