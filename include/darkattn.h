@@ -122,6 +122,20 @@ darkattn_status_t darkattn_backward(darkattn_plan_t plan, const void *Q, const v
 darkattn_status_t darkattn_backward_dw(darkattn_plan_t plan, const void *M, float *dW, void *workspace,
                                        void *cuda_stream);
 
+/* One decode step of causal attention in its recurrent form. Section 2 ("Efficient Attention via Random Feature
+ * Kernels") evaluates the attention as phi(Q) (phi(K)^T V) without forming the L x L matrix; with the causal mask the
+ * same ordering, taken one token at a time, needs only the running sums S = sum_{j<=i} phi(k_j) v_j^T and
+ * z = sum_{j<=i} phi(k_j) (the Discussion names long-context use as a direction). For every (batch, head) this call
+ * adds the new token's key and value to the caller's running state and returns the new token's output,
+ *     S += phi(k) v^T,   z += phi(k),   o = phi(q)^T S / phi(q)^T z.
+ * q, k [B, H, d] and v, o [B, H, dv] in desc.dtype; S [B, H, m, dv] and z [B, H, m] float32, owned by the caller and
+ * updated in place: zero them before the first token. The features are scaled by exp(-|w_l|^2/2) (keys) and its
+ * inverse (queries), which cancels in o, is the same at every step and keeps every key feature <= 1; the state is
+ * therefore only meaningful to this call. Needs a causal plan (B, H, d, r, m, dv, dtype, scale, w_per_head are taken
+ * from it; N is not used) with dv a multiple of 32. No workspace. Asynchronous on `cuda_stream`.                  */
+darkattn_status_t darkattn_decode_step(darkattn_plan_t plan, const void *q, const void *k, const void *v, const void *M,
+                                       const void *W, float *S, float *z, void *o, void *cuda_stream);
+
 /* Synchronise `cuda_stream`, then read the device status word kept at the start of `workspace`
  * (written by kernels whose bounded waits gave up, or that met a normaliser that is zero or not
  * finite). Returns DARKATTN_OK, DARKATTN_ERR_TIMEOUT, DARKATTN_ERR_NONFINITE or DARKATTN_ERR_CUDA.  */

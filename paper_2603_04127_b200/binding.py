@@ -24,7 +24,7 @@ EXPORTS = [
     "darkattn_plan_launches", "darkattn_forward", "darkattn_backward", "darkattn_last_device_status",
     "darkattn_destroy", "darkattn_status_string", "darkattn_last_cuda_error", "darkattn_measure_alu_peak",
     "darkattn_static_scratch_needed", "darkattn_forward_static", "darkattn_kernel_timing", "darkattn_kernel_times",
-    "darkattn_backward_dw",
+    "darkattn_backward_dw", "darkattn_decode_step",
 ]
 STATIC_SCRATCH_BYTES = 16 << 20
 
@@ -58,6 +58,8 @@ lib.darkattn_backward.argtypes = [_vp] * 15
 lib.darkattn_backward.restype = ctypes.c_int
 lib.darkattn_backward_dw.argtypes = [_vp] * 5
 lib.darkattn_backward_dw.restype = ctypes.c_int
+lib.darkattn_decode_step.argtypes = [_vp] * 10
+lib.darkattn_decode_step.restype = ctypes.c_int
 lib.darkattn_last_device_status.argtypes = [_vp, _vp, _vp]
 lib.darkattn_last_device_status.restype = ctypes.c_int
 lib.darkattn_destroy.argtypes = [_vp]
@@ -169,6 +171,14 @@ def darkattn_backward_dw(plan: Plan, M, dW, workspace, stream=None):
     _check(lib.darkattn_backward_dw(plan.handle, _ptr(M), _ptr(dW), _ptr(workspace), _stream(stream)),
            "darkattn_backward_dw")
     return dW
+
+
+def darkattn_decode_step(plan: Plan, q, k, v, M, W, S, z, o, stream=None):
+    """One recurrent step: S, z (float32, caller-owned running state) are updated in place, o receives the output."""
+    assert S.dtype == torch.float32 and z.dtype == torch.float32
+    _check(lib.darkattn_decode_step(plan.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(M), _ptr(W), _ptr(S), _ptr(z), _ptr(o),
+                                    _stream(stream)), "darkattn_decode_step")
+    return o
 
 
 def darkattn_last_device_status(plan: Plan, workspace, stream=None) -> int:

@@ -1,0 +1,128 @@
+// Single-token decode step of causal DARK attention: the recurrent form of the causal scan. Per (batch, head) the
+// caller keeps the running state S = sum_j phi(k_j) v_j^T (m x dv) and z = sum_j phi(k_j) (m), both float32; one step
+// adds the new token's key and value and reads the new token's query out:
+//     S += phi(k) v^T,   z += phi(k),   o = phi(q)^T S / phi(q)^T z          (Section 2's ordering phi(Q) (phi(K)^T V), one row at a time)
+// Stabiliser (cancels in o, and is the same at every step, so the state of one step is valid for the next): keys use
+// the per-feature shift c_l = |w_l|^2 / 2, i.e. phi(k)_l = exp(u_l - |x~|^2/2 - c_l) = exp(-|x~ - w_l|^2 / 2) <= 1;
+// queries use exp(u_l + c_l - max_l(u_l + c_l)).
+// The step is bound by the traffic of the state (read and written once): plain SIMT, FP32, coalesced over dv.
+#include "common.cuh"
+
+#include <math.h>
+
+namespace darkattn {
+
+namespace {
+
+template <typename T>
+__device__ __forceinline__ float ldf(const T *p, size_t i)
+{
+    if constexpr (sizeof(T) == 2) return __bfloat162float(p[i]);
+    else return p[i];
+}
+
+// grid = (dv / 32 column blocks, B*H); block = 256 threads = 32 columns x 8 groups of features.
+template <typename T>
+__global__ void __launch_bounds__(256) decode_step_kernel(const T *q, const T *k, const T *v, const T *M, const T *W, float *S,
+                                                           float *z, T *o, int H, int d, int r, int m, int dv, int w_per_head,
+                                                           float s)
+{
+    extern __shared__ float sm[];
+    float *xq = sm, *xk = xq + r, *fq = xk + r, *fk = fq + m, *red = fk + m;   // red: 8 x 32 partial numerators + 8 partial normalisers + scratch
+    const int bh = blockIdx.y, h = bh % H, tid = threadIdx.x;
+    const T *Mh = M + (size_t)h * r * d, *Wh = W + (size_t)(w_per_head ? h : 0) * m * r;
+    const T *qv = q + (size_t)bh * d, *kv = k + (size_t)bh * d;
+
+    for (int a = tid; a < r; a += 256) {            // x~ = s M x for the query and the key
+        float aq = 0.f, ak = 0.f;
+        for (int c = 0; c < d; ++c) {
+            const float mv = ldf(Mh, (size_t)a * d + c);
+            aq = fmaf(mv, ldf(qv, c), aq);
+            ak = fmaf(mv, ldf(kv, c), ak);
+        }
+        xq[a] = s * aq;
+        xk[a] = s * ak;
+    }
+    __syncthreads();
+    float nk = 0.f;
+    for (int a = 0; a < r; ++a) nk = fmaf(xk[a], xk[a], nk);
+    nk *= 0.5f;
+    float mx = -INFINITY;
+    for (int l = tid; l < m; l += 256) {            // exponents of the features
+        float uq = 0.f, uk = 0.f, c = 0.f;
+        for (int a = 0; a < r; ++a) {
+            const float w = ldf(Wh, (size_t)l * r + a);
+            uq = fmaf(w, xq[a], uq);
+            uk = fmaf(w, xk[a], uk);
+            c = fmaf(w, w, c);
+        }
+        c *= 0.5f;
+        fk[l] = __expf(uk - nk - c);
+        fq[l] = uq + c;
+        mx = fmaxf(mx, fq[l]);
+    }
+    for (int off = 16; off; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+    if ((tid & 31) == 0) red[tid >> 5] = mx;
+    __syncthreads();
+    mx = red[0];
+    for (int w = 1; w < 8; ++w) mx = fmaxf(mx, red[w]);
+    __syncthreads();
+    for (int l = tid; l < m; l += 256) fq[l] = __expf(fq[l] - mx);
+    __syncthreads();
+
+    // state update and read-out: thread = (column, feature group)
+    const int col = blockIdx.x * 32 + (tid & 31), grp = tid >> 5;
+    const float vv = ldf(v, (size_t)bh * dv + col);
+    float *Sb = S + (size_t)bh * m * dv;
+    float *zb = z + (size_t)bh * m;
+    float num = 0.f, den = 0.f;
+    for (int l = grp; l < m; l += 8) {
+        const float snew = fmaf(fk[l], vv, Sb[(size_t)l * dv + col]);
+        Sb[(size_t)l * dv + col] = snew;
+        num = fmaf(fq[l], snew, num);
+        if ((tid & 31) == 0) {                       // one lane per group carries the normaliser
+            const float znew = zb[l] + fk[l];
+            if (blockIdx.x == 0) zb[l] = znew;       // every column block needs z; one of them stores it
+            den = fmaf(fq[l], znew, den);
+        }
+    }
+    red[grp * 32 + (tid & 31)] = num;
+    if ((tid & 31) == 0) red[256 + grp] = den;
+    __syncthreads();
+    if (tid < 32) {
+        float n = 0.f, dn = 0.f;
+        for (int g = 0; g < 8; ++g) { n += red[g * 32 + tid]; dn += red[256 + g]; }
+        const float out = n / dn;
+        if constexpr (sizeof(T) == 2) o[(size_t)bh * dv + blockIdx.x * 32 + tid] = __float2bfloat16_rn(out);
+        else o[(size_t)bh * dv + blockIdx.x * 32 + tid] = out;
+    }
+}
+
+}  // namespace
+
+}  // namespace darkattn
+
+using namespace darkattn;
+
+extern "C" darkattn_status_t darkattn_decode_step(darkattn_plan_t plan, const void *q, const void *k, const void *v, const void *M,
+                                                  const void *W, float *S, float *z, void *o, void *cuda_stream)
+{
+    if (!plan || !q || !k || !v || !M || !W || !S || !z || !o) return DARKATTN_ERR_INVALID_ARG;
+    const Dims &D = plan->dims;
+    if (!D.causal) return DARKATTN_ERR_UNSUPPORTED;          // the recurrent form is the causal one
+    if (D.dv % 32) return DARKATTN_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const size_t smem = (size_t)(2 * D.r + 2 * D.m + 256 + 16) * sizeof(float);
+    if (smem > 48 * 1024) return DARKATTN_ERR_UNSUPPORTED;
+    const dim3 grid(D.dv / 32, D.BH);
+    if (D.bf16)
+        decode_step_kernel<__nv_bfloat16><<<grid, 256, smem, st>>>((const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k, (const __nv_bfloat16 *)v,
+                                                                  (const __nv_bfloat16 *)M, (const __nv_bfloat16 *)W, S, z, (__nv_bfloat16 *)o,
+                                                                  D.H, D.d, D.r, D.m, D.dv, D.w_per_head, D.s);
+    else
+        decode_step_kernel<float><<<grid, 256, smem, st>>>((const float *)q, (const float *)k, (const float *)v, (const float *)M,
+                                                           (const float *)W, S, z, (float *)o, D.H, D.d, D.r, D.m, D.dv, D.w_per_head, D.s);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { set_cuda_error(e, "decode_step"); return DARKATTN_ERR_CUDA; }
+    return DARKATTN_OK;
+}

@@ -190,6 +190,29 @@ def test_gradient_of_the_projection_rows(binding, case):
     assert_close(got["dW"], want, TOL[wl.dtype], f"{case}: dW")
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_decode_steps_reproduce_the_causal_forward(binding, dtype):
+    """Token by token through the recurrent entry point: step t's output is row t of the causal attention."""
+    import torch
+    from tests.util import to_dev, torch_dtype
+    wl = inputs.small(name="decode", wid=83, B=2, H=3, N=40, d=32, m=96, r=16, dv=64, causal=True, dtype=dtype, backward=False)
+    t = inputs.generate(wl)
+    dt = torch_dtype(dtype)
+    Q, K, V, M, W = (to_dev(x, dt) for x in (t.Q, t.K, t.V, t.M, t.W))
+    plan = binding.darkattn_plan(2, 3, 40, 32, 96, r=16, dv=64, dtype=binding.F32 if dtype == "f32" else binding.BF16, causal=True)
+    S = torch.zeros(2, 3, 96, 64, dtype=torch.float32, device="cuda")
+    z = torch.zeros(2, 3, 96, dtype=torch.float32, device="cuda")
+    rows = []
+    for i in range(wl.N):
+        o = torch.empty(2, 3, 64, dtype=dt, device="cuda")
+        binding.darkattn_decode_step(plan, Q[:, :, i].contiguous(), K[:, :, i].contiguous(), V[:, :, i].contiguous(), M, W, S, z, o)
+        rows.append(o.float().cpu().numpy().astype(np.float64))
+    got = np.stack(rows, axis=2)
+    want = ref.forward(t.Q, t.K, t.V, t.M, t.W, causal=True)
+    assert_close(got, want, 1e-4 if dtype == "f32" else 1e-2, f"decode {dtype}")
+    plan.destroy()
+
+
 def test_headline_backward_sampled_heads(binding):
     """Forward + backward at the benchmark's full size; dQ, dK, dV of sampled (batch, head) pairs and
     the gradient of M of one head (summed over the whole batch) against the oracle."""
