@@ -29,7 +29,7 @@ if ROOT not in sys.path:
 # DRAM bytes (read + write) per (token, head) of the scan kernels at d = dv = 128, m = 256 from their ncu capture on the
 # small profiling workload (profiles/scan_kernels_d128_small.md); traffic is proportional to the (token, head) count.
 # A kernel that changed since its capture has no entry.
-NCU_TRAFFIC_PER_TOKEN_HEAD = {"tc_fwd_causal_kernel": 1073.0, "tc_bwd_q_kernel": 1503.0, "tc_bwd_k_kernel": 1965.0}
+NCU_TRAFFIC_PER_TOKEN_HEAD = {"tc_fwd_causal_kernel": 1083.0, "tc_bwd_q_kernel": 1516.0, "tc_bwd_k_kernel": 1966.0}
 
 METRIC = "DARK-attention fwd+bwd tokens/s"
 UNIT = "tokens/s"
