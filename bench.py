@@ -69,6 +69,8 @@ def kernel_work(d, r, m, dv, C, nslab, causal):
         "tc_fwd_queries_kernel": (feat // 2 + 2 * m * dv, m, (d + dv) * e, "tensor"),
         "tc_bwd_q_kernel": (feat // 2 + 4 * m * dv + tri * (m + dv) + 2 * m * r + 4 * r * d, m, (3 * d + 2 * dv) * e, "tensor"),
         "tc_bwd_k_kernel": (feat // 2 + 6 * m * dv + tri * (2 * m + dv) + 2 * m * r + 4 * r * d, m, (3 * d + 3 * dv) * e, "tensor"),
+        "tc_bwd_nc_q_kernel": (feat // 2 + 4 * m * dv + 2 * m * r + 4 * r * d, m, (2 * d + dv) * e, "tensor"),
+        "tc_bwd_nc_k_kernel": (feat // 2 + 4 * m * dv + 2 * m * r + 4 * r * d, m, (2 * d + 2 * dv) * e, "tensor"),
         "tc_bwd_finish_k_kernel": (6 * r * d, 0, 3 * d * e, "hbm"),
         "tc_key_norms_kernel": (2 * r * d, 0, d * e + 4, "hbm"),
         "combine_kernel": (0, 0, (nslab * dv + dv) * e + nslab * 8, "hbm"),

@@ -85,7 +85,8 @@ size_t darkattn_workspace_bytes(darkattn_plan_t plan);
 
 /* Bytes of the forward->backward stash (`saved`): what the forward pass computed and the backward
  * pass needs again (on the tensor-core path the per-row normalisers, the key norms, the folded
- * projections and the key-side shifts). 0 means there is none. `saved` may always be NULL in both
+ * projections, the key-side shifts and the key-side sums: z before every chunk when causal, S and
+ * z of the whole sequence otherwise). 0 means there is none. `saved` may always be NULL in both
  * calls: backward then recomputes what it needs, at the cost of running the forward kernels again. */
 size_t darkattn_saved_bytes(darkattn_plan_t plan);
 

@@ -69,9 +69,12 @@ struct TensorLayout {
     size_t espart;  // partials of rowsum(E_K) per slab and 32-column group, fp32 [4 nslab, BH, N]
     size_t Tacc;    // sum_i E_i^T x_i over both sides and the batch, fp32 [H, m, d]
     size_t dMn;     // gradient of M through the key norm term, fp32 [H, r, d]
+    size_t Racc;    // non-causal backward: sum of A^^T dO, fp32 [BH, m, dv]; rhot directly behind it
+    size_t rhot;    // non-causal backward: -sum of A^^T delta, fp32 [BH, m]
+    size_t Rb;      // bf16 copy of Racc
     size_t total_bytes;
     // the forward -> backward stash (`saved`): per-row normalisers, key norms, folded projections, key shifts
-    size_t sv_sv, sv_nK, sv_Om, sv_cs, sv_zc, sv_bytes;
+    size_t sv_sv, sv_nK, sv_Om, sv_cs, sv_zc, sv_Sb, sv_zt, sv_bytes;
     size_t zc;      // workspace copy of the stash's per-chunk z (causal): sum_j phi(K)_jl over the chunks before t, fp32 [BH, T, m]
     int nslab, T, nsplit;
 };
@@ -84,19 +87,23 @@ struct Stash {
     __nv_bfloat16 *Om;
     float *cs;
     float *zc;      // causal: z before chunk t, [BH, T, m] (row t = 0 is not written: it is zero)
+    __nv_bfloat16 *Sb;   // non-causal: S of the whole sequence, bf16 [BH, m, dv]
+    float *zt;      // non-causal: z of the whole sequence, [BH, m]
 };
 inline Stash stash_in_workspace(const TensorLayout &Y, char *ws)
 {
     return Stash{reinterpret_cast<float2 *>(ws + Y.sv), reinterpret_cast<float *>(ws + Y.nK),
                  reinterpret_cast<__nv_bfloat16 *>(ws + Y.Om), reinterpret_cast<float *>(ws + Y.cs),
-                 reinterpret_cast<float *>(ws + Y.zc)};
+                 reinterpret_cast<float *>(ws + Y.zc), reinterpret_cast<__nv_bfloat16 *>(ws + Y.Sb),
+                 reinterpret_cast<float *>(ws + Y.zacc)};
 }
 inline Stash stash_in_saved(const TensorLayout &Y, void *saved)
 {
     char *b = static_cast<char *>(saved);
     return Stash{reinterpret_cast<float2 *>(b + Y.sv_sv), reinterpret_cast<float *>(b + Y.sv_nK),
                  reinterpret_cast<__nv_bfloat16 *>(b + Y.sv_Om), reinterpret_cast<float *>(b + Y.sv_cs),
-                 reinterpret_cast<float *>(b + Y.sv_zc)};
+                 reinterpret_cast<float *>(b + Y.sv_zc), reinterpret_cast<__nv_bfloat16 *>(b + Y.sv_Sb),
+                 reinterpret_cast<float *>(b + Y.sv_zt)};
 }
 
 }  // namespace darkattn
@@ -157,6 +164,8 @@ cudaError_t tensor_prologue(const darkattn_plan_s *plan, const void *K, const vo
                             const Stash &out, cudaStream_t st);
 // dW from what the last backward call left in the workspace
 darkattn_status_t simt_backward_dw(const darkattn_plan_s *plan, float *dW, char *ws, cudaStream_t st);
+cudaError_t tensor_backward_nc_passes(const darkattn_plan_s *plan, const void *Q, const void *K, const void *V, const void *dO,
+                                      const Stash &stash, void *dQ, void *dK, void *dV, char *ws, cudaStream_t st);
 darkattn_status_t tensor_backward_dw(const darkattn_plan_s *plan, const void *M, float *dW, char *ws, cudaStream_t st);
 darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, const void *K, const void *V,
                                   const void *M, const void *W, const void *O, const void *dO, const void *saved,

@@ -933,10 +933,6 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
 {
     const Dims &D = plan->dims;
     const TensorLayout &Y = plan->tensor;
-    if (!D.causal) {   // the non-causal backward has no tensor-core kernels: FP32 path, same workspace
-        timer_mark(plan, st, "simt_backward (all kernels)");
-        return simt_backward(plan, Q, K, V, M, W, dO, dQ, dK, dV, dM, ws, st);
-    }
     const size_t BH = D.BH, N = D.N;
     auto bf = [&](size_t off) { return reinterpret_cast<__nv_bfloat16 *>(ws + off); };
     auto fl = [&](size_t off) { return reinterpret_cast<float *>(ws + off); };
@@ -982,32 +978,38 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
         keep(cudaMemsetAsync(dQ, 0, BH * N * D.d * 2, st));
     }
 
-    BwdParams P;
-    memset(&P, 0, sizeof(P));
-    bool ok = make_map(&P.mapQ, Q, BH * N, D.d, 128) && make_map(&P.mapK, K, BH * N, D.d, 128) &&
-              make_map(&P.mapV, V, BH * N, D.dv, 128) && make_map(&P.mapG, dO, BH * N, D.dv, 128) &&
-              make_map(&P.mapOm, stash.Om, (size_t)D.H * D.m, D.d, 128) &&
-              make_map(&P.mapDQ, dQ, BH * N, D.d, 128) && make_map(&P.mapDK, dK, BH * N, D.d, 128) &&
-              make_map(&P.mapDV, dV, BH * N, D.dv, 128);
     FinishParams F;
     memset(&F, 0, sizeof(F));
-    ok = ok && make_map(&F.mapM, M, (size_t)D.H * D.r, D.d, 128);
-    if (!ok) { set_cuda_error(cudaErrorInvalidValue, "tensor_backward: tensor map encode"); return DARKATTN_ERR_CUDA; }
-    F.mapK = P.mapK;
-    P.sv = stash.sv; P.delta = fl(Y.delta); P.nK = stash.nK; P.cs = stash.cs; P.zc = stash.zc; P.rhoc = fl(Y.rhoc);
-    P.espart = fl(Y.espart); P.Tacc = fl(Y.Tacc);
-    P.status = reinterpret_cast<int *>(ws + Y.status);
-    P.N = D.N; P.H = D.H; P.BH = D.BH; P.m = D.m; P.nslab = Y.nslab; P.T = Y.T;
-    const int units = (int)(BH * Y.nslab);
-    if (D.d == 64 && D.dv == 64) keep(launch_scan<64, 64>(plan, P, units, st));
-    else if (D.d == 128 && D.dv == 128) keep(launch_scan<128, 128>(plan, P, units, st));
-    else if (D.d == 64 && D.dv == 128) keep(launch_scan<64, 128>(plan, P, units, st));
-    else keep(launch_scan<128, 64>(plan, P, units, st));
+    if (!make_map(&F.mapM, M, (size_t)D.H * D.r, D.d, 128) || !make_map(&F.mapK, K, BH * N, D.d, 128) ||
+        !make_map(&F.mapP, dK, BH * N, D.d, 128)) {
+        set_cuda_error(cudaErrorInvalidValue, "tensor_backward: tensor map encode");
+        return DARKATTN_ERR_CUDA;
+    }
+    if (D.causal) {
+        BwdParams P;
+        memset(&P, 0, sizeof(P));
+        const bool ok = make_map(&P.mapQ, Q, BH * N, D.d, 128) && make_map(&P.mapK, K, BH * N, D.d, 128) &&
+                        make_map(&P.mapV, V, BH * N, D.dv, 128) && make_map(&P.mapG, dO, BH * N, D.dv, 128) &&
+                        make_map(&P.mapOm, stash.Om, (size_t)D.H * D.m, D.d, 128) &&
+                        make_map(&P.mapDQ, dQ, BH * N, D.d, 128) && make_map(&P.mapDK, dK, BH * N, D.d, 128) &&
+                        make_map(&P.mapDV, dV, BH * N, D.dv, 128);
+        if (!ok) { set_cuda_error(cudaErrorInvalidValue, "tensor_backward: tensor map encode"); return DARKATTN_ERR_CUDA; }
+        P.sv = stash.sv; P.delta = fl(Y.delta); P.nK = stash.nK; P.cs = stash.cs; P.zc = stash.zc; P.rhoc = fl(Y.rhoc);
+        P.espart = fl(Y.espart); P.Tacc = fl(Y.Tacc);
+        P.status = reinterpret_cast<int *>(ws + Y.status);
+        P.N = D.N; P.H = D.H; P.BH = D.BH; P.m = D.m; P.nslab = Y.nslab; P.T = Y.T;
+        const int units = (int)(BH * Y.nslab);
+        if (D.d == 64 && D.dv == 64) keep(launch_scan<64, 64>(plan, P, units, st));
+        else if (D.d == 128 && D.dv == 128) keep(launch_scan<128, 128>(plan, P, units, st));
+        else if (D.d == 64 && D.dv == 128) keep(launch_scan<64, 128>(plan, P, units, st));
+        else keep(launch_scan<128, 64>(plan, P, units, st));
+    } else {
+        keep(tensor_backward_nc_passes(plan, Q, K, V, dO, stash, dQ, dK, dV, ws, st));
+    }
 
-    F.mapP = P.mapDK;
     if (!make_map(&F.mapOut, dK, BH * N, D.d, 128)) { set_cuda_error(cudaErrorInvalidValue, "tensor_backward: tensor map encode"); return DARKATTN_ERR_CUDA; }
     F.espart = fl(Y.espart); F.dMn = fl(Y.dMn);
-    F.status = P.status;
+    F.status = reinterpret_cast<int *>(ws + Y.status);
     F.N = D.N; F.H = D.H; F.BH = D.BH; F.T = Y.T; F.r = D.r; F.nslab = 1; F.nes = 4 * Y.nslab; F.s2 = D.s * D.s;
     F.nsplit = pick_splits((long long)BH, Y.T, 3.5, 5.0, 64);
     timer_mark(plan, st, "tc_bwd_finish_k_kernel");
@@ -1026,7 +1028,6 @@ darkattn_status_t tensor_backward_dw(const darkattn_plan_s *plan, const void *M,
 {
     const Dims &D = plan->dims;
     const TensorLayout &Y = plan->tensor;
-    if (!D.causal) return simt_backward_dw(plan, dW, ws, st);     // that backward ran on the FP32 path
     timer_mark(plan, st, "dw_kernel");
     dw_kernel<<<dim3(D.m, D.w_per_head ? D.H : 1), D.r, 0, st>>>(reinterpret_cast<const float *>(ws + Y.Tacc), (const __nv_bfloat16 *)M, dW,
                                                                 D.H, D.m, D.r, D.d, D.w_per_head, D.s);

@@ -798,11 +798,14 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_queries_kernel(const __gri
     if (warp == kEpiWarps) tmem_dealloc(tmem, 512);
 }
 
-// Sb[bh,l,:] = bf16(Sacc[bh,l,:])  (operand of the query pass)
-__global__ void state_to_bf16_kernel(const float *S, __nv_bfloat16 *Sb, long long n)
+// Sb[bh,l,:] = bf16(Sacc[bh,l,:])  (operand of the query pass); z is copied beside it where the backward pass
+// will look for it (zout == z when that is the workspace itself)
+__global__ void state_to_bf16_kernel(const float *S, __nv_bfloat16 *Sb, long long n, const float *z, float *zout, long long nz)
 {
-    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
-        Sb[i] = __float2bfloat16_rn(S[i]);
+    const long long i0 = blockIdx.x * (long long)blockDim.x + threadIdx.x, step = (long long)gridDim.x * blockDim.x;
+    for (long long i = i0; i < n; i += step) Sb[i] = __float2bfloat16_rn(S[i]);
+    if (zout != z)
+        for (long long i = i0; i < nz; i += step) zout[i] = z[i];
 }
 
 // In-place exclusive prefix over the segments of S[bh, seg, e] (e over m*dv) and z[bh, seg, l]; Sb receives the bf16
@@ -989,22 +992,26 @@ void tensor_make_layout(darkattn_plan_s *plan)
         Y.sv_Om = take(so, (size_t)D.H * m * d * 2);
         Y.sv_cs = take(so, BH * Y.nslab * 4);
         Y.sv_zc = take(so, D.causal ? BH * (size_t)Y.T * m * 4 : 0);
+        Y.sv_Sb = take(so, D.causal ? 0 : BH * m * dv * 2);
+        Y.sv_zt = take(so, D.causal ? 0 : BH * m * 4);
         Y.sv_bytes = so;
         plan->saved_bytes = so;
     }
-    if (D.causal) {       // tensor-core backward (the non-causal backward runs on the FP32 path)
-        Y.Oscr = take(off, BH * N * dv * 2);
-        Y.delta = take(off, BH * N * 4);
-        Y.rhoc = take(off, BH * (size_t)Y.T * m * 4);
-        Y.espart = take(off, (size_t)4 * Y.nslab * BH * N * 4);
-        Y.Tacc = take(off, (size_t)D.H * m * d * 4);
-        Y.dMn = take(off, (size_t)D.H * D.r * d * 4);
-        plan->launches_bwd = 1 + 2 + 1 + 1;   // delta, two scan kernels, dK finishing, dM (with `saved`; without it the forward launches come on top)
-    }
+    // backward pass
+    Y.Oscr = take(off, BH * N * dv * 2);
+    Y.delta = take(off, BH * N * 4);
+    Y.rhoc = take(off, D.causal ? BH * (size_t)Y.T * m * 4 : 0);
+    Y.espart = take(off, (size_t)4 * Y.nslab * BH * N * 4);
+    Y.Tacc = take(off, (size_t)D.H * m * d * 4);
+    Y.dMn = take(off, (size_t)D.H * D.r * d * 4);
+    Y.Racc = take(off, D.causal ? 0 : BH * m * dv * 4);
+    Y.rhot = take(off, D.causal ? 0 : BH * m * 4);
+    Y.Rb = take(off, D.causal ? 0 : BH * m * dv * 2);
+    // with `saved`; without it the forward launches come on top. Causal: delta, two scan kernels, dK finishing, dM;
+    // non-causal: one more for the rounding of R between the two passes.
+    plan->launches_bwd = D.causal ? 5 : 6;
     Y.total_bytes = off;
-    // causal plans run entirely on the tensor kernels; the non-causal backward still needs the FP32 path's layout
-    if (D.causal) plan->workspace_bytes = Y.total_bytes;
-    else if (Y.total_bytes > plan->workspace_bytes) plan->workspace_bytes = Y.total_bytes;
+    plan->workspace_bytes = Y.total_bytes;
 }
 
 cudaError_t tensor_prologue(const darkattn_plan_s *plan, const void *K, const void *M, const void *W, char *ws,
@@ -1060,7 +1067,7 @@ darkattn_status_t tensor_forward(const darkattn_plan_s *plan, const void *Q, con
     memset(&P, 0, sizeof(P));
     bool ok = make_map(&P.mapQ, Q, BH * N, D.d, 128) && make_map(&P.mapK, K, BH * N, D.d, 128) &&
               make_map(&P.mapV, V, BH * N, D.dv, 128) && make_map(&P.mapOm, stash.Om, (size_t)D.H * D.m, D.d, 128) &&
-              make_map(&P.mapSb, bf(Y.Sb), BH * (D.causal ? Y.nsplit : 1) * D.m, D.dv, 128) &&
+              make_map(&P.mapSb, D.causal ? bf(Y.Sb) : stash.Sb, BH * (D.causal ? Y.nsplit : 1) * D.m, D.dv, 128) &&
               make_map(&P.mapPN, bf(Y.pnum), (size_t)Y.nslab * BH * N, D.dv, 128);
     if (!ok) { set_cuda_error(cudaErrorInvalidValue, "tensor_forward: tensor map encode"); return DARKATTN_ERR_CUDA; }
 
@@ -1092,7 +1099,7 @@ darkattn_status_t tensor_forward(const darkattn_plan_s *plan, const void *Q, con
         if (x != cudaSuccess && e == cudaSuccess) e = x;
         const long long n = (long long)BH * D.m * D.dv;
         timer_mark(plan, st, "state_to_bf16_kernel");
-        state_to_bf16_kernel<<<(unsigned)((n + 1023) / 1024), 256, 0, st>>>(fl(Y.Sacc), bf(Y.Sb), n);
+        state_to_bf16_kernel<<<(unsigned)((n + 1023) / 1024), 256, 0, st>>>(fl(Y.Sacc), stash.Sb, n, fl(Y.zacc), stash.zt, (long long)BH * D.m);
         chk();
         timer_mark(plan, st, "tc_fwd_queries_kernel");
         x = launch_main_shape<MODE_QUERIES>(D.d, D.dv, P, units * Y.nsplit, st);

@@ -48,6 +48,8 @@ WORKLOADS = {
     "c4": Workload("c4", 4, 1, 8, 65536, 64, 512, "bf16", True, top_scale=4.0),
     "c5": Workload("c5", 5, 8, 12, 2048, 64, 256, "bf16", True, backward=True),
     "headline": Workload("headline", 3, 4, 16, 8192, 128, 256, "bf16", True, backward=True, rho=0.95),
+    # the headline shape without the causal mask (bidirectional attention), forward + backward
+    "headline_nc": Workload("headline_nc", 6, 4, 16, 8192, 128, 256, "bf16", False, backward=True, rho=0.95),
     # the headline's per-head shape on fewer, shorter sequences: one CTA per SM (2 * 37 heads * 2 slabs = 148),
     # inputs still larger than L2; small enough for a full profiler capture
     "profile_small": Workload("profile_small", 3, 2, 37, 2048, 128, 256, "bf16", True, backward=True, rho=0.95),

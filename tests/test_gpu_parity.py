@@ -153,6 +153,13 @@ TENSOR_BWD = [
     ("b_d128_dv64_r64", dict(B=1, H=2, N=256, d=128, m=128, dv=64, r=64, causal=True)),
     ("b_d64_dv128_r32", dict(B=2, H=2, N=384, d=64, m=256, dv=128, r=32, causal=True)),
     ("b_segmented_fwd", dict(B=1, H=2, N=1024, d=64, m=128, causal=True)),
+    # no causal mask: one pass over the queries, one over the keys
+    ("b_nc_one_tile", dict(B=1, H=1, N=128, d=64, m=128, causal=False)),
+    ("b_nc_d64_m256", dict(B=2, H=3, N=640, d=64, m=256, causal=False)),
+    ("b_nc_d128_m256", dict(B=1, H=2, N=384, d=128, m=256, causal=False)),
+    ("b_nc_d128_dv64_r64", dict(B=1, H=2, N=256, d=128, m=128, dv=64, r=64, causal=False)),
+    ("b_nc_d64_dv128_r32", dict(B=2, H=2, N=384, d=64, m=512, dv=128, r=32, causal=False)),
+    ("b_nc_pieces", dict(B=1, H=1, N=2048, d=64, m=128, causal=False)),
 ]
 
 
@@ -174,11 +181,11 @@ def test_tensor_path_per_head_projections_and_scale(binding):
     _compare(got, _oracle(t, wl, scale=0.2), TOL["bf16"], "t_wph")
 
 
-@pytest.mark.parametrize("case", ["simt_f32", "simt_f32_noncausal_wph", "tensor", "tensor_wph"])
+@pytest.mark.parametrize("case", ["simt_f32", "simt_f32_noncausal_wph", "tensor", "tensor_wph", "tensor_noncausal"])
 def test_gradient_of_the_projection_rows(binding, case):
     wph = case.endswith("wph")
     tensor = case.startswith("tensor")
-    kw = dict(B=2, H=3, N=384, d=64, m=256, causal=True) if tensor else dict(B=2, H=2, N=150, d=24, m=40, r=16, causal="noncausal" not in case)
+    kw = dict(B=2, H=3, N=384, d=64, m=256, causal="noncausal" not in case) if tensor else dict(B=2, H=2, N=150, d=24, m=40, r=16, causal="noncausal" not in case)
     wl = inputs.small(name=case, wid=81, dtype="bf16" if tensor else "f32", backward=True, **kw)
     t = inputs.generate(wl)
     if wph:
