@@ -69,6 +69,8 @@ struct TensorLayout {
     size_t espart;  // partials of rowsum(E_K) per slab and 32-column group, fp32 [4 nslab, BH, N]
     size_t Tacc;    // sum_i E_i^T x_i over both sides and the batch, fp32 [H, m, d]
     size_t dMn;     // gradient of M through the key norm term, fp32 [H, r, d]
+    size_t Ahat;    // causal backward: A^ of every (token, feature), bf16 [BH, N, m] (query-side kernel -> key-side kernel)
+    size_t Bphi;    // causal backward: Bf likewise
     size_t Racc;    // non-causal backward: sum of A^^T dO, fp32 [BH, m, dv]; rhot directly behind it
     size_t rhot;    // non-causal backward: -sum of A^^T delta, fp32 [BH, m]
     size_t Rb;      // bf16 copy of Racc

@@ -36,6 +36,7 @@ constexpr float kLn2 = 0.6931471805599453f;
 
 struct BwdParams {
     CUtensorMap mapQ, mapK, mapV, mapG, mapOm, mapDQ, mapDK, mapDV;   // the last three: the gradients, for the (adding) stores
+    CUtensorMap mapAh, mapBf;   // A^ and Bf as [BH*N, m] bf16: written by the query-side kernel, read by the key-side one
     const float2 *sv;     // [BH*N]  (normaliser, exponent it is scaled by) from the forward pass
     const float *delta;   // [BH*N]  dO_i . O_i
     const float *nK;      // [BH*N]  key norms, log2 units
@@ -110,6 +111,11 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                 mbar_expect_tx(bar, 128 * width * 2);
                 for (int a = 0; a < width / 64; ++a) tma_load_2d(dst + a * 16384, map, bar, a * 64, row0 + t * 128);
             };
+            auto store_features = [&](unsigned char *src, const CUtensorMap *map, int t) {
+                tma_store_2d(map, src, slab * 128, row0 + t * 128);
+                tma_store_2d(map, src + 16384, slab * 128 + 64, row0 + t * 128);
+                tma_store_commit();
+            };
             const TileDesc tOm(sOm), tQA(sQA), tKB(sKB), tV(sV), tG(sG), tSt(sSt), tDel(sStg);
             const uint32_t id_kk = make_idesc(128, 128, 0, 0);
             const uint32_t id_vec = make_idesc(128, 16, 1, 0);
@@ -146,12 +152,14 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                 _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R1, kdesc(tQA, k), kdesc(tOm, k), id_kk, k > 0);       // U_Q
                 mma_commit(bars + QM1);
                 QWAIT(QE0); if (!ok) break;                                                                      // Bf in smem, R2 read
+                store_features(sKB, &p.mapBf, t);                                                                // kept for the key-side kernel
                 QWAIT(QB_V); if (!ok) break;
                 QWAIT(QB_G); if (!ok) break;
                 tc_fence_after();
                 _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R2, kdesc(tG, k), kdesc(tV, k), id_kk, k > 0);         // dO V^T
                 mma_commit(bars + QM3);
                 QWAIT(QE1); if (!ok) break;                                                                      // A^ in smem, R1 read
+                store_features(sQA, &p.mapAh, t);
                 QWAIT(QE2A); if (!ok) break;                                                                     // dO V^T read out of R2
                 tc_fence_after();
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R2 + 64, mndesc(tQA, k), vecdesc(tDel, k), id_vec, k > 0);  // rho_c = -A^^T delta (columns 0, 1)
@@ -160,6 +168,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R1, R2 + k * 8, mndesc(tKB, k), id_tm, k > 0);               // dP Bf
                 if (!first)
                     _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R1, kdesc(tG, k), kdesc(tSt, k), id_kk, 1);        // + dO S_prev^T
+                tma_store_wait_read();          // both feature tiles have left shared memory: E may overwrite A^, the next K tile Bf
                 mma_commit(bars + QM4);
                 // the state update is not on the chunk's critical path: it runs while the epilogue forms E
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColState, mndesc(tKB, k), mndesc(tV, k), id_state, (!first) || k > 0);   // S += Bf^T V
@@ -186,6 +195,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                 QWAIT(QE4); if (!ok) break;
 #undef QWAIT
             }
+            tma_store_wait_all();
         }
     } else {
         // ============================== epilogue threads (see kEpiWarps)
@@ -333,7 +343,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
     if (warp == kEpiWarps) tmem_dealloc(tmem, 512);
 }
 
-enum KBars { KB_OM, KB_Q, KB_K, KB_V, KB_G, KB_X2, KM1, KM2, KM3, KM4, KM5, KM6, KM7, KM8, KM9, KE0, KE1, KE2, KE3, KE4, KE5, KNBARS };
+enum KBars { KB_OM, KB_A, KB_B, KB_V, KB_G, KB_X2, KM3, KM4, KM5, KM6, KM7, KM8, KM9, KE2, KE3, KE4, KE5, KNBARS };
 
 // ------------------------------------------------------------------ key side (reverse direction)
 template <int D, int DV>
@@ -353,8 +363,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
     const int row0 = bh * p.N, T = p.T;
 
     if (tid == 0) {
-        for (int i = 0; i < KE0; ++i) mbar_init(bars + i, 1);
-        for (int i = KE0; i < KNBARS; ++i) mbar_init(bars + i, kEpiWarps);
+        for (int i = 0; i < KE2; ++i) mbar_init(bars + i, 1);
+        for (int i = KE2; i < KNBARS; ++i) mbar_init(bars + i, kEpiWarps);
         *abort_flag = (smem_u32(smem) & 1023u) ? 1 : 0;
         fence_mbar_init();
     }
@@ -374,6 +384,11 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
                 mbar_expect_tx(bar, 128 * width * 2);
                 for (int a = 0; a < width / 64; ++a) tma_load_2d(dst + a * 16384, map, bar, a * 64, row0 + t * 128);
             };
+            auto load_features = [&](unsigned char *dst, const CUtensorMap *map, uint64_t *bar, int t) {
+                mbar_expect_tx(bar, 32768);
+                tma_load_2d(dst, map, bar, slab * 128, row0 + t * 128);
+                tma_load_2d(dst + 16384, map, bar, slab * 128 + 64, row0 + t * 128);
+            };
             const TileDesc tOm(sOm), tQA(sQA), tKB(sKB), tV(sV), tG(sG), tSt(sSt);
             const uint32_t id_kk = make_idesc(128, 128, 0, 0);
             const uint32_t id_state = make_idesc(128, DV, 1, 1);
@@ -385,42 +400,36 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
 
             mbar_expect_tx(bars + KB_OM, 128 * D * 2);
             for (int a = 0; a < D / 64; ++a) tma_load_2d(sOm + a * 16384, &p.mapOm, bars + KB_OM, a * 64, h * p.m + slab * 128);
-            load_tile(sQA, &p.mapQ, bars + KB_Q, D, T - 1);
-            load_tile(sKB, &p.mapK, bars + KB_K, D, T - 1);
             load_tile(sV, &p.mapV, bars + KB_V, DV, T - 1);
             load_tile(sG, &p.mapG, bars + KB_G, DV, T - 1);
+            load_features(sQA, &p.mapAh, bars + KB_A, T - 1);
+            load_features(sKB, &p.mapBf, bars + KB_B, T - 1);
 
-            // Schedule of one chunk. U_Q of the next chunk is issued in the tail of the current one, and V dO^T
-            // runs while the epilogue is still busy with Bf.
-            //   R1: U_Q -> (A^ read) -> V dO^T -> packed dP^T [0,64) and P^^T [64,128) (A operands) -> U_Q of the next chunk
-            //   R2: U_K -> (Bf read) -> Bf A^^T -> dV -> dBf -> dK partial
+            // Schedule of one chunk. A^ and Bf come from the query-side kernel through the workspace; V dO^T of
+            // the next chunk is issued in the tail of the current one.
+            //   R1: V dO^T -> packed dP^T [0,64) and P^^T [64,128) (A operands) -> V dO^T of the next chunk
+            //   R2: Bf A^^T -> (read) -> dV -> (read) -> dBf -> (E formed) -> dK partial -> (read)
+            // Shared memory: the K tile that T += E^T K needs takes the place of A^ once dP^T A^ is done, so that
+            // V and dO of the next chunk can be fetched early; A^ and Bf of the next chunk follow after T.
             bool ok = wait_or_abort(bars + KB_OM, 0, status, abort_flag);
-            if (ok) ok = wait_or_abort(bars + KB_Q, 0, status, abort_flag);
+            if (ok) ok = wait_or_abort(bars + KB_V, 0, status, abort_flag);
+            if (ok) ok = wait_or_abort(bars + KB_G, 0, status, abort_flag);
             if (ok) {
                 tc_fence_after();
-                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R1, kdesc(tQA, k), kdesc(tOm, k), id_kk, k > 0);       // U_Q of the last chunk
-                mma_commit(bars + KM1);
+                _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R1, kdesc(tV, k), kdesc(tG, k), id_kk, k > 0);         // V dO^T of the last chunk
+                mma_commit(bars + KM3);
             }
             for (int it = 0; it < T && ok; ++it) {
                 const int t = T - 1 - it;
                 const uint32_t ph = it & 1;
                 const bool first = (it == 0), last = (it + 1 == T);
 #define KWAIT(b) do { ok = wait_or_abort(bars + (b), ph, status, abort_flag); } while (0)
-                KWAIT(KB_K); if (!ok) break;
-                tc_fence_after();
-                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R2, kdesc(tKB, k), kdesc(tOm, k), id_kk, k > 0);       // U_K
-                mma_commit(bars + KM2);
-                KWAIT(KE0); if (!ok) break;                                                                      // A^ in smem, R1 read
-                KWAIT(KB_V); if (!ok) break;
-                KWAIT(KB_G); if (!ok) break;
-                tc_fence_after();
-                _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R1, kdesc(tV, k), kdesc(tG, k), id_kk, k > 0);         // V dO^T
-                mma_commit(bars + KM3);
-                KWAIT(KE1); if (!ok) break;                                                                      // Bf in smem, R2 read
+                KWAIT(KB_A); if (!ok) break;
+                KWAIT(KB_B); if (!ok) break;
                 tc_fence_after();
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R2, kdesc(tKB, k), kdesc(tQA, k), id_kk, k > 0);             // P^^T = Bf A^^T
                 mma_commit(bars + KM4);
-                KWAIT(KE2); if (!ok) break;
+                KWAIT(KE2); if (!ok) break;                                                                      // dP^T and P^^T packed in R1
                 tc_fence_after();
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R2, R1 + 64 + k * 8, mndesc(tG, k), id_dv_t, k > 0);         // P^^T dO
                 if (!first)
@@ -435,25 +444,26 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
                 if (!first)
                     _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R2, kdesc(tV, k), kdesc(tSt, k), id_kk, 1);        // + V R_next^T
                 mma_commit(bars + KM7);
-                KWAIT(KM7); if (!ok) break;
-                load_tile(sG, &p.mapK, bars + KB_X2, D, t);                                                     // K again, for T
-                if (!last) { load_tile(sQA, &p.mapQ, bars + KB_Q, D, t - 1); load_tile(sV, &p.mapV, bars + KB_V, DV, t - 1); }
+                KWAIT(KM7); if (!ok) break;                                                                      // A^, V and dO of this chunk are done with
+                load_tile(sQA, &p.mapK, bars + KB_X2, D, t);                                                    // the K tile, for T
+                if (!last) { load_tile(sV, &p.mapV, bars + KB_V, DV, t - 1); load_tile(sG, &p.mapG, bars + KB_G, DV, t - 1); }
                 KWAIT(KE4); if (!ok) break;
                 KWAIT(KB_X2); if (!ok) break;
                 tc_fence_after();
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R2, kdesc(tKB, k), mndesc(tOm, k), id_dx, k > 0);            // E Omega
                 mma_commit(bars + KM8);
-                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColT, mndesc(tKB, k), mndesc(tG, k), id_t, (!first) || k > 0);   // T += E^T K
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColT, mndesc(tKB, k), mndesc(tQA, k), id_t, (!first) || k > 0);   // T += E^T K
                 mma_commit(bars + KM9);
                 if (!last) {
-                    ok = wait_or_abort(bars + KB_Q, ph ^ 1, status, abort_flag);
+                    ok = wait_or_abort(bars + KB_V, ph ^ 1, status, abort_flag);
+                    if (ok) ok = wait_or_abort(bars + KB_G, ph ^ 1, status, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R1, kdesc(tQA, k), kdesc(tOm, k), id_kk, k > 0);   // U_Q of the next chunk
-                    mma_commit(bars + KM1);
+                    _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R1, kdesc(tV, k), kdesc(tG, k), id_kk, k > 0);     // V dO^T of the next chunk
+                    mma_commit(bars + KM3);
                 }
                 KWAIT(KM9); if (!ok) break;
-                if (!last) { load_tile(sKB, &p.mapK, bars + KB_K, D, t - 1); load_tile(sG, &p.mapG, bars + KB_G, DV, t - 1); }
+                if (!last) { load_features(sQA, &p.mapAh, bars + KB_A, t - 1); load_features(sKB, &p.mapBf, bars + KB_B, t - 1); }
                 KWAIT(KE5); if (!ok) break;
 #undef KWAIT
             }
@@ -464,7 +474,6 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
         const bool g0 = (col0 == 0);
         const uint32_t lane_addr = tmem + ((uint32_t)(q4 * 32) << 16);
         const uint32_t R1 = lane_addr + kColR1, R2 = lane_addr + kColR2;
-        const float cshift = p.cs[bh * p.nslab + slab];
         const size_t rows = (size_t)p.BH * p.N;
         bool ok = true;
         for (int it = 0; it < T && ok; ++it) {
@@ -473,27 +482,12 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
             const bool last = (it + 1 == T);
             const size_t row = (size_t)row0 + (size_t)t * 128 + r;
 #define EWAIT(b) do { ok = __all_sync(0xffffffffu, wait_or_abort(bars + (b), ph, status, abort_flag)); } while (0)
-            const float2 svv = p.sv[row];
-            const float nk = p.nK[row] + cshift;
-            const float aq = svv.y - cshift + log2f(svv.x);
             float rho_c = 0.f;
             if (g0) {
                 rho_c = p.rhoc[((size_t)bh * T + t) * p.m + slab * 128 + r];
                 sDel[r] = p.delta[row];
             }
-            EWAIT(KM1); if (!ok) break;
-            tc_fence_after();
-            features_to_tile(R1 + col0, aq, sQA, r, col0);
-            fence_async_smem();
             if (tid == 0) tma_store_wait_read();      // the previous chunk's dK store has left the staging tile
-            tc_fence_before();
-            mbar_arrive_warp(bars + KE0);
-            EWAIT(KM2); if (!ok) break;
-            tc_fence_after();
-            features_to_tile(R2 + col0, nk, sKB, r, col0);
-            fence_async_smem();
-            tc_fence_before();
-            mbar_arrive_warp(bars + KE1);
 
             EWAIT(KM3); if (!ok) break;
             tc_fence_after();
@@ -501,7 +495,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
                 uint32_t v[32], pk[16];
                 tmem_ld32(R1 + col0, v);
                 tmem_wait_ld();
-                quarter_sync(q4);
+                epi_sync();          // every column group has read before anyone overwrites; delta of every row is in place
 #pragma unroll
                 for (int j = 0; j < 32; j += 2) {
                     const float2 dl = *reinterpret_cast<const float2 *>(sDel + col0 + j);
@@ -992,7 +986,8 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
                         make_map(&P.mapV, V, BH * N, D.dv, 128) && make_map(&P.mapG, dO, BH * N, D.dv, 128) &&
                         make_map(&P.mapOm, stash.Om, (size_t)D.H * D.m, D.d, 128) &&
                         make_map(&P.mapDQ, dQ, BH * N, D.d, 128) && make_map(&P.mapDK, dK, BH * N, D.d, 128) &&
-                        make_map(&P.mapDV, dV, BH * N, D.dv, 128);
+                        make_map(&P.mapDV, dV, BH * N, D.dv, 128) &&
+                        make_map(&P.mapAh, bf(Y.Ahat), BH * N, D.m, 128) && make_map(&P.mapBf, bf(Y.Bphi), BH * N, D.m, 128);
         if (!ok) { set_cuda_error(cudaErrorInvalidValue, "tensor_backward: tensor map encode"); return DARKATTN_ERR_CUDA; }
         P.sv = stash.sv; P.delta = fl(Y.delta); P.nK = stash.nK; P.cs = stash.cs; P.zc = stash.zc; P.rhoc = fl(Y.rhoc);
         P.espart = fl(Y.espart); P.Tacc = fl(Y.Tacc);

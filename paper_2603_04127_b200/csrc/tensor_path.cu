@@ -1004,6 +1004,8 @@ void tensor_make_layout(darkattn_plan_s *plan)
     Y.espart = take(off, (size_t)4 * Y.nslab * BH * N * 4);
     Y.Tacc = take(off, (size_t)D.H * m * d * 4);
     Y.dMn = take(off, (size_t)D.H * D.r * d * 4);
+    Y.Ahat = take(off, D.causal ? BH * N * m * 2 : 0);
+    Y.Bphi = take(off, D.causal ? BH * N * m * 2 : 0);
     Y.Racc = take(off, D.causal ? 0 : BH * m * dv * 4);
     Y.rhot = take(off, D.causal ? 0 : BH * m * 4);
     Y.Rb = take(off, D.causal ? 0 : BH * m * dv * 2);

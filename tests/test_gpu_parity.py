@@ -220,10 +220,11 @@ def test_decode_steps_reproduce_the_causal_forward(binding, dtype):
     plan.destroy()
 
 
-def test_headline_backward_sampled_heads(binding):
+@pytest.mark.parametrize("name", ["headline", "headline_nc"])
+def test_headline_backward_sampled_heads(binding, name):
     """Forward + backward at the benchmark's full size; dQ, dK, dV of sampled (batch, head) pairs and
     the gradient of M of one head (summed over the whole batch) against the oracle."""
-    wl = inputs.WORKLOADS["headline"]
+    wl = inputs.WORKLOADS[name]
     B, H = wl.B, wl.H
     t = inputs.generate(wl)
     got = run_gpu(binding, wl, t, use_saved=True)
@@ -233,8 +234,8 @@ def test_headline_backward_sampled_heads(binding):
     want = _oracle(sub, wl)
     for k in ("O", "dQ", "dK", "dV"):
         g = np.stack([got[k][b, h] for b in range(B)])[:, None]
-        assert_close(g, want[k], TOL["bf16"], f"headline head {h}: {k}")
-    assert_close(got["dM"][h], want["dM"][0], TOL["bf16"], f"headline head {h}: dM")
+        assert_close(g, want[k], TOL["bf16"], f"{name} head {h}: {k}")
+    assert_close(got["dM"][h], want["dM"][0], TOL["bf16"], f"{name} head {h}: dM")
 
 
 def test_tensor_path_is_deterministic(binding):
