@@ -69,6 +69,7 @@ struct TensorLayout {
     size_t espart;  // partials of rowsum(E_K) per slab and 32-column group, fp32 [4 nslab, BH, N]
     size_t Tacc;    // sum_i E_i^T x_i over both sides and the batch, fp32 [H, m, d]
     size_t dMn;     // gradient of M through the key norm term, fp32 [H, r, d]
+    size_t Sst;     // workspace copy of the stash's per-chunk S (causal): bf16 [BH, T, m, dv], S before chunk t (t = 0 not written)
     size_t Ahat;    // causal backward: A^ of every (token, feature), bf16 [BH, N, m] (query-side kernel -> key-side kernel)
     size_t Bphi;    // causal backward: Bf likewise
     size_t Racc;    // non-causal backward: sum of A^^T dO, fp32 [BH, m, dv]; rhot directly behind it
@@ -76,7 +77,7 @@ struct TensorLayout {
     size_t Rb;      // bf16 copy of Racc
     size_t total_bytes;
     // the forward -> backward stash (`saved`): per-row normalisers, key norms, folded projections, key shifts
-    size_t sv_sv, sv_nK, sv_Om, sv_cs, sv_zc, sv_Sb, sv_zt, sv_bytes;
+    size_t sv_sv, sv_nK, sv_Om, sv_cs, sv_zc, sv_Sb, sv_zt, sv_Sst, sv_bytes;
     size_t zc;      // workspace copy of the stash's per-chunk z (causal): sum_j phi(K)_jl over the chunks before t, fp32 [BH, T, m]
     int nslab, T, nsplit;
 };
@@ -91,13 +92,14 @@ struct Stash {
     float *zc;      // causal: z before chunk t, [BH, T, m] (row t = 0 is not written: it is zero)
     __nv_bfloat16 *Sb;   // non-causal: S of the whole sequence, bf16 [BH, m, dv]
     float *zt;      // non-causal: z of the whole sequence, [BH, m]
+    __nv_bfloat16 *Sst;  // causal: S before chunk t, bf16 [BH, T, m, dv] (t = 0 is not written: it is zero)
 };
 inline Stash stash_in_workspace(const TensorLayout &Y, char *ws)
 {
     return Stash{reinterpret_cast<float2 *>(ws + Y.sv), reinterpret_cast<float *>(ws + Y.nK),
                  reinterpret_cast<__nv_bfloat16 *>(ws + Y.Om), reinterpret_cast<float *>(ws + Y.cs),
                  reinterpret_cast<float *>(ws + Y.zc), reinterpret_cast<__nv_bfloat16 *>(ws + Y.Sb),
-                 reinterpret_cast<float *>(ws + Y.zacc)};
+                 reinterpret_cast<float *>(ws + Y.zacc), reinterpret_cast<__nv_bfloat16 *>(ws + Y.Sst)};
 }
 inline Stash stash_in_saved(const TensorLayout &Y, void *saved)
 {
@@ -105,7 +107,7 @@ inline Stash stash_in_saved(const TensorLayout &Y, void *saved)
     return Stash{reinterpret_cast<float2 *>(b + Y.sv_sv), reinterpret_cast<float *>(b + Y.sv_nK),
                  reinterpret_cast<__nv_bfloat16 *>(b + Y.sv_Om), reinterpret_cast<float *>(b + Y.sv_cs),
                  reinterpret_cast<float *>(b + Y.sv_zc), reinterpret_cast<__nv_bfloat16 *>(b + Y.sv_Sb),
-                 reinterpret_cast<float *>(b + Y.sv_zt)};
+                 reinterpret_cast<float *>(b + Y.sv_zt), reinterpret_cast<__nv_bfloat16 *>(b + Y.sv_Sst)};
 }
 
 }  // namespace darkattn
@@ -160,7 +162,7 @@ darkattn_status_t simt_backward(const darkattn_plan_s *plan, const void *Q, cons
 bool tensor_supported(const darkattn_plan_s *plan);
 void tensor_make_layout(darkattn_plan_s *plan);
 darkattn_status_t tensor_forward(const darkattn_plan_s *plan, const void *Q, const void *K, const void *V,
-                                 const void *M, const void *W, void *O, void *saved, char *ws, cudaStream_t st);
+                                 const void *M, const void *W, void *O, void *saved, char *ws, cudaStream_t st, bool stash_states);
 // Folded projections, key-side shifts and key norms (written to `out`).
 cudaError_t tensor_prologue(const darkattn_plan_s *plan, const void *K, const void *M, const void *W, char *ws,
                             const Stash &out, cudaStream_t st);

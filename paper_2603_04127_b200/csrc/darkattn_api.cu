@@ -104,7 +104,7 @@ darkattn_status_t darkattn_forward(darkattn_plan_t plan, const void *Q, const vo
     DARKATTN_CUDA_TRY(cudaMemsetAsync(workspace, 0, 256, st), "forward: clear status word");
     darkattn_status_t rc;
     if (plan->path == DARKATTN_PATH_TENSOR) {
-        rc = tensor_forward(plan, Q, K, V, M, W, O, saved, static_cast<char *>(workspace), st);
+        rc = tensor_forward(plan, Q, K, V, M, W, O, saved, static_cast<char *>(workspace), st, saved != nullptr);
     } else {
         timer_mark(plan, st, "simt_forward (all kernels)");
         rc = simt_forward(plan, Q, K, V, M, W, O, static_cast<char *>(workspace), st, false);

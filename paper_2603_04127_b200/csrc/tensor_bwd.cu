@@ -37,6 +37,7 @@ constexpr float kLn2 = 0.6931471805599453f;
 struct BwdParams {
     CUtensorMap mapQ, mapK, mapV, mapG, mapOm, mapDQ, mapDK, mapDV;   // the last three: the gradients, for the (adding) stores
     CUtensorMap mapAh, mapBf;   // A^ and Bf as [BH*N, m] bf16: written by the query-side kernel, read by the key-side one
+    CUtensorMap mapSst;         // S before every chunk as [BH*T*m, dv] bf16, from the forward pass
     const float2 *sv;     // [BH*N]  (normaliser, exponent it is scaled by) from the forward pass
     const float *delta;   // [BH*N]  dO_i . O_i
     const float *nK;      // [BH*N]  key norms, log2 units
@@ -70,9 +71,12 @@ constexpr uint32_t kColState = 0, kColT = 128, kColR1 = 256, kColR2 = 384;
 // K-major 16 x 128 bf16 operand (two atoms of 2 KB): step k covers 16 elements of K
 __device__ __forceinline__ uint64_t vecdesc(const TileDesc &t, int k) { return t.kmaj + (uint64_t)(((k / 4) * 2048 + (k % 4) * 32) >> 4); }
 
-enum QBars { QB_OM, QB_Q, QB_K, QB_V, QB_G, QB_X2, QM1, QM2, QM3, QMS, QM4, QM5, QM6, QE0, QE1, QE2A, QE2, QE3, QE4, QNBARS };
+enum QBars { QB_OM, QB_Q, QB_K, QB_V, QB_G, QB_S, QB_X2, QM1, QM2, QM3, QM4, QM5, QM6, QE0, QE1, QE2A, QE2, QE3, QE4, QET, QNBARS };
 
-// ------------------------------------------------------------------ query side (forward direction)
+// ------------------------------------------------------------------ query side
+// The state S before every chunk comes from the forward pass (bf16, through the stash), so the chunks are
+// independent of one another here: the chunks of all (batch, head) pairs form one line that is cut evenly over groups
+// of nslab CTAs, and a CTA walks its piece run by run (a run = consecutive chunks of one (batch, head) pair).
 template <int D, int DV>
 __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_constant__ BwdParams p)
 {
@@ -86,8 +90,12 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + QNBARS + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5;
-    const int bh = blockIdx.x / p.nslab, slab = blockIdx.x % p.nslab, h = bh % p.H;
-    const int row0 = bh * p.N, T = p.T;
+    const int T = p.T;
+    // CTAs work in groups of nslab (one per slab of the head) on the same piece of the line of (batch, head, chunk)
+    // items, so that the Q, K, V, dO tiles a group reads are fetched from HBM once
+    const int slab = blockIdx.x % p.nslab, group = blockIdx.x / p.nslab, ngroups = gridDim.x / p.nslab;
+    const long long total = (long long)p.BH * T;
+    const long long lbeg = total * group / ngroups, lend = total * (group + 1) / ngroups;
 
     if (tid == 0) {
         for (int i = 0; i < QE0; ++i) mbar_init(bars + i, 1);
@@ -95,7 +103,6 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
         *abort_flag = (smem_u32(smem) & 1023u) ? 1 : 0;
         fence_mbar_init();
     }
-    if (tid < 128) sZ[tid] = 0.f;
     if (warp == kEpiWarps) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
@@ -107,93 +114,109 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
         if (tid == 0) atomicExch(status, (int)DARKATTN_ERR_CUDA);
     } else if (warp == kEpiWarps) {
         if ((tid & 31) == 0) {
-            auto load_tile = [&](unsigned char *dst, const CUtensorMap *map, uint64_t *bar, int width, int t) {
-                mbar_expect_tx(bar, 128 * width * 2);
-                for (int a = 0; a < width / 64; ++a) tma_load_2d(dst + a * 16384, map, bar, a * 64, row0 + t * 128);
-            };
-            auto store_features = [&](unsigned char *src, const CUtensorMap *map, int t) {
-                tma_store_2d(map, src, slab * 128, row0 + t * 128);
-                tma_store_2d(map, src + 16384, slab * 128 + 64, row0 + t * 128);
-                tma_store_commit();
-            };
             const TileDesc tOm(sOm), tQA(sQA), tKB(sKB), tV(sV), tG(sG), tSt(sSt), tDel(sStg);
             const uint32_t id_kk = make_idesc(128, 128, 0, 0);
             const uint32_t id_vec = make_idesc(128, 16, 1, 0);
-            const uint32_t id_state = make_idesc(128, DV, 1, 1);
             const uint32_t id_tm = make_idesc(128, 128, 0, 1);
             const uint32_t id_dx = make_idesc(128, D, 0, 1);
             const uint32_t id_t = make_idesc(128, D, 1, 1);
             const uint32_t R1 = tmem + kColR1, R2 = tmem + kColR2;
 
-            mbar_expect_tx(bars + QB_OM, 128 * D * 2);
-            for (int a = 0; a < D / 64; ++a) tma_load_2d(sOm + a * 16384, &p.mapOm, bars + QB_OM, a * 64, h * p.m + slab * 128);
-            load_tile(sQA, &p.mapQ, bars + QB_Q, D, 0);
-            load_tile(sKB, &p.mapK, bars + QB_K, D, 0);
-            load_tile(sV, &p.mapV, bars + QB_V, DV, 0);
-            load_tile(sG, &p.mapG, bars + QB_G, DV, 0);
-
             // Schedule of one chunk (R1, R2: the two scratch regions of TMEM). U_K of the next chunk is issued in
             // the tail of the current one, and dO V^T runs while the epilogue is still busy with A^.
             //   R2: U_K -> (Bf read) -> dO V^T -> packed dP in [0,64) (A operand of dP Bf), rho_c in [64,80) -> U_K of the next chunk
             //   R1: U_Q -> (A^ read) -> dP Bf + dO S^T -> (E read) -> E Omega -> (dQ read)
-            bool ok = wait_or_abort(bars + QB_OM, 0, status, abort_flag);
-            if (ok) ok = wait_or_abort(bars + QB_K, 0, status, abort_flag);
-            if (ok) {
-                tc_fence_after();
-                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R2, kdesc(tKB, k), kdesc(tOm, k), id_kk, k > 0);       // U_K of chunk 0
-                mma_commit(bars + QM2);
-            }
-            for (int t = 0; t < T && ok; ++t) {
-                const uint32_t ph = t & 1;
-                const bool first = (t == 0), last = (t + 1 == T);
-#define QWAIT(b) do { ok = wait_or_abort(bars + (b), ph, status, abort_flag); } while (0)
-                QWAIT(QB_Q); if (!ok) break;
-                tc_fence_after();
-                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R1, kdesc(tQA, k), kdesc(tOm, k), id_kk, k > 0);       // U_Q
-                mma_commit(bars + QM1);
-                QWAIT(QE0); if (!ok) break;                                                                      // Bf in smem, R2 read
-                store_features(sKB, &p.mapBf, t);                                                                // kept for the key-side kernel
-                QWAIT(QB_V); if (!ok) break;
-                QWAIT(QB_G); if (!ok) break;
-                tc_fence_after();
-                _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R2, kdesc(tG, k), kdesc(tV, k), id_kk, k > 0);         // dO V^T
-                mma_commit(bars + QM3);
-                QWAIT(QE1); if (!ok) break;                                                                      // A^ in smem, R1 read
-                store_features(sQA, &p.mapAh, t);
-                QWAIT(QE2A); if (!ok) break;                                                                     // dO V^T read out of R2
-                tc_fence_after();
-                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R2 + 64, mndesc(tQA, k), vecdesc(tDel, k), id_vec, k > 0);  // rho_c = -A^^T delta (columns 0, 1)
-                QWAIT(QE2); if (!ok) break;                                                                      // dP packed in R2
-                tc_fence_after();
-                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R1, R2 + k * 8, mndesc(tKB, k), id_tm, k > 0);               // dP Bf
-                if (!first)
-                    _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R1, kdesc(tG, k), kdesc(tSt, k), id_kk, 1);        // + dO S_prev^T
-                tma_store_wait_read();          // both feature tiles have left shared memory: E may overwrite A^, the next K tile Bf
-                mma_commit(bars + QM4);
-                // the state update is not on the chunk's critical path: it runs while the epilogue forms E
-                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColState, mndesc(tKB, k), mndesc(tV, k), id_state, (!first) || k > 0);   // S += Bf^T V
-                mma_commit(bars + QMS);
-                QWAIT(QMS); if (!ok) break;                                                                      // (also: dP Bf before it is done)
-                load_tile(sG, &p.mapQ, bars + QB_X2, D, t);                                                     // Q again, for T
-                if (!last) { load_tile(sV, &p.mapV, bars + QB_V, DV, t + 1); load_tile(sKB, &p.mapK, bars + QB_K, D, t + 1); }
-                QWAIT(QE3); if (!ok) break;
-                QWAIT(QB_X2); if (!ok) break;
-                tc_fence_after();
-                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R1, kdesc(tQA, k), mndesc(tOm, k), id_dx, k > 0);            // E Omega
-                mma_commit(bars + QM5);
-                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColT, mndesc(tQA, k), mndesc(tG, k), id_t, (!first) || k > 0);   // T += E^T Q
-                mma_commit(bars + QM6);
-                if (!last) {
-                    ok = wait_or_abort(bars + QB_K, ph ^ 1, status, abort_flag);
-                    if (!ok) break;
+            bool ok = true;
+            int it = 0, run = 0;        // chunks and runs done so far: the parities of the barriers
+            for (long long l0 = lbeg; l0 < lend && ok; ++run) {
+                const int bh = (int)(l0 / T), t0 = (int)(l0 % T);
+                long long l1 = (long long)(bh + 1) * T;
+                if (l1 > lend) l1 = lend;
+                const int nrun = (int)(l1 - l0);
+                l0 = l1;
+                const int h = bh % p.H, row0 = bh * p.N;
+                auto load_tile = [&](unsigned char *dst, const CUtensorMap *map, uint64_t *bar, int width, int t) {
+                    mbar_expect_tx(bar, 128 * width * 2);
+                    for (int a = 0; a < width / 64; ++a) tma_load_2d(dst + a * 16384, map, bar, a * 64, row0 + t * 128);
+                };
+                auto load_state = [&](int t) {     // S before chunk t (for t = 0 the tile is loaded but not used)
+                    mbar_expect_tx(bars + QB_S, 128 * DV * 2);
+                    for (int a = 0; a < DV / 64; ++a) tma_load_2d(sSt + a * 16384, &p.mapSst, bars + QB_S, a * 64, (bh * T + t) * p.m + slab * 128);
+                };
+                auto store_features = [&](unsigned char *src, const CUtensorMap *map, int t) {
+                    tma_store_2d(map, src, slab * 128, row0 + t * 128);
+                    tma_store_2d(map, src + 16384, slab * 128 + 64, row0 + t * 128);
+                    tma_store_commit();
+                };
+                mbar_expect_tx(bars + QB_OM, 128 * D * 2);
+                for (int a = 0; a < D / 64; ++a) tma_load_2d(sOm + a * 16384, &p.mapOm, bars + QB_OM, a * 64, h * p.m + slab * 128);
+                load_tile(sQA, &p.mapQ, bars + QB_Q, D, t0);
+                load_tile(sKB, &p.mapK, bars + QB_K, D, t0);
+                load_tile(sV, &p.mapV, bars + QB_V, DV, t0);
+                load_tile(sG, &p.mapG, bars + QB_G, DV, t0);
+                load_state(t0);
+                ok = wait_or_abort(bars + QB_OM, run & 1, status, abort_flag);
+                if (ok) ok = wait_or_abort(bars + QB_K, it & 1, status, abort_flag);
+                if (ok) {
                     tc_fence_after();
-                    _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R2, kdesc(tKB, k), kdesc(tOm, k), id_kk, k > 0);   // U_K of the next chunk
+                    _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R2, kdesc(tKB, k), kdesc(tOm, k), id_kk, k > 0);   // U_K of the run's first chunk
                     mma_commit(bars + QM2);
                 }
-                QWAIT(QM6); if (!ok) break;
-                if (!last) { load_tile(sQA, &p.mapQ, bars + QB_Q, D, t + 1); load_tile(sG, &p.mapG, bars + QB_G, DV, t + 1); }
-                QWAIT(QE4); if (!ok) break;
+                for (int c = 0; c < nrun && ok; ++c, ++it) {
+                    const int t = t0 + c;
+                    const uint32_t ph = it & 1;
+                    const bool first = (t == 0), last = (c + 1 == nrun);
+#define QWAIT(b) do { ok = wait_or_abort(bars + (b), ph, status, abort_flag); } while (0)
+                    QWAIT(QB_Q); if (!ok) break;
+                    tc_fence_after();
+                    _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R1, kdesc(tQA, k), kdesc(tOm, k), id_kk, k > 0);   // U_Q
+                    mma_commit(bars + QM1);
+                    QWAIT(QE0); if (!ok) break;                                                                  // Bf in smem, R2 read
+                    store_features(sKB, &p.mapBf, t);                                                            // kept for the key-side kernel
+                    QWAIT(QB_V); if (!ok) break;
+                    QWAIT(QB_G); if (!ok) break;
+                    tc_fence_after();
+                    _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R2, kdesc(tG, k), kdesc(tV, k), id_kk, k > 0);     // dO V^T
+                    mma_commit(bars + QM3);
+                    QWAIT(QE1); if (!ok) break;                                                                  // A^ in smem, R1 read
+                    store_features(sQA, &p.mapAh, t);
+                    QWAIT(QE2A); if (!ok) break;                                                                 // dO V^T read out of R2
+                    tc_fence_after();
+                    _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R2 + 64, mndesc(tQA, k), vecdesc(tDel, k), id_vec, k > 0);  // rho_c = -A^^T delta (columns 0, 1)
+                    QWAIT(QE2); if (!ok) break;                                                                  // dP packed in R2
+                    QWAIT(QB_S); if (!ok) break;
+                    tc_fence_after();
+                    _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R1, R2 + k * 8, mndesc(tKB, k), id_tm, k > 0);           // dP Bf
+                    if (!first)
+                        _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R1, kdesc(tG, k), kdesc(tSt, k), id_kk, 1);    // + dO S_prev^T
+                    tma_store_wait_read();      // both feature tiles have left shared memory: E may overwrite A^, the next K tile Bf
+                    mma_commit(bars + QM4);
+                    QWAIT(QM4); if (!ok) break;                                                                  // Bf, V, dO and S of this chunk are done with
+                    load_tile(sG, &p.mapQ, bars + QB_X2, D, t);                                                 // Q again, for T
+                    if (!last) { load_tile(sV, &p.mapV, bars + QB_V, DV, t + 1); load_tile(sKB, &p.mapK, bars + QB_K, D, t + 1); load_state(t + 1); }
+                    QWAIT(QE3); if (!ok) break;
+                    QWAIT(QB_X2); if (!ok) break;
+                    if (c == 0 && run > 0) {                                                                     // T of the previous run has been read out
+                        ok = wait_or_abort(bars + QET, (run - 1) & 1, status, abort_flag);
+                        if (!ok) break;
+                    }
+                    tc_fence_after();
+                    _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R1, kdesc(tQA, k), mndesc(tOm, k), id_dx, k > 0);        // E Omega
+                    mma_commit(bars + QM5);
+                    _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColT, mndesc(tQA, k), mndesc(tG, k), id_t, (c > 0) || k > 0);   // T += E^T Q
+                    mma_commit(bars + QM6);
+                    if (!last) {
+                        ok = wait_or_abort(bars + QB_K, ph ^ 1, status, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R2, kdesc(tKB, k), kdesc(tOm, k), id_kk, k > 0);   // U_K of the next chunk
+                        mma_commit(bars + QM2);
+                    }
+                    QWAIT(QM6); if (!ok) break;
+                    if (!last) { load_tile(sQA, &p.mapQ, bars + QB_Q, D, t + 1); load_tile(sG, &p.mapG, bars + QB_G, DV, t + 1); }
+                    QWAIT(QE4); if (!ok) break;
 #undef QWAIT
+                }
             }
             tma_store_wait_all();
         }
@@ -204,138 +227,150 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
         const bool g0 = (col0 == 0);                         // these 128 threads: row r also stands for feature r of the slab
         const uint32_t lane_addr = tmem + ((uint32_t)(q4 * 32) << 16);
         const uint32_t R1 = lane_addr + kColR1, R2 = lane_addr + kColR2;
-        const float cshift = p.cs[bh * p.nslab + slab];
         bool ok = true;
-        for (int t = 0; t < T && ok; ++t) {
-            const uint32_t ph = t & 1;
-            const bool last = (t + 1 == T);
-            const size_t row = (size_t)row0 + (size_t)t * 128 + r;
-#define EWAIT(b) do { ok = __all_sync(0xffffffffu, wait_or_abort(bars + (b), ph, status, abort_flag)); } while (0)
-            const float2 svv = p.sv[row];
-            const float del = p.delta[row];
-            const float nk = p.nK[row] + cshift;
-            const float aq = svv.y - cshift + log2f(svv.x);
-            // z before the next chunk, from the forward pass (loaded early, used at the end of the chunk)
-            const float znext = (g0 && !last) ? __ldg(p.zc + ((size_t)bh * T + t + 1) * p.m + slab * 128 + r) : 0.f;
-            float dtile[4] = {0.f, 0.f, 0.f, 0.f};       // warp 0: -delta of rows lane, lane + 32, ... for the operand of rho_c
-            if (warp == 0) {
-#pragma unroll
-                for (int i = 0; i < 4; ++i) dtile[i] = -__ldg(p.delta + (size_t)row0 + (size_t)t * 128 + i * 32 + lane);
-            }
-            EWAIT(QM2); if (!ok) break;
-            tc_fence_after();
-            features_to_tile(R2 + col0, nk, sKB, r, col0);                             // Bf
-            if (warp == 0) {
-                // 16 x 128 K-major operand of rho_c = -A^^T delta at the start of the staging tile: row 0 = -delta rounded
-                // to bf16, row 1 = the rounding's remainder. Written by the warp whose first lane has just seen the
-                // previous chunk's store leave the tile.
-                if (tid == 0) tma_store_wait_read();
-                __syncwarp();
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int k = i * 32 + lane;
-                    const float dk = dtile[i];
-                    const __nv_bfloat16 hi = __float2bfloat16_rn(dk);
-                    const __nv_bfloat16 lo = __float2bfloat16_rn(dk - __bfloat162float(hi));
-                    const int atom = k >> 6, kk = k & 63, ch = kk >> 3;
-                    *reinterpret_cast<__nv_bfloat16 *>(sStg + atom * 2048 + (ch << 4) + (kk & 7) * 2) = hi;
-                    *reinterpret_cast<__nv_bfloat16 *>(sStg + atom * 2048 + 128 + ((ch ^ 1) << 4) + (kk & 7) * 2) = lo;
-                }
-            }
-            fence_async_smem();
-            tc_fence_before();
-            mbar_arrive_warp(bars + QE0);
-            EWAIT(QM1); if (!ok) break;
-            tc_fence_after();
-            features_to_tile(R1 + col0, aq, sQA, r, col0);                             // A^
-            fence_async_smem();
-            tc_fence_before();
-            mbar_arrive_warp(bars + QE1);
-
-            EWAIT(QM3); if (!ok) break;
-            tc_fence_after();
-            {   // dP = tril(dO V^T - delta) as a bf16 operand in TMEM (packed over the fp32 tile)
-                uint32_t v[32], pk[16];
-                tmem_ld32(R2 + col0, v);
-                tmem_wait_ld();
-                tc_fence_before();
-                mbar_arrive_warp(bars + QE2A);
-                quarter_sync(q4);                         // every column group has read before anyone overwrites
-#pragma unroll
-                for (int j = 0; j < 32; j += 2) {
-                    const float x0 = (col0 + j <= r) ? __uint_as_float(v[j]) - del : 0.f;
-                    const float x1 = (col0 + j + 1 <= r) ? __uint_as_float(v[j + 1]) - del : 0.f;
-                    pk[j / 2] = pack_bf16(x0, x1);
-                }
-                tmem_st16(R2 + col0 / 2, pk);
-            }
-            tmem_wait_st();
-            tc_fence_before();
-            mbar_arrive_warp(bars + QE2);
-
-            EWAIT(QM4); if (!ok) break;
-            tc_fence_after();
-            if (g0) {       // rho_c of feature r (TMEM lane r; its MMAs ran ahead of dP Bf), for the key-side kernel
-                uint32_t v[16];
-                tmem_ld16(R2 + 64, v);
-                tmem_wait_ld();
-                p.rhoc[((size_t)bh * T + t) * p.m + slab * 128 + r] = __uint_as_float(v[0]) + __uint_as_float(v[1]);
-            }
-            {   // E = A^ .* (dP Bf + dO S^T - delta z^T), in place over A^
-                uint32_t v[32];
-                tmem_ld32(R1 + col0, v);
-                tmem_wait_ld();
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    uint4 *cell = reinterpret_cast<uint4 *>(tile_chunk(sQA, r, col0 / 8 + q));
-                    float a[8];
-                    unpack8(*cell, a);
-                    const float4 z0 = *reinterpret_cast<const float4 *>(sZ + col0 + 8 * q);
-                    const float4 z1 = *reinterpret_cast<const float4 *>(sZ + col0 + 8 * q + 4);
-                    const float zz[8] = {z0.x, z0.y, z0.z, z0.w, z1.x, z1.y, z1.z, z1.w};
-                    float e[8];
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) e[j] = a[j] * fmaf(-del, zz[j], __uint_as_float(v[8 * q + j]));
-                    *cell = make_uint4(pack_bf16(e[0], e[1]), pack_bf16(e[2], e[3]), pack_bf16(e[4], e[5]), pack_bf16(e[6], e[7]));
-                }
-            }
-            fence_async_smem();
-            tc_fence_before();
-            mbar_arrive_warp(bars + QE3);
-
-            EWAIT(QM5); if (!ok) break;
-            tc_fence_after();
-            if (col0 < D) tmem_row_to_tile(R1 + col0, sStg, r, col0, kLn2);  // this slab's part of dQ -> staging -> added into dQ
-            fence_async_smem();
+        int it = 0, run = 0;
+        for (long long l0 = lbeg; l0 < lend && ok; ++run) {
+            const int bh = (int)(l0 / T), t0 = (int)(l0 % T);
+            long long l1 = (long long)(bh + 1) * T;
+            if (l1 > lend) l1 = lend;
+            const int nrun = (int)(l1 - l0);
+            l0 = l1;
+            const int h = bh % p.H, row0 = bh * p.N;
+            const float cshift = p.cs[bh * p.nslab + slab];
+            if (g0) sZ[r] = (t0 > 0) ? __ldg(p.zc + ((size_t)bh * T + t0) * p.m + slab * 128 + r) : 0.f;
             epi_sync();
-            if (tid == 0) {
-                for (int a = 0; a < D / 64; ++a) {
-                    if (p.nslab > 1) tma_reduce_add_2d(&p.mapDQ, sStg + a * 16384, a * 64, row0 + t * 128);
-                    else tma_store_2d(&p.mapDQ, sStg + a * 16384, a * 64, row0 + t * 128);
+            for (int c = 0; c < nrun && ok; ++c, ++it) {
+                const int t = t0 + c;
+                const uint32_t ph = it & 1;
+                const bool last = (c + 1 == nrun);
+                const size_t row = (size_t)row0 + (size_t)t * 128 + r;
+#define EWAIT(b) do { ok = __all_sync(0xffffffffu, wait_or_abort(bars + (b), ph, status, abort_flag)); } while (0)
+                const float2 svv = p.sv[row];
+                const float del = p.delta[row];
+                const float nk = p.nK[row] + cshift;
+                const float aq = svv.y - cshift + log2f(svv.x);
+                // z before the next chunk, from the forward pass (loaded early, used at the end of the chunk)
+                const float znext = (g0 && !last) ? __ldg(p.zc + ((size_t)bh * T + t + 1) * p.m + slab * 128 + r) : 0.f;
+                float dtile[4] = {0.f, 0.f, 0.f, 0.f};       // warp 0: -delta of rows lane, lane + 32, ... for the operand of rho_c
+                if (warp == 0) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) dtile[i] = -__ldg(p.delta + (size_t)row0 + (size_t)t * 128 + i * 32 + lane);
                 }
-                tma_store_commit();
-            }
-            EWAIT(QMS); if (!ok) break;
-            if (!last) {
-                if (col0 < DV) tmem_row_to_tile(lane_addr + kColState + col0, sSt, r, col0);
-                if (g0) sZ[r] = znext;
+                EWAIT(QM2); if (!ok) break;
+                tc_fence_after();
+                features_to_tile(R2 + col0, nk, sKB, r, col0);                             // Bf
+                if (warp == 0) {
+                    // 16 x 128 K-major operand of rho_c = -A^^T delta at the start of the staging tile: row 0 = -delta rounded
+                    // to bf16, row 1 = the rounding's remainder. Written by the warp whose first lane has just seen the
+                    // previous chunk's store leave the tile.
+                    if (tid == 0) tma_store_wait_read();
+                    __syncwarp();
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int k = i * 32 + lane;
+                        const float dk = dtile[i];
+                        const __nv_bfloat16 hi = __float2bfloat16_rn(dk);
+                        const __nv_bfloat16 lo = __float2bfloat16_rn(dk - __bfloat162float(hi));
+                        const int atom = k >> 6, kk = k & 63, ch = kk >> 3;
+                        *reinterpret_cast<__nv_bfloat16 *>(sStg + atom * 2048 + (ch << 4) + (kk & 7) * 2) = hi;
+                        *reinterpret_cast<__nv_bfloat16 *>(sStg + atom * 2048 + 128 + ((ch ^ 1) << 4) + (kk & 7) * 2) = lo;
+                    }
+                }
                 fence_async_smem();
-            }
-            tc_fence_before();
-            mbar_arrive_warp(bars + QE4);
+                tc_fence_before();
+                mbar_arrive_warp(bars + QE0);
+                EWAIT(QM1); if (!ok) break;
+                tc_fence_after();
+                features_to_tile(R1 + col0, aq, sQA, r, col0);                             // A^
+                fence_async_smem();
+                tc_fence_before();
+                mbar_arrive_warp(bars + QE1);
+
+                EWAIT(QM3); if (!ok) break;
+                tc_fence_after();
+                {   // dP = tril(dO V^T - delta) as a bf16 operand in TMEM (packed over the fp32 tile)
+                    uint32_t v[32], pk[16];
+                    tmem_ld32(R2 + col0, v);
+                    tmem_wait_ld();
+                    tc_fence_before();
+                    mbar_arrive_warp(bars + QE2A);
+                    quarter_sync(q4);                         // every column group has read before anyone overwrites
+#pragma unroll
+                    for (int j = 0; j < 32; j += 2) {
+                        const float x0 = (col0 + j <= r) ? __uint_as_float(v[j]) - del : 0.f;
+                        const float x1 = (col0 + j + 1 <= r) ? __uint_as_float(v[j + 1]) - del : 0.f;
+                        pk[j / 2] = pack_bf16(x0, x1);
+                    }
+                    tmem_st16(R2 + col0 / 2, pk);
+                }
+                tmem_wait_st();
+                tc_fence_before();
+                mbar_arrive_warp(bars + QE2);
+
+                EWAIT(QM4); if (!ok) break;
+                tc_fence_after();
+                if (g0) {       // rho_c of feature r (TMEM lane r; its MMAs ran ahead of dP Bf), for the key-side kernel
+                    uint32_t v[16];
+                    tmem_ld16(R2 + 64, v);
+                    tmem_wait_ld();
+                    p.rhoc[((size_t)bh * T + t) * p.m + slab * 128 + r] = __uint_as_float(v[0]) + __uint_as_float(v[1]);
+                }
+                {   // E = A^ .* (dP Bf + dO S^T - delta z^T), in place over A^
+                    uint32_t v[32];
+                    tmem_ld32(R1 + col0, v);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        uint4 *cell = reinterpret_cast<uint4 *>(tile_chunk(sQA, r, col0 / 8 + q));
+                        float a[8];
+                        unpack8(*cell, a);
+                        const float4 z0 = *reinterpret_cast<const float4 *>(sZ + col0 + 8 * q);
+                        const float4 z1 = *reinterpret_cast<const float4 *>(sZ + col0 + 8 * q + 4);
+                        const float zz[8] = {z0.x, z0.y, z0.z, z0.w, z1.x, z1.y, z1.z, z1.w};
+                        float e[8];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) e[j] = a[j] * fmaf(-del, zz[j], __uint_as_float(v[8 * q + j]));
+                        *cell = make_uint4(pack_bf16(e[0], e[1]), pack_bf16(e[2], e[3]), pack_bf16(e[4], e[5]), pack_bf16(e[6], e[7]));
+                    }
+                }
+                fence_async_smem();
+                tc_fence_before();
+                mbar_arrive_warp(bars + QE3);
+
+                EWAIT(QM5); if (!ok) break;
+                tc_fence_after();
+                if (col0 < D) tmem_row_to_tile(R1 + col0, sStg, r, col0, kLn2);  // this slab's part of dQ -> staging -> added into dQ
+                fence_async_smem();
+                epi_sync();
+                if (tid == 0) {
+                    for (int a = 0; a < D / 64; ++a) {
+                        if (p.nslab > 1) tma_reduce_add_2d(&p.mapDQ, sStg + a * 16384, a * 64, row0 + t * 128);
+                        else tma_store_2d(&p.mapDQ, sStg + a * 16384, a * 64, row0 + t * 128);
+                    }
+                    tma_store_commit();
+                }
+                if (g0 && !last) sZ[r] = znext;       // every reader of z is past its E step (E Omega was issued behind all of them)
+                tc_fence_before();
+                mbar_arrive_warp(bars + QE4);
 #undef EWAIT
+            }
+            // the run's T: every MMA of the run completed before its last T += E^T Q did
+            if (ok) ok = __all_sync(0xffffffffu, wait_or_abort(bars + QM6, (it - 1) & 1, status, abort_flag));
+            if (ok) {
+                tc_fence_after();
+                if (col0 < D) {
+                    float *dst = p.Tacc + ((size_t)h * p.m + slab * 128 + r) * D + col0;
+                    uint32_t v[32];
+                    tmem_ld32(lane_addr + kColT + col0, v);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) atomicAdd(dst + j, __uint_as_float(v[j]));
+                }
+                tc_fence_before();
+                mbar_arrive_warp(bars + QET);
+            }
         }
         if (tid == 0) tma_store_wait_all();
-        if (ok) ok = wait_or_abort(bars + QM6, (T - 1) & 1, status, abort_flag);
-        if (ok && col0 < D) {
-            tc_fence_after();
-            float *dst = p.Tacc + ((size_t)h * p.m + slab * 128 + r) * D + col0;
-            uint32_t v[32];
-            tmem_ld32(lane_addr + kColT + col0, v);
-            tmem_wait_ld();
-#pragma unroll
-            for (int j = 0; j < 32; ++j) atomicAdd(dst + j, __uint_as_float(v[j]));
-        }
     }
     if (*abort_flag) __nanosleep(200000);   // error path only: let copies and MMAs in flight drain
     tc_fence_before();
@@ -884,6 +919,17 @@ __global__ void dw_kernel(const float *Tacc, const __nv_bfloat16 *M, float *dW, 
     dW[((size_t)(w_per_head ? blockIdx.y : 0) * m + l) * r + a] = s * acc;
 }
 
+int sm_count()
+{
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) n = v;
+        else n = 148;
+    }
+    return n;
+}
+
 template <int D, int DV>
 cudaError_t launch_scan(const darkattn_plan_s *plan, const BwdParams &P, int grid, cudaStream_t st)
 {
@@ -893,8 +939,13 @@ cudaError_t launch_scan(const darkattn_plan_s *plan, const BwdParams &P, int gri
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(tc_bwd_k_kernel<D, DV>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
     if (e != cudaSuccess) return e;
+    // the query-side kernel divides all chunks evenly over the SMs: groups of nslab CTAs, one group per piece
+    long long groups = sm_count() / P.nslab;
+    if (groups < 1) groups = 1;
+    if (groups > (long long)P.BH * P.T) groups = (long long)P.BH * P.T;
+    const int qgrid = (int)groups * P.nslab;
     timer_mark(plan, st, "tc_bwd_q_kernel");
-    tc_bwd_q_kernel<D, DV><<<grid, kThreads, L::kTotal, st>>>(P);
+    tc_bwd_q_kernel<D, DV><<<qgrid, kThreads, L::kTotal, st>>>(P);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (P.nslab > 1) {
@@ -941,7 +992,7 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
     // workspace by running the forward kernels again.
     Stash stash;
     if (!O || !saved) {
-        darkattn_status_t s = tensor_forward(plan, Q, K, V, M, W, bf(Y.Oscr), nullptr, ws, st);
+        darkattn_status_t s = tensor_forward(plan, Q, K, V, M, W, bf(Y.Oscr), nullptr, ws, st, true);
         if (s != DARKATTN_OK) return s;
         O = bf(Y.Oscr);
         stash = stash_in_workspace(Y, ws);
@@ -987,7 +1038,8 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
                         make_map(&P.mapOm, stash.Om, (size_t)D.H * D.m, D.d, 128) &&
                         make_map(&P.mapDQ, dQ, BH * N, D.d, 128) && make_map(&P.mapDK, dK, BH * N, D.d, 128) &&
                         make_map(&P.mapDV, dV, BH * N, D.dv, 128) &&
-                        make_map(&P.mapAh, bf(Y.Ahat), BH * N, D.m, 128) && make_map(&P.mapBf, bf(Y.Bphi), BH * N, D.m, 128);
+                        make_map(&P.mapAh, bf(Y.Ahat), BH * N, D.m, 128) && make_map(&P.mapBf, bf(Y.Bphi), BH * N, D.m, 128) &&
+                        make_map(&P.mapSst, stash.Sst, BH * Y.T * D.m, D.dv, 128);
         if (!ok) { set_cuda_error(cudaErrorInvalidValue, "tensor_backward: tensor map encode"); return DARKATTN_ERR_CUDA; }
         P.sv = stash.sv; P.delta = fl(Y.delta); P.nK = stash.nK; P.cs = stash.cs; P.zc = stash.zc; P.rhoc = fl(Y.rhoc);
         P.espart = fl(Y.espart); P.Tacc = fl(Y.Tacc);

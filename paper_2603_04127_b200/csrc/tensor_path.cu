@@ -169,6 +169,8 @@ __global__ void __launch_bounds__(160, 1) tc_key_norms_kernel(const __grid_const
 // ------------------------------------------------------------------ the main kernel
 struct MainParams {
     CUtensorMap mapQ, mapK, mapV, mapOm, mapSb, mapPN;
+    CUtensorMap mapSst;  // causal, when stash_S: S before every chunk as [BH*T*m, dv] bf16, for the backward pass
+    int stash_S;
     const float *nK;     // [BH, N]      key norms in log2 units
     const float *cs;     // [BH, nslab]  key-side shift per slab (log2 units)
     float *pdr;          // [nslab, BH*N, 2]  partial normaliser and the exponent the partial is scaled by
@@ -367,6 +369,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
                 mma_commit(bars + CM4);
                 // the state update is not on the chunk's critical path: it runs while the output tile is read out
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColS, mndesc(tFK, k), mndesc(tV, k), id_s, (!first) || k > 0);   // S += phi(K)^T V
+                if (p.stash_S) tma_store_wait_read();       // the stash copy of the state before this chunk has left its tile
                 mma_commit(bars + CMS);
                 if (!last) {
                     ok = wait_or_abort(bars + CB_Q, ph ^ 1, status, abort_flag);
@@ -379,8 +382,13 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
                 if (!last) load_tile(sV, &p.mapV, bars + CB_V, DV, t + 1);
                 CWAIT(CE3); if (!ok) break;
                 CWAIT(CE4); if (!ok) break;
+                if (p.stash_S && t + 1 < p.T) {         // the state through this chunk, bf16: what the backward pass starts chunk t + 1 from
+                    for (int a = 0; a < DV / 64; ++a) tma_store_2d(&p.mapSst, sSb + a * 16384, a * 64, (bh * p.T + t + 1) * p.m + slab * 128);
+                    tma_store_commit();
+                }
 #undef CWAIT
             }
+            tma_store_wait_all();
         }
     } else {
         const int lane = tid & 31, q4 = warp & 3, g = warp >> 2, col0 = g * 32;
@@ -462,7 +470,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
             quarter_sync(q4);                      // the exchange array is free for the next chunk's maxima
             EWAIT(CMS); if (!ok) break;
             tc_fence_after();
-            if (!last) {
+            if (!last || (p.stash_S && t + 1 < p.T)) {
                 if (col0 < DV) tmem_row_to_tile(lane_addr + kColS + col0, sSb, r, col0);
                 fence_async_smem();
             }
@@ -994,6 +1002,7 @@ void tensor_make_layout(darkattn_plan_s *plan)
         Y.sv_zc = take(so, D.causal ? BH * (size_t)Y.T * m * 4 : 0);
         Y.sv_Sb = take(so, D.causal ? 0 : BH * m * dv * 2);
         Y.sv_zt = take(so, D.causal ? 0 : BH * m * 4);
+        Y.sv_Sst = take(so, D.causal ? BH * (size_t)Y.T * m * dv * 2 : 0);
         Y.sv_bytes = so;
         plan->saved_bytes = so;
     }
@@ -1004,6 +1013,7 @@ void tensor_make_layout(darkattn_plan_s *plan)
     Y.espart = take(off, (size_t)4 * Y.nslab * BH * N * 4);
     Y.Tacc = take(off, (size_t)D.H * m * d * 4);
     Y.dMn = take(off, (size_t)D.H * D.r * d * 4);
+    Y.Sst = take(off, D.causal ? BH * (size_t)Y.T * m * dv * 2 : 0);
     Y.Ahat = take(off, D.causal ? BH * N * m * 2 : 0);
     Y.Bphi = take(off, D.causal ? BH * N * m * 2 : 0);
     Y.Racc = take(off, D.causal ? 0 : BH * m * dv * 4);
@@ -1055,7 +1065,7 @@ cudaError_t tensor_prologue(const darkattn_plan_s *plan, const void *K, const vo
 }
 
 darkattn_status_t tensor_forward(const darkattn_plan_s *plan, const void *Q, const void *K, const void *V,
-                                 const void *M, const void *W, void *O, void *saved, char *ws, cudaStream_t st)
+                                 const void *M, const void *W, void *O, void *saved, char *ws, cudaStream_t st, bool stash_states)
 {
     const Dims &D = plan->dims;
     const TensorLayout &Y = plan->tensor;
@@ -1079,6 +1089,11 @@ darkattn_status_t tensor_forward(const darkattn_plan_s *plan, const void *Q, con
     P.nK = stash.nK; P.cs = stash.cs; P.zc = stash.zc; P.pdr = fl(Y.pdr); P.Sacc = fl(Y.Sacc); P.zacc = fl(Y.zacc);
     P.status = reinterpret_cast<int *>(ws + Y.status);
     P.N = D.N; P.H = D.H; P.BH = D.BH; P.m = D.m; P.nslab = Y.nslab; P.T = Y.T; P.nsplit = Y.nsplit;
+    P.stash_S = (D.causal && stash_states) ? 1 : 0;
+    if (P.stash_S && !make_map(&P.mapSst, stash.Sst, BH * Y.T * D.m, D.dv, 128)) {
+        set_cuda_error(cudaErrorInvalidValue, "tensor_forward: tensor map encode");
+        return DARKATTN_ERR_CUDA;
+    }
     const int units = (int)(BH * Y.nslab);
     if (D.causal) {
         if (Y.nsplit > 1) {      // segment states, then their exclusive prefix
