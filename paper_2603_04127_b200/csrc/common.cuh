@@ -146,6 +146,16 @@ struct darkattn_plan_s {
 namespace darkattn {
 
 void set_cuda_error(cudaError_t e, const char *where);
+// The plan's side stream and the two events that fork work onto it and join it back (created on first use).
+inline cudaError_t ensure_aux(const darkattn_plan_s *plan)
+{
+    if (plan->aux_stream) return cudaSuccess;
+    cudaError_t e = cudaStreamCreateWithFlags(&plan->aux_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&plan->aux_fork, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&plan->aux_join, cudaEventDisableTiming);
+    return e;
+}
+
 // Records an event in front of the kernel `name` (nullptr: after the last kernel of a call) when timing is on.
 void timer_mark(const darkattn_plan_s *plan, cudaStream_t st, const char *name);
 

@@ -894,9 +894,16 @@ __global__ void dm_kernel(const __nv_bfloat16 *W, const float *Tacc, const float
     for (int j = 0; j < 8; ++j)
         if (a0 + j < r) {
             float v = s * acc[j];
-            if (lb == 0) v += dMn[((size_t)h * r + a0 + j) * d + c];
+            if (lb == 0 && dMn) v += dMn[((size_t)h * r + a0 + j) * d + c];
             atomicAdd(dM + ((size_t)h * r + a0 + j) * d + c, v);
         }
+}
+
+// dM += dMn (the norm term's part, when dm_kernel ran beside the kernel that produces it)
+__global__ void dm_add_kernel(float *dM, const float *dMn, int n)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) dM[i] += dMn[i];
 }
 
 // dW[(h,) l, a] = s * sum_c T[h,l,c] M[h,a,c], summed over the heads when W is shared: through the folded projection
@@ -1009,12 +1016,8 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
     if (Y.nslab > 1) {
         // The slabs of a head add their parts into the gradients, which therefore start at zero. dQ is needed first;
         // dK and dV are zeroed on a side stream while the query-side scan runs (it leaves SMs and bandwidth free).
-        if (!plan->aux_stream) {
-            keep(cudaStreamCreateWithFlags(&plan->aux_stream, cudaStreamNonBlocking));
-            keep(cudaEventCreateWithFlags(&plan->aux_fork, cudaEventDisableTiming));
-            keep(cudaEventCreateWithFlags(&plan->aux_join, cudaEventDisableTiming));
-            if (e != cudaSuccess) { set_cuda_error(e, "tensor_backward: side stream"); return DARKATTN_ERR_CUDA; }
-        }
+        keep(ensure_aux(plan));
+        if (e != cudaSuccess) { set_cuda_error(e, "tensor_backward: side stream"); return DARKATTN_ERR_CUDA; }
         keep(cudaEventRecord(plan->aux_fork, st));
         keep(cudaStreamWaitEvent(plan->aux_stream, plan->aux_fork, 0));
         keep(cudaMemsetAsync(dK, 0, BH * N * D.d * 2, plan->aux_stream));
@@ -1059,14 +1062,34 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
     F.status = reinterpret_cast<int *>(ws + Y.status);
     F.N = D.N; F.H = D.H; F.BH = D.BH; F.T = Y.T; F.r = D.r; F.nslab = 1; F.nes = 4 * Y.nslab; F.s2 = D.s * D.s;
     F.nsplit = pick_splits((long long)BH, Y.T, 3.5, 5.0, 64);
+    // dM = s W^T T + (norm term). T is complete once the key-side pass is done, so its product runs on the side
+    // stream next to the kernel that produces the norm term, and a small kernel adds the two. (With per-kernel
+    // timing on, everything stays on one stream.)
+    const dim3 dm_grid((D.r + 7) / 8, D.H, D.m / 64);
+    const bool beside = !plan->timer.on && ensure_aux(plan) == cudaSuccess;
+    if (beside) {
+        keep(cudaEventRecord(plan->aux_fork, st));
+        keep(cudaStreamWaitEvent(plan->aux_stream, plan->aux_fork, 0));
+        keep(cudaMemsetAsync(dM, 0, (size_t)D.H * D.r * D.d * 4, plan->aux_stream));
+        dm_kernel<<<dm_grid, D.d, 0, plan->aux_stream>>>((const __nv_bfloat16 *)W, fl(Y.Tacc), nullptr, dM, D.m, D.r, D.d, D.w_per_head, D.s);
+        chk();
+        keep(cudaEventRecord(plan->aux_join, plan->aux_stream));
+    }
     timer_mark(plan, st, "tc_bwd_finish_k_kernel");
     if (D.d == 64) keep(launch_finish<64>(F, (int)(BH * F.nsplit), st));
     else keep(launch_finish<128>(F, (int)(BH * F.nsplit), st));
 
-    timer_mark(plan, st, "dm_kernel");
-    keep(cudaMemsetAsync(dM, 0, (size_t)D.H * D.r * D.d * 4, st));
-    dm_kernel<<<dim3((D.r + 7) / 8, D.H, D.m / 64), D.d, 0, st>>>((const __nv_bfloat16 *)W, fl(Y.Tacc), fl(Y.dMn), dM, D.m, D.r, D.d, D.w_per_head, D.s);
-    chk();
+    if (beside) {
+        keep(cudaStreamWaitEvent(st, plan->aux_join, 0));
+        const int n = D.H * D.r * D.d;
+        dm_add_kernel<<<(n + 255) / 256, 256, 0, st>>>(dM, fl(Y.dMn), n);
+        chk();
+    } else {
+        timer_mark(plan, st, "dm_kernel");
+        keep(cudaMemsetAsync(dM, 0, (size_t)D.H * D.r * D.d * 4, st));
+        dm_kernel<<<dm_grid, D.d, 0, st>>>((const __nv_bfloat16 *)W, fl(Y.Tacc), fl(Y.dMn), dM, D.m, D.r, D.d, D.w_per_head, D.s);
+        chk();
+    }
     if (e != cudaSuccess) { set_cuda_error(e, "tensor_backward"); return DARKATTN_ERR_CUDA; }
     return DARKATTN_OK;
 }

@@ -1039,13 +1039,22 @@ cudaError_t tensor_prologue(const darkattn_plan_s *plan, const void *K, const vo
     cudaError_t e = cudaSuccess;
     auto chk = [&]() { cudaError_t x = cudaGetLastError(); if (x != cudaSuccess && e == cudaSuccess) e = x; };
 
+    // The two small kernels that read only M and W run on the side stream next to the key-norm kernel (with
+    // per-kernel timing on, everything stays on one stream).
+    const bool beside = !plan->timer.on && ensure_aux(plan) == cudaSuccess;
+    cudaStream_t sp = beside ? plan->aux_stream : st;
+    if (beside) {
+        e = cudaEventRecord(plan->aux_fork, st);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(sp, plan->aux_fork, 0);
+    }
     timer_mark(plan, st, "fold_omega_kernel");
-    fold_omega_kernel<<<dim3(D.m / 4, D.H), D.d, 0, st>>>((const __nv_bfloat16 *)W, (const __nv_bfloat16 *)M, out.Om, D.m, D.r, D.d,
+    fold_omega_kernel<<<dim3(D.m / 4, D.H), D.d, 0, sp>>>((const __nv_bfloat16 *)W, (const __nv_bfloat16 *)M, out.Om, D.m, D.r, D.d,
                                                       D.w_per_head, kLog2e * D.s);
     chk();
     timer_mark(plan, st, "slab_shift_kernel");
-    slab_shift_kernel<<<(unsigned)(BH * Y.nslab), 128, 0, st>>>((const __nv_bfloat16 *)W, out.cs, D.H, D.m, D.r, Y.nslab, D.w_per_head);
+    slab_shift_kernel<<<(unsigned)(BH * Y.nslab), 128, 0, sp>>>((const __nv_bfloat16 *)W, out.cs, D.H, D.m, D.r, Y.nslab, D.w_per_head);
     chk();
+    if (beside && e == cudaSuccess) e = cudaEventRecord(plan->aux_join, sp);
 
     NP.nK = out.nK; NP.status = reinterpret_cast<int *>(ws + Y.status);
     NP.N = D.N; NP.H = D.H; NP.T = Y.T; NP.r = D.r;
@@ -1061,6 +1070,7 @@ cudaError_t tensor_prologue(const darkattn_plan_s *plan, const void *K, const vo
         tc_key_norms_kernel<128><<<(unsigned)(BH * NP.nsplit), 160, smem_bytes, st>>>(NP);
     }
     chk();
+    if (beside && e == cudaSuccess) e = cudaStreamWaitEvent(st, plan->aux_join, 0);
     return e;
 }
 
