@@ -29,7 +29,7 @@ if ROOT not in sys.path:
 # DRAM bytes (read + write) per (token, head) of the scan kernels at d = dv = 128, m = 256 from their ncu capture on the
 # small profiling workload (profiles/scan_kernels_d128_small.md); traffic is proportional to the (token, head) count.
 # A kernel that changed since its capture has no entry.
-NCU_TRAFFIC_PER_TOKEN_HEAD = {"tc_fwd_causal_kernel": 1083.0, "tc_bwd_q_kernel": 1516.0, "tc_bwd_k_kernel": 1966.0}
+NCU_TRAFFIC_PER_TOKEN_HEAD = {"tc_fwd_causal_kernel": 1472.0, "tc_bwd_q_kernel": 2899.0, "tc_bwd_k_kernel": 2796.0}
 
 METRIC = "DARK-attention fwd+bwd tokens/s"
 UNIT = "tokens/s"
@@ -37,12 +37,14 @@ UNIT = "tokens/s"
 
 def flops_per_token_head(d, r, m, dv, C, causal, backward):
     """Algorithmic floating-point operations per (token, head); intra-chunk terms count the lower
-    triangle only."""
+    triangle only. Backward: the features are computed once more (query-side kernel; the key-side
+    kernel reads them back), and the state before each chunk comes from the forward stash instead of
+    being recomputed, so the state terms are dO S^T, R += A^T dO, V R^T and Bf R: 8 m dv."""
     feat = 2 * (2 * d * r + 2 * r * m)                 # both sides: x~ = M x and u = W x~
     fwd = feat + 4 * m * dv + ((C + 1) * (m + dv) if causal else 0)
     if not backward:
         return fwd
-    bwd = feat + 10 * m * dv + ((C + 1) * (3 * m + 2 * dv) if causal else 0) + 4 * m * r + 8 * r * d
+    bwd = feat + 8 * m * dv + ((C + 1) * (3 * m + 2 * dv) if causal else 0) + 4 * m * r + 8 * r * d
     return fwd + bwd
 
 
@@ -57,9 +59,11 @@ def exps_per_token_head(m, backward):
 
 def kernel_work(d, r, m, dv, C, nslab, causal):
     """Algorithmic work per (token, head) of each kernel of the tensor-core path: (flops, exps, bytes,
-    bound). The scan kernels split the step's total of flops_per_token_head() between them (each is
-    charged half of the backward feature recompute and of the feature-map backward); the helper kernels
-    are HBM-bound and are charged the tensors they read and write once."""
+    bound). The scan kernels split the step's total of flops_per_token_head() between them: the causal
+    query-side backward kernel is charged the whole feature recompute (the key-side kernel reads its
+    feature tiles back), each backward kernel half of the feature-map backward; bytes count what the
+    kernel has to move once (inputs, outputs, and the stashed tiles it reads or writes). The helper
+    kernels are HBM-bound and are charged the tensors they read and write once."""
     feat = 2 * (2 * d * r + 2 * r * m)
     tri = C + 1
     e = 2
@@ -67,8 +71,9 @@ def kernel_work(d, r, m, dv, C, nslab, causal):
         "tc_fwd_causal_kernel": (feat + 4 * m * dv + tri * (m + dv), 2 * m, (2 * d + 2 * dv) * e, "tensor"),
         "tc_fwd_keys_kernel": (feat // 2 + 2 * m * dv, m, (d + dv) * e, "tensor"),
         "tc_fwd_queries_kernel": (feat // 2 + 2 * m * dv, m, (d + dv) * e, "tensor"),
-        "tc_bwd_q_kernel": (feat // 2 + 4 * m * dv + tri * (m + dv) + 2 * m * r + 4 * r * d, m, (3 * d + 2 * dv) * e, "tensor"),
-        "tc_bwd_k_kernel": (feat // 2 + 6 * m * dv + tri * (2 * m + dv) + 2 * m * r + 4 * r * d, m, (3 * d + 3 * dv) * e, "tensor"),
+        "tc_bwd_q_kernel": (feat + 2 * m * dv + tri * (m + dv) + 2 * m * r + 4 * r * d, 2 * m,
+                            (3 * d + 2 * dv + 2 * m) * e + m * dv * e // C, "tensor"),
+        "tc_bwd_k_kernel": (6 * m * dv + tri * (2 * m + dv) + 2 * m * r + 4 * r * d, 0, (2 * d + 3 * dv + 2 * m) * e, "tensor"),
         "tc_bwd_nc_q_kernel": (feat // 2 + 4 * m * dv + 2 * m * r + 4 * r * d, m, (2 * d + dv) * e, "tensor"),
         "tc_bwd_nc_k_kernel": (feat // 2 + 4 * m * dv + 2 * m * r + 4 * r * d, m, (2 * d + 2 * dv) * e, "tensor"),
         "tc_bwd_finish_k_kernel": (6 * r * d, 0, 3 * d * e, "hbm"),
@@ -344,6 +349,10 @@ def main():
     flops = flops_per_token_head(d, r, m, dv, 128, wl.causal, wl.backward) * th
     nbytes = bytes_per_token_head(d, dv, wl.backward) * th
     nexp = exps_per_token_head(m, wl.backward) * th
+    # cycles per 128x128x16 MMA with both operands in shared memory, alone and beside busy epilogue warps, and the
+    # fixed cycles a batch pays between its first issue and the arrival of its commit
+    mma_alone, mma_fixed = binding.darkattn_measure_mma_cycles(0, False)
+    mma_busy, _ = binding.darkattn_measure_mma_cycles(2, True)
     ex2_peak = binding.darkattn_measure_alu_peak(0, 10)
     fma_peak = binding.darkattn_measure_alu_peak(1, 10)
     legs = {"tensor_us": flops / (peaks["bf16_tflops_sustained"] * 1e12) * 1e6,
@@ -385,6 +394,7 @@ def main():
         roofline = dict(whole, traffic=None, kernel="whole step")
     roofline.update(peak_source=peaks["source"] + " (sustained bf16 GEMM / copy bandwidth)", whole_step=whole, kernels=kernels,
                     ex2_per_s_measured=ex2_peak, fma_per_s_measured=fma_peak, forward_ms=fwd_ms,
+                    mma_cycles={"ss_alone": mma_alone, "ss_mn_beside_epilogue": mma_busy, "per_batch_fixed": mma_fixed},
                     forward_tokens_per_s=world * tokens / (fwd_ms * 1e-3))
 
     out = {

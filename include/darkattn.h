@@ -156,6 +156,18 @@ const char *darkattn_last_cuda_error(void);
 darkattn_status_t darkattn_measure_alu_peak(int32_t which, int32_t iters, double *ops_per_second,
                                             void *cuda_stream);
 
+/* Measure what one tcgen05.mma (bf16, M = 128, K = 16) costs on this GPU in the forms the scan kernels
+ * issue, so that their tensor-pipe time can be told apart from the hand-over between MMA batches and
+ * the warps that consume them. variant: 0 both operands in shared memory, K-major, N = 128; 1 B MN-major;
+ * 2 A and B MN-major; 3 A in tensor memory, B K-major; 4 A in tensor memory, B MN-major; 5 as 0 with
+ * N = 256; 6 as 0 with N = 64; 7 A MN-major, N = 16. One CTA per SM issues two batches of dependent MMAs
+ * (32 and 288) and waits for each batch's commit with a bounded wait; busy_epilogue != 0 makes the 16
+ * other warps read tensor memory and write shared memory meanwhile. Writes the SM-clock cycles per MMA
+ * (slope) and the fixed cycles per batch (intercept) to the two host pointers. Synchronises the
+ * stream. DARKATTN_ERR_TIMEOUT if a commit did not arrive within the wait's limit.                 */
+darkattn_status_t darkattn_measure_mma_cycles(int32_t variant, int32_t busy_epilogue, double *cycles_per_mma,
+                                              double *batch_overhead_cycles, void *cuda_stream);
+
 /* Per-kernel device times, for benchmarks. While enabled, forward and backward record a CUDA event on
  * the call's stream in front of every kernel they launch and one behind the last (events are host
  * objects created by the first enabling call; no device memory is involved). Enabling also clears the

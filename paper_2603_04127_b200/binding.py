@@ -24,7 +24,7 @@ EXPORTS = [
     "darkattn_plan_launches", "darkattn_forward", "darkattn_backward", "darkattn_last_device_status",
     "darkattn_destroy", "darkattn_status_string", "darkattn_last_cuda_error", "darkattn_measure_alu_peak",
     "darkattn_static_scratch_needed", "darkattn_forward_static", "darkattn_kernel_timing", "darkattn_kernel_times",
-    "darkattn_backward_dw", "darkattn_decode_step",
+    "darkattn_backward_dw", "darkattn_decode_step", "darkattn_measure_mma_cycles",
 ]
 STATIC_SCRATCH_BYTES = 16 << 20
 
@@ -70,6 +70,9 @@ lib.darkattn_last_cuda_error.argtypes = []
 lib.darkattn_last_cuda_error.restype = ctypes.c_char_p
 lib.darkattn_measure_alu_peak.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(ctypes.c_double), _vp]
 lib.darkattn_measure_alu_peak.restype = ctypes.c_int
+lib.darkattn_measure_mma_cycles.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(ctypes.c_double),
+                                            ctypes.POINTER(ctypes.c_double), _vp]
+lib.darkattn_measure_mma_cycles.restype = ctypes.c_int
 lib.darkattn_kernel_timing.argtypes = [_vp, ctypes.c_int32]
 lib.darkattn_kernel_timing.restype = ctypes.c_int
 lib.darkattn_kernel_times.argtypes = [_vp, ctypes.c_int32, ctypes.c_char_p, ctypes.POINTER(ctypes.c_float),
@@ -190,6 +193,14 @@ def darkattn_measure_alu_peak(which: int, iters: int = 20, stream=None) -> float
     _check(lib.darkattn_measure_alu_peak(which, iters, ctypes.byref(out), _stream(stream)),
            "darkattn_measure_alu_peak")
     return out.value
+
+
+def darkattn_measure_mma_cycles(variant: int, busy_epilogue: bool = False, stream=None):
+    """(cycles per MMA, fixed cycles per batch) of one tcgen05.mma form; see the header for the variants."""
+    per, fixed = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    _check(lib.darkattn_measure_mma_cycles(variant, int(bool(busy_epilogue)), ctypes.byref(per), ctypes.byref(fixed),
+                                           _stream(stream)), "darkattn_measure_mma_cycles")
+    return per.value, fixed.value
 
 
 def darkattn_kernel_timing(plan: Plan, enable: bool):

@@ -254,6 +254,19 @@ def test_tensor_path_is_deterministic(binding):
             assert worst < 2.0 ** -7, f"{k} differs between runs by {worst:.2e} of its largest value"
 
 
+def test_mma_cycle_measurement_is_sane(binding):
+    """The instrument behind the scan kernels' tensor-pipe accounting: a 128x128x16 bf16 MMA cannot beat the
+    pipe's 8192 flop per clock (64 cycles), and none of the forms the kernels use should cost twice that."""
+    for variant in range(5):
+        per, fixed = binding.darkattn_measure_mma_cycles(variant, False)
+        assert 60.0 < per < 128.0, (variant, per)
+        assert 0.0 < fixed < 5000.0, (variant, fixed)
+    per256, _ = binding.darkattn_measure_mma_cycles(5, False)
+    assert 120.0 < per256 < 256.0, per256
+    busy, _ = binding.darkattn_measure_mma_cycles(2, True)
+    assert 60.0 < busy < 128.0, busy
+
+
 def test_kernel_timing_reports_every_kernel_of_a_step(binding):
     import torch
     wl = inputs.small(name="timing", wid=91, B=1, H=2, N=512, d=64, m=256, causal=True, dtype="bf16", backward=True)
