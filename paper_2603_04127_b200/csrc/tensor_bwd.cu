@@ -121,6 +121,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
             const uint32_t id_dx = make_idesc(128, D, 0, 1);
             const uint32_t id_t = make_idesc(128, D, 1, 1);
             const uint32_t R1 = tmem + kColR1, R2 = tmem + kColR2;
+            // The Q tile that T += E^T Q needs is fetched again into the V tile's buffer as soon as dO V^T is done (where
+            // it fits), so that dO of the next chunk can follow early into its own buffer; otherwise into dO's buffer.
+            constexpr bool kQinV = (D <= DV);
 
             // Schedule of one chunk (R1, R2: the two scratch regions of TMEM). U_K of the next chunk is issued in
             // the tail of the current one, and dO V^T runs while the epilogue is still busy with A^.
@@ -181,6 +184,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                     QWAIT(QE1); if (!ok) break;                                                                  // A^ in smem, R1 read
                     store_features(sQA, &p.mapAh, t);
                     QWAIT(QE2A); if (!ok) break;                                                                 // dO V^T read out of R2
+                    if (kQinV) load_tile(sV, &p.mapQ, bars + QB_X2, D, t);                                      // V is done with: Q again, for T
                     tc_fence_after();
                     _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R2 + 64, mndesc(tQA, k), vecdesc(tDel, k), id_vec, k > 0);  // rho_c = -A^^T delta (columns 0, 1)
                     QWAIT(QE2); if (!ok) break;                                                                  // dP packed in R2
@@ -192,8 +196,13 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                     tma_store_wait_read();      // both feature tiles have left shared memory: E may overwrite A^, the next K tile Bf
                     mma_commit(bars + QM4);
                     QWAIT(QM4); if (!ok) break;                                                                  // Bf, V, dO and S of this chunk are done with
-                    load_tile(sG, &p.mapQ, bars + QB_X2, D, t);                                                 // Q again, for T
-                    if (!last) { load_tile(sV, &p.mapV, bars + QB_V, DV, t + 1); load_tile(sKB, &p.mapK, bars + QB_K, D, t + 1); load_state(t + 1); }
+                    if (!kQinV) load_tile(sG, &p.mapQ, bars + QB_X2, D, t);                                     // Q again, for T
+                    if (!last) {
+                        if (kQinV) load_tile(sG, &p.mapG, bars + QB_G, DV, t + 1);
+                        else load_tile(sV, &p.mapV, bars + QB_V, DV, t + 1);
+                        load_tile(sKB, &p.mapK, bars + QB_K, D, t + 1);
+                        load_state(t + 1);
+                    }
                     QWAIT(QE3); if (!ok) break;
                     QWAIT(QB_X2); if (!ok) break;
                     if (c == 0 && run > 0) {                                                                     // T of the previous run has been read out
@@ -203,7 +212,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                     tc_fence_after();
                     _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R1, kdesc(tQA, k), mndesc(tOm, k), id_dx, k > 0);        // E Omega
                     mma_commit(bars + QM5);
-                    _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColT, mndesc(tQA, k), mndesc(tG, k), id_t, (c > 0) || k > 0);   // T += E^T Q
+                    _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColT, mndesc(tQA, k), mndesc(kQinV ? tV : tG, k), id_t, (c > 0) || k > 0);   // T += E^T Q
                     mma_commit(bars + QM6);
                     if (!last) {
                         ok = wait_or_abort(bars + QB_K, ph ^ 1, status, abort_flag);
@@ -213,7 +222,11 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                         mma_commit(bars + QM2);
                     }
                     QWAIT(QM6); if (!ok) break;
-                    if (!last) { load_tile(sQA, &p.mapQ, bars + QB_Q, D, t + 1); load_tile(sG, &p.mapG, bars + QB_G, DV, t + 1); }
+                    if (!last) {
+                        load_tile(sQA, &p.mapQ, bars + QB_Q, D, t + 1);
+                        if (kQinV) load_tile(sV, &p.mapV, bars + QB_V, DV, t + 1);
+                        else load_tile(sG, &p.mapG, bars + QB_G, DV, t + 1);
+                    }
                     QWAIT(QE4); if (!ok) break;
 #undef QWAIT
                 }
