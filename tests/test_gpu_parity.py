@@ -153,6 +153,9 @@ TENSOR_BWD = [
     ("b_d128_dv64_r64", dict(B=1, H=2, N=256, d=128, m=128, dv=64, r=64, causal=True)),
     ("b_d64_dv128_r32", dict(B=2, H=2, N=384, d=64, m=256, dv=128, r=32, causal=True)),
     ("b_segmented_fwd", dict(B=1, H=2, N=1024, d=64, m=128, causal=True)),
+    # more (batch, head, chunk) items than CTA groups: a query-side CTA walks several runs, across heads
+    ("b_m512_runs", dict(B=2, H=4, N=2048, d=64, m=512, causal=True)),
+    ("b_d128_dv64_runs", dict(B=2, H=20, N=1024, d=128, m=128, dv=64, causal=True)),
     # no causal mask: one pass over the queries, one over the keys
     ("b_nc_one_tile", dict(B=1, H=1, N=128, d=64, m=128, causal=False)),
     ("b_nc_d64_m256", dict(B=2, H=3, N=640, d=64, m=256, causal=False)),
