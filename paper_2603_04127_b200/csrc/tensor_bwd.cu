@@ -657,34 +657,34 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
 //   w_j  = -s^2 rowsum(E^K)_j x~'_j   (bf16 operand)
 //   dK_j = (dK_j as the scan kernel left it) + w_j M          dMn += w^T K
 struct FinishParams {
-    CUtensorMap mapK, mapM, mapP, mapOut;   // K, M, dK without the norm term (nslab tensors stacked; here one: dK itself), dK
+    CUtensorMap mapK, mapM, mapOut;   // K, M, dK (the norm term's part is added into it)
     const float *espart;  // [nes, BH*N]
     float *dMn;           // [H, r, D]
     int *status;
-    int N, H, BH, T, nsplit, r, nslab, nes, pbufs;   // pbufs: partial tiles resident at a time
+    int N, H, BH, T, nsplit, r, nes;
     float s2;
 };
 
-// Shared memory: M tile, two K tiles, the w tile (32 KB), the output staging tile, pbufs partial tiles, barriers.
+// Shared memory: M tile, two K tiles, the w tile (32 KB), the output staging tile, barriers. The norm term's part of
+// dK is added into dK (which holds what the key-side pass added up) by TMA reduce-add stores.
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __grid_constant__ FinishParams p)
 {
     extern __shared__ __align__(1024) unsigned char smem[];
     constexpr int kTile = 128 * D * 2;
-    unsigned char *sM = smem, *sK0 = smem + kTile, *sW = smem + 3 * kTile, *sOut = sW + 32768, *sP = sOut + kTile;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(sP + (size_t)p.pbufs * kTile);
-    uint64_t *bar_m = bars, *bar_k = bars + 1 /* two */, *bar_p = bars + 3, *m1 = bars + 4, *m2 = bars + 5, *m3 = bars + 6;
-    uint64_t *e1 = bars + 7, *e2 = bars + 8, *e_p = bars + 9;
+    unsigned char *sM = smem, *sK0 = smem + kTile, *sW = smem + 3 * kTile, *sOut = sW + 32768;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(sOut + kTile);
+    uint64_t *bar_m = bars, *bar_k = bars + 1 /* two */, *m1 = bars + 4, *m2 = bars + 5, *m3 = bars + 6;
+    uint64_t *e1 = bars + 7, *e2 = bars + 8;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 10);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 11);
     const int tid = threadIdx.x, warp = tid >> 5;
     const int bh = blockIdx.x / p.nsplit, split = blockIdx.x % p.nsplit, h = bh % p.H;
     const int t0 = (int)((long long)p.T * split / p.nsplit), t1 = (int)((long long)p.T * (split + 1) / p.nsplit);
-    const int nrounds = (p.nslab + p.pbufs - 1) / p.pbufs;
     const size_t rows = (size_t)p.BH * p.N;
     if (tid == 0) {
         for (int i = 0; i < 7; ++i) mbar_init(bars + i, 1);
-        mbar_init(e1, kEpiWarps); mbar_init(e2, kEpiWarps); mbar_init(e_p, kEpiWarps);
+        mbar_init(e1, kEpiWarps); mbar_init(e2, kEpiWarps);
         *abort_flag = (smem_u32(smem) & 1023u) ? 1 : 0;
         fence_mbar_init();
     }
@@ -706,13 +706,6 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __gr
                 mbar_expect_tx(bar_k + b, kTile);
                 for (int a = 0; a < D / 64; ++a) tma_load_2d(sK0 + b * kTile + a * 16384, &p.mapK, bar_k + b, a * 64, bh * p.N + t * 128);
             };
-            auto load_partials = [&](int t, int round) {
-                const int s0 = round * p.pbufs, n = min(p.pbufs, p.nslab - s0);
-                mbar_expect_tx(bar_p, n * kTile);
-                for (int j = 0; j < n; ++j)
-                    for (int a = 0; a < D / 64; ++a)
-                        tma_load_2d(sP + (size_t)j * kTile + a * 16384, &p.mapP, bar_p, a * 64, (int)((size_t)(s0 + j) * rows + (size_t)bh * p.N + (size_t)t * 128));
-            };
             mbar_expect_tx(bar_m, kTile);
             for (int a = 0; a < D / 64; ++a) tma_load_2d(sM + a * 16384, &p.mapM, bar_m, a * 64, h * p.r);
             load_k(t0);
@@ -720,7 +713,6 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __gr
             // K M^T of tile i+1 is issued right behind the two products of tile i, so that it runs while the epilogue
             // warps still write tile i out.
             bool ok = wait_or_abort(bar_m, 0, p.status, abort_flag);
-            uint32_t np = 0;                             // rounds of partial loads issued so far
             if (t0 + 1 < t1) load_k(t0 + 1);
             if (ok) ok = wait_or_abort(bar_k, 0, p.status, abort_flag);
             if (ok) {
@@ -732,9 +724,6 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __gr
                 const int i = t - t0, b = i & 1;
                 const uint32_t ph = i & 1;
                 const TileDesc &tK = b ? tK1 : tK0;
-                if (np > 0) ok = wait_or_abort(e_p, (np - 1) & 1, p.status, abort_flag);   // partial tiles consumed
-                if (!ok) break;
-                load_partials(t, 0); ++np;
                 ok = wait_or_abort(e1, ph, p.status, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
@@ -750,11 +739,6 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __gr
                     _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(tmem + C1, kdesc(tKn, k), kdesc(tM, k), id_x, k > 0);
                     mma_commit(m1);
                 }
-                for (int round = 1; round < nrounds && ok; ++round) {
-                    ok = wait_or_abort(e_p, (np - 1) & 1, p.status, abort_flag);
-                    if (ok) { load_partials(t, round); ++np; }
-                }
-                if (!ok) break;
                 ok = wait_or_abort(m3, ph, p.status, abort_flag);
                 if (!ok) break;
                 if (t + 2 < t1) load_k(t + 2);          // this tile's K buffer has been read by both of its products
@@ -766,7 +750,6 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __gr
         const int r = q4 * 32 + lane;
         const uint32_t lane_addr = tmem + ((uint32_t)(q4 * 32) << 16);
         bool ok = true;
-        uint32_t np = 0;
         // rowsum(E) of a tile's row: its partials are loaded one tile ahead (their latency is hidden behind a tile's work)
         auto row_sum = [&](int t) {
             const size_t rw = (size_t)bh * p.N + (size_t)t * 128 + r;
@@ -801,26 +784,6 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __gr
             mbar_arrive_warp(e1);
             if (t + 1 < t1) es_next = row_sum(t + 1);
 
-            float acc[32];
-#pragma unroll
-            for (int j = 0; j < 32; ++j) acc[j] = 0.f;
-            for (int round = 0; round < nrounds && ok; ++round, ++np) {
-                ok = __all_sync(0xffffffffu, wait_or_abort(bar_p, np & 1, p.status, abort_flag));
-                if (!ok) break;
-                const int n = min(p.pbufs, p.nslab - round * p.pbufs);
-                if (col0 < D)
-                    for (int j = 0; j < n; ++j) {
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            float f[8];
-                            unpack8(*reinterpret_cast<const uint4 *>(tile_chunk(sP + (size_t)j * kTile, r, col0 / 8 + q)), f);
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) acc[8 * q + e] += f[e];
-                        }
-                    }
-                mbar_arrive_warp(e_p);
-            }
-            if (!ok) break;
             ok = __all_sync(0xffffffffu, wait_or_abort(m2, ph, p.status, abort_flag));
             if (!ok) break;
             tc_fence_after();
@@ -829,14 +792,12 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __gr
                 tmem_ld32(lane_addr + C2 + col0, v);
                 tmem_wait_ld();
 #pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(acc[j] + __uint_as_float(v[j]));
-#pragma unroll
                 for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4 *>(tile_chunk(sOut, r, col0 / 8 + q)) = pack8(v + 8 * q);
             }
             fence_async_smem();
             epi_sync();
             if (tid == 0) {
-                for (int a = 0; a < D / 64; ++a) tma_store_2d(&p.mapOut, sOut + a * 16384, a * 64, (int)(row - r));
+                for (int a = 0; a < D / 64; ++a) tma_reduce_add_2d(&p.mapOut, sOut + a * 16384, a * 64, (int)(row - r));
                 tma_store_commit();
             }
             tc_fence_before();
@@ -980,10 +941,7 @@ cudaError_t launch_scan(const darkattn_plan_s *plan, const BwdParams &P, int gri
 template <int D>
 cudaError_t launch_finish(FinishParams &P, int grid, cudaStream_t st)
 {
-    constexpr int kTile = 128 * D * 2, kFixed = 4 * kTile + 32768 + 128;
-    P.pbufs = (232448 - kFixed) / kTile;
-    if (P.pbufs > P.nslab) P.pbufs = P.nslab;
-    const int smem_bytes = kFixed + P.pbufs * kTile;
+    constexpr int kTile = 128 * D * 2, smem_bytes = 4 * kTile + 32768 + 128;    // M, two K tiles, staging; w; barriers
     cudaError_t e = cudaFuncSetAttribute(tc_bwd_finish_k_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
     if (e != cudaSuccess) return e;
     tc_bwd_finish_k_kernel<D><<<grid, kThreads, smem_bytes, st>>>(P);
@@ -1041,8 +999,7 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
 
     FinishParams F;
     memset(&F, 0, sizeof(F));
-    if (!make_map(&F.mapM, M, (size_t)D.H * D.r, D.d, 128) || !make_map(&F.mapK, K, BH * N, D.d, 128) ||
-        !make_map(&F.mapP, dK, BH * N, D.d, 128)) {
+    if (!make_map(&F.mapM, M, (size_t)D.H * D.r, D.d, 128) || !make_map(&F.mapK, K, BH * N, D.d, 128)) {
         set_cuda_error(cudaErrorInvalidValue, "tensor_backward: tensor map encode");
         return DARKATTN_ERR_CUDA;
     }
@@ -1073,7 +1030,7 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
     if (!make_map(&F.mapOut, dK, BH * N, D.d, 128)) { set_cuda_error(cudaErrorInvalidValue, "tensor_backward: tensor map encode"); return DARKATTN_ERR_CUDA; }
     F.espart = fl(Y.espart); F.dMn = fl(Y.dMn);
     F.status = reinterpret_cast<int *>(ws + Y.status);
-    F.N = D.N; F.H = D.H; F.BH = D.BH; F.T = Y.T; F.r = D.r; F.nslab = 1; F.nes = 4 * Y.nslab; F.s2 = D.s * D.s;
+    F.N = D.N; F.H = D.H; F.BH = D.BH; F.T = Y.T; F.r = D.r; F.nes = 4 * Y.nslab; F.s2 = D.s * D.s;
     F.nsplit = pick_splits((long long)BH, Y.T, 3.5, 5.0, 64);
     // dM = s W^T T + (norm term). T is complete once the key-side pass is done, so its product runs on the side
     // stream next to the kernel that produces the norm term, and a small kernel adds the two. (With per-kernel
