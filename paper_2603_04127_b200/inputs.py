@@ -86,6 +86,57 @@ def random_orthogonal(d: int, rng: np.random.Generator) -> np.ndarray:
     return q * np.sign(np.diag(rr))[None, :]
 
 
+def orthogonal_projection_rows(m: int, r: int, rng: np.random.Generator) -> np.ndarray:
+    """W [m, r] in blocks of r rows: each block is a Haar-random orthogonal basis whose rows are rescaled to the
+    norms of independent N(0, I_r) vectors, so every row is marginally N(0, I_r) while the rows of a block are
+    exactly orthogonal (the orthogonal random features Section 2 mentions). Blocks are independent."""
+    blocks = []
+    for _ in range((m + r - 1) // r):
+        q = random_orthogonal(r, rng)
+        norms = np.linalg.norm(rng.standard_normal((r, r)), axis=1)
+        blocks.append(q * norms[:, None])
+    return np.concatenate(blocks, axis=0)[:m]
+
+
+def optimal_proposal_spectrum(lam: np.ndarray) -> np.ndarray:
+    """Eigenvalues of Sigma* = (I + 2 Lambda)(I - 2 Lambda)^-1 (Theorem 3.2) for the eigenvalues ``lam`` of the
+    input covariance Lambda; a valid covariance only while max(lam) < 1/2."""
+    lam = np.asarray(lam, dtype=np.float64)
+    if not (lam.max() < 0.5 and lam.min() >= 0.0):
+        raise ValueError("Sigma* is a covariance only for 0 <= lambda < 1/2")
+    return (1.0 + 2.0 * lam) / (1.0 - 2.0 * lam)
+
+
+def aligned_M(U: np.ndarray, lam: np.ndarray) -> np.ndarray:
+    """M [d, d] with M^T M = U diag(sigma*) U^T, sigma* = optimal_proposal_spectrum(lam): the geometry of the
+    variance-optimal Gaussian proposal for inputs of covariance U diag(lam) U^T."""
+    return np.sqrt(optimal_proposal_spectrum(lam))[:, None] * U.T
+
+
+def variance_workload(wid: int, B: int, H: int, N: int, d: int, m: int, lam_max: float = 0.2, aligned: bool = True,
+                      causal: bool = False, dtype: str = "bf16", backward: bool = True, dv: int = 0) -> "Tensors":
+    """The second synthetic workload: Gaussian queries and keys of covariance Lambda = U diag(lam) U^T with a
+    geometric spectrum below 1/2 (lam_i = lam_max * 0.9**i), orthogonal projection rows W, and M either the
+    identity (isotropic sampling) or aligned_M(U, lam) (data-aligned sampling, the same for every head). Use it
+    with scale = 1."""
+    wl = Workload(f"variance_{'aligned' if aligned else 'isotropic'}", wid, B, H, N, d, m, dtype, causal, backward, 0.9, 1.0, 0, dv)
+    _, _, _, _, r, _, dvv = wl.dims()
+    U = random_orthogonal(d, _rng(wid, "U"))
+    lam = lam_max * 0.9 ** np.arange(d, dtype=np.float64)
+    draw = lambda stream, width, aniso: np.stack([
+        (anisotropic_rows(wid, stream, N, U, lam, b * H + h) if aniso else _rng(wid, stream, b * H + h).standard_normal((N, width)))
+        for b in range(B) for h in range(H)]).reshape(B, H, N, width)
+    Q, K, V = draw("Q", d, True), draw("K", d, True), draw("V", dvv, False)
+    dO = draw("dO", dvv, False) if backward else None
+    M = np.broadcast_to((aligned_M(U, lam) if aligned else np.eye(d))[None], (H, d, d)).copy()
+    W = orthogonal_projection_rows(m, r, _rng(wid, "W"))
+    if dtype == "bf16":
+        rt = lambda a: None if a is None else round_to_bf16(a).astype(np.float64)
+    else:
+        rt = lambda a: None if a is None else a.astype(np.float32).astype(np.float64)
+    return Tensors(wl, rt(Q), rt(K), rt(V), rt(M), rt(W), rt(dO), [(b, h) for b in range(B) for h in range(H)])
+
+
 def _rng(wid: int, stream: str, extra: int = 0) -> np.random.Generator:
     return np.random.default_rng([1000 * wid + _STREAMS[stream], extra])
 

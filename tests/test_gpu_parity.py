@@ -257,6 +257,16 @@ def test_tensor_path_is_deterministic(binding):
             assert worst < 2.0 ** -7, f"{k} differs between runs by {worst:.2e} of its largest value"
 
 
+@pytest.mark.parametrize("causal", [False, True], ids=["noncausal", "causal"])
+@pytest.mark.parametrize("aligned", [False, True], ids=["isotropic", "aligned"])
+def test_variance_workload_on_the_tensor_path(binding, aligned, causal):
+    """The second synthetic workload (Gaussian inputs below the Theorem 3.2 bound, orthogonal projection rows, M the
+    identity or the variance-optimal geometry, scale 1), forward and backward, against the oracle."""
+    t = inputs.variance_workload(wid=23, B=2, H=2, N=512, d=64, m=256, lam_max=0.2, aligned=aligned, causal=causal)
+    got = run_gpu(binding, t.wl, t, path=binding.PATH_TENSOR, scale=1.0, use_saved=True)
+    _compare(got, _oracle(t, t.wl, scale=1.0), TOL["bf16"], t.wl.name)
+
+
 def test_mma_cycle_measurement_is_sane(binding):
     """The instrument behind the scan kernels' tensor-pipe accounting: a 128x128x16 bf16 MMA cannot beat the
     pipe's 8192 flop per clock (64 cycles), and none of the forms the kernels use should cost twice that."""
