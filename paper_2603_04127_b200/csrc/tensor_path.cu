@@ -1019,9 +1019,10 @@ void tensor_make_layout(darkattn_plan_s *plan)
     Y.Racc = take(off, D.causal ? 0 : BH * m * dv * 4);
     Y.rhot = take(off, D.causal ? 0 : BH * m * 4);
     Y.Rb = take(off, D.causal ? 0 : BH * m * dv * 2);
-    // with `saved`; without it the forward launches come on top. Causal: delta, two scan kernels, dK finishing, dM;
-    // non-causal: one more for the rounding of R between the two passes.
-    plan->launches_bwd = D.causal ? 5 : 6;
+    // with `saved`; without it the forward launches come on top. Causal: delta, two scan kernels, dK finishing, the
+    // dM product and the small kernel that adds the norm term's part; non-causal: one more for the rounding of R
+    // between the two passes. (With per-kernel timing on, dM is one kernel.)
+    plan->launches_bwd = D.causal ? 6 : 7;
     Y.total_bytes = off;
     plan->workspace_bytes = Y.total_bytes;
 }
