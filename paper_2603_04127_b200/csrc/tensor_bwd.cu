@@ -805,14 +805,16 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __gr
         }
         if (tid == 0) tma_store_wait_all();
         if (ok) ok = wait_or_abort(m3, (t1 - 1 - t0) & 1, p.status, abort_flag);
-        if (ok && r < p.r && col0 < D) {
+        if (ok && q4 * 32 < p.r && col0 < D) {      // whole warps: the tensor-memory load is a warp-wide instruction
             tc_fence_after();
             float *dst = p.dMn + ((size_t)h * p.r + r) * D + col0;
             uint32_t v[32];
             tmem_ld32(lane_addr + C3 + col0, v);
             tmem_wait_ld();
+            if (r < p.r) {                           // r may end inside the warp's 32 rows (r = 16, 48, ...)
 #pragma unroll
-            for (int j = 0; j < 32; ++j) atomicAdd(dst + j, __uint_as_float(v[j]));
+                for (int j = 0; j < 32; ++j) atomicAdd(dst + j, __uint_as_float(v[j]));
+            }
         }
     }
     if (*abort_flag) __nanosleep(200000);

@@ -153,6 +153,12 @@ TENSOR_BWD = [
     ("b_d128_dv64_r64", dict(B=1, H=2, N=256, d=128, m=128, dv=64, r=64, causal=True)),
     ("b_d64_dv128_r32", dict(B=2, H=2, N=384, d=64, m=256, dv=128, r=32, causal=True)),
     ("b_segmented_fwd", dict(B=1, H=2, N=1024, d=64, m=128, causal=True)),
+    # eight slabs of features (the general-slab-count code paths), smallest projection rank
+    ("b_m1024_r16", dict(B=1, H=2, N=256, d=64, m=1024, r=16, causal=True)),
+    ("b_nc_m1024", dict(B=1, H=1, N=256, d=64, m=1024, causal=False)),
+    # projection ranks that end inside a warp's 32 rows
+    ("b_r48", dict(B=1, H=2, N=256, d=64, m=128, r=48, causal=True)),
+    ("b_nc_r16_d128", dict(B=1, H=2, N=256, d=128, m=256, r=16, causal=False)),
     # more (batch, head, chunk) items than CTA groups: a query-side CTA walks several runs, across heads
     ("b_m512_runs", dict(B=2, H=4, N=2048, d=64, m=512, causal=True)),
     ("b_d128_dv64_runs", dict(B=2, H=20, N=1024, d=128, m=128, dv=64, causal=True)),
