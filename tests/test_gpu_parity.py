@@ -181,6 +181,35 @@ def test_tensor_path_backward(binding, name, kw, use_saved):
     _compare(got, _oracle(t, wl), TOL["bf16"], name)
 
 
+# Shapes drawn at random over everything the tensor-core path accepts (three and five feature slabs, projection ranks
+# that are not multiples of 32 or exceed d, d != dv, per-head projection rows, recompute and stash), kept as a fixed list.
+MIXED = [
+    dict(B=1, H=1, N=128, d=64, dv=128, m=640, r=16, causal=False, saved=True, wph=False),
+    dict(B=2, H=1, N=256, d=128, dv=64, m=384, r=32, causal=False, saved=False, wph=True),
+    dict(B=3, H=2, N=384, d=128, dv=128, m=640, r=96, causal=True, saved=False, wph=True),
+    dict(B=2, H=1, N=640, d=128, dv=128, m=640, r=48, causal=True, saved=False, wph=False),
+    dict(B=2, H=1, N=256, d=64, dv=128, m=256, r=80, causal=True, saved=False, wph=True),
+    dict(B=1, H=1, N=256, d=64, dv=128, m=512, r=112, causal=True, saved=False, wph=False),
+    dict(B=3, H=3, N=640, d=64, dv=128, m=128, r=80, causal=True, saved=True, wph=False),
+    dict(B=1, H=3, N=384, d=128, dv=64, m=256, r=112, causal=False, saved=True, wph=False),
+    dict(B=1, H=2, N=3072, d=64, dv=64, m=384, r=128, causal=True, saved=True, wph=False),
+    dict(B=1, H=1, N=4096, d=128, dv=64, m=256, r=64, causal=True, saved=False, wph=False),
+]
+
+
+@pytest.mark.parametrize("i", range(len(MIXED)))
+def test_tensor_path_mixed_shapes(binding, i):
+    kw = dict(MIXED[i])
+    saved, wph = kw.pop("saved"), kw.pop("wph")
+    wl = inputs.small(name=f"mixed{i}", wid=300 + i, dtype="bf16", backward=True, **kw)
+    t = inputs.generate(wl)
+    if wph:
+        rng = np.random.default_rng(300 + i)
+        t.W = inputs.round_to_bf16(rng.standard_normal((wl.H,) + t.W.shape)).astype(np.float64)
+    got = run_gpu(binding, wl, t, path=binding.PATH_TENSOR, use_saved=saved, w_per_head=wph)
+    _compare(got, _oracle(t, wl), TOL["bf16"], wl.name)
+
+
 def test_tensor_path_per_head_projections_and_scale(binding):
     wl = inputs.small(name="t_wph", wid=77, B=2, H=3, N=384, d=64, m=256, causal=True, dtype="bf16", backward=True)
     t = inputs.generate(wl)
