@@ -94,7 +94,8 @@ size_t darkattn_saved_bytes(darkattn_plan_t plan);
 int32_t darkattn_plan_path(darkattn_plan_t plan);
 
 /* Number of kernel launches one forward (which = 0) or one backward (which = 1) call enqueues
- * (backward: when it is given O and `saved`; otherwise the forward launches come on top).        */
+ * (backward: when it is given O and `saved`; otherwise the forward launches come on top), in the
+ * plan's current mode: with per-kernel timing on, the tensor-core backward launches one fewer.   */
 int32_t darkattn_plan_launches(darkattn_plan_t plan, int32_t which);
 
 /* O = normalised random-feature attention (formulas at the top of this file).                   */

@@ -88,7 +88,9 @@ int32_t darkattn_plan_path(darkattn_plan_t plan) { return plan ? plan->path : -1
 int32_t darkattn_plan_launches(darkattn_plan_t plan, int32_t which)
 {
     if (!plan) return -1;
-    return which ? plan->launches_bwd : plan->launches_fwd;
+    if (!which) return plan->launches_fwd;
+    // with per-kernel timing on, the tensor-core backward keeps everything on one stream and dM is one kernel, not two
+    return plan->launches_bwd - ((plan->path == DARKATTN_PATH_TENSOR && plan->timer.on) ? 1 : 0);
 }
 
 darkattn_status_t darkattn_forward(darkattn_plan_t plan, const void *Q, const void *K, const void *V,
