@@ -170,6 +170,13 @@ darkattn_status_t darkattn_measure_alu_peak(int32_t which, int32_t iters, double
 darkattn_status_t darkattn_measure_mma_cycles(int32_t variant, int32_t busy_epilogue, double *cycles_per_mma,
                                               double *batch_overhead_cycles, void *cuda_stream);
 
+/* Self-test of the bounded device-side wait the scan kernels rely on: launches one small kernel whose
+ * only thread waits on a barrier nobody arrives on. The wait must give up after its limit (2 s),
+ * record DARKATTN_ERR_TIMEOUT in a device status word and let the kernel end normally. Writes that
+ * status word and the kernel's device time in seconds to the two host pointers; synchronises the
+ * stream. Nothing faults, the context stays usable. Returns DARKATTN_OK when the launch itself ran. */
+darkattn_status_t darkattn_selftest_wait_limit(int32_t *device_status, double *seconds, void *cuda_stream);
+
 /* Per-kernel device times, for benchmarks. While enabled, forward and backward record a CUDA event on
  * the call's stream in front of every kernel they launch and one behind the last (events are host
  * objects created by the first enabling call; no device memory is involved). Enabling also clears the

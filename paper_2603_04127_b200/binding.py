@@ -24,7 +24,7 @@ EXPORTS = [
     "darkattn_plan_launches", "darkattn_forward", "darkattn_backward", "darkattn_last_device_status",
     "darkattn_destroy", "darkattn_status_string", "darkattn_last_cuda_error", "darkattn_measure_alu_peak",
     "darkattn_static_scratch_needed", "darkattn_forward_static", "darkattn_kernel_timing", "darkattn_kernel_times",
-    "darkattn_backward_dw", "darkattn_decode_step", "darkattn_measure_mma_cycles",
+    "darkattn_backward_dw", "darkattn_decode_step", "darkattn_measure_mma_cycles", "darkattn_selftest_wait_limit",
 ]
 STATIC_SCRATCH_BYTES = 16 << 20
 
@@ -73,6 +73,8 @@ lib.darkattn_measure_alu_peak.restype = ctypes.c_int
 lib.darkattn_measure_mma_cycles.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(ctypes.c_double),
                                             ctypes.POINTER(ctypes.c_double), _vp]
 lib.darkattn_measure_mma_cycles.restype = ctypes.c_int
+lib.darkattn_selftest_wait_limit.argtypes = [ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_double), _vp]
+lib.darkattn_selftest_wait_limit.restype = ctypes.c_int
 lib.darkattn_kernel_timing.argtypes = [_vp, ctypes.c_int32]
 lib.darkattn_kernel_timing.restype = ctypes.c_int
 lib.darkattn_kernel_times.argtypes = [_vp, ctypes.c_int32, ctypes.c_char_p, ctypes.POINTER(ctypes.c_float),
@@ -201,6 +203,13 @@ def darkattn_measure_mma_cycles(variant: int, busy_epilogue: bool = False, strea
     _check(lib.darkattn_measure_mma_cycles(variant, int(bool(busy_epilogue)), ctypes.byref(per), ctypes.byref(fixed),
                                            _stream(stream)), "darkattn_measure_mma_cycles")
     return per.value, fixed.value
+
+
+def darkattn_selftest_wait_limit(stream=None):
+    """(device status word, kernel seconds) of a wait on a barrier nobody arrives on."""
+    st, sec = ctypes.c_int32(0), ctypes.c_double(0.0)
+    _check(lib.darkattn_selftest_wait_limit(ctypes.byref(st), ctypes.byref(sec), _stream(stream)), "darkattn_selftest_wait_limit")
+    return st.value, sec.value
 
 
 def darkattn_kernel_timing(plan: Plan, enable: bool):

@@ -302,6 +302,17 @@ def test_variance_workload_on_the_tensor_path(binding, aligned, causal):
     _compare(got, _oracle(t, t.wl, scale=1.0), TOL["bf16"], t.wl.name)
 
 
+def test_a_wait_that_nothing_ends_gives_up_and_reports_it(binding):
+    """The bounded wait of the scan kernels, on a barrier nobody arrives on: it must run out after its limit, leave
+    DARKATTN_ERR_TIMEOUT in the status word, and the kernel must end normally (the next call works)."""
+    status, seconds = binding.darkattn_selftest_wait_limit()
+    assert status == binding.ERR_TIMEOUT
+    assert 1.5 < seconds < 6.0, seconds
+    wl = inputs.small(name="after_timeout", wid=5, B=1, H=1, N=128, d=64, m=128, causal=True, dtype="bf16", backward=False)
+    t = inputs.generate(wl)
+    _compare(run_gpu(binding, wl, t, path=binding.PATH_TENSOR), _oracle(t, wl), TOL["bf16"], "after_timeout")
+
+
 def test_mma_cycle_measurement_is_sane(binding):
     """The instrument behind the scan kernels' tensor-pipe accounting: a 128x128x16 bf16 MMA cannot beat the
     pipe's 8192 flop per clock (64 cycles), and none of the forms the kernels use should cost twice that."""
