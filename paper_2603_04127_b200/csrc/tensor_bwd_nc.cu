@@ -62,7 +62,7 @@ __device__ __forceinline__ uint64_t vecdesc(const TileDesc &t, int k) { return t
 enum NBars { NB_OM, NB_X0, NB_X1, NB_Y, NM1, NMA, NM2, NM3, NE1, NE2, NE3, NNBARS };
 
 // Both passes share one schedule per tile t (R1, R2: scratch regions of tensor memory):
-//   R1: U = X Omega^T -> (features read) -> query pass: rho_c | key pass: dV = Bf R -> (read)
+//   R1: U = X Omega^T (issued in the tail of the tile before) -> (features read) -> query pass: rho_c | key pass: dV = Bf R -> (read)
 //   R2: dO S^T | V R^T (independent of the features, issued at once) -> (E formed) -> E Omega -> (read, stored)
 // and the state updates R += A^^T dO, T += E^T X run behind them. KEYS selects the key pass.
 template <int D, int DV, bool KEYS>
@@ -124,16 +124,18 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_nc_kernel(const __grid_con
             load_tile(sY, &p.mapY, bars + NB_Y, DV, tbeg);
 
             bool ok = wait_or_abort(bars + NB_OM, 0, status, abort_flag);
+            if (ok) ok = wait_or_abort(bars + NB_X0, 0, status, abort_flag);
+            if (ok) {
+                tc_fence_after();
+                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R1, kdesc(tX0, k), kdesc(tOm, k), id_kk, k > 0);      // U of the first tile
+                mma_commit(bars + NM1);
+            }
             for (int it = 0; it < nt && ok; ++it) {
                 const int t = tbeg + it;
-                const uint32_t ph = it & 1, phx = (it >> 1) & 1;
+                const uint32_t ph = it & 1;
                 const bool first = (it == 0), last = (it + 1 == nt);
                 const TileDesc &tX = (it & 1) ? tX1 : tX0;
 #define NWAIT(b, q) do { ok = wait_or_abort(bars + (b), (q), status, abort_flag); } while (0)
-                NWAIT(NB_X0 + (it & 1), phx); if (!ok) break;
-                tc_fence_after();
-                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R1, kdesc(tX, k), kdesc(tOm, k), id_kk, k > 0);       // U
-                mma_commit(bars + NM1);
                 if (!first) { NWAIT(NM3, ph ^ 1); if (!ok) break; }                 // T += E^T X of the tile before: its X buffer is free
                 if (!last) load_tile(sX + ((it + 1) & 1) * 128 * D * 2, &p.mapX, bars + NB_X0 + ((it + 1) & 1), D, t + 1);
                 NWAIT(NB_Y, ph); if (!ok) break;
@@ -156,6 +158,13 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_nc_kernel(const __grid_con
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R2, kdesc(tA, k), mndesc(tOm, k), id_dx, k > 0);            // E Omega
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColT, mndesc(tA, k), mndesc(tX, k), id_t, (!first) || k > 0);   // T += E^T X
                 mma_commit(bars + NM3);
+                if (!last) {       // U of the next tile behind them (R1 has been read): its features can be formed at once
+                    NWAIT(NB_X0 + ((it + 1) & 1), ((it + 1) >> 1) & 1); if (!ok) break;
+                    tc_fence_after();
+                    const TileDesc &tXn = ((it + 1) & 1) ? tX1 : tX0;
+                    _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R1, kdesc(tXn, k), kdesc(tOm, k), id_kk, k > 0);
+                    mma_commit(bars + NM1);
+                }
 #undef NWAIT
             }
         }
