@@ -59,7 +59,8 @@ struct BwdSmem {
     static constexpr int kV = kKB + 32768;                 // V tile                            [128, DV]
     static constexpr int kG = kV + 128 * DV * 2;           // dO tile; later the reloaded Q / K tile
     static constexpr int kSt = kG + 128 * kDmax * 2;       // bf16 copy of the scan state       [128 l, DV]
-    static constexpr int kStg = kSt + 128 * DV * 2;        // staging tile of the TMA stores of the partials
+    static constexpr int kStg = kSt + 32768;               // (32 KB: the query-side kernel also keeps a 128 x 128 feature tile there)
+                                                           // staging tile of the TMA stores of the partials
     static constexpr int kVec = kStg + 128 * kDmax * 2;    // three float[128]
     static constexpr int kBars = kVec + 1536;
     static constexpr int kTotal = kBars + 256;
@@ -125,10 +126,15 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
             // it fits), so that dO of the next chunk can follow early into its own buffer; otherwise into dO's buffer.
             constexpr bool kQinV = (D <= DV);
 
-            // Schedule of one chunk (R1, R2: the two scratch regions of TMEM). U_K of the next chunk is issued in
+            // Schedule of one chunk (R1, R2, R3: scratch regions of TMEM). U_K and U_Q of the next chunk are issued in
             // the tail of the current one, and dO V^T runs while the epilogue is still busy with A^.
             //   R2: U_K -> (Bf read) -> dO V^T -> packed dP in [0,64) (A operand of dP Bf), rho_c in [64,80) -> U_K of the next chunk
-            //   R1: U_Q -> (A^ read) -> dP Bf + dO S^T -> (E read) -> E Omega -> (dQ read)
+            //   R3: U_Q -> (A^ read) -> U_Q of the next chunk
+            //   R1: dP Bf + dO S^T -> (E read) -> E Omega -> (dQ read)
+            // Two tile buffers swap roles from chunk to chunk: X holds Q, then A^, then E; S holds the state before the
+            // chunk. S is free first (after dO S^T) and takes the next chunk's Q, so that its projection can be issued
+            // in the tail; X is free last (after T += E^T Q) and takes the next chunk's state, which is needed late.
+            const uint32_t R3 = tmem + kColState;
             bool ok = true;
             int it = 0, run = 0;        // chunks and runs done so far: the parities of the barriers
             for (long long l0 = lbeg; l0 < lend && ok; ++run) {
@@ -142,9 +148,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                     mbar_expect_tx(bar, 128 * width * 2);
                     for (int a = 0; a < width / 64; ++a) tma_load_2d(dst + a * 16384, map, bar, a * 64, row0 + t * 128);
                 };
-                auto load_state = [&](int t) {     // S before chunk t (for t = 0 the tile is loaded but not used)
+                auto load_state = [&](unsigned char *dst, int t) {     // S before chunk t (for t = 0 the tile is loaded but not used)
                     mbar_expect_tx(bars + QB_S, 128 * DV * 2);
-                    for (int a = 0; a < DV / 64; ++a) tma_load_2d(sSt + a * 16384, &p.mapSst, bars + QB_S, a * 64, (bh * T + t) * p.m + slab * 128);
+                    for (int a = 0; a < DV / 64; ++a) tma_load_2d(dst + a * 16384, &p.mapSst, bars + QB_S, a * 64, (bh * T + t) * p.m + slab * 128);
                 };
                 auto store_features = [&](unsigned char *src, const CUtensorMap *map, int t) {
                     tma_store_2d(map, src, slab * 128, row0 + t * 128);
@@ -153,27 +159,32 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                 };
                 mbar_expect_tx(bars + QB_OM, 128 * D * 2);
                 for (int a = 0; a < D / 64; ++a) tma_load_2d(sOm + a * 16384, &p.mapOm, bars + QB_OM, a * 64, h * p.m + slab * 128);
-                load_tile(sQA, &p.mapQ, bars + QB_Q, D, t0);
+                load_tile((it & 1) ? sSt : sQA, &p.mapQ, bars + QB_Q, D, t0);
                 load_tile(sKB, &p.mapK, bars + QB_K, D, t0);
                 load_tile(sV, &p.mapV, bars + QB_V, DV, t0);
                 load_tile(sG, &p.mapG, bars + QB_G, DV, t0);
-                load_state(t0);
+                load_state((it & 1) ? sQA : sSt, t0);
                 ok = wait_or_abort(bars + QB_OM, run & 1, status, abort_flag);
                 if (ok) ok = wait_or_abort(bars + QB_K, it & 1, status, abort_flag);
                 if (ok) {
                     tc_fence_after();
                     _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R2, kdesc(tKB, k), kdesc(tOm, k), id_kk, k > 0);   // U_K of the run's first chunk
                     mma_commit(bars + QM2);
+                    ok = wait_or_abort(bars + QB_Q, it & 1, status, abort_flag);
+                }
+                if (ok) {
+                    tc_fence_after();
+                    const TileDesc &tX0 = (it & 1) ? tSt : tQA;
+                    _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R3, kdesc(tX0, k), kdesc(tOm, k), id_kk, k > 0);   // U_Q of the run's first chunk
+                    mma_commit(bars + QM1);
                 }
                 for (int c = 0; c < nrun && ok; ++c, ++it) {
                     const int t = t0 + c;
                     const uint32_t ph = it & 1;
                     const bool first = (t == 0), last = (c + 1 == nrun);
+                    unsigned char *bX = ph ? sSt : sQA, *bS = ph ? sQA : sSt;
+                    const TileDesc &tX = ph ? tSt : tQA, &tS = ph ? tQA : tSt;
 #define QWAIT(b) do { ok = wait_or_abort(bars + (b), ph, status, abort_flag); } while (0)
-                    QWAIT(QB_Q); if (!ok) break;
-                    tc_fence_after();
-                    _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R1, kdesc(tQA, k), kdesc(tOm, k), id_kk, k > 0);   // U_Q
-                    mma_commit(bars + QM1);
                     QWAIT(QE0); if (!ok) break;                                                                  // Bf in smem, R2 read
                     store_features(sKB, &p.mapBf, t);                                                            // kept for the key-side kernel
                     QWAIT(QB_V); if (!ok) break;
@@ -181,18 +192,18 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                     tc_fence_after();
                     _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R2, kdesc(tG, k), kdesc(tV, k), id_kk, k > 0);     // dO V^T
                     mma_commit(bars + QM3);
-                    QWAIT(QE1); if (!ok) break;                                                                  // A^ in smem, R1 read
-                    store_features(sQA, &p.mapAh, t);
+                    QWAIT(QE1); if (!ok) break;                                                                  // A^ in X, R3 read
+                    store_features(bX, &p.mapAh, t);
                     QWAIT(QE2A); if (!ok) break;                                                                 // dO V^T read out of R2
                     if (kQinV) load_tile(sV, &p.mapQ, bars + QB_X2, D, t);                                      // V is done with: Q again, for T
                     tc_fence_after();
-                    _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R2 + 64, mndesc(tQA, k), vecdesc(tDel, k), id_vec, k > 0);  // rho_c = -A^^T delta (columns 0, 1)
+                    _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R2 + 64, mndesc(tX, k), vecdesc(tDel, k), id_vec, k > 0);  // rho_c = -A^^T delta (columns 0, 1)
                     QWAIT(QE2); if (!ok) break;                                                                  // dP packed in R2
                     QWAIT(QB_S); if (!ok) break;
                     tc_fence_after();
                     _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R1, R2 + k * 8, mndesc(tKB, k), id_tm, k > 0);           // dP Bf
                     if (!first)
-                        _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R1, kdesc(tG, k), kdesc(tSt, k), id_kk, 1);    // + dO S_prev^T
+                        _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R1, kdesc(tG, k), kdesc(tS, k), id_kk, 1);     // + dO S_prev^T
                     tma_store_wait_read();      // both feature tiles have left shared memory: E may overwrite A^, the next K tile Bf
                     mma_commit(bars + QM4);
                     QWAIT(QM4); if (!ok) break;                                                                  // Bf, V, dO and S of this chunk are done with
@@ -201,7 +212,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                         if (kQinV) load_tile(sG, &p.mapG, bars + QB_G, DV, t + 1);
                         else load_tile(sV, &p.mapV, bars + QB_V, DV, t + 1);
                         load_tile(sKB, &p.mapK, bars + QB_K, D, t + 1);
-                        load_state(t + 1);
+                        load_tile(bS, &p.mapQ, bars + QB_Q, D, t + 1);                                          // the state tile is done with: the next chunk's Q
                     }
                     QWAIT(QE3); if (!ok) break;
                     QWAIT(QB_X2); if (!ok) break;
@@ -210,9 +221,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                         if (!ok) break;
                     }
                     tc_fence_after();
-                    _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R1, kdesc(tQA, k), mndesc(tOm, k), id_dx, k > 0);        // E Omega
+                    _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R1, kdesc(tX, k), mndesc(tOm, k), id_dx, k > 0);         // E Omega
                     mma_commit(bars + QM5);
-                    _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColT, mndesc(tQA, k), mndesc(kQinV ? tV : tG, k), id_t, (c > 0) || k > 0);   // T += E^T Q
+                    _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColT, mndesc(tX, k), mndesc(kQinV ? tV : tG, k), id_t, (c > 0) || k > 0);   // T += E^T Q
                     mma_commit(bars + QM6);
                     if (!last) {
                         ok = wait_or_abort(bars + QB_K, ph ^ 1, status, abort_flag);
@@ -220,10 +231,15 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                         tc_fence_after();
                         _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R2, kdesc(tKB, k), kdesc(tOm, k), id_kk, k > 0);   // U_K of the next chunk
                         mma_commit(bars + QM2);
+                        ok = wait_or_abort(bars + QB_Q, ph ^ 1, status, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R3, kdesc(tS, k), kdesc(tOm, k), id_kk, k > 0);    // U_Q of the next chunk (its Q sits in S)
+                        mma_commit(bars + QM1);
                     }
                     QWAIT(QM6); if (!ok) break;
                     if (!last) {
-                        load_tile(sQA, &p.mapQ, bars + QB_Q, D, t + 1);
+                        load_state(bX, t + 1);                                                                   // E is done with: the next chunk's state
                         if (kQinV) load_tile(sV, &p.mapV, bars + QB_V, DV, t + 1);
                         else load_tile(sG, &p.mapG, bars + QB_G, DV, t + 1);
                     }
@@ -269,6 +285,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
 #pragma unroll
                     for (int i = 0; i < 4; ++i) dtile[i] = -__ldg(p.delta + (size_t)row0 + (size_t)t * 128 + i * 32 + lane);
                 }
+                unsigned char *bX = ph ? sSt : sQA;          // this chunk's Q / A^ / E tile
                 EWAIT(QM2); if (!ok) break;
                 tc_fence_after();
                 features_to_tile(R2 + col0, nk, sKB, r, col0);                             // Bf
@@ -294,7 +311,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                 mbar_arrive_warp(bars + QE0);
                 EWAIT(QM1); if (!ok) break;
                 tc_fence_after();
-                features_to_tile(R1 + col0, aq, sQA, r, col0);                             // A^
+                features_to_tile(lane_addr + kColState + col0, aq, bX, r, col0);           // A^
                 fence_async_smem();
                 tc_fence_before();
                 mbar_arrive_warp(bars + QE1);
@@ -334,7 +351,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                     tmem_wait_ld();
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
-                        uint4 *cell = reinterpret_cast<uint4 *>(tile_chunk(sQA, r, col0 / 8 + q));
+                        uint4 *cell = reinterpret_cast<uint4 *>(tile_chunk(bX, r, col0 / 8 + q));
                         float a[8];
                         unpack8(*cell, a);
                         const float4 z0 = *reinterpret_cast<const float4 *>(sZ + col0 + 8 * q);
