@@ -29,7 +29,7 @@ if ROOT not in sys.path:
 # DRAM bytes (read + write) per (token, head) of the scan kernels at d = dv = 128, m = 256 from their ncu capture on the
 # small profiling workload (profiles/scan_kernels_d128_small.md); traffic is proportional to the (token, head) count.
 # A kernel that changed since its capture has no entry.
-NCU_TRAFFIC_PER_TOKEN_HEAD = {"tc_fwd_causal_kernel": 1471.0, "tc_bwd_q_kernel": 2904.0, "tc_bwd_k_kernel": 2800.0}
+NCU_TRAFFIC_PER_TOKEN_HEAD = {"tc_fwd_causal_kernel": 1469.0, "tc_bwd_q_kernel": 2916.0, "tc_bwd_k_kernel": 2797.0}
 
 METRIC = "DARK-attention fwd+bwd tokens/s"
 UNIT = "tokens/s"
