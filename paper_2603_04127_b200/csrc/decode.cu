@@ -21,23 +21,18 @@ __device__ __forceinline__ float ldf(const T *p, size_t i)
     else return p[i];
 }
 
-// grid = (dv / 32 column blocks, B*H); block = 256 threads = 32 columns x 8 groups of features.
-template <typename T>
-__global__ void __launch_bounds__(256) decode_step_kernel(const T *q, const T *k, const T *v, const T *M, const T *W, float *S,
-                                                           float *z, T *o, int H, int d, int r, int m, int dv, int w_per_head,
-                                                           float s)
+// Features of one (batch, head)'s new token, by a block of 256 threads: fk[l] = phi(k)_l and, when WITH_Q, fq[l] = phi(q)_l
+// (shared memory: xq[r], xk[r], fq[m], fk[m], red[...]).
+template <typename T, bool WITH_Q>
+__device__ __forceinline__ void token_features(const T *qv, const T *kv, const T *Mh, const T *Wh, float *xq, float *xk, float *fq,
+                                               float *fk, float *red, int d, int r, int m, float s)
 {
-    extern __shared__ float sm[];
-    float *xq = sm, *xk = xq + r, *fq = xk + r, *fk = fq + m, *red = fk + m;   // red: 8 x 32 partial numerators + 8 partial normalisers + scratch
-    const int bh = blockIdx.y, h = bh % H, tid = threadIdx.x;
-    const T *Mh = M + (size_t)h * r * d, *Wh = W + (size_t)(w_per_head ? h : 0) * m * r;
-    const T *qv = q + (size_t)bh * d, *kv = k + (size_t)bh * d;
-
+    const int tid = threadIdx.x;
     for (int a = tid; a < r; a += 256) {            // x~ = s M x for the query and the key
         float aq = 0.f, ak = 0.f;
         for (int c = 0; c < d; ++c) {
             const float mv = ldf(Mh, (size_t)a * d + c);
-            aq = fmaf(mv, ldf(qv, c), aq);
+            if constexpr (WITH_Q) aq = fmaf(mv, ldf(qv, c), aq);
             ak = fmaf(mv, ldf(kv, c), ak);
         }
         xq[a] = s * aq;
@@ -52,7 +47,7 @@ __global__ void __launch_bounds__(256) decode_step_kernel(const T *q, const T *k
         float uq = 0.f, uk = 0.f, c = 0.f;
         for (int a = 0; a < r; ++a) {
             const float w = ldf(Wh, (size_t)l * r + a);
-            uq = fmaf(w, xq[a], uq);
+            if constexpr (WITH_Q) uq = fmaf(w, xq[a], uq);
             uk = fmaf(w, xk[a], uk);
             c = fmaf(w, w, c);
         }
@@ -61,29 +56,44 @@ __global__ void __launch_bounds__(256) decode_step_kernel(const T *q, const T *k
         fq[l] = uq + c;
         mx = fmaxf(mx, fq[l]);
     }
-    for (int off = 16; off; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-    if ((tid & 31) == 0) red[tid >> 5] = mx;
+    if constexpr (WITH_Q) {
+        for (int off = 16; off; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+        if ((tid & 31) == 0) red[tid >> 5] = mx;
+        __syncthreads();
+        mx = red[0];
+        for (int w = 1; w < 8; ++w) mx = fmaxf(mx, red[w]);
+        __syncthreads();
+        for (int l = tid; l < m; l += 256) fq[l] = __expf(fq[l] - mx);
+    }
     __syncthreads();
-    mx = red[0];
-    for (int w = 1; w < 8; ++w) mx = fmaxf(mx, red[w]);
-    __syncthreads();
-    for (int l = tid; l < m; l += 256) fq[l] = __expf(fq[l] - mx);
-    __syncthreads();
+}
+
+// grid = (dv / 32 column blocks, B*H); block = 256 threads = 32 columns x 8 groups of features. Every column block of a
+// (batch, head) needs z + phi(k) for the normaliser; none of them stores it (the blocks are not ordered among themselves):
+// decode_z_kernel, launched behind this one on the same stream, applies z += phi(k).
+template <typename T>
+__global__ void __launch_bounds__(256) decode_step_kernel(const T *q, const T *k, const T *v, const T *M, const T *W, float *S,
+                                                           const float *z, T *o, int H, int d, int r, int m, int dv, int w_per_head,
+                                                           float s)
+{
+    extern __shared__ float sm[];
+    float *xq = sm, *xk = xq + r, *fq = xk + r, *fk = fq + m, *red = fk + m;   // red: 8 x 32 partial numerators + 8 partial normalisers + scratch
+    const int bh = blockIdx.y, h = bh % H, tid = threadIdx.x;
+    token_features<T, true>(q + (size_t)bh * d, k + (size_t)bh * d, M + (size_t)h * r * d, W + (size_t)(w_per_head ? h : 0) * m * r,
+                            xq, xk, fq, fk, red, d, r, m, s);
 
     // state update and read-out: thread = (column, feature group)
     const int col = blockIdx.x * 32 + (tid & 31), grp = tid >> 5;
     const float vv = ldf(v, (size_t)bh * dv + col);
     float *Sb = S + (size_t)bh * m * dv;
-    float *zb = z + (size_t)bh * m;
+    const float *zb = z + (size_t)bh * m;
     float num = 0.f, den = 0.f;
     for (int l = grp; l < m; l += 8) {
         const float snew = fmaf(fk[l], vv, Sb[(size_t)l * dv + col]);
         Sb[(size_t)l * dv + col] = snew;
         num = fmaf(fq[l], snew, num);
         if ((tid & 31) == 0) {                       // one lane per group carries the normaliser
-            const float znew = zb[l] + fk[l];
-            if (blockIdx.x == 0) zb[l] = znew;       // every column block needs z; one of them stores it
-            den = fmaf(fq[l], znew, den);
+            den = fmaf(fq[l], zb[l] + fk[l], den);
         }
     }
     red[grp * 32 + (tid & 31)] = num;
@@ -96,6 +106,19 @@ __global__ void __launch_bounds__(256) decode_step_kernel(const T *q, const T *k
         if constexpr (sizeof(T) == 2) o[(size_t)bh * dv + blockIdx.x * 32 + tid] = __float2bfloat16_rn(out);
         else o[(size_t)bh * dv + blockIdx.x * 32 + tid] = out;
     }
+}
+
+// z += phi(k) of the new token; one block per (batch, head).
+template <typename T>
+__global__ void __launch_bounds__(256) decode_z_kernel(const T *k, const T *M, const T *W, float *z, int H, int d, int r, int m,
+                                                        int w_per_head, float s)
+{
+    extern __shared__ float sm[];
+    float *xq = sm, *xk = xq + r, *fq = xk + r, *fk = fq + m, *red = fk + m;
+    const int bh = blockIdx.x, h = bh % H;
+    token_features<T, false>(nullptr, k + (size_t)bh * d, M + (size_t)h * r * d, W + (size_t)(w_per_head ? h : 0) * m * r, xq, xk, fq,
+                             fk, red, d, r, m, s);
+    for (int l = threadIdx.x; l < m; l += 256) z[(size_t)bh * m + l] += fk[l];
 }
 
 }  // namespace
@@ -122,6 +145,12 @@ extern "C" darkattn_status_t darkattn_decode_step(darkattn_plan_t plan, const vo
     else
         decode_step_kernel<float><<<grid, 256, smem, st>>>((const float *)q, (const float *)k, (const float *)v, (const float *)M,
                                                            (const float *)W, S, z, (float *)o, D.H, D.d, D.r, D.m, D.dv, D.w_per_head, D.s);
+    if (D.bf16)
+        decode_z_kernel<__nv_bfloat16><<<D.BH, 256, smem, st>>>((const __nv_bfloat16 *)k, (const __nv_bfloat16 *)M, (const __nv_bfloat16 *)W, z,
+                                                              D.H, D.d, D.r, D.m, D.w_per_head, D.s);
+    else
+        decode_z_kernel<float><<<D.BH, 256, smem, st>>>((const float *)k, (const float *)M, (const float *)W, z, D.H, D.d, D.r, D.m,
+                                                        D.w_per_head, D.s);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_cuda_error(e, "decode_step"); return DARKATTN_ERR_CUDA; }
     return DARKATTN_OK;

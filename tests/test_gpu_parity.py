@@ -235,26 +235,35 @@ def test_gradient_of_the_projection_rows(binding, case):
     assert_close(got["dW"], want, TOL[wl.dtype], f"{case}: dW")
 
 
+DECODE = [
+    ("few_heads", dict(B=2, H=3, N=40, d=32, m=96, r=16, dv=64)),
+    # several thousand (batch, head) pairs with four column blocks each: the blocks of one pair land in different waves
+    ("many_heads_dv128", dict(B=64, H=48, N=5, d=32, m=64, r=16, dv=128)),
+]
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-def test_decode_steps_reproduce_the_causal_forward(binding, dtype):
+@pytest.mark.parametrize("name,kw", DECODE, ids=[s[0] for s in DECODE])
+def test_decode_steps_reproduce_the_causal_forward(binding, name, kw, dtype):
     """Token by token through the recurrent entry point: step t's output is row t of the causal attention."""
     import torch
     from tests.util import to_dev, torch_dtype
-    wl = inputs.small(name="decode", wid=83, B=2, H=3, N=40, d=32, m=96, r=16, dv=64, causal=True, dtype=dtype, backward=False)
+    wl = inputs.small(name="decode_" + name, wid=83, causal=True, dtype=dtype, backward=False, **kw)
     t = inputs.generate(wl)
     dt = torch_dtype(dtype)
+    B, H, N, d, m, r, dv = (kw[k] for k in ("B", "H", "N", "d", "m", "r", "dv"))
     Q, K, V, M, W = (to_dev(x, dt) for x in (t.Q, t.K, t.V, t.M, t.W))
-    plan = binding.darkattn_plan(2, 3, 40, 32, 96, r=16, dv=64, dtype=binding.F32 if dtype == "f32" else binding.BF16, causal=True)
-    S = torch.zeros(2, 3, 96, 64, dtype=torch.float32, device="cuda")
-    z = torch.zeros(2, 3, 96, dtype=torch.float32, device="cuda")
+    plan = binding.darkattn_plan(B, H, N, d, m, r=r, dv=dv, dtype=binding.F32 if dtype == "f32" else binding.BF16, causal=True)
+    S = torch.zeros(B, H, m, dv, dtype=torch.float32, device="cuda")
+    z = torch.zeros(B, H, m, dtype=torch.float32, device="cuda")
     rows = []
-    for i in range(wl.N):
-        o = torch.empty(2, 3, 64, dtype=dt, device="cuda")
+    for i in range(N):
+        o = torch.empty(B, H, dv, dtype=dt, device="cuda")
         binding.darkattn_decode_step(plan, Q[:, :, i].contiguous(), K[:, :, i].contiguous(), V[:, :, i].contiguous(), M, W, S, z, o)
         rows.append(o.float().cpu().numpy().astype(np.float64))
     got = np.stack(rows, axis=2)
     want = ref.forward(t.Q, t.K, t.V, t.M, t.W, causal=True)
-    assert_close(got, want, 1e-4 if dtype == "f32" else 1e-2, f"decode {dtype}")
+    assert_close(got, want, 1e-4 if dtype == "f32" else 1e-2, f"decode {name} {dtype}")
     plan.destroy()
 
 
