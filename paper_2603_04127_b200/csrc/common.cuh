@@ -54,10 +54,12 @@ struct SimtLayout {
 struct TensorLayout {
     size_t status;
     size_t Om;      // folded projections log2(e) s W M, bf16 [H, m, d]
+    size_t Oml;     // what the rounding of Om to bf16 left out, bf16 [H, m, d]: the projections are taken against Om + Oml
     size_t cs;      // key-side shift per (bh, slab), fp32
     size_t nK;      // key norms, fp32 [BH, N]
     size_t pnum;    // partial numerators, bf16 [nslab, BH, N, dv]
-    size_t pdr;     // partial normaliser and scale exponent, fp32 [nslab, BH, N, 2]
+    size_t pdr;     // per slab and row: the partial normalisers of the four 32-column groups and the exponent the partial is
+                    // scaled by, fp32 [nslab, BH, N, 8] (entries 0..3 and 4; 5..7 unused)
     size_t Sacc;    // non-causal state sums, fp32 [BH, m, dv]
     size_t zacc;    // fp32 [BH, m]
     size_t Sb;      // bf16 copy of the state, [BH, m, dv]
@@ -77,7 +79,7 @@ struct TensorLayout {
     size_t Rb;      // bf16 copy of Racc
     size_t total_bytes;
     // the forward -> backward stash (`saved`): per-row normalisers, key norms, folded projections, key shifts
-    size_t sv_sv, sv_nK, sv_Om, sv_cs, sv_zc, sv_Sb, sv_zt, sv_Sst, sv_bytes;
+    size_t sv_sv, sv_nK, sv_Om, sv_Oml, sv_cs, sv_zc, sv_Sb, sv_zt, sv_Sst, sv_bytes;
     size_t zc;      // workspace copy of the stash's per-chunk z (causal): sum_j phi(K)_jl over the chunks before t, fp32 [BH, T, m]
     int nslab, T, nsplit;
 };
@@ -87,7 +89,7 @@ struct TensorLayout {
 struct Stash {
     float2 *sv;
     float *nK;
-    __nv_bfloat16 *Om;
+    __nv_bfloat16 *Om, *Oml;
     float *cs;
     float *zc;      // causal: z before chunk t, [BH, T, m] (row t = 0 is not written: it is zero)
     __nv_bfloat16 *Sb;   // non-causal: S of the whole sequence, bf16 [BH, m, dv]
@@ -97,7 +99,8 @@ struct Stash {
 inline Stash stash_in_workspace(const TensorLayout &Y, char *ws)
 {
     return Stash{reinterpret_cast<float2 *>(ws + Y.sv), reinterpret_cast<float *>(ws + Y.nK),
-                 reinterpret_cast<__nv_bfloat16 *>(ws + Y.Om), reinterpret_cast<float *>(ws + Y.cs),
+                 reinterpret_cast<__nv_bfloat16 *>(ws + Y.Om), reinterpret_cast<__nv_bfloat16 *>(ws + Y.Oml),
+                 reinterpret_cast<float *>(ws + Y.cs),
                  reinterpret_cast<float *>(ws + Y.zc), reinterpret_cast<__nv_bfloat16 *>(ws + Y.Sb),
                  reinterpret_cast<float *>(ws + Y.zacc), reinterpret_cast<__nv_bfloat16 *>(ws + Y.Sst)};
 }
@@ -105,7 +108,8 @@ inline Stash stash_in_saved(const TensorLayout &Y, void *saved)
 {
     char *b = static_cast<char *>(saved);
     return Stash{reinterpret_cast<float2 *>(b + Y.sv_sv), reinterpret_cast<float *>(b + Y.sv_nK),
-                 reinterpret_cast<__nv_bfloat16 *>(b + Y.sv_Om), reinterpret_cast<float *>(b + Y.sv_cs),
+                 reinterpret_cast<__nv_bfloat16 *>(b + Y.sv_Om), reinterpret_cast<__nv_bfloat16 *>(b + Y.sv_Oml),
+                 reinterpret_cast<float *>(b + Y.sv_cs),
                  reinterpret_cast<float *>(b + Y.sv_zc), reinterpret_cast<__nv_bfloat16 *>(b + Y.sv_Sb),
                  reinterpret_cast<float *>(b + Y.sv_zt), reinterpret_cast<__nv_bfloat16 *>(b + Y.sv_Sst)};
 }

@@ -5,7 +5,9 @@
 // quantity of the attention is a sum over features, so a slab CTA produces, for its 128 features, the
 // partial numerator rows, the partial normaliser and the exponent its rows were scaled by; a small
 // combine kernel adds the slabs. Per 128-token tile a slab CTA computes
-//     U = X Omega_slab^T            Omega = log2(e) s W M folded once per call (u = w.(sMx) = (sM^T w).x)
+//     U = X Omega_slab^T            Omega = log2(e) s W M folded once per call (u = w.(sMx) = (sM^T w).x), kept as the
+//                                   sum of two bf16 matrices (its rounding and what the rounding left out), so that the
+//                                   exponent's argument is as accurate as its fp32 accumulation
 //     phi(Q) = 2^(U - rowmax U)     any per-row factor cancels in O, including exp(-|Mq|^2/2)
 //     phi(K) = 2^(U - n - c)        n = log2(e) |sMk|^2/2 per key (from the norms kernel), c per slab
 // and then, causal:   P = tril(phi(Q) phi(K)^T),  O = P V + phi(Q) S_prev,  S += phi(K)^T V,  z += phi(K)^T 1
@@ -29,10 +31,11 @@ constexpr int kMaxNsplit = 64;
 // ------------------------------------------------------------------ small helpers
 
 // ------------------------------------------------------------------ prologue kernels (SIMT, tiny)
-// Omega[h,l,c] = log2(e) * s * sum_a W[l,a] M[h,a,c]  (bf16). One block per (head, 4 rows l), one thread per column c
+// Omega[h,l,c] = log2(e) * s * sum_a W[l,a] M[h,a,c], stored as its bf16 rounding Om and the bf16 rounding Oml of what
+// that left out (Om + Oml carries 16 bits of Omega). One block per (head, 4 rows l), one thread per column c
 // (the block has d threads); many small blocks, because the kernel is bound by the latency of its loads.
-__global__ void fold_omega_kernel(const __nv_bfloat16 *W, const __nv_bfloat16 *M, __nv_bfloat16 *Om, int m, int r, int d,
-                                  int w_per_head, float coef)
+__global__ void fold_omega_kernel(const __nv_bfloat16 *W, const __nv_bfloat16 *M, __nv_bfloat16 *Om, __nv_bfloat16 *Oml, int m, int r,
+                                  int d, int w_per_head, float coef)
 {
     __shared__ __align__(16) float sw[4][128];
     const int h = blockIdx.y, l0 = blockIdx.x * 4, c = threadIdx.x;
@@ -57,7 +60,12 @@ __global__ void fold_omega_kernel(const __nv_bfloat16 *W, const __nv_bfloat16 *M
         }
     }
 #pragma unroll
-    for (int i = 0; i < 4; ++i) Om[((size_t)h * m + l0 + i) * d + c] = __float2bfloat16_rn(coef * acc[i]);
+    for (int i = 0; i < 4; ++i) {
+        const float om = coef * acc[i];
+        const __nv_bfloat16 hi = __float2bfloat16_rn(om);
+        Om[((size_t)h * m + l0 + i) * d + c] = hi;
+        Oml[((size_t)h * m + l0 + i) * d + c] = __float2bfloat16_rn(om - __bfloat162float(hi));
+    }
 }
 
 // Key-side shift of a slab, in log2 units: c = log2(e) * max(0, max_l |w_l|^2/2 - 40).
@@ -168,12 +176,12 @@ __global__ void __launch_bounds__(160, 1) tc_key_norms_kernel(const __grid_const
 
 // ------------------------------------------------------------------ the main kernel
 struct MainParams {
-    CUtensorMap mapQ, mapK, mapV, mapOm, mapSb, mapPN;
+    CUtensorMap mapQ, mapK, mapV, mapOm, mapOml, mapSb, mapPN;
     CUtensorMap mapSst;  // causal, when stash_S: S before every chunk as [BH*T*m, dv] bf16, for the backward pass
     int stash_S;
     const float *nK;     // [BH, N]      key norms in log2 units
     const float *cs;     // [BH, nslab]  key-side shift per slab (log2 units)
-    float *pdr;          // [nslab, BH*N, 2]  partial normaliser and the exponent the partial is scaled by
+    float *pdr;          // [nslab, BH*N, 8]  partial normalisers of the four column groups (0..3), exponent the partial is scaled by (4)
     float *Sacc;         // [BH, m, DV]  fp32 state sums (non-causal key pass, atomics)
     float *zacc;         // [BH, m]
     // causal scan cut into nsplit segments of the sequence: the key pass stores one state per segment
@@ -200,8 +208,9 @@ __device__ __forceinline__ void store_row_f32x32_bf16(const uint32_t (&v)[32], u
 }
 
 // phi(Q) of one row segment: row maximum over the slab's 128 features (exchanged with the three other warps
-// of the lane quarter through red[4][128]), 2^(u - max) packed to bf16 into TMEM columns fq + col0/2,
-// returns sum_l phi(Q)_l z_l over the segment. rmax receives the row maximum.
+// of the lane quarter through red[4][128]), 2^(u - max) packed to bf16 into TMEM columns fq + col0/2.
+// rmax receives the row maximum. WITH_Z: returns sum_l phi(Q)_l z_l over the segment (else 0).
+template <bool WITH_Z>
 __device__ __forceinline__ float query_features_to_tmem(uint32_t u_addr, uint32_t fq_addr, float *red, const float *z, int q4,
                                                         int g, int r, int col0, float &rmax)
 {
@@ -218,9 +227,11 @@ __device__ __forceinline__ float query_features_to_tmem(uint32_t u_addr, uint32_
 #pragma unroll
     for (int j = 0; j < 32; j += 2) {
         const float f0 = ex2f(__uint_as_float(v[j]) - rmax), f1 = ex2f(__uint_as_float(v[j + 1]) - rmax);
-        const float2 zz = *reinterpret_cast<const float2 *>(z + col0 + j);
-        dz = fmaf(f0, zz.x, dz);
-        dz = fmaf(f1, zz.y, dz);
+        if constexpr (WITH_Z) {
+            const float2 zz = *reinterpret_cast<const float2 *>(z + col0 + j);
+            dz = fmaf(f0, zz.x, dz);
+            dz = fmaf(f1, zz.y, dz);
+        }
         pk[j / 2] = pack_bf16(f0, f1);
     }
     tmem_st16(fq_addr + col0 / 2, pk);
@@ -230,34 +241,49 @@ __device__ __forceinline__ float query_features_to_tmem(uint32_t u_addr, uint32_
 
 template <int D, int DV>
 struct FwdCausalSmem {
-    static constexpr int kOm = 0;
-    static constexpr int kQ = kOm + 128 * D * 2;
+    static constexpr int kOm = 0;                          // folded projections of the slab, rounded    [128 l, D]
+    static constexpr int kOml = kOm + 128 * D * 2;         // ... and what the rounding left out         [128 l, D]
+    static constexpr int kQ = kOml + 128 * D * 2;
     static constexpr int kK = kQ + 128 * D * 2;
     static constexpr int kV = kK + 128 * D * 2;
     static constexpr int kFK = kV + 128 * DV * 2;          // phi(K)                              [128, 128]
     static constexpr int kSb = kFK + 32768;                // bf16 copy of the state              [128 l, DV]
-    static constexpr int kStg = kSb + 128 * DV * 2;        // output staging; its first 2 KB hold the ones operand mid-chunk
-    static constexpr int kZ = kStg + 128 * DV * 2;         // z_prev, float[128]
-    static constexpr int kRed = kZ + 512;                  // float[4][128] exchange between the warps of a row
-    static constexpr int kBars = kRed + 2048;
+    static constexpr int kRed = kSb + 128 * DV * 2;        // float[4][128]: row maxima exchanged between the warps of a row;
+                                                           // mid-chunk the same 2 KB hold the ones operand of z += phi(K)^T 1
+    static constexpr int kZ = kRed + 2048;                 // z_prev, float[128]
+    static constexpr int kBars = kZ + 512;
     static constexpr int kTotal = kBars + 256;
 };
 
-// TMEM columns of the causal kernel: state S at 0 (DV), z at 128 (16), packed phi(Q) at 160 (64), R1 at 256, R2 at 384.
-constexpr uint32_t kColS = 0, kColZ = 128, kColFQ = 160, kColR1 = 256, kColR2 = 384;
+// TMEM columns of the causal kernel: state S at 0 (DV), four partial sums of z at 128 (16 each: consecutive MMAs of
+// z += phi(K)^T 1 go to different ones, so that none has to wait for the one before), packed phi(Q) at 192 (64),
+// R1 at 256, R2 at 384.
+constexpr uint32_t kColS = 0, kColZ = 128, kColFQ = 192, kColR1 = 256, kColR2 = 384;
 
-enum CBars { CB_OM, CB_Q, CB_K, CB_V, CM1, CM2, CM3, CMS, CM4, CE0, CE1, CE2, CE3, CE4, CNBARS };
+enum CBars { CB_OM, CB_Q, CB_K, CB_V, CB_ST, CM1, CM2, CM3, CMS, CM4, CE0, CE1, CE2, CE3, CE4, CNBARS };
+
+// X (Om + Oml)^T into a TMEM region: the projection against both halves of the folded matrix
+template <int D>
+__device__ __forceinline__ void issue_projection(uint32_t dst, const TileDesc &tX, const TileDesc &tOm, const TileDesc &tOml, uint32_t idesc)
+{
+    _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(dst, kdesc(tX, k), kdesc(tOm, k), idesc, k > 0);
+    _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(dst, kdesc(tX, k), kdesc(tOml, k), idesc, 1);
+}
 
 // Causal: one CTA per (b, h, slab) walks the chunks of the sequence.
 //   R1: U_Q -> (phi(Q) read) -> P = phi(Q) phi(K)^T -> packed tril(P) (A operand of P V) -> U_Q of the next chunk
-//   R2: U_K -> (phi(K) read) -> O = phi(Q) S_prev + P V -> (O read)
+//   R2: U_K -> (phi(K) read) -> O = phi(Q) S_prev + P V -> (O read) -> U_K of the next chunk
+// The epilogue warps work in this order: phi(K) of chunk t; the bf16 copy of the state through chunk t - 1 (while P
+// runs); tril(P); the output tile and z; phi(Q) of chunk t + 1 (both projections of the next chunk are issued behind
+// the output MMAs and run while the output is read). The state tile's buffer doubles as the staging tile of the
+// output's TMA store: between the output MMAs of chunk t and the copy of the state through chunk t nobody reads it.
 template <int D, int DV>
 __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid_constant__ MainParams p)
 {
     using L = FwdCausalSmem<D, DV>;
     extern __shared__ __align__(1024) unsigned char smem[];
-    unsigned char *sOm = smem + L::kOm, *sQ = smem + L::kQ, *sK = smem + L::kK, *sV = smem + L::kV;
-    unsigned char *sFK = smem + L::kFK, *sSb = smem + L::kSb, *sStg = smem + L::kStg;
+    unsigned char *sOm = smem + L::kOm, *sOml = smem + L::kOml, *sQ = smem + L::kQ, *sK = smem + L::kK, *sV = smem + L::kV;
+    unsigned char *sFK = smem + L::kFK, *sSb = smem + L::kSb;
     float *sZ = reinterpret_cast<float *>(smem + L::kZ), *sRed = reinterpret_cast<float *>(smem + L::kRed);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::kBars);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + CNBARS);
@@ -269,6 +295,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
     const int row0 = bh * p.N;
     const int tbeg = (int)((long long)p.T * seg / p.nsplit), tend = (int)((long long)p.T * (seg + 1) / p.nsplit);
     const bool fresh = (seg == 0);                 // the scan state starts at zero (else at the segment's prefix state)
+    // the state through the segment's last chunk is also copied (and stored) when the backward pass will start the
+    // next segment from it
+    const bool copy_last = p.stash_S && tend < p.T;
 
     if (tid == 0) {
         for (int i = 0; i < CE0; ++i) mbar_init(bars + i, 1);
@@ -298,11 +327,12 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
             }
             tmem_st32(lane_addr + kColS + col0, v);
         }
-        if (col0 == 0) {
+        {       // z: the prefix into the first partial sum, zero into the three others (one per column group's warp)
             uint32_t v[16];
+            const uint32_t zv = (col0 == 0) ? __float_as_uint(sZ[r]) : 0u;
 #pragma unroll
-            for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(sZ[r]);
-            tmem_st16(lane_addr + kColZ, v);
+            for (int j = 0; j < 16; ++j) v[j] = zv;
+            tmem_st16(lane_addr + kColZ + (col0 / 32) * 16, v);
         }
         tmem_wait_st();
     }
@@ -319,16 +349,28 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
                 mbar_expect_tx(bar, 128 * width * 2);
                 for (int a = 0; a < width / 64; ++a) tma_load_2d(dst + a * 16384, map, bar, a * 64, row0 + t * 128);
             };
-            const TileDesc tOm(sOm), tQ(sQ), tK(sK), tV(sV), tFK(sFK), tSb(sSb);
-            const uint64_t ones_desc = make_sdesc(smem_u32(sStg), 16384, 1024);
+            const int prow0 = (slab * p.BH + bh) * p.N;
+            auto store_output = [&](int t) {       // this slab's part of the output rows of chunk t, staged in the state tile's buffer
+                for (int a = 0; a < DV / 64; ++a) tma_store_2d(&p.mapPN, sSb + a * 16384, a * 64, prow0 + t * 128);
+                tma_store_commit();
+            };
+            auto store_state = [&](int t) {        // the bf16 state before chunk t, for the backward pass
+                for (int a = 0; a < DV / 64; ++a) tma_store_2d(&p.mapSst, sSb + a * 16384, a * 64, (bh * p.T + t) * p.m + slab * 128);
+                tma_store_commit();
+            };
+            const TileDesc tOm(sOm), tOml(sOml), tQ(sQ), tK(sK), tV(sV), tFK(sFK), tSb(sSb);
+            const uint64_t ones_desc = make_sdesc(smem_u32(sRed), 16384, 1024);
             const uint32_t id_kk = make_idesc(128, 128, 0, 0);
             const uint32_t id_o = make_idesc(128, DV, 0, 1);
             const uint32_t id_s = make_idesc(128, DV, 1, 1);
             const uint32_t id_z = make_idesc(128, 16, 1, 1);
             const uint32_t R1 = tmem + kColR1, R2 = tmem + kColR2, FQ = tmem + kColFQ;
 
-            mbar_expect_tx(bars + CB_OM, 128 * D * 2 + (fresh ? 0 : 128 * DV * 2));
-            for (int a = 0; a < D / 64; ++a) tma_load_2d(sOm + a * 16384, &p.mapOm, bars + CB_OM, a * 64, h * p.m + slab * 128);
+            mbar_expect_tx(bars + CB_OM, 2 * 128 * D * 2 + (fresh ? 0 : 128 * DV * 2));
+            for (int a = 0; a < D / 64; ++a) {
+                tma_load_2d(sOm + a * 16384, &p.mapOm, bars + CB_OM, a * 64, h * p.m + slab * 128);
+                tma_load_2d(sOml + a * 16384, &p.mapOml, bars + CB_OM, a * 64, h * p.m + slab * 128);
+            }
             if (!fresh)     // bf16 copy of the segment's prefix state
                 for (int a = 0; a < DV / 64; ++a)
                     tma_load_2d(sSb + a * 16384, &p.mapSb, bars + CB_OM, a * 64, (bh * p.nsplit + seg) * p.m + slab * 128);
@@ -336,58 +378,75 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
             load_tile(sK, &p.mapK, bars + CB_K, D, tbeg);
             load_tile(sV, &p.mapV, bars + CB_V, DV, tbeg);
 
-            bool ok = wait_or_abort(bars + CB_OM, 0, status, abort_flag);
-            if (ok) ok = wait_or_abort(bars + CB_Q, 0, status, abort_flag);
+#define CWAIT(b, q) do { ok = wait_or_abort(bars + (b), (q), status, abort_flag); } while (0)
+            bool ok = true;
+            CWAIT(CB_OM, 0);
+            if (ok) CWAIT(CB_Q, 0);
             if (ok) {
                 tc_fence_after();
-                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R1, kdesc(tQ, k), kdesc(tOm, k), id_kk, k > 0);         // U_Q of chunk 0
+                issue_projection<D>(R1, tQ, tOm, tOml, id_kk);                                                    // U_Q of the first chunk
                 mma_commit(bars + CM1);
+                CWAIT(CB_K, 0);
             }
+            if (ok) {
+                tc_fence_after();
+                issue_projection<D>(R2, tK, tOm, tOml, id_kk);                                                    // U_K of the first chunk
+                mma_commit(bars + CM2);
+                CWAIT(CE0, 0);                                                  // phi(Q) packed, Q tile consumed
+            }
+            if (ok && tbeg + 1 < tend) load_tile(sQ, &p.mapQ, bars + CB_Q, D, tbeg + 1);
             for (int t = tbeg; t < tend && ok; ++t) {
                 const uint32_t ph = (t - tbeg) & 1;
                 const bool first = (t == tbeg) && fresh, last = (t + 1 == tend);
-#define CWAIT(b) do { ok = wait_or_abort(bars + (b), ph, status, abort_flag); } while (0)
-                CWAIT(CB_K); if (!ok) break;
-                tc_fence_after();
-                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R2, kdesc(tK, k), kdesc(tOm, k), id_kk, k > 0);         // U_K
-                mma_commit(bars + CM2);
-                CWAIT(CE0); if (!ok) break;                                     // phi(Q) packed in TMEM, R1 read, Q tile consumed
-                if (!last) load_tile(sQ, &p.mapQ, bars + CB_Q, D, t + 1);
-                CWAIT(CE1); if (!ok) break;                                     // phi(K) in smem, R2 read, K tile consumed
+                CWAIT(CE1, ph); if (!ok) break;                                 // phi(K) and the ones in smem, R2 read, K tile consumed
                 if (!last) load_tile(sK, &p.mapK, bars + CB_K, D, t + 1);
                 tc_fence_after();
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R1, FQ + k * 8, kdesc(tFK, k), id_kk, k > 0);                // P = phi(Q) phi(K)^T
                 mma_commit(bars + CM3);
-                if (!first)
+                if (!first) {
+                    if (t > tbeg) {                                             // the bf16 state through chunk t - 1 is in smem
+                        CWAIT(CE4, ph ^ 1); if (!ok) break;
+                        if (p.stash_S) store_state(t);
+                    }
                     _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R2, FQ + k * 8, mndesc(tSb, k), id_o, k > 0);            // O = phi(Q) S_prev
-                // z += phi(K)^T 1 now: its operand of ones lies in the staging tile, which the output read-out overwrites
-                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColZ, mndesc(tFK, k), ones_desc, id_z, (!first) || k > 0);
-                CWAIT(CB_V); if (!ok) break;
-                CWAIT(CE2); if (!ok) break;                                     // tril(P) packed in R1
+                }
+                _Pragma("unroll") for (int k = 0; k < 8; ++k)                                                                     // z += phi(K)^T 1
+                    mma_ss(tmem + kColZ + 16 * (k & 3), mndesc(tFK, k), ones_desc, id_z, (!first) || k >= 4);
+                CWAIT(CB_V, ph); if (!ok) break;
+                CWAIT(CE2, ph); if (!ok) break;                                 // tril(P) packed in R1
                 tc_fence_after();
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R2, R1 + k * 8, mndesc(tV, k), id_o, (!first) || k > 0);     // O += P V
+                if (p.stash_S) tma_store_wait_read();       // the stash copy of the state before this chunk has left its tile: the output may be staged there
                 mma_commit(bars + CM4);
-                // the state update is not on the chunk's critical path: it runs while the output tile is read out
-                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColS, mndesc(tFK, k), mndesc(tV, k), id_s, (!first) || k > 0);   // S += phi(K)^T V
-                if (p.stash_S) tma_store_wait_read();       // the stash copy of the state before this chunk has left its tile
-                mma_commit(bars + CMS);
-                if (!last) {
-                    ok = wait_or_abort(bars + CB_Q, ph ^ 1, status, abort_flag);
-                    if (!ok) break;
+                if (!last) {        // U_Q of the next chunk, while the epilogue warps read the output tile out
+                    CWAIT(CB_Q, ph ^ 1); if (!ok) break;
                     tc_fence_after();
-                    _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R1, kdesc(tQ, k), kdesc(tOm, k), id_kk, k > 0);     // U_Q of the next chunk
+                    issue_projection<D>(R1, tQ, tOm, tOml, id_kk);
                     mma_commit(bars + CM1);
                 }
-                CWAIT(CMS); if (!ok) break;                                     // (also: the output MMAs before it are done)
-                if (!last) load_tile(sV, &p.mapV, bars + CB_V, DV, t + 1);
-                CWAIT(CE3); if (!ok) break;
-                CWAIT(CE4); if (!ok) break;
-                if (p.stash_S && t + 1 < p.T) {         // the state through this chunk, bf16: what the backward pass starts chunk t + 1 from
-                    for (int a = 0; a < DV / 64; ++a) tma_store_2d(&p.mapSst, sSb + a * 16384, a * 64, (bh * p.T + t + 1) * p.m + slab * 128);
-                    tma_store_commit();
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColS, mndesc(tFK, k), mndesc(tV, k), id_s, (!first) || k > 0);   // S += phi(K)^T V
+                mma_commit(bars + CMS);
+                CWAIT(CE3, ph); if (!ok) break;                                 // the output tile has been read out of R2 and staged
+                store_output(t);
+                if (!last) {
+                    CWAIT(CB_K, ph ^ 1); if (!ok) break;
+                    tc_fence_after();
+                    issue_projection<D>(R2, tK, tOm, tOml, id_kk);                                                // U_K of the next chunk
+                    mma_commit(bars + CM2);
                 }
-#undef CWAIT
+                if (!last || copy_last) { tma_store_wait_read(); mbar_arrive(bars + CB_ST); }     // the staged output has left the state tile's buffer
+                CWAIT(CMS, ph); if (!ok) break;                                 // V tile consumed
+                if (!last) {
+                    load_tile(sV, &p.mapV, bars + CB_V, DV, t + 1);
+                    CWAIT(CE0, ph ^ 1); if (!ok) break;                         // phi(Q) of the next chunk packed, its Q tile consumed
+                    if (t + 2 < tend) load_tile(sQ, &p.mapQ, bars + CB_Q, D, t + 2);
+                }
             }
+            if (ok && copy_last) {      // the state through the segment's last chunk: what the backward pass starts the next segment from
+                CWAIT(CE4, (tend - 1 - tbeg) & 1);
+                if (ok) store_state(tend);
+            }
+#undef CWAIT
             tma_store_wait_all();
         }
     } else {
@@ -397,41 +456,62 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
         const uint32_t R1 = lane_addr + kColR1, R2 = lane_addr + kColR2;
         const float cshift = p.cs[bh * p.nslab + slab];
         const size_t prow0 = ((size_t)slab * p.BH + bh) * p.N;
+        uint32_t *sOnes = reinterpret_cast<uint32_t *>(sRed);
         bool ok = true;
-        for (int t = tbeg; t < tend && ok; ++t) {
-            const uint32_t ph = (t - tbeg) & 1;
-            const bool last = (t + 1 == tend);
-#define EWAIT(b) do { ok = __all_sync(0xffffffffu, wait_or_abort(bars + (b), ph, status, abort_flag)); } while (0)
-            const float nk = p.nK[(size_t)row0 + (size_t)t * 128 + r] + cshift;
-            float rmax;
-            EWAIT(CM1); if (!ok) break;
+        float rmax = 0.f;                           // row maximum of the chunk whose phi(Q) was formed last
+#define EWAIT(b, q) do { ok = __all_sync(0xffffffffu, wait_or_abort(bars + (b), (q), status, abort_flag)); } while (0)
+        // phi(K): once the four warps of these rows are done with the exchanged maxima the array is filled with bf16 ones,
+        // the B operand of z += phi(K)^T 1
+        auto key_features = [&](float nk) {
             tc_fence_after();
-            const float dz = query_features_to_tmem(R1, lane_addr + kColFQ, sRed, sZ, q4, g, r, col0, rmax);
-            tc_fence_before();
-            mbar_arrive_warp(bars + CE0);
-
-            EWAIT(CM2); if (!ok) break;
-            tc_fence_after();
+            quarter_sync(q4);
+            sOnes[g * 128 + r] = 0x3F803F80u;
             features_to_tile(R2 + col0, nk, sFK, r, col0);
-            if (warp == 0) {  // 2 KB of bf16 ones at the start of the staging tile: B operand of z += phi(K)^T 1
-                if (tid == 0) tma_store_wait_read();       // once the previous chunk's store has left the tile
-                __syncwarp();
-#pragma unroll
-                for (int i = 0; i < 4; ++i)
-                    *reinterpret_cast<uint4 *>(sStg + (i * 32 + tid) * 16) = make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
-            }
             fence_async_smem();
             tc_fence_before();
             mbar_arrive_warp(bars + CE1);
+        };
+        float dz = 0.f;                             // phi(Q) z_prev over this thread's features, of the chunk whose phi(Q) was formed last
+        auto query_features = [&]() {
+            tc_fence_after();
+            dz = query_features_to_tmem<true>(R1, lane_addr + kColFQ, sRed, sZ, q4, g, r, col0, rmax);
+            tc_fence_before();
+            mbar_arrive_warp(bars + CE0);
+        };
+        // the state through chunk t as the bf16 operand of phi(Q) S, once the staged output of chunk t has left the tile
+        auto copy_state = [&](int t) -> bool {
+            const uint32_t q = (t - tbeg) & 1;
+            EWAIT(CB_ST, q); if (!ok) return false;
+            EWAIT(CMS, q); if (!ok) return false;
+            tc_fence_after();
+            if (col0 < DV) tmem_row_to_tile(lane_addr + kColS + col0, sSb, r, col0);
+            fence_async_smem();
+            tc_fence_before();
+            mbar_arrive_warp(bars + CE4);
+            return true;
+        };
+        EWAIT(CM1, 0);
+        if (ok) query_features();
+        float nk_next = p.nK[(size_t)row0 + (size_t)tbeg * 128 + r] + cshift;
+        for (int t = tbeg; t < tend && ok; ++t) {
+            const uint32_t ph = (t - tbeg) & 1;
+            const bool last = (t + 1 == tend);
+            const size_t prow = prow0 + (size_t)t * 128 + r;
+            const float nk = nk_next;
+            if (!last) nk_next = p.nK[(size_t)row0 + (size_t)(t + 1) * 128 + r] + cshift;     // needed a chunk from now
 
-            EWAIT(CM3); if (!ok) break;
+            EWAIT(CM2, ph); if (!ok) break;
+            key_features(nk);
+            if (t > tbeg && !copy_state(t - 1)) break;      // while P runs
+
+            EWAIT(CM3, ph); if (!ok) break;
             tc_fence_after();
             float rowsum = 0.f;
             {
                 uint32_t v[32], pk[16];
                 tmem_ld32(R1 + col0, v);
                 tmem_wait_ld();
-                quarter_sync(q4);
+                quarter_sync(q4);                   // every column group has read P before anyone overwrites it
 #pragma unroll
                 for (int j = 0; j < 32; j += 2) {
                     const float x0 = (col0 + j <= r) ? __uint_as_float(v[j]) : 0.f;
@@ -445,48 +525,36 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
             tc_fence_before();
             mbar_arrive_warp(bars + CE2);
 
-            EWAIT(CM4); if (!ok) break;
+            EWAIT(CM4, ph); if (!ok) break;         // the output tile; z through this chunk (its MMAs ran ahead of the output's)
             tc_fence_after();
             if (col0 < DV) {
                 uint32_t v[32];
                 tmem_ld32(R2 + col0, v);
                 tmem_wait_ld();
-                store_row_f32x32_bf16(v, sStg, r, col0);
+                store_row_f32x32_bf16(v, sSb, r, col0);
             }
-            sRed[g * 128 + r] = rowsum + dz;
+            if (g == 0 && t + 1 < p.T) {            // (also after a segment's last chunk: the next segment's backward needs it)
+                const uint32_t z0 = tmem_ld1(lane_addr + kColZ), z1 = tmem_ld1(lane_addr + kColZ + 16);
+                const uint32_t z2 = tmem_ld1(lane_addr + kColZ + 32), z3 = tmem_ld1(lane_addr + kColZ + 48);
+                tmem_wait_ld();
+                const float zv = (__uint_as_float(z0) + __uint_as_float(z1)) + (__uint_as_float(z2) + __uint_as_float(z3));
+                sZ[r] = zv;
+                p.zc[((size_t)bh * p.T + t + 1) * p.m + slab * 128 + r] = zv;
+            }
             fence_async_smem();
             tc_fence_before();
             mbar_arrive_warp(bars + CE3);
-            epi_sync();
-            if (tid == 0) {
-                for (int a = 0; a < DV / 64; ++a) tma_store_2d(&p.mapPN, sStg + a * 16384, a * 64, (int)(prow0 + (size_t)t * 128));
-                tma_store_commit();
+            p.pdr[8 * prow + g] = rowsum + dz;
+            if (g == 0) p.pdr[8 * prow + 4] = rmax + cshift;
+            epi_sync();                             // every z is in place before anyone forms the next chunk's phi(Q)
+
+            if (!last) {
+                EWAIT(CM1, ph ^ 1); if (!ok) break;
+                query_features();
             }
-            if (g == 0) {
-                const float den = sRed[r] + sRed[128 + r] + sRed[256 + r] + sRed[384 + r];
-                if (!(den > 0.f) || !isfinite(den)) atomicCAS(status, 0, (int)DARKATTN_ERR_NONFINITE);
-                *reinterpret_cast<float2 *>(p.pdr + 2 * (prow0 + (size_t)t * 128 + r)) = make_float2(den, rmax + cshift);
-            }
-            quarter_sync(q4);                      // the exchange array is free for the next chunk's maxima
-            EWAIT(CMS); if (!ok) break;
-            tc_fence_after();
-            if (!last || (p.stash_S && t + 1 < p.T)) {
-                if (col0 < DV) tmem_row_to_tile(lane_addr + kColS + col0, sSb, r, col0);
-                fence_async_smem();
-            }
-            if (g == 0 && t + 1 < p.T) {        // z through this chunk: the next chunk's normaliser term, and the backward pass's
-                uint32_t v[16];                 // (also after a segment's last chunk: the next segment's backward needs it)
-                tmem_ld16(lane_addr + kColZ, v);
-                tmem_wait_ld();
-                sZ[r] = __uint_as_float(v[0]);
-                p.zc[((size_t)bh * p.T + t + 1) * p.m + slab * 128 + r] = __uint_as_float(v[0]);
-            }
-            epi_sync();       // a warp that runs ahead into the next chunk reads every z right away
-            tc_fence_before();
-            mbar_arrive_warp(bars + CE4);
-#undef EWAIT
         }
-        if (tid == 0) tma_store_wait_all();
+        if (ok && copy_last) copy_state(tend - 1);
+#undef EWAIT
     }
     if (*abort_flag) __nanosleep(200000);   // error path only: let copies and MMAs in flight drain
     tc_fence_before();
@@ -498,13 +566,16 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
 template <int D, int DV>
 struct FwdKeysSmem {
     // K and V tiles sit in rings of kStages buffers (4 where they are small enough), so that a tile's load is issued
-    // several tiles before its use; phi(K) tiles and TMEM regions alternate between two.
-    static constexpr int kStages = (3 * 128 * (D + DV) * 2 + 128 * D * 2 + 2 * 32768 + 4096 <= 232448) ? 4 : 2;
+    // several tiles before its use; TMEM regions alternate between two, and so do the phi(K) tiles where two fit.
+    static constexpr int kFixed = 2 * 128 * D * 2 + 2048 + 256;       // both halves of the folded projections, ones, barriers
+    static constexpr int kStages = (kFixed + 4 * 128 * (D + DV) * 2 + 2 * 32768 <= 232448) ? 4 : 2;
+    static constexpr int kFKs = (kFixed + kStages * 128 * (D + DV) * 2 + 2 * 32768 <= 232448) ? 2 : 1;
     static constexpr int kOm = 0;
-    static constexpr int kK = kOm + 128 * D * 2;
+    static constexpr int kOml = kOm + 128 * D * 2;
+    static constexpr int kK = kOml + 128 * D * 2;
     static constexpr int kV = kK + kStages * 128 * D * 2;
-    static constexpr int kFK = kV + kStages * 128 * DV * 2;   // two phi(K) tiles
-    static constexpr int kOnes = kFK + 2 * 32768;
+    static constexpr int kFK = kV + kStages * 128 * DV * 2;   // phi(K) tiles
+    static constexpr int kOnes = kFK + kFKs * 32768;
     static constexpr int kBars = kOnes + 2048;
     static constexpr int kTotal = kBars + 256;
 };
@@ -520,7 +591,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_keys_kernel(const __grid_c
     using L = FwdKeysSmem<D, DV>;
     extern __shared__ __align__(1024) unsigned char smem[];
     constexpr int kXT = 128 * D * 2, kVT = 128 * DV * 2;
-    unsigned char *sOm = smem + L::kOm, *sK = smem + L::kK, *sV = smem + L::kV, *sFK = smem + L::kFK, *sOnes = smem + L::kOnes;
+    unsigned char *sOm = smem + L::kOm, *sOml = smem + L::kOml, *sK = smem + L::kK, *sV = smem + L::kV, *sFK = smem + L::kFK, *sOnes = smem + L::kOnes;
+    constexpr int kFKstride = (L::kFKs == 2) ? 32768 : 0;     // one phi(K) tile: tile i + 1 is written once the state update of tile i is done
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::kBars);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + YNBARS);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + YNBARS + 1);
@@ -564,19 +636,22 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_keys_kernel(const __grid_c
                 mbar_expect_tx(bars + YB_V0 + b, kVT);
                 for (int a = 0; a < DV / 64; ++a) tma_load_2d(sV + b * kVT + a * 16384, &p.mapV, bars + YB_V0 + b, a * 64, row0 + (t0 + i) * 128);
             };
-            const TileDesc tOm(sOm), tF0(sFK), tF1(sFK + 32768);
+            const TileDesc tOm(sOm), tOml(sOml), tF0(sFK), tF1(sFK + kFKstride);
             const uint64_t ones_desc = make_sdesc(smem_u32(sOnes), 16384, 1024);
             const uint32_t id_kk = make_idesc(128, 128, 0, 0), id_s = make_idesc(128, DV, 1, 1), id_z = make_idesc(128, 16, 1, 1);
 
-            mbar_expect_tx(bars + YB_OM, 128 * D * 2);
-            for (int a = 0; a < D / 64; ++a) tma_load_2d(sOm + a * 16384, &p.mapOm, bars + YB_OM, a * 64, h * p.m + slab * 128);
+            mbar_expect_tx(bars + YB_OM, 2 * 128 * D * 2);
+            for (int a = 0; a < D / 64; ++a) {
+                tma_load_2d(sOm + a * 16384, &p.mapOm, bars + YB_OM, a * 64, h * p.m + slab * 128);
+                tma_load_2d(sOml + a * 16384, &p.mapOml, bars + YB_OM, a * 64, h * p.m + slab * 128);
+            }
             for (int i = 0; i < NST && i < n; ++i) { load_k(i); load_v(i); }
             bool ok = wait_or_abort(bars + YB_OM, 0, status, abort_flag);
             if (ok) ok = wait_or_abort(bars + YB_K0, 0, status, abort_flag);
             if (ok) {
                 tc_fence_after();
                 const TileDesc tK0(sK);
-                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(tmem + kColR1, kdesc(tK0, k), kdesc(tOm, k), id_kk, k > 0);
+                issue_projection<D>(tmem + kColR1, tK0, tOm, tOml, id_kk);
                 mma_commit(bars + YM2_0);
             }
             for (int i = 0; i < n && ok; ++i) {
@@ -588,7 +663,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_keys_kernel(const __grid_c
                     if (!ok) break;
                     tc_fence_after();
                     const TileDesc tKn(sK + sn * kXT);
-                    _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(tmem + (b ? kColR1 : kColR2), kdesc(tKn, k), kdesc(tOm, k), id_kk, k > 0);
+                    issue_projection<D>(tmem + (b ? kColR1 : kColR2), tKn, tOm, tOml, id_kk);
                     mma_commit(bars + YM2_0 + (b ^ 1));
                 }
                 ok = wait_or_abort(bars + YE1_0 + b, phb, status, abort_flag);      // phi(K) of tile i in smem; its K tile is consumed
@@ -619,8 +694,12 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_keys_kernel(const __grid_c
             const float nk = p.nK[(size_t)row0 + (size_t)(t0 + i) * 128 + r] + cshift;
             ok = __all_sync(0xffffffffu, wait_or_abort(bars + YM2_0 + b, phb, status, abort_flag));
             if (!ok) break;
+            if (L::kFKs == 1 && i > 0) {       // the one phi(K) tile is free once the state update of the tile before is done
+                ok = __all_sync(0xffffffffu, wait_or_abort(bars + YMS_0 + (b ^ 1), ((i - 1) >> 1) & 1, status, abort_flag));
+                if (!ok) break;
+            }
             tc_fence_after();
-            features_to_tile(lane_addr + (b ? kColR2 : kColR1) + col0, nk, sFK + b * 32768, r, col0);
+            features_to_tile(lane_addr + (b ? kColR2 : kColR1) + col0, nk, sFK + b * kFKstride, r, col0);
             fence_async_smem();
             tc_fence_before();
             mbar_arrive_warp(bars + YE1_0 + b);
@@ -662,9 +741,11 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_keys_kernel(const __grid_c
 // ------------------------------------------------------------------ non-causal, query pass: partial O = phi(Q) S, den = phi(Q) z
 template <int D, int DV>
 struct FwdQueriesSmem {
-    static constexpr int kStages = 4;                      // ring of Q tiles
+    // ring of Q tiles: 4 where they fit beside both halves of the folded projections, else 3
+    static constexpr int kStages = (2 * 128 * D * 2 + 4 * 128 * D * 2 + 2 * 128 * DV * 2 + 512 + 2048 + 256 <= 232448) ? 4 : 3;
     static constexpr int kOm = 0;
-    static constexpr int kQ = kOm + 128 * D * 2;
+    static constexpr int kOml = kOm + 128 * D * 2;
+    static constexpr int kQ = kOml + 128 * D * 2;
     static constexpr int kSb = kQ + kStages * 128 * D * 2; // bf16 state of the slab [128 l, DV]
     static constexpr int kStg = kSb + 128 * DV * 2;
     static constexpr int kZ = kStg + 128 * DV * 2;
@@ -682,7 +763,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_queries_kernel(const __gri
     using L = FwdQueriesSmem<D, DV>;
     extern __shared__ __align__(1024) unsigned char smem[];
     constexpr int kXT = 128 * D * 2;
-    unsigned char *sOm = smem + L::kOm, *sQ = smem + L::kQ, *sSb = smem + L::kSb, *sStg = smem + L::kStg;
+    unsigned char *sOm = smem + L::kOm, *sOml = smem + L::kOml, *sQ = smem + L::kQ, *sSb = smem + L::kSb, *sStg = smem + L::kStg;
     float *sZ = reinterpret_cast<float *>(smem + L::kZ), *sRed = reinterpret_cast<float *>(smem + L::kRed);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::kBars);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + UNBARS);
@@ -719,17 +800,20 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_queries_kernel(const __gri
                 mbar_expect_tx(bars + UB_Q0 + b, kXT);
                 for (int a = 0; a < D / 64; ++a) tma_load_2d(sQ + b * kXT + a * 16384, &p.mapQ, bars + UB_Q0 + b, a * 64, row0 + (t0 + i) * 128);
             };
-            const TileDesc tOm(sOm), tQ0(sQ), tSb(sSb);
+            const TileDesc tOm(sOm), tOml(sOml), tQ0(sQ), tSb(sSb);
             const uint32_t id_kk = make_idesc(128, 128, 0, 0), id_o = make_idesc(128, DV, 0, 1);
-            mbar_expect_tx(bars + UB_OM, 128 * D * 2 + 128 * DV * 2);
-            for (int a = 0; a < D / 64; ++a) tma_load_2d(sOm + a * 16384, &p.mapOm, bars + UB_OM, a * 64, h * p.m + slab * 128);
+            mbar_expect_tx(bars + UB_OM, 2 * 128 * D * 2 + 128 * DV * 2);
+            for (int a = 0; a < D / 64; ++a) {
+                tma_load_2d(sOm + a * 16384, &p.mapOm, bars + UB_OM, a * 64, h * p.m + slab * 128);
+                tma_load_2d(sOml + a * 16384, &p.mapOml, bars + UB_OM, a * 64, h * p.m + slab * 128);
+            }
             for (int a = 0; a < DV / 64; ++a) tma_load_2d(sSb + a * 16384, &p.mapSb, bars + UB_OM, a * 64, bh * p.m + slab * 128);
             for (int i = 0; i < NST && i < n; ++i) load_q(i);
             bool ok = wait_or_abort(bars + UB_OM, 0, status, abort_flag);
             if (ok) ok = wait_or_abort(bars + UB_Q0, 0, status, abort_flag);
             if (ok) {
                 tc_fence_after();
-                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(tmem + kColR1, kdesc(tQ0, k), kdesc(tOm, k), id_kk, k > 0);
+                issue_projection<D>(tmem + kColR1, tQ0, tOm, tOml, id_kk);
                 mma_commit(bars + UM1_0);
             }
             for (int i = 0; i < n && ok; ++i) {
@@ -741,7 +825,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_queries_kernel(const __gri
                     if (!ok) break;
                     tc_fence_after();
                     const TileDesc tQn(sQ + ((i + 1) % NST) * kXT);
-                    _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(tmem + (b ? kColR1 : kColR2), kdesc(tQn, k), kdesc(tOm, k), id_kk, k > 0);
+                    issue_projection<D>(tmem + (b ? kColR1 : kColR2), tQn, tOm, tOml, id_kk);
                     mma_commit(bars + UM1_0 + (b ^ 1));
                 }
                 ok = wait_or_abort(bars + UE0_0 + b, phb, status, abort_flag);      // phi(Q) packed; U read; Q tile consumed
@@ -767,7 +851,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_queries_kernel(const __gri
             ok = __all_sync(0xffffffffu, wait_or_abort(bars + UM1_0 + b, phb, status, abort_flag));
             if (!ok) break;
             tc_fence_after();
-            const float dz = query_features_to_tmem(R, lane_addr + b * 64, sRed, sZ, q4, g, r, col0, rmax);
+            const float dz = query_features_to_tmem<true>(R, lane_addr + b * 64, sRed, sZ, q4, g, r, col0, rmax);
             tc_fence_before();
             mbar_arrive_warp(bars + UE0_0 + b);
 
@@ -793,8 +877,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_queries_kernel(const __gri
             }
             if (g == 0) {
                 const float den = sRed[r] + sRed[128 + r] + sRed[256 + r] + sRed[384 + r];
-                if (!(den > 0.f) || !isfinite(den)) atomicCAS(status, 0, (int)DARKATTN_ERR_NONFINITE);
-                *reinterpret_cast<float2 *>(p.pdr + 2 * (prow0 + (size_t)(t0 + i) * 128 + r)) = make_float2(den, rmax + cshift);
+                float *dst = p.pdr + 8 * (prow0 + (size_t)(t0 + i) * 128 + r);
+                *reinterpret_cast<float4 *>(dst) = make_float4(den, 0.f, 0.f, 0.f);
+                dst[4] = rmax + cshift;
             }
             quarter_sync(q4);
         }
@@ -842,12 +927,13 @@ __global__ void segment_prefix_kernel(float *S, __nv_bfloat16 *Sb, float *z, int
     }
 }
 
-// O[row,:] = sum_s num_s[row,:] 2^(rho_s - rho) / sum_s den_s 2^(rho_s - rho), rho = max_s rho_s.
-// One thread per 8 output columns. The combined normaliser and rho are also written to sv for the backward pass.
+// O[row,:] = sum_s num_s[row,:] 2^(rho_s - rho) / sum_s den_s 2^(rho_s - rho), rho = max_s rho_s; den_s is the sum of
+// the slab's four partial normalisers. One thread per 8 output columns. The combined normaliser and rho are also
+// written to sv for the backward pass; a normaliser that is zero or not finite is reported through the status word.
 // NS > 0: the number of slabs at compile time (all loads of a thread are issued before the first use).
 template <int NS>
 __global__ void combine_kernel(const __nv_bfloat16 *pnum, const float *pdr, __nv_bfloat16 *O, float2 *sv,
-                               long long rows, int dv, int nslab_rt)
+                               long long rows, int dv, int nslab_rt, int *status)
 {
     const long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;
     const int per_row = dv / 8;
@@ -855,20 +941,24 @@ __global__ void combine_kernel(const __nv_bfloat16 *pnum, const float *pdr, __nv
     const long long row = i / per_row;
     const int c0 = (int)(i % per_row) * 8;
     float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}, den = 0.f, rho = -INFINITY;
+    auto slab_den = [](const float4 &d4) { return (d4.x + d4.y) + (d4.z + d4.w); };
     if constexpr (NS > 0) {
-        float2 dr[NS];
+        float4 d4[NS];
+        float rh[NS];
         uint4 raw[NS];
 #pragma unroll
         for (int s = 0; s < NS; ++s) {
-            dr[s] = *reinterpret_cast<const float2 *>(pdr + 2 * ((size_t)s * rows + row));
+            const float *q = pdr + 8 * ((size_t)s * rows + row);
+            d4[s] = *reinterpret_cast<const float4 *>(q);
+            rh[s] = q[4];
             raw[s] = *reinterpret_cast<const uint4 *>(pnum + ((size_t)s * rows + row) * dv + c0);
         }
 #pragma unroll
-        for (int s = 0; s < NS; ++s) rho = fmaxf(rho, dr[s].y);
+        for (int s = 0; s < NS; ++s) rho = fmaxf(rho, rh[s]);
 #pragma unroll
         for (int s = 0; s < NS; ++s) {
-            const float w = exp2f(dr[s].y - rho);
-            den = fmaf(dr[s].x, w, den);
+            const float w = exp2f(rh[s] - rho);
+            den = fmaf(slab_den(d4[s]), w, den);
             const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&raw[s]);
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
@@ -878,22 +968,25 @@ __global__ void combine_kernel(const __nv_bfloat16 *pnum, const float *pdr, __nv
             }
         }
     } else {
-        for (int s = 0; s < nslab_rt; ++s) rho = fmaxf(rho, pdr[2 * ((size_t)s * rows + row) + 1]);
+        for (int s = 0; s < nslab_rt; ++s) rho = fmaxf(rho, pdr[8 * ((size_t)s * rows + row) + 4]);
         for (int s = 0; s < nslab_rt; ++s) {
-            const float2 dr = *reinterpret_cast<const float2 *>(pdr + 2 * ((size_t)s * rows + row));
-            const float w = exp2f(dr.y - rho);
-            den = fmaf(dr.x, w, den);
+            const float *q = pdr + 8 * ((size_t)s * rows + row);
+            const float w = exp2f(q[4] - rho);
+            den = fmaf(slab_den(*reinterpret_cast<const float4 *>(q)), w, den);
             const uint4 raw = *reinterpret_cast<const uint4 *>(pnum + ((size_t)s * rows + row) * dv + c0);
             const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const float2 f = __bfloat1622float2(h2[q]);
-                acc[2 * q] = fmaf(f.x, w, acc[2 * q]);
-                acc[2 * q + 1] = fmaf(f.y, w, acc[2 * q + 1]);
+            for (int q2 = 0; q2 < 4; ++q2) {
+                const float2 f = __bfloat1622float2(h2[q2]);
+                acc[2 * q2] = fmaf(f.x, w, acc[2 * q2]);
+                acc[2 * q2 + 1] = fmaf(f.y, w, acc[2 * q2 + 1]);
             }
         }
     }
-    if (c0 == 0) sv[row] = make_float2(den, rho);
+    if (c0 == 0) {
+        sv[row] = make_float2(den, rho);
+        if (!(den > 0.f) || !isfinite(den)) atomicCAS(status, 0, (int)DARKATTN_ERR_NONFINITE);
+    }
     const float inv = 1.f / den;
     uint4 out;
     out.x = pack_bf16(acc[0] * inv, acc[1] * inv); out.y = pack_bf16(acc[2] * inv, acc[3] * inv);
@@ -983,10 +1076,11 @@ void tensor_make_layout(darkattn_plan_s *plan)
     size_t off = 0;
     Y.status = take(off, 256);
     Y.Om = take(off, (size_t)D.H * m * d * 2);
+    Y.Oml = take(off, (size_t)D.H * m * d * 2);
     Y.cs = take(off, BH * Y.nslab * 4);
     Y.nK = take(off, BH * N * 4);
     Y.pnum = take(off, (size_t)Y.nslab * BH * N * dv * 2);
-    Y.pdr = take(off, (size_t)Y.nslab * BH * N * 8);
+    Y.pdr = take(off, (size_t)Y.nslab * BH * N * 32);
     Y.Sacc = take(off, BH * nstate * m * dv * 4);
     Y.zacc = take(off, BH * nstate * m * 4);
     Y.Sb = take(off, BH * nstate * m * dv * 2);
@@ -998,6 +1092,7 @@ void tensor_make_layout(darkattn_plan_s *plan)
         Y.sv_sv = take(so, BH * N * 8);
         Y.sv_nK = take(so, BH * N * 4);
         Y.sv_Om = take(so, (size_t)D.H * m * d * 2);
+        Y.sv_Oml = take(so, (size_t)D.H * m * d * 2);
         Y.sv_cs = take(so, BH * Y.nslab * 4);
         Y.sv_zc = take(so, D.causal ? BH * (size_t)Y.T * m * 4 : 0);
         Y.sv_Sb = take(so, D.causal ? 0 : BH * m * dv * 2);
@@ -1049,8 +1144,8 @@ cudaError_t tensor_prologue(const darkattn_plan_s *plan, const void *K, const vo
         if (e == cudaSuccess) e = cudaStreamWaitEvent(sp, plan->aux_fork, 0);
     }
     timer_mark(plan, st, "fold_omega_kernel");
-    fold_omega_kernel<<<dim3(D.m / 4, D.H), D.d, 0, sp>>>((const __nv_bfloat16 *)W, (const __nv_bfloat16 *)M, out.Om, D.m, D.r, D.d,
-                                                      D.w_per_head, kLog2e * D.s);
+    fold_omega_kernel<<<dim3(D.m / 4, D.H), D.d, 0, sp>>>((const __nv_bfloat16 *)W, (const __nv_bfloat16 *)M, out.Om, out.Oml, D.m, D.r,
+                                                      D.d, D.w_per_head, kLog2e * D.s);
     chk();
     timer_mark(plan, st, "slab_shift_kernel");
     slab_shift_kernel<<<(unsigned)(BH * Y.nslab), 128, 0, sp>>>((const __nv_bfloat16 *)W, out.cs, D.H, D.m, D.r, Y.nslab, D.w_per_head);
@@ -1090,6 +1185,7 @@ darkattn_status_t tensor_forward(const darkattn_plan_s *plan, const void *Q, con
     memset(&P, 0, sizeof(P));
     bool ok = make_map(&P.mapQ, Q, BH * N, D.d, 128) && make_map(&P.mapK, K, BH * N, D.d, 128) &&
               make_map(&P.mapV, V, BH * N, D.dv, 128) && make_map(&P.mapOm, stash.Om, (size_t)D.H * D.m, D.d, 128) &&
+              make_map(&P.mapOml, stash.Oml, (size_t)D.H * D.m, D.d, 128) &&
               make_map(&P.mapSb, D.causal ? bf(Y.Sb) : stash.Sb, BH * (D.causal ? Y.nsplit : 1) * D.m, D.dv, 128) &&
               make_map(&P.mapPN, bf(Y.pnum), (size_t)Y.nslab * BH * N, D.dv, 128);
     if (!ok) { set_cuda_error(cudaErrorInvalidValue, "tensor_forward: tensor map encode"); return DARKATTN_ERR_CUDA; }
@@ -1138,10 +1234,10 @@ darkattn_status_t tensor_forward(const darkattn_plan_s *plan, const void *Q, con
         timer_mark(plan, st, "combine_kernel");
         const unsigned grid = (unsigned)((threads + 255) / 256);
         __nv_bfloat16 *Ob = (__nv_bfloat16 *)O;
-        if (Y.nslab == 1) combine_kernel<1><<<grid, 256, 0, st>>>(bf(Y.pnum), fl(Y.pdr), Ob, stash.sv, rows, D.dv, 1);
-        else if (Y.nslab == 2) combine_kernel<2><<<grid, 256, 0, st>>>(bf(Y.pnum), fl(Y.pdr), Ob, stash.sv, rows, D.dv, 2);
-        else if (Y.nslab == 4) combine_kernel<4><<<grid, 256, 0, st>>>(bf(Y.pnum), fl(Y.pdr), Ob, stash.sv, rows, D.dv, 4);
-        else combine_kernel<0><<<grid, 256, 0, st>>>(bf(Y.pnum), fl(Y.pdr), Ob, stash.sv, rows, D.dv, Y.nslab);
+        if (Y.nslab == 1) combine_kernel<1><<<grid, 256, 0, st>>>(bf(Y.pnum), fl(Y.pdr), Ob, stash.sv, rows, D.dv, 1, P.status);
+        else if (Y.nslab == 2) combine_kernel<2><<<grid, 256, 0, st>>>(bf(Y.pnum), fl(Y.pdr), Ob, stash.sv, rows, D.dv, 2, P.status);
+        else if (Y.nslab == 4) combine_kernel<4><<<grid, 256, 0, st>>>(bf(Y.pnum), fl(Y.pdr), Ob, stash.sv, rows, D.dv, 4, P.status);
+        else combine_kernel<0><<<grid, 256, 0, st>>>(bf(Y.pnum), fl(Y.pdr), Ob, stash.sv, rows, D.dv, Y.nslab, P.status);
         chk();
     }
     if (e != cudaSuccess) { set_cuda_error(e, "tensor_forward"); return DARKATTN_ERR_CUDA; }
