@@ -339,6 +339,15 @@ __device__ __forceinline__ uint64_t kdesc(const TileDesc &t, int k) { return t.k
 // MN-major operand: step k covers 16 K-rows of 128 bytes
 __device__ __forceinline__ uint64_t mndesc(const TileDesc &t, int k) { return t.mnmaj + (uint64_t)((k * 2048) >> 4); }
 
+// X (Om + Oml)^T into a TMEM region: the projection against both halves of the folded matrix (its bf16 rounding and
+// the bf16 rounding of what that left out), accumulated in fp32
+template <int D>
+__device__ __forceinline__ void issue_projection(uint32_t dst, const TileDesc &tX, const TileDesc &tOm, const TileDesc &tOml, uint32_t idesc)
+{
+    _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(dst, kdesc(tX, k), kdesc(tOm, k), idesc, k > 0);
+    _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(dst, kdesc(tX, k), kdesc(tOml, k), idesc, 1);
+}
+
 // ---------------------------------------------------------------- host side: tensor maps
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,

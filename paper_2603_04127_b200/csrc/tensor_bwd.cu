@@ -35,7 +35,7 @@ namespace {
 constexpr float kLn2 = 0.6931471805599453f;
 
 struct BwdParams {
-    CUtensorMap mapQ, mapK, mapV, mapG, mapOm, mapDQ, mapDK, mapDV;   // the last three: the gradients, for the (adding) stores
+    CUtensorMap mapQ, mapK, mapV, mapG, mapOm, mapOml, mapDQ, mapDK, mapDV;   // the last three: the gradients, for the (adding) stores
     CUtensorMap mapAh, mapBf;   // A^ and Bf as [BH*N, m] bf16: written by the query-side kernel, read by the key-side one
     CUtensorMap mapSst;         // S before every chunk as [BH*T*m, dv] bf16, from the forward pass
     const float2 *sv;     // [BH*N]  (normaliser, exponent it is scaled by) from the forward pass
@@ -54,23 +54,31 @@ template <int D, int DV>
 struct BwdSmem {
     static constexpr int kDmax = D > DV ? D : DV;
     static constexpr int kOm = 0;                          // folded projections of the slab [128 l, D]
-    static constexpr int kQA = kOm + 128 * D * 2;          // Q tile, then A^ (then E^Q)       [128, 128]
+    static constexpr int kAux = kOm + 128 * D * 2;         // query side: what the rounding of the folded projections left out [128 l, D];
+                                                           // key side: staging tile of the TMA stores of dV and dK
+    static constexpr int kQA = kAux + 32768;               // Q tile, then A^ (then E^Q)       [128, 128]
     static constexpr int kKB = kQA + 32768;                // K tile, then Bf (then E^K)        [128, 128]
     static constexpr int kV = kKB + 32768;                 // V tile                            [128, DV]
     static constexpr int kG = kV + 128 * DV * 2;           // dO tile; later the reloaded Q / K tile
     static constexpr int kSt = kG + 128 * kDmax * 2;       // bf16 copy of the scan state       [128 l, DV]
-    static constexpr int kStg = kSt + 32768;               // (32 KB: the query-side kernel also keeps a 128 x 128 feature tile there)
-                                                           // staging tile of the TMA stores of the partials
-    static constexpr int kVec = kStg + 128 * kDmax * 2;    // three float[128]
-    static constexpr int kBars = kVec + 1536;
-    static constexpr int kTotal = kBars + 256;
+                                                           // (32 KB: the query-side kernel also keeps a 128 x 128 feature tile there)
+    // 3 KB of small things. Query side: the 16 x 128 K-major operand holding -delta (two swizzle atoms of which only the
+    // rows 0 and 1, 256 bytes each, carry data: the MMA also reads the 768 bytes behind each and the kilobyte behind the
+    // second atom as rows 2..15, whose products land in output columns nobody reads), barriers and z in between.
+    static constexpr int kSmall = kSt + 32768;
+    static constexpr int kDel0 = kSmall;                   // rows 0, 1 of the first atom (k = 0..63)
+    static constexpr int kBars = kSmall + 256;
+    static constexpr int kVec = kSmall + 512;              // query side: float[128] (z); key side: two float[128] (rho, delta)
+    static constexpr int kDel1 = kSmall + 1024;            // rows 0, 1 of the second atom (k = 64..127)
+    static constexpr int kTotal = kSmall + 3072;
+    static_assert(kDel1 == kDel0 + 1024, "the two atoms of the -delta operand are 1 KB apart");
 };
 
 // TMEM columns (512 allocated): scan state at 0, T at 128, scratch R1 at 256 and R2 at 384.
 constexpr uint32_t kColState = 0, kColT = 128, kColR1 = 256, kColR2 = 384;
 
-// K-major 16 x 128 bf16 operand (two atoms of 2 KB): step k covers 16 elements of K
-__device__ __forceinline__ uint64_t vecdesc(const TileDesc &t, int k) { return t.kmaj + (uint64_t)(((k / 4) * 2048 + (k % 4) * 32) >> 4); }
+// K-major 16 x 128 bf16 operand (two atoms 1 KB apart): step k covers 16 elements of K
+__device__ __forceinline__ uint64_t vecdesc(const TileDesc &t, int k) { return t.kmaj + (uint64_t)(((k / 4) * 1024 + (k % 4) * 32) >> 4); }
 
 enum QBars { QB_OM, QB_Q, QB_K, QB_V, QB_G, QB_S, QB_X2, QM1, QM2, QM3, QM4, QM5, QM6, QE0, QE1, QE2A, QE2, QE3, QE4, QET, QNBARS };
 
@@ -83,8 +91,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
 {
     using L = BwdSmem<D, DV>;
     extern __shared__ __align__(1024) unsigned char smem[];
-    unsigned char *sOm = smem + L::kOm, *sQA = smem + L::kQA, *sKB = smem + L::kKB, *sV = smem + L::kV;
-    unsigned char *sG = smem + L::kG, *sSt = smem + L::kSt, *sStg = smem + L::kStg;
+    unsigned char *sOm = smem + L::kOm, *sOml = smem + L::kAux, *sQA = smem + L::kQA, *sKB = smem + L::kKB, *sV = smem + L::kV;
+    unsigned char *sG = smem + L::kG, *sSt = smem + L::kSt, *sDelOp = smem + L::kDel0;
     float *sZ = reinterpret_cast<float *>(smem + L::kVec);      // z before this chunk
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::kBars);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + QNBARS);
@@ -115,7 +123,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
         if (tid == 0) atomicExch(status, (int)DARKATTN_ERR_CUDA);
     } else if (warp == kEpiWarps) {
         if ((tid & 31) == 0) {
-            const TileDesc tOm(sOm), tQA(sQA), tKB(sKB), tV(sV), tG(sG), tSt(sSt), tDel(sStg);
+            const TileDesc tOm(sOm), tOml(sOml), tQA(sQA), tKB(sKB), tV(sV), tG(sG), tSt(sSt), tDel(sDelOp);
             const uint32_t id_kk = make_idesc(128, 128, 0, 0);
             const uint32_t id_vec = make_idesc(128, 16, 1, 0);
             const uint32_t id_tm = make_idesc(128, 128, 0, 1);
@@ -157,8 +165,12 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                     tma_store_2d(map, src + 16384, slab * 128 + 64, row0 + t * 128);
                     tma_store_commit();
                 };
-                mbar_expect_tx(bars + QB_OM, 128 * D * 2);
-                for (int a = 0; a < D / 64; ++a) tma_load_2d(sOm + a * 16384, &p.mapOm, bars + QB_OM, a * 64, h * p.m + slab * 128);
+                tma_store_wait_read();      // the last dQ tile of the run before has left its buffer
+                mbar_expect_tx(bars + QB_OM, 2 * 128 * D * 2);
+                for (int a = 0; a < D / 64; ++a) {
+                    tma_load_2d(sOm + a * 16384, &p.mapOm, bars + QB_OM, a * 64, h * p.m + slab * 128);
+                    tma_load_2d(sOml + a * 16384, &p.mapOml, bars + QB_OM, a * 64, h * p.m + slab * 128);
+                }
                 load_tile((it & 1) ? sSt : sQA, &p.mapQ, bars + QB_Q, D, t0);
                 load_tile(sKB, &p.mapK, bars + QB_K, D, t0);
                 load_tile(sV, &p.mapV, bars + QB_V, DV, t0);
@@ -168,14 +180,14 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                 if (ok) ok = wait_or_abort(bars + QB_K, it & 1, status, abort_flag);
                 if (ok) {
                     tc_fence_after();
-                    _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R2, kdesc(tKB, k), kdesc(tOm, k), id_kk, k > 0);   // U_K of the run's first chunk
+                    issue_projection<D>(R2, tKB, tOm, tOml, id_kk);                                              // U_K of the run's first chunk
                     mma_commit(bars + QM2);
                     ok = wait_or_abort(bars + QB_Q, it & 1, status, abort_flag);
                 }
                 if (ok) {
                     tc_fence_after();
                     const TileDesc &tX0 = (it & 1) ? tSt : tQA;
-                    _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R3, kdesc(tX0, k), kdesc(tOm, k), id_kk, k > 0);   // U_Q of the run's first chunk
+                    issue_projection<D>(R3, tX0, tOm, tOml, id_kk);                                              // U_Q of the run's first chunk
                     mma_commit(bars + QM1);
                 }
                 for (int c = 0; c < nrun && ok; ++c, ++it) {
@@ -229,21 +241,29 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                         ok = wait_or_abort(bars + QB_K, ph ^ 1, status, abort_flag);
                         if (!ok) break;
                         tc_fence_after();
-                        _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R2, kdesc(tKB, k), kdesc(tOm, k), id_kk, k > 0);   // U_K of the next chunk
+                        issue_projection<D>(R2, tKB, tOm, tOml, id_kk);                                          // U_K of the next chunk
                         mma_commit(bars + QM2);
                         ok = wait_or_abort(bars + QB_Q, ph ^ 1, status, abort_flag);
                         if (!ok) break;
                         tc_fence_after();
-                        _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R3, kdesc(tS, k), kdesc(tOm, k), id_kk, k > 0);    // U_Q of the next chunk (its Q sits in S)
+                        issue_projection<D>(R3, tS, tOm, tOml, id_kk);                                           // U_Q of the next chunk (its Q sits in S)
                         mma_commit(bars + QM1);
                     }
                     QWAIT(QM6); if (!ok) break;
                     if (!last) {
-                        load_state(bX, t + 1);                                                                   // E is done with: the next chunk's state
                         if (kQinV) load_tile(sV, &p.mapV, bars + QB_V, DV, t + 1);
                         else load_tile(sG, &p.mapG, bars + QB_G, DV, t + 1);
                     }
-                    QWAIT(QE4); if (!ok) break;
+                    QWAIT(QE4); if (!ok) break;                                                                  // this slab's part of dQ is staged where E was
+                    for (int a = 0; a < D / 64; ++a) {
+                        if (p.nslab > 1) tma_reduce_add_2d(&p.mapDQ, bX + a * 16384, a * 64, row0 + t * 128);
+                        else tma_store_2d(&p.mapDQ, bX + a * 16384, a * 64, row0 + t * 128);
+                    }
+                    tma_store_commit();
+                    if (!last) {
+                        tma_store_wait_read();
+                        load_state(bX, t + 1);                                                                   // the next chunk's state (needed late in it)
+                    }
 #undef QWAIT
                 }
             }
@@ -290,11 +310,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                 tc_fence_after();
                 features_to_tile(R2 + col0, nk, sKB, r, col0);                             // Bf
                 if (warp == 0) {
-                    // 16 x 128 K-major operand of rho_c = -A^^T delta at the start of the staging tile: row 0 = -delta rounded
-                    // to bf16, row 1 = the rounding's remainder. Written by the warp whose first lane has just seen the
-                    // previous chunk's store leave the tile.
-                    if (tid == 0) tma_store_wait_read();
-                    __syncwarp();
+                    // 16 x 128 K-major operand of rho_c = -A^^T delta: row 0 = -delta rounded to bf16, row 1 = the rounding's
+                    // remainder (its last reader, the chunk before's MMAs, completed before that chunk's E was formed)
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         const int k = i * 32 + lane;
@@ -302,8 +319,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                         const __nv_bfloat16 hi = __float2bfloat16_rn(dk);
                         const __nv_bfloat16 lo = __float2bfloat16_rn(dk - __bfloat162float(hi));
                         const int atom = k >> 6, kk = k & 63, ch = kk >> 3;
-                        *reinterpret_cast<__nv_bfloat16 *>(sStg + atom * 2048 + (ch << 4) + (kk & 7) * 2) = hi;
-                        *reinterpret_cast<__nv_bfloat16 *>(sStg + atom * 2048 + 128 + ((ch ^ 1) << 4) + (kk & 7) * 2) = lo;
+                        *reinterpret_cast<__nv_bfloat16 *>(sDelOp + atom * 1024 + (ch << 4) + (kk & 7) * 2) = hi;
+                        *reinterpret_cast<__nv_bfloat16 *>(sDelOp + atom * 1024 + 128 + ((ch ^ 1) << 4) + (kk & 7) * 2) = lo;
                     }
                 }
                 fence_async_smem();
@@ -369,16 +386,22 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
 
                 EWAIT(QM5); if (!ok) break;
                 tc_fence_after();
-                if (col0 < D) tmem_row_to_tile(R1 + col0, sStg, r, col0, kLn2);  // this slab's part of dQ -> staging -> added into dQ
-                fence_async_smem();
-                epi_sync();
-                if (tid == 0) {
-                    for (int a = 0; a < D / 64; ++a) {
-                        if (p.nslab > 1) tma_reduce_add_2d(&p.mapDQ, sStg + a * 16384, a * 64, row0 + t * 128);
-                        else tma_store_2d(&p.mapDQ, sStg + a * 16384, a * 64, row0 + t * 128);
+                {   // this slab's part of dQ: out of tensor memory, then (once T += E^T Q has read E) staged over E; the control
+                    // thread adds the tile into dQ
+                    uint32_t v[32];
+                    if (col0 < D) {
+                        tmem_ld32(R1 + col0, v);
+                        tmem_wait_ld();
                     }
-                    tma_store_commit();
+                    EWAIT(QM6); if (!ok) break;
+                    if (col0 < D) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(kLn2 * __uint_as_float(v[j]));
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4 *>(tile_chunk(bX, r, col0 / 8 + q)) = pack8(v + 8 * q);
+                    }
                 }
+                fence_async_smem();
                 if (g0 && !last) sZ[r] = znext;       // every reader of z is past its E step (E Omega was issued behind all of them)
                 tc_fence_before();
                 mbar_arrive_warp(bars + QE4);
@@ -400,7 +423,6 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                 mbar_arrive_warp(bars + QET);
             }
         }
-        if (tid == 0) tma_store_wait_all();
     }
     if (*abort_flag) __nanosleep(200000);   // error path only: let copies and MMAs in flight drain
     tc_fence_before();
@@ -417,7 +439,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
     using L = BwdSmem<D, DV>;
     extern __shared__ __align__(1024) unsigned char smem[];
     unsigned char *sOm = smem + L::kOm, *sQA = smem + L::kQA, *sKB = smem + L::kKB, *sV = smem + L::kV;
-    unsigned char *sG = smem + L::kG, *sSt = smem + L::kSt, *sStg = smem + L::kStg;
+    unsigned char *sG = smem + L::kG, *sSt = smem + L::kSt, *sStg = smem + L::kAux;
     float *sRho = reinterpret_cast<float *>(smem + L::kVec), *sDel = sRho + 128;
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::kBars);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + KNBARS);
@@ -1028,6 +1050,7 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
         const bool ok = make_map(&P.mapQ, Q, BH * N, D.d, 128) && make_map(&P.mapK, K, BH * N, D.d, 128) &&
                         make_map(&P.mapV, V, BH * N, D.dv, 128) && make_map(&P.mapG, dO, BH * N, D.dv, 128) &&
                         make_map(&P.mapOm, stash.Om, (size_t)D.H * D.m, D.d, 128) &&
+                        make_map(&P.mapOml, stash.Oml, (size_t)D.H * D.m, D.d, 128) &&
                         make_map(&P.mapDQ, dQ, BH * N, D.d, 128) && make_map(&P.mapDK, dK, BH * N, D.d, 128) &&
                         make_map(&P.mapDV, dV, BH * N, D.dv, 128) &&
                         make_map(&P.mapAh, bf(Y.Ahat), BH * N, D.m, 128) && make_map(&P.mapBf, bf(Y.Bphi), BH * N, D.m, 128) &&

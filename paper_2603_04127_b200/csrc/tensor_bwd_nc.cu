@@ -27,7 +27,7 @@ namespace {
 constexpr float kLn2 = 0.6931471805599453f;
 
 struct NcParams {
-    CUtensorMap mapX, mapY, mapOm, mapSt, mapOut, mapDV;   // X: Q or K; Y: dO or V; St: S or R (bf16); Out: dQ or dK
+    CUtensorMap mapX, mapY, mapOm, mapOml, mapSt, mapOut, mapDV;   // X: Q or K; Y: dO or V; St: S or R (bf16); Out: dQ or dK
     const float2 *sv;     // [BH*N]  (normaliser, exponent it is scaled by) from the forward pass
     const float *delta;   // [BH*N]  dO_i . O_i
     const float *nK;      // [BH*N]  key norms, log2 units
@@ -43,21 +43,26 @@ struct NcParams {
 
 template <int D, int DV>
 struct NcSmem {
-    static constexpr int kDmax = D > DV ? D : DV;
     static constexpr int kOm = 0;                          // folded projections of the slab [128 l, D]
-    static constexpr int kX = kOm + 128 * D * 2;           // two buffers of the Q (K) tile     [128, D]
+    static constexpr int kOml = kOm + 128 * D * 2;         // what their rounding to bf16 left out [128 l, D]
+    static constexpr int kX = kOml + 128 * D * 2;          // two buffers of the Q (K) tile     [128, D]; a tile's buffer also
+                                                           // stages the tile's part of dQ (dK) once T += E^T X has read it
     static constexpr int kA = kX + 2 * 128 * D * 2;        // A^ (Bf), then E                   [128, 128]
-    static constexpr int kY = kA + 32768;                  // dO (V) tile                       [128, DV]
+    static constexpr int kY = kA + 32768;                  // dO (V) tile                       [128, DV]; key pass: then the staged dV tile
     static constexpr int kSt = kY + 128 * DV * 2;          // S (R) of the slab, bf16           [128 l, DV]
-    static constexpr int kStg = kSt + 128 * DV * 2;        // staging tile of the TMA stores
-    static constexpr int kVec = kStg + 128 * kDmax * 2;    // float[128]: z (rho) of the slab
-    static constexpr int kBars = kVec + 512;
-    static constexpr int kTotal = kBars + 256;
+    // 3 KB of small things; query pass: the 16 x 128 K-major operand holding -delta (two swizzle atoms 1 KB apart of
+    // which only rows 0 and 1, 256 bytes each, carry data; the MMA reads what lies behind them as rows 2..15, whose
+    // products land in output columns nobody reads), barriers and z (rho) in between
+    static constexpr int kSmall = kSt + 128 * DV * 2;
+    static constexpr int kDel0 = kSmall;
+    static constexpr int kBars = kSmall + 256;
+    static constexpr int kVec = kSmall + 512;              // float[128]: z (rho) of the slab
+    static constexpr int kTotal = kSmall + 3072;
 };
 
 constexpr uint32_t kColState = 0, kColT = 128, kColR1 = 256, kColR2 = 384;
 
-__device__ __forceinline__ uint64_t vecdesc(const TileDesc &t, int k) { return t.kmaj + (uint64_t)(((k / 4) * 2048 + (k % 4) * 32) >> 4); }
+__device__ __forceinline__ uint64_t vecdesc(const TileDesc &t, int k) { return t.kmaj + (uint64_t)(((k / 4) * 1024 + (k % 4) * 32) >> 4); }
 
 enum NBars { NB_OM, NB_X0, NB_X1, NB_Y, NM1, NMA, NM2, NM3, NE1, NE2, NE3, NNBARS };
 
@@ -70,8 +75,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_nc_kernel(const __grid_con
 {
     using L = NcSmem<D, DV>;
     extern __shared__ __align__(1024) unsigned char smem[];
-    unsigned char *sOm = smem + L::kOm, *sX = smem + L::kX, *sA = smem + L::kA, *sY = smem + L::kY;
-    unsigned char *sSt = smem + L::kSt, *sStg = smem + L::kStg;
+    unsigned char *sOm = smem + L::kOm, *sOml = smem + L::kOml, *sX = smem + L::kX, *sA = smem + L::kA, *sY = smem + L::kY;
+    unsigned char *sSt = smem + L::kSt, *sDelOp = smem + L::kDel0;
     float *sVec = reinterpret_cast<float *>(smem + L::kVec);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::kBars);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + NNBARS);
@@ -108,7 +113,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_nc_kernel(const __grid_con
                 mbar_expect_tx(bar, 128 * width * 2);
                 for (int a = 0; a < width / 64; ++a) tma_load_2d(dst + a * 16384, map, bar, a * 64, row0 + t * 128);
             };
-            const TileDesc tOm(sOm), tX0(sX), tX1(sX + 128 * D * 2), tA(sA), tY(sY), tSt(sSt), tDel(sStg);
+            const TileDesc tOm(sOm), tOml(sOml), tX0(sX), tX1(sX + 128 * D * 2), tA(sA), tY(sY), tSt(sSt), tDel(sDelOp);
             const uint32_t id_kk = make_idesc(128, 128, 0, 0);
             const uint32_t id_vec = make_idesc(128, 16, 1, 0);
             const uint32_t id_state = make_idesc(128, DV, 1, 1);
@@ -117,8 +122,11 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_nc_kernel(const __grid_con
             const uint32_t id_t = make_idesc(128, D, 1, 1);
             const uint32_t R1 = tmem + kColR1, R2 = tmem + kColR2;
 
-            mbar_expect_tx(bars + NB_OM, 128 * D * 2 + 128 * DV * 2);
-            for (int a = 0; a < D / 64; ++a) tma_load_2d(sOm + a * 16384, &p.mapOm, bars + NB_OM, a * 64, h * p.m + slab * 128);
+            mbar_expect_tx(bars + NB_OM, 2 * 128 * D * 2 + 128 * DV * 2);
+            for (int a = 0; a < D / 64; ++a) {
+                tma_load_2d(sOm + a * 16384, &p.mapOm, bars + NB_OM, a * 64, h * p.m + slab * 128);
+                tma_load_2d(sOml + a * 16384, &p.mapOml, bars + NB_OM, a * 64, h * p.m + slab * 128);
+            }
             for (int a = 0; a < DV / 64; ++a) tma_load_2d(sSt + a * 16384, &p.mapSt, bars + NB_OM, a * 64, bh * p.m + slab * 128);
             load_tile(sX, &p.mapX, bars + NB_X0, D, tbeg);
             load_tile(sY, &p.mapY, bars + NB_Y, DV, tbeg);
@@ -127,7 +135,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_nc_kernel(const __grid_con
             if (ok) ok = wait_or_abort(bars + NB_X0, 0, status, abort_flag);
             if (ok) {
                 tc_fence_after();
-                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R1, kdesc(tX0, k), kdesc(tOm, k), id_kk, k > 0);      // U of the first tile
+                issue_projection<D>(R1, tX0, tOm, tOml, id_kk);                                                  // U of the first tile
                 mma_commit(bars + NM1);
             }
             for (int it = 0; it < nt && ok; ++it) {
@@ -136,13 +144,23 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_nc_kernel(const __grid_con
                 const bool first = (it == 0), last = (it + 1 == nt);
                 const TileDesc &tX = (it & 1) ? tX1 : tX0;
 #define NWAIT(b, q) do { ok = wait_or_abort(bars + (b), (q), status, abort_flag); } while (0)
-                if (!first) { NWAIT(NM3, ph ^ 1); if (!ok) break; }                 // T += E^T X of the tile before: its X buffer is free
-                if (!last) load_tile(sX + ((it + 1) & 1) * 128 * D * 2, &p.mapX, bars + NB_X0 + ((it + 1) & 1), D, t + 1);
+                auto store_out = [&](const CUtensorMap *map, unsigned char *src, int width, int tt) {     // (adds into the gradient when the head has several slabs)
+                    for (int a = 0; a < width / 64; ++a) {
+                        if (p.nslab > 1) tma_reduce_add_2d(map, src + a * 16384, a * 64, row0 + tt * 128);
+                        else tma_store_2d(map, src + a * 16384, a * 64, row0 + tt * 128);
+                    }
+                    tma_store_commit();
+                };
                 NWAIT(NB_Y, ph); if (!ok) break;
-                if (!first) { NWAIT(NE3, ph ^ 1); if (!ok) break; }                 // R2 read out
+                if (!first) {                                                       // the tile before: R2 read out, its part of dQ | dK staged in its X buffer
+                    NWAIT(NE3, ph ^ 1); if (!ok) break;
+                    store_out(&p.mapOut, sX + ((it + 1) & 1) * 128 * D * 2, D, t - 1);
+                }
                 tc_fence_after();
                 _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R2, kdesc(tY, k), kdesc(tSt, k), id_kk, k > 0);      // dO S^T | V R^T
                 mma_commit(bars + NMA);
+                if (!first) tma_store_wait_read();                                  // the staged tile has left the X buffer
+                if (!last) load_tile(sX + ((it + 1) & 1) * 128 * D * 2, &p.mapX, bars + NB_X0 + ((it + 1) & 1), D, t + 1);
                 NWAIT(NE1, ph); if (!ok) break;                                     // features in smem, R1 read
                 tc_fence_after();
                 if (KEYS) {
@@ -152,8 +170,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_nc_kernel(const __grid_con
                     _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColState, mndesc(tA, k), mndesc(tY, k), id_state, (!first) || k > 0);   // R += A^^T dO
                 }
                 mma_commit(bars + NM2);
-                NWAIT(NE2, ph); if (!ok) break;                                     // E in smem; R1 and R2 read
-                if (!last) load_tile(sY, &p.mapY, bars + NB_Y, DV, t + 1);
+                NWAIT(NE2, ph); if (!ok) break;                                     // E in smem; R1 and R2 read; key pass: dV staged over the V tile
+                if (KEYS) store_out(&p.mapDV, sY, DV, t);
+                else if (!last) load_tile(sY, &p.mapY, bars + NB_Y, DV, t + 1);
                 tc_fence_after();
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R2, kdesc(tA, k), mndesc(tOm, k), id_dx, k > 0);            // E Omega
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColT, mndesc(tA, k), mndesc(tX, k), id_t, (!first) || k > 0);   // T += E^T X
@@ -162,11 +181,17 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_nc_kernel(const __grid_con
                     NWAIT(NB_X0 + ((it + 1) & 1), ((it + 1) >> 1) & 1); if (!ok) break;
                     tc_fence_after();
                     const TileDesc &tXn = ((it + 1) & 1) ? tX1 : tX0;
-                    _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(R1, kdesc(tXn, k), kdesc(tOm, k), id_kk, k > 0);
+                    issue_projection<D>(R1, tXn, tOm, tOml, id_kk);
                     mma_commit(bars + NM1);
+                }
+                if (KEYS && !last) { tma_store_wait_read(); load_tile(sY, &p.mapY, bars + NB_Y, DV, t + 1); }     // the staged dV has left the V tile's buffer
+                if (last) {        // the last tile's part of dQ | dK
+                    NWAIT(NE3, ph); if (!ok) break;
+                    store_out(&p.mapOut, sX + (it & 1) * 128 * D * 2, D, t);
                 }
 #undef NWAIT
             }
+            tma_store_wait_all();
         }
     } else {
         const int lane = tid & 31, q4 = warp & 3, g = warp >> 2, col0 = g * 32;
@@ -200,11 +225,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_nc_kernel(const __grid_con
             tc_fence_after();
             features_to_tile(R1 + col0, offset, sA, r, col0);                          // A^ | Bf
             if (warp == 0) {
-                if (tid == 0) tma_store_wait_read();      // the staging tile is free again
-                __syncwarp();
                 if (!KEYS) {
-                    // 16 x 128 K-major operand of rho_c at the start of the staging tile: row 0 = -delta rounded to
-                    // bf16, row 1 = the rounding's remainder
+                    // 16 x 128 K-major operand of rho_c: row 0 = -delta rounded to bf16, row 1 = the rounding's remainder
+                    // (its last reader, the MMAs of the tile before, completed before that tile's E was formed)
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         const int k = i * 32 + lane;
@@ -212,8 +235,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_nc_kernel(const __grid_con
                         const __nv_bfloat16 hi = __float2bfloat16_rn(dk);
                         const __nv_bfloat16 lo = __float2bfloat16_rn(dk - __bfloat162float(hi));
                         const int atom = k >> 6, kk = k & 63, ch = kk >> 3;
-                        *reinterpret_cast<__nv_bfloat16 *>(sStg + atom * 2048 + (ch << 4) + (kk & 7) * 2) = hi;
-                        *reinterpret_cast<__nv_bfloat16 *>(sStg + atom * 2048 + 128 + ((ch ^ 1) << 4) + (kk & 7) * 2) = lo;
+                        *reinterpret_cast<__nv_bfloat16 *>(sDelOp + atom * 1024 + (ch << 4) + (kk & 7) * 2) = hi;
+                        *reinterpret_cast<__nv_bfloat16 *>(sDelOp + atom * 1024 + 128 + ((ch ^ 1) << 4) + (kk & 7) * 2) = lo;
                     }
                 }
             }
@@ -225,7 +248,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_nc_kernel(const __grid_con
             EWAIT(NM2); if (!ok) break;
             tc_fence_after();
             if (KEYS) {
-                if (col0 < DV) tmem_row_to_tile(R1 + col0, sStg, r, col0);             // this slab's part of dV
+                if (col0 < DV) tmem_row_to_tile(R1 + col0, sY, r, col0);               // this slab's part of dV, staged over the V tile (V R^T is done)
             } else if (g0) {
                 uint32_t v[16];
                 tmem_ld16(R1, v);
@@ -257,37 +280,17 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_nc_kernel(const __grid_con
                 if (KEYS) p.espart[((size_t)slab * 4 + g) * rows + row] = es;
             }
             fence_async_smem();
-            if (KEYS) {
-                epi_sync();
-                if (tid == 0) {
-                    for (int a = 0; a < DV / 64; ++a) {
-                        if (p.nslab > 1) tma_reduce_add_2d(&p.mapDV, sStg + a * 16384, a * 64, row0 + t * 128);
-                        else tma_store_2d(&p.mapDV, sStg + a * 16384, a * 64, row0 + t * 128);
-                    }
-                    tma_store_commit();
-                    tma_store_wait_read();                // staging free again before anyone passes NE2
-                }
-            }
             tc_fence_before();
             mbar_arrive_warp(bars + NE2);
 
-            EWAIT(NM3); if (!ok) break;
+            EWAIT(NM3); if (!ok) break;     // E Omega in R2; T += E^T X has read this tile's X buffer: the control thread stores from there
             tc_fence_after();
-            if (col0 < D) tmem_row_to_tile(R2 + col0, sStg, r, col0, kLn2);  // this slab's part of dQ | dK (without the norm term)
+            if (col0 < D) tmem_row_to_tile(R2 + col0, sX + (it & 1) * 128 * D * 2, r, col0, kLn2);  // this slab's part of dQ | dK (without the norm term)
             fence_async_smem();
             tc_fence_before();
             mbar_arrive_warp(bars + NE3);
-            epi_sync();
-            if (tid == 0) {
-                for (int a = 0; a < D / 64; ++a) {
-                    if (p.nslab > 1) tma_reduce_add_2d(&p.mapOut, sStg + a * 16384, a * 64, row0 + t * 128);
-                    else tma_store_2d(&p.mapOut, sStg + a * 16384, a * 64, row0 + t * 128);
-                }
-                tma_store_commit();
-            }
 #undef EWAIT
         }
-        if (tid == 0) tma_store_wait_all();
         // every MMA of this CTA completed before the last NM3 did: the accumulators can be read
         if (ok) {
             tc_fence_after();
@@ -377,12 +380,14 @@ cudaError_t tensor_backward_nc_passes(const darkattn_plan_s *plan, const void *Q
     PQ.nsplit = pick_splits((long long)BH * Y.nslab, Y.T, 3.0, 6.0, 64);
     NcParams PK = PQ;
     const bool ok = make_map(&PQ.mapX, Q, BH * N, D.d, 128) && make_map(&PQ.mapY, dO, BH * N, D.dv, 128) &&
-                    make_map(&PQ.mapOm, stash.Om, (size_t)D.H * D.m, D.d, 128) && make_map(&PQ.mapSt, stash.Sb, BH * D.m, D.dv, 128) &&
+                    make_map(&PQ.mapOm, stash.Om, (size_t)D.H * D.m, D.d, 128) && make_map(&PQ.mapOml, stash.Oml, (size_t)D.H * D.m, D.d, 128) &&
+                    make_map(&PQ.mapSt, stash.Sb, BH * D.m, D.dv, 128) &&
                     make_map(&PQ.mapOut, dQ, BH * N, D.d, 128) && make_map(&PQ.mapDV, dV, BH * N, D.dv, 128) &&
                     make_map(&PK.mapX, K, BH * N, D.d, 128) && make_map(&PK.mapY, V, BH * N, D.dv, 128) &&
                     make_map(&PK.mapSt, Rb, BH * D.m, D.dv, 128) && make_map(&PK.mapOut, dK, BH * N, D.d, 128);
     if (!ok) return cudaErrorInvalidValue;
     PK.mapOm = PQ.mapOm;
+    PK.mapOml = PQ.mapOml;
     PK.mapDV = PQ.mapDV;
     const long long nstate = (long long)BH * D.m * D.dv;
     cudaError_t e = cudaMemsetAsync(ws + Y.Racc, 0, (Y.rhot - Y.Racc) + BH * D.m * 4, st);      // R and rho sums (adjacent)

@@ -262,14 +262,6 @@ constexpr uint32_t kColS = 0, kColZ = 128, kColFQ = 192, kColR1 = 256, kColR2 = 
 
 enum CBars { CB_OM, CB_Q, CB_K, CB_V, CB_ST, CM1, CM2, CM3, CMS, CM4, CE0, CE1, CE2, CE3, CE4, CNBARS };
 
-// X (Om + Oml)^T into a TMEM region: the projection against both halves of the folded matrix
-template <int D>
-__device__ __forceinline__ void issue_projection(uint32_t dst, const TileDesc &tX, const TileDesc &tOm, const TileDesc &tOml, uint32_t idesc)
-{
-    _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(dst, kdesc(tX, k), kdesc(tOm, k), idesc, k > 0);
-    _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(dst, kdesc(tX, k), kdesc(tOml, k), idesc, 1);
-}
-
 // Causal: one CTA per (b, h, slab) walks the chunks of the sequence.
 //   R1: U_Q -> (phi(Q) read) -> P = phi(Q) phi(K)^T -> packed tril(P) (A operand of P V) -> U_Q of the next chunk
 //   R2: U_K -> (phi(K) read) -> O = phi(Q) S_prev + P V -> (O read) -> U_K of the next chunk
