@@ -73,13 +73,13 @@ struct TensorLayout {
     size_t dMn;     // gradient of M through the key norm term, fp32 [H, r, d]
     size_t Sst;     // workspace copy of the stash's per-chunk S (causal): bf16 [BH, T, m, dv], S before chunk t (t = 0 not written)
     size_t Ahat;    // causal backward: A^ of every (token, feature), bf16 [BH, N, m] (query-side kernel -> key-side kernel)
-    size_t Bphi;    // causal backward: Bf likewise
+    size_t Bphi;    // workspace copy of the stash's key features Bf (causal), bf16 [BH, N, m]: forward scan -> both backward kernels
     size_t Racc;    // non-causal backward: sum of A^^T dO, fp32 [BH, m, dv]; rhot directly behind it
     size_t rhot;    // non-causal backward: -sum of A^^T delta, fp32 [BH, m]
     size_t Rb;      // bf16 copy of Racc
     size_t total_bytes;
     // the forward -> backward stash (`saved`): per-row normalisers, key norms, folded projections, key shifts
-    size_t sv_sv, sv_nK, sv_Om, sv_Oml, sv_cs, sv_zc, sv_Sb, sv_zt, sv_Sst, sv_bytes;
+    size_t sv_sv, sv_nK, sv_Om, sv_Oml, sv_cs, sv_zc, sv_Sb, sv_zt, sv_Sst, sv_Bphi, sv_bytes;
     size_t zc;      // workspace copy of the stash's per-chunk z (causal): sum_j phi(K)_jl over the chunks before t, fp32 [BH, T, m]
     int nslab, T, nsplit;
 };
@@ -95,6 +95,7 @@ struct Stash {
     __nv_bfloat16 *Sb;   // non-causal: S of the whole sequence, bf16 [BH, m, dv]
     float *zt;      // non-causal: z of the whole sequence, [BH, m]
     __nv_bfloat16 *Sst;  // causal: S before chunk t, bf16 [BH, T, m, dv] (t = 0 is not written: it is zero)
+    __nv_bfloat16 *Bphi; // causal: the key features Bf of every (token, feature), bf16 [BH, N, m], as the forward scan formed them
 };
 inline Stash stash_in_workspace(const TensorLayout &Y, char *ws)
 {
@@ -102,7 +103,8 @@ inline Stash stash_in_workspace(const TensorLayout &Y, char *ws)
                  reinterpret_cast<__nv_bfloat16 *>(ws + Y.Om), reinterpret_cast<__nv_bfloat16 *>(ws + Y.Oml),
                  reinterpret_cast<float *>(ws + Y.cs),
                  reinterpret_cast<float *>(ws + Y.zc), reinterpret_cast<__nv_bfloat16 *>(ws + Y.Sb),
-                 reinterpret_cast<float *>(ws + Y.zacc), reinterpret_cast<__nv_bfloat16 *>(ws + Y.Sst)};
+                 reinterpret_cast<float *>(ws + Y.zacc), reinterpret_cast<__nv_bfloat16 *>(ws + Y.Sst),
+                 reinterpret_cast<__nv_bfloat16 *>(ws + Y.Bphi)};
 }
 inline Stash stash_in_saved(const TensorLayout &Y, void *saved)
 {
@@ -111,7 +113,8 @@ inline Stash stash_in_saved(const TensorLayout &Y, void *saved)
                  reinterpret_cast<__nv_bfloat16 *>(b + Y.sv_Om), reinterpret_cast<__nv_bfloat16 *>(b + Y.sv_Oml),
                  reinterpret_cast<float *>(b + Y.sv_cs),
                  reinterpret_cast<float *>(b + Y.sv_zc), reinterpret_cast<__nv_bfloat16 *>(b + Y.sv_Sb),
-                 reinterpret_cast<float *>(b + Y.sv_zt), reinterpret_cast<__nv_bfloat16 *>(b + Y.sv_Sst)};
+                 reinterpret_cast<float *>(b + Y.sv_zt), reinterpret_cast<__nv_bfloat16 *>(b + Y.sv_Sst),
+                 reinterpret_cast<__nv_bfloat16 *>(b + Y.sv_Bphi)};
 }
 
 }  // namespace darkattn

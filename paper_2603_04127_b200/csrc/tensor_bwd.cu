@@ -36,7 +36,8 @@ constexpr float kLn2 = 0.6931471805599453f;
 
 struct BwdParams {
     CUtensorMap mapQ, mapK, mapV, mapG, mapOm, mapOml, mapDQ, mapDK, mapDV;   // the last three: the gradients, for the (adding) stores
-    CUtensorMap mapAh, mapBf;   // A^ and Bf as [BH*N, m] bf16: written by the query-side kernel, read by the key-side one
+    CUtensorMap mapAh, mapBf;   // A^ and Bf as [BH*N, m] bf16: A^ is written by the query-side kernel and read by the key-side one, Bf comes
+                                // from the forward pass (through the stash) and is read by both
     CUtensorMap mapSst;         // S before every chunk as [BH*T*m, dv] bf16, from the forward pass
     const float2 *sv;     // [BH*N]  (normaliser, exponent it is scaled by) from the forward pass
     const float *delta;   // [BH*N]  dO_i . O_i
@@ -80,12 +81,12 @@ constexpr uint32_t kColState = 0, kColT = 128, kColR1 = 256, kColR2 = 384;
 // K-major 16 x 128 bf16 operand (two atoms 1 KB apart): step k covers 16 elements of K
 __device__ __forceinline__ uint64_t vecdesc(const TileDesc &t, int k) { return t.kmaj + (uint64_t)(((k / 4) * 1024 + (k % 4) * 32) >> 4); }
 
-enum QBars { QB_OM, QB_Q, QB_K, QB_V, QB_G, QB_S, QB_X2, QM1, QM2, QM3, QM4, QM5, QM6, QE0, QE1, QE2A, QE2, QE3, QE4, QET, QNBARS };
+enum QBars { QB_OM, QB_Q, QB_B, QB_V, QB_G, QB_S, QB_X2, QM1, QM3, QM4, QM5, QM6, QE1, QE2A, QE2, QE3, QE4, QET, QNBARS };
 
 // ------------------------------------------------------------------ query side
-// The state S before every chunk comes from the forward pass (bf16, through the stash), so the chunks are
-// independent of one another here: the chunks of all (batch, head) pairs form one line that is cut evenly over groups
-// of nslab CTAs, and a CTA walks its piece run by run (a run = consecutive chunks of one (batch, head) pair).
+// The state S before every chunk and the key features Bf come from the forward pass (bf16, through the stash), so the
+// chunks are independent of one another here: the chunks of all (batch, head) pairs form one line that is cut evenly
+// over groups of nslab CTAs, and a CTA walks its piece run by run (a run = consecutive chunks of one (batch, head) pair).
 template <int D, int DV>
 __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_constant__ BwdParams p)
 {
@@ -101,14 +102,14 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
     const int tid = threadIdx.x, warp = tid >> 5;
     const int T = p.T;
     // CTAs work in groups of nslab (one per slab of the head) on the same piece of the line of (batch, head, chunk)
-    // items, so that the Q, K, V, dO tiles a group reads are fetched from HBM once
+    // items, so that the Q, V, dO tiles a group reads are fetched from HBM once
     const int slab = blockIdx.x % p.nslab, group = blockIdx.x / p.nslab, ngroups = gridDim.x / p.nslab;
     const long long total = (long long)p.BH * T;
     const long long lbeg = total * group / ngroups, lend = total * (group + 1) / ngroups;
 
     if (tid == 0) {
-        for (int i = 0; i < QE0; ++i) mbar_init(bars + i, 1);
-        for (int i = QE0; i < QNBARS; ++i) mbar_init(bars + i, kEpiWarps);
+        for (int i = 0; i < QE1; ++i) mbar_init(bars + i, 1);
+        for (int i = QE1; i < QNBARS; ++i) mbar_init(bars + i, kEpiWarps);
         *abort_flag = (smem_u32(smem) & 1023u) ? 1 : 0;
         fence_mbar_init();
     }
@@ -134,14 +135,14 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
             // it fits), so that dO of the next chunk can follow early into its own buffer; otherwise into dO's buffer.
             constexpr bool kQinV = (D <= DV);
 
-            // Schedule of one chunk (R1, R2, R3: scratch regions of TMEM). U_K and U_Q of the next chunk are issued in
-            // the tail of the current one, and dO V^T runs while the epilogue is still busy with A^.
-            //   R2: U_K -> (Bf read) -> dO V^T -> packed dP in [0,64) (A operand of dP Bf), rho_c in [64,80) -> U_K of the next chunk
+            // Schedule of one chunk (R1, R2, R3: scratch regions of TMEM). U_Q of the next chunk is issued in the tail of
+            // the current one, dO V^T runs while the epilogue warps are busy with A^, dO S^T while they mask dP.
             //   R3: U_Q -> (A^ read) -> U_Q of the next chunk
-            //   R1: dP Bf + dO S^T -> (E read) -> E Omega -> (dQ read)
-            // Two tile buffers swap roles from chunk to chunk: X holds Q, then A^, then E; S holds the state before the
-            // chunk. S is free first (after dO S^T) and takes the next chunk's Q, so that its projection can be issued
-            // in the tail; X is free last (after T += E^T Q) and takes the next chunk's state, which is needed late.
+            //   R2: dO V^T -> packed dP in [0,64) (A operand of dP Bf), rho_c in [64,80)
+            //   R1: dO S^T + dP Bf -> (E read) -> E Omega -> (dQ read)
+            // Two tile buffers swap roles from chunk to chunk: X holds Q, then A^, then E, then the staged dQ tile; S holds
+            // the state before the chunk. S is free first (after dO S^T) and takes the next chunk's Q, so that its
+            // projection can be issued in the tail; X is free last and takes the next chunk's state, which is needed late.
             const uint32_t R3 = tmem + kColState;
             bool ok = true;
             int it = 0, run = 0;        // chunks and runs done so far: the parities of the barriers
@@ -156,14 +157,14 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                     mbar_expect_tx(bar, 128 * width * 2);
                     for (int a = 0; a < width / 64; ++a) tma_load_2d(dst + a * 16384, map, bar, a * 64, row0 + t * 128);
                 };
+                auto load_key_features = [&](int t) {                  // Bf of chunk t, as the forward pass formed it
+                    mbar_expect_tx(bars + QB_B, 32768);
+                    tma_load_2d(sKB, &p.mapBf, bars + QB_B, slab * 128, row0 + t * 128);
+                    tma_load_2d(sKB + 16384, &p.mapBf, bars + QB_B, slab * 128 + 64, row0 + t * 128);
+                };
                 auto load_state = [&](unsigned char *dst, int t) {     // S before chunk t (for t = 0 the tile is loaded but not used)
                     mbar_expect_tx(bars + QB_S, 128 * DV * 2);
                     for (int a = 0; a < DV / 64; ++a) tma_load_2d(dst + a * 16384, &p.mapSst, bars + QB_S, a * 64, (bh * T + t) * p.m + slab * 128);
-                };
-                auto store_features = [&](unsigned char *src, const CUtensorMap *map, int t) {
-                    tma_store_2d(map, src, slab * 128, row0 + t * 128);
-                    tma_store_2d(map, src + 16384, slab * 128 + 64, row0 + t * 128);
-                    tma_store_commit();
                 };
                 tma_store_wait_read();      // the last dQ tile of the run before has left its buffer
                 mbar_expect_tx(bars + QB_OM, 2 * 128 * D * 2);
@@ -172,18 +173,13 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                     tma_load_2d(sOml + a * 16384, &p.mapOml, bars + QB_OM, a * 64, h * p.m + slab * 128);
                 }
                 load_tile((it & 1) ? sSt : sQA, &p.mapQ, bars + QB_Q, D, t0);
-                load_tile(sKB, &p.mapK, bars + QB_K, D, t0);
                 load_tile(sV, &p.mapV, bars + QB_V, DV, t0);
                 load_tile(sG, &p.mapG, bars + QB_G, DV, t0);
+                load_key_features(t0);
                 load_state((it & 1) ? sQA : sSt, t0);
                 ok = wait_or_abort(bars + QB_OM, run & 1, status, abort_flag);
-                if (ok) ok = wait_or_abort(bars + QB_K, it & 1, status, abort_flag);
-                if (ok) {
-                    tc_fence_after();
-                    issue_projection<D>(R2, tKB, tOm, tOml, id_kk);                                              // U_K of the run's first chunk
-                    mma_commit(bars + QM2);
-                    ok = wait_or_abort(bars + QB_Q, it & 1, status, abort_flag);
-                }
+                if (ok) ok = wait_or_abort(bars + QB_Q, it & 1, status, abort_flag);
+                if (ok && run > 0) ok = wait_or_abort(bars + QET, (run - 1) & 1, status, abort_flag);       // T of the previous run has been read out
                 if (ok) {
                     tc_fence_after();
                     const TileDesc &tX0 = (it & 1) ? tSt : tQA;
@@ -197,52 +193,48 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                     unsigned char *bX = ph ? sSt : sQA, *bS = ph ? sQA : sSt;
                     const TileDesc &tX = ph ? tSt : tQA, &tS = ph ? tQA : tSt;
 #define QWAIT(b) do { ok = wait_or_abort(bars + (b), ph, status, abort_flag); } while (0)
-                    QWAIT(QE0); if (!ok) break;                                                                  // Bf in smem, R2 read
-                    store_features(sKB, &p.mapBf, t);                                                            // kept for the key-side kernel
                     QWAIT(QB_V); if (!ok) break;
                     QWAIT(QB_G); if (!ok) break;
                     tc_fence_after();
                     _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R2, kdesc(tG, k), kdesc(tV, k), id_kk, k > 0);     // dO V^T
                     mma_commit(bars + QM3);
-                    QWAIT(QE1); if (!ok) break;                                                                  // A^ in X, R3 read
-                    store_features(bX, &p.mapAh, t);
+                    if (!first) {
+                        QWAIT(QB_S); if (!ok) break;
+                        tc_fence_after();
+                        _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R1, kdesc(tG, k), kdesc(tS, k), id_kk, k > 0); // dO S_prev^T
+                    }
+                    QWAIT(QE1); if (!ok) break;                                                                  // A^ in X, R3 read, -delta operand written
+                    tma_store_2d(&p.mapAh, bX, slab * 128, row0 + t * 128);                                      // A^ kept for the key-side kernel
+                    tma_store_2d(&p.mapAh, bX + 16384, slab * 128 + 64, row0 + t * 128);
+                    tma_store_commit();
                     QWAIT(QE2A); if (!ok) break;                                                                 // dO V^T read out of R2
                     if (kQinV) load_tile(sV, &p.mapQ, bars + QB_X2, D, t);                                      // V is done with: Q again, for T
                     tc_fence_after();
                     _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R2 + 64, mndesc(tX, k), vecdesc(tDel, k), id_vec, k > 0);  // rho_c = -A^^T delta (columns 0, 1)
                     QWAIT(QE2); if (!ok) break;                                                                  // dP packed in R2
-                    QWAIT(QB_S); if (!ok) break;
+                    if (first) { QWAIT(QB_S); if (!ok) break; }                                                  // (keeps the barrier's phases in step)
+                    QWAIT(QB_B); if (!ok) break;
                     tc_fence_after();
-                    _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R1, R2 + k * 8, mndesc(tKB, k), id_tm, k > 0);           // dP Bf
-                    if (!first)
-                        _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R1, kdesc(tG, k), kdesc(tS, k), id_kk, 1);     // + dO S_prev^T
-                    tma_store_wait_read();      // both feature tiles have left shared memory: E may overwrite A^, the next K tile Bf
+                    _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R1, R2 + k * 8, mndesc(tKB, k), id_tm, (!first) || k > 0);   // + dP Bf
+                    tma_store_wait_read();      // the A^ tile has left shared memory: E may overwrite it
                     mma_commit(bars + QM4);
                     QWAIT(QM4); if (!ok) break;                                                                  // Bf, V, dO and S of this chunk are done with
                     if (!kQinV) load_tile(sG, &p.mapQ, bars + QB_X2, D, t);                                     // Q again, for T
                     if (!last) {
                         if (kQinV) load_tile(sG, &p.mapG, bars + QB_G, DV, t + 1);
                         else load_tile(sV, &p.mapV, bars + QB_V, DV, t + 1);
-                        load_tile(sKB, &p.mapK, bars + QB_K, D, t + 1);
+                        load_key_features(t + 1);
                         load_tile(bS, &p.mapQ, bars + QB_Q, D, t + 1);                                          // the state tile is done with: the next chunk's Q
                     }
                     QWAIT(QE3); if (!ok) break;
-                    QWAIT(QB_X2); if (!ok) break;
-                    if (c == 0 && run > 0) {                                                                     // T of the previous run has been read out
-                        ok = wait_or_abort(bars + QET, (run - 1) & 1, status, abort_flag);
-                        if (!ok) break;
-                    }
                     tc_fence_after();
                     _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R1, kdesc(tX, k), mndesc(tOm, k), id_dx, k > 0);         // E Omega
                     mma_commit(bars + QM5);
+                    QWAIT(QB_X2); if (!ok) break;
+                    tc_fence_after();
                     _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColT, mndesc(tX, k), mndesc(kQinV ? tV : tG, k), id_t, (c > 0) || k > 0);   // T += E^T Q
                     mma_commit(bars + QM6);
                     if (!last) {
-                        ok = wait_or_abort(bars + QB_K, ph ^ 1, status, abort_flag);
-                        if (!ok) break;
-                        tc_fence_after();
-                        issue_projection<D>(R2, tKB, tOm, tOml, id_kk);                                          // U_K of the next chunk
-                        mma_commit(bars + QM2);
                         ok = wait_or_abort(bars + QB_Q, ph ^ 1, status, abort_flag);
                         if (!ok) break;
                         tc_fence_after();
@@ -262,7 +254,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                     tma_store_commit();
                     if (!last) {
                         tma_store_wait_read();
-                        load_state(bX, t + 1);                                                                   // the next chunk's state (needed late in it)
+                        load_state(bX, t + 1);                                                                   // the next chunk's state
                     }
 #undef QWAIT
                 }
@@ -296,7 +288,6 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
 #define EWAIT(b) do { ok = __all_sync(0xffffffffu, wait_or_abort(bars + (b), ph, status, abort_flag)); } while (0)
                 const float2 svv = p.sv[row];
                 const float del = p.delta[row];
-                const float nk = p.nK[row] + cshift;
                 const float aq = svv.y - cshift + log2f(svv.x);
                 // z before the next chunk, from the forward pass (loaded early, used at the end of the chunk)
                 const float znext = (g0 && !last) ? __ldg(p.zc + ((size_t)bh * T + t + 1) * p.m + slab * 128 + r) : 0.f;
@@ -306,9 +297,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                     for (int i = 0; i < 4; ++i) dtile[i] = -__ldg(p.delta + (size_t)row0 + (size_t)t * 128 + i * 32 + lane);
                 }
                 unsigned char *bX = ph ? sSt : sQA;          // this chunk's Q / A^ / E tile
-                EWAIT(QM2); if (!ok) break;
+                EWAIT(QM1); if (!ok) break;
                 tc_fence_after();
-                features_to_tile(R2 + col0, nk, sKB, r, col0);                             // Bf
+                features_to_tile(lane_addr + kColState + col0, aq, bX, r, col0);           // A^
                 if (warp == 0) {
                     // 16 x 128 K-major operand of rho_c = -A^^T delta: row 0 = -delta rounded to bf16, row 1 = the rounding's
                     // remainder (its last reader, the chunk before's MMAs, completed before that chunk's E was formed)
@@ -323,12 +314,6 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                         *reinterpret_cast<__nv_bfloat16 *>(sDelOp + atom * 1024 + 128 + ((ch ^ 1) << 4) + (kk & 7) * 2) = lo;
                     }
                 }
-                fence_async_smem();
-                tc_fence_before();
-                mbar_arrive_warp(bars + QE0);
-                EWAIT(QM1); if (!ok) break;
-                tc_fence_after();
-                features_to_tile(lane_addr + kColState + col0, aq, bX, r, col0);           // A^
                 fence_async_smem();
                 tc_fence_before();
                 mbar_arrive_warp(bars + QE1);
@@ -1053,7 +1038,7 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
                         make_map(&P.mapOml, stash.Oml, (size_t)D.H * D.m, D.d, 128) &&
                         make_map(&P.mapDQ, dQ, BH * N, D.d, 128) && make_map(&P.mapDK, dK, BH * N, D.d, 128) &&
                         make_map(&P.mapDV, dV, BH * N, D.dv, 128) &&
-                        make_map(&P.mapAh, bf(Y.Ahat), BH * N, D.m, 128) && make_map(&P.mapBf, bf(Y.Bphi), BH * N, D.m, 128) &&
+                        make_map(&P.mapAh, bf(Y.Ahat), BH * N, D.m, 128) && make_map(&P.mapBf, stash.Bphi, BH * N, D.m, 128) &&
                         make_map(&P.mapSst, stash.Sst, BH * Y.T * D.m, D.dv, 128);
         if (!ok) { set_cuda_error(cudaErrorInvalidValue, "tensor_backward: tensor map encode"); return DARKATTN_ERR_CUDA; }
         P.sv = stash.sv; P.delta = fl(Y.delta); P.nK = stash.nK; P.cs = stash.cs; P.zc = stash.zc; P.rhoc = fl(Y.rhoc);

@@ -178,6 +178,7 @@ __global__ void __launch_bounds__(160, 1) tc_key_norms_kernel(const __grid_const
 struct MainParams {
     CUtensorMap mapQ, mapK, mapV, mapOm, mapOml, mapSb, mapPN;
     CUtensorMap mapSst;  // causal, when stash_S: S before every chunk as [BH*T*m, dv] bf16, for the backward pass
+    CUtensorMap mapBf;   // causal, when stash_S: the key features as [BH*N, m] bf16, for the backward pass
     int stash_S;
     const float *nK;     // [BH, N]      key norms in log2 units
     const float *cs;     // [BH, nslab]  key-side shift per slab (log2 units)
@@ -392,6 +393,11 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
                 const bool first = (t == tbeg) && fresh, last = (t + 1 == tend);
                 CWAIT(CE1, ph); if (!ok) break;                                 // phi(K) and the ones in smem, R2 read, K tile consumed
                 if (!last) load_tile(sK, &p.mapK, bars + CB_K, D, t + 1);
+                if (p.stash_S) {        // the backward kernels read the key features back instead of forming them again
+                    tma_store_2d(&p.mapBf, sFK, slab * 128, row0 + t * 128);
+                    tma_store_2d(&p.mapBf, sFK + 16384, slab * 128 + 64, row0 + t * 128);
+                    tma_store_commit();
+                }
                 tc_fence_after();
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R1, FQ + k * 8, kdesc(tFK, k), id_kk, k > 0);                // P = phi(Q) phi(K)^T
                 mma_commit(bars + CM3);
@@ -408,7 +414,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
                 CWAIT(CE2, ph); if (!ok) break;                                 // tril(P) packed in R1
                 tc_fence_after();
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R2, R1 + k * 8, mndesc(tV, k), id_o, (!first) || k > 0);     // O += P V
-                if (p.stash_S) tma_store_wait_read();       // the stash copy of the state before this chunk has left its tile: the output may be staged there
+                if (p.stash_S) tma_store_wait_read();       // the stash copies of the state before this chunk and of phi(K) have left their tiles: the output may be
+                                                            // staged in the first, the next phi(K) written to the second
                 mma_commit(bars + CM4);
                 if (!last) {        // U_Q of the next chunk, while the epilogue warps read the output tile out
                     CWAIT(CB_Q, ph ^ 1); if (!ok) break;
@@ -1090,6 +1097,7 @@ void tensor_make_layout(darkattn_plan_s *plan)
         Y.sv_Sb = take(so, D.causal ? 0 : BH * m * dv * 2);
         Y.sv_zt = take(so, D.causal ? 0 : BH * m * 4);
         Y.sv_Sst = take(so, D.causal ? BH * (size_t)Y.T * m * dv * 2 : 0);
+        Y.sv_Bphi = take(so, D.causal ? BH * N * m * 2 : 0);
         Y.sv_bytes = so;
         plan->saved_bytes = so;
     }
@@ -1189,7 +1197,7 @@ darkattn_status_t tensor_forward(const darkattn_plan_s *plan, const void *Q, con
     P.status = reinterpret_cast<int *>(ws + Y.status);
     P.N = D.N; P.H = D.H; P.BH = D.BH; P.m = D.m; P.nslab = Y.nslab; P.T = Y.T; P.nsplit = Y.nsplit;
     P.stash_S = (D.causal && stash_states) ? 1 : 0;
-    if (P.stash_S && !make_map(&P.mapSst, stash.Sst, BH * Y.T * D.m, D.dv, 128)) {
+    if (P.stash_S && !(make_map(&P.mapSst, stash.Sst, BH * Y.T * D.m, D.dv, 128) && make_map(&P.mapBf, stash.Bphi, BH * N, D.m, 128))) {
         set_cuda_error(cudaErrorInvalidValue, "tensor_forward: tensor map encode");
         return DARKATTN_ERR_CUDA;
     }
