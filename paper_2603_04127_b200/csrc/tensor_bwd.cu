@@ -415,7 +415,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
     if (warp == kEpiWarps) tmem_dealloc(tmem, 512);
 }
 
-enum KBars { KB_OM, KB_A, KB_B, KB_V, KB_G, KB_X2, KM3, KM4, KM5, KM6, KM7, KM8, KM9, KE2, KE3, KE4, KE5, KNBARS };
+enum KBars { KB_OM, KB_A, KB_B, KB_V, KB_G, KB_X2, KM3, KM4, KM5, KM6, KM7, KM8, KE2, KE3, KE4, KE5, KNBARS };
 
 // ------------------------------------------------------------------ key side (reverse direction)
 template <int D, int DV>
@@ -461,7 +461,11 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
                 tma_load_2d(dst, map, bar, slab * 128, row0 + t * 128);
                 tma_load_2d(dst + 16384, map, bar, slab * 128 + 64, row0 + t * 128);
             };
-            const TileDesc tOm(sOm), tQA(sQA), tKB(sKB), tV(sV), tG(sG), tSt(sSt);
+            auto prefetch_features = [&](const CUtensorMap *map, int t) {
+                tma_prefetch_l2_2d(map, slab * 128, row0 + t * 128);
+                tma_prefetch_l2_2d(map, slab * 128 + 64, row0 + t * 128);
+            };
+            const TileDesc tOm(sOm), tQA(sQA), tKB(sKB), tV(sV), tG(sG), tSt(sSt), tStg(sStg);
             const uint32_t id_kk = make_idesc(128, 128, 0, 0);
             const uint32_t id_state = make_idesc(128, DV, 1, 1);
             const uint32_t id_dv_t = make_idesc(128, DV, 0, 1);
@@ -477,12 +481,19 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
             load_features(sQA, &p.mapAh, bars + KB_A, T - 1);
             load_features(sKB, &p.mapBf, bars + KB_B, T - 1);
 
-            // Schedule of one chunk. A^ and Bf come from the query-side kernel through the workspace; V dO^T of
-            // the next chunk is issued in the tail of the current one.
+            // Schedule of one chunk. A^ comes from the query-side kernel through the workspace, Bf from the forward pass
+            // through the stash; V dO^T of the next chunk is issued in the tail of the current one.
             //   R1: V dO^T -> packed dP^T [0,64) and P^^T [64,128) (A operands) -> V dO^T of the next chunk
             //   R2: Bf A^^T -> (read) -> dV -> (read) -> dBf -> (E formed) -> dK partial -> (read)
-            // Shared memory: the K tile that T += E^T K needs takes the place of A^ once dP^T A^ is done, so that
-            // V and dO of the next chunk can be fetched early; A^ and Bf of the next chunk follow after T.
+            // Shared memory: the spare tile stages dV, then holds the K tile that T += E^T K needs, then stages dK; so
+            // A^ of the next chunk can be fetched as soon as dP^T A^ is done, V and dO with it, Bf once E Omega is done.
+            auto store_out = [&](const CUtensorMap *map, int width, int t) {     // the staged tile into (or, with several slabs, added into) the gradient
+                for (int a = 0; a < width / 64; ++a) {
+                    if (p.nslab > 1) tma_reduce_add_2d(map, sStg + a * 16384, a * 64, row0 + t * 128);
+                    else tma_store_2d(map, sStg + a * 16384, a * 64, row0 + t * 128);
+                }
+                tma_store_commit();
+            };
             bool ok = wait_or_abort(bars + KB_OM, 0, status, abort_flag);
             if (ok) ok = wait_or_abort(bars + KB_V, 0, status, abort_flag);
             if (ok) ok = wait_or_abort(bars + KB_G, 0, status, abort_flag);
@@ -501,31 +512,38 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
                 tc_fence_after();
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R2, kdesc(tKB, k), kdesc(tQA, k), id_kk, k > 0);             // P^^T = Bf A^^T
                 mma_commit(bars + KM4);
+                if (!last) prefetch_features(&p.mapBf, t - 1);      // into L2 now: its load can only be issued late in the chunk
                 KWAIT(KE2); if (!ok) break;                                                                      // dP^T and P^^T packed in R1
                 tc_fence_after();
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R2, R1 + 64 + k * 8, mndesc(tG, k), id_dv_t, k > 0);         // P^^T dO
                 if (!first)
                     _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R2, kdesc(tKB, k), mndesc(tSt, k), id_dv_t, 1);          // + Bf R_next
+                tma_store_wait_read();      // the dK tile of the chunk before has left the spare tile: dV may be staged there
                 mma_commit(bars + KM6);
                 // the state update is not on the chunk's critical path: it runs while dV is read out
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColState, mndesc(tQA, k), mndesc(tG, k), id_state, (!first) || k > 0);   // R += A^^T dO
                 mma_commit(bars + KM5);
-                KWAIT(KE3); if (!ok) break;
+                KWAIT(KE3); if (!ok) break;                                                                      // dV read out of R2 and staged
+                store_out(&p.mapDV, DV, t);
                 tc_fence_after();
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R2, R1 + k * 8, mndesc(tQA, k), id_tm, k > 0);               // dP^T A^
                 if (!first)
                     _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R2, kdesc(tV, k), kdesc(tSt, k), id_kk, 1);        // + V R_next^T
                 mma_commit(bars + KM7);
                 KWAIT(KM7); if (!ok) break;                                                                      // A^, V and dO of this chunk are done with
-                load_tile(sQA, &p.mapK, bars + KB_X2, D, t);                                                    // the K tile, for T
-                if (!last) { load_tile(sV, &p.mapV, bars + KB_V, DV, t - 1); load_tile(sG, &p.mapG, bars + KB_G, DV, t - 1); }
-                KWAIT(KE4); if (!ok) break;
+                tma_store_wait_read();                                                                           // the staged dV has left the spare tile:
+                load_tile(sStg, &p.mapK, bars + KB_X2, D, t);                                                   // the K tile, for T
+                if (!last) {
+                    load_features(sQA, &p.mapAh, bars + KB_A, t - 1);
+                    load_tile(sV, &p.mapV, bars + KB_V, DV, t - 1);
+                    load_tile(sG, &p.mapG, bars + KB_G, DV, t - 1);
+                }
+                KWAIT(KE4); if (!ok) break;                                                                      // E in smem, R2 read
                 KWAIT(KB_X2); if (!ok) break;
                 tc_fence_after();
+                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColT, mndesc(tKB, k), mndesc(tStg, k), id_t, (!first) || k > 0);   // T += E^T K
                 _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R2, kdesc(tKB, k), mndesc(tOm, k), id_dx, k > 0);            // E Omega
                 mma_commit(bars + KM8);
-                _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColT, mndesc(tKB, k), mndesc(tQA, k), id_t, (!first) || k > 0);   // T += E^T K
-                mma_commit(bars + KM9);
                 if (!last) {
                     ok = wait_or_abort(bars + KB_V, ph ^ 1, status, abort_flag);
                     if (ok) ok = wait_or_abort(bars + KB_G, ph ^ 1, status, abort_flag);
@@ -534,11 +552,13 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
                     _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R1, kdesc(tV, k), kdesc(tG, k), id_kk, k > 0);     // V dO^T of the next chunk
                     mma_commit(bars + KM3);
                 }
-                KWAIT(KM9); if (!ok) break;
-                if (!last) { load_features(sQA, &p.mapAh, bars + KB_A, t - 1); load_features(sKB, &p.mapBf, bars + KB_B, t - 1); }
-                KWAIT(KE5); if (!ok) break;
+                KWAIT(KM8); if (!ok) break;                                                                      // E and the K tile are done with
+                if (!last) load_features(sKB, &p.mapBf, bars + KB_B, t - 1);
+                KWAIT(KE5); if (!ok) break;                                                                      // dK read out of R2 and staged; bf16 copy of R in place
+                store_out(&p.mapDK, D, t);
 #undef KWAIT
             }
+            tma_store_wait_all();
         }
     } else {
         const int lane = tid & 31, q4 = warp & 3, g = warp >> 2, col0 = g * 32;
@@ -559,8 +579,6 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
                 rho_c = p.rhoc[((size_t)bh * T + t) * p.m + slab * 128 + r];
                 sDel[r] = p.delta[row];
             }
-            if (tid == 0) tma_store_wait_read();      // the previous chunk's dK store has left the staging tile
-
             EWAIT(KM3); if (!ok) break;
             tc_fence_after();
             {   // dP^T = (V dO^T - delta_i) masked to queries i >= this key, packed over the fp32 tile
@@ -597,18 +615,10 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
 
             EWAIT(KM6); if (!ok) break;
             tc_fence_after();
-            if (col0 < DV) tmem_row_to_tile(R2 + col0, sStg, r, col0);      // this slab's part of dV -> staging -> added into dV
+            if (col0 < DV) tmem_row_to_tile(R2 + col0, sStg, r, col0);      // this slab's part of dV, staged: the control thread adds it into dV
             fence_async_smem();
             tc_fence_before();
             mbar_arrive_warp(bars + KE3);
-            epi_sync();
-            if (tid == 0) {
-                for (int a = 0; a < DV / 64; ++a) {
-                    if (p.nslab > 1) tma_reduce_add_2d(&p.mapDV, sStg + a * 16384, a * 64, row0 + t * 128);
-                    else tma_store_2d(&p.mapDV, sStg + a * 16384, a * 64, row0 + t * 128);
-                }
-                tma_store_commit();
-            }
 
             EWAIT(KM7); if (!ok) break;
             tc_fence_after();
@@ -633,33 +643,21 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
                 p.espart[((size_t)slab * 4 + g) * rows + row] = es;
             }
             fence_async_smem();
-            if (tid == 0) tma_store_wait_read();      // staging free again before anyone passes KE4
             tc_fence_before();
             mbar_arrive_warp(bars + KE4);
+            // while T += E^T K and E Omega run: R (updated behind the dV MMAs, its last reader V R^T done before E was formed) -> bf16 copy
+            if (!last && col0 < DV) tmem_row_to_tile(lane_addr + kColState + col0, sSt, r, col0);
 
-            EWAIT(KM8); if (!ok) break;
+            EWAIT(KM8); if (!ok) break;     // (T += E^T K, issued ahead of E Omega, has read the K tile in the spare tile)
             tc_fence_after();
-            if (col0 < D) tmem_row_to_tile(R2 + col0, sStg, r, col0, kLn2); // this slab's part of dK (without the norm term) -> added into dK
+            if (col0 < D) tmem_row_to_tile(R2 + col0, sStg, r, col0, kLn2); // this slab's part of dK (without the norm term), staged: the control thread adds it into dK
+            if (g0 && !last) sRho[r] += rho_c;      // rho_next for the chunk below (every reader of rho is past its E step)
             fence_async_smem();
-            epi_sync();
-            if (tid == 0) {
-                for (int a = 0; a < D / 64; ++a) {
-                    if (p.nslab > 1) tma_reduce_add_2d(&p.mapDK, sStg + a * 16384, a * 64, row0 + t * 128);
-                    else tma_store_2d(&p.mapDK, sStg + a * 16384, a * 64, row0 + t * 128);
-                }
-                tma_store_commit();
-            }
-            if (!last) {     // R (updated behind the dV MMAs, before KM7) -> bf16 copy; rho_next for the chunk below
-                if (col0 < DV) tmem_row_to_tile(lane_addr + kColState + col0, sSt, r, col0);
-                if (g0) sRho[r] += rho_c;
-                fence_async_smem();
-            }
             tc_fence_before();
             mbar_arrive_warp(bars + KE5);
 #undef EWAIT
         }
-        if (tid == 0) tma_store_wait_all();
-        if (ok) ok = wait_or_abort(bars + KM9, (T - 1) & 1, status, abort_flag);
+        if (ok) ok = wait_or_abort(bars + KM8, (T - 1) & 1, status, abort_flag);
         if (ok && col0 < D) {
             tc_fence_after();
             float *dst = p.Tacc + ((size_t)h * p.m + slab * 128 + r) * D + col0;
