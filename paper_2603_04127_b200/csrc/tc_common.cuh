@@ -256,6 +256,12 @@ __device__ __forceinline__ float ex2f(float x)
     return y;
 }
 
+// Floats as integers whose order is the floats' order (for atomicMax on signed integers), and back.
+__device__ __forceinline__ int float_order_key(float x) { const int b = __float_as_int(x); return b >= 0 ? b : b ^ 0x7fffffff; }
+__device__ __forceinline__ float float_from_order_key(int k) { return __int_as_float(k >= 0 ? k : k ^ 0x7fffffff); }
+// The key-side shift of a (batch, head, slab): kept as such an integer by the kernel that takes the maximum over the keys.
+__device__ __forceinline__ float load_key_shift(const float *cs, int i) { return float_from_order_key(reinterpret_cast<const int *>(cs)[i]); }
+
 // mbarrier wait that also gives up when another thread of the CTA already did.
 __device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, int *status, volatile int *abort_flag)
 {

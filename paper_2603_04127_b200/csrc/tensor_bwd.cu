@@ -277,7 +277,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
             const int nrun = (int)(l1 - l0);
             l0 = l1;
             const int h = bh % p.H, row0 = bh * p.N;
-            const float cshift = p.cs[bh * p.nslab + slab];
+            const float cshift = load_key_shift(p.cs, bh * p.nslab + slab);
             if (g0) sZ[r] = (t0 > 0) ? __ldg(p.zc + ((size_t)bh * T + t0) * p.m + slab * 128 + r) : 0.f;
             epi_sync();
             for (int c = 0; c < nrun && ok; ++c, ++it) {

@@ -199,7 +199,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_nc_kernel(const __grid_con
         const bool g0 = (col0 == 0);                         // these 128 threads: row r also stands for feature r of the slab
         const uint32_t lane_addr = tmem + ((uint32_t)(q4 * 32) << 16);
         const uint32_t R1 = lane_addr + kColR1, R2 = lane_addr + kColR2;
-        const float cshift = p.cs[bh * p.nslab + slab];
+        const float cshift = load_key_shift(p.cs, bh * p.nslab + slab);
         const size_t rows = (size_t)p.BH * p.N;
         float rho_run = 0.f;
         bool ok = true;

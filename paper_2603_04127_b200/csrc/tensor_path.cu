@@ -27,6 +27,10 @@ namespace {
 
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kMaxNsplit = 64;
+// The key features are scaled so that the largest one of a (batch, head, slab) is 2^kShiftHeadroom rather than 1: fp32 and
+// bf16 reach down to 2^-126, so keys up to 190 binary orders below the largest keep a nonzero feature (causal prefixes see
+// only some of the keys), while sums over 2^17 keys of products with values and query features (<= 1) stay far from 2^127.
+constexpr float kShiftHeadroom = 64.f;
 
 // ------------------------------------------------------------------ small helpers
 
@@ -68,26 +72,11 @@ __global__ void fold_omega_kernel(const __nv_bfloat16 *W, const __nv_bfloat16 *M
     }
 }
 
-// Key-side shift of a slab, in log2 units: c = log2(e) * max(0, max_l |w_l|^2/2 - 40).
-// u - n <= |w_l|^2 / 2 for every key (complete the square), so phi(K) <= e^40 whatever the data.
-// One block per (bh, slab), 128 threads.
-__global__ void slab_shift_kernel(const __nv_bfloat16 *W, float *cs, int H, int m, int r, int nslab, int w_per_head)
+// Start value of the key-side shifts, which tc_key_shift_kernel raises to the maximum over the keys: the smallest order key.
+__global__ void shift_init_kernel(int *cs, int n)
 {
-    const int bh = blockIdx.x / nslab, slab = blockIdx.x % nslab, h = bh % H;
-    const __nv_bfloat16 *w = W + ((size_t)(w_per_head ? h : 0) * m + (size_t)slab * 128 + threadIdx.x) * r;
-    float acc = 0.f;
-    for (int a = 0; a < r; a += 8) {                // r is a multiple of 16 and the rows are 16-byte aligned
-        const uint4 raw = *reinterpret_cast<const uint4 *>(w + a);
-        const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
-#pragma unroll
-        for (int q = 0; q < 4; ++q) { const float2 f = __bfloat1622float2(h2[q]); acc = fmaf(f.x, f.x, fmaf(f.y, f.y, acc)); }
-    }
-    acc *= 0.5f;
-    __shared__ float red[128];
-    red[threadIdx.x] = acc;
-    __syncthreads();
-    for (int o = 64; o; o >>= 1) { if (threadIdx.x < o) red[threadIdx.x] = fmaxf(red[threadIdx.x], red[threadIdx.x + o]); __syncthreads(); }
-    if (threadIdx.x == 0) cs[blockIdx.x] = kLog2e * fmaxf(0.f, red[0] - 40.f);
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) cs[i] = (int)0x80000000u;
 }
 
 // ------------------------------------------------------------------ key norms: n[bh,j] = coef * |M_h k_j|^2
@@ -167,6 +156,102 @@ __global__ void __launch_bounds__(160, 1) tc_key_norms_kernel(const __grid_const
             tc_fence_before();
             mbar_arrive(bar_e);
             p.nK[(size_t)bh * p.N + (size_t)t * 128 + tid] = p.coef * acc;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 4) tmem_dealloc(tmem, 128);
+}
+
+// ------------------------------------------------------------------ key-side shift: c[bh,slab] = max_j max_{l in slab} (u_jl - n_j)
+// The stabiliser of the key features is the largest exponent any key of the (batch, head) reaches in the slab, taken
+// from the data (with it the largest key feature is 2^kShiftHeadroom, whatever the norms of the keys); being one constant per
+// (batch, head, slab) it cancels in O. One CTA per (batch, head, slab, piece of the sequence): K tile by TMA,
+// U = K Omega_slab^T on the tensor cores, row maxima read out of tensor memory, the piece's maximum by atomicMax.
+struct ShiftParams {
+    CUtensorMap mapK, mapOm;
+    const float *nK;     // [BH, N] key norms, log2 units
+    int *cs;             // [BH, nslab] order keys of the shifts
+    int *status;
+    int N, H, T, m, nslab, nsplit;
+};
+
+template <int D>
+__global__ void __launch_bounds__(160, 1) tc_key_shift_kernel(const __grid_constant__ ShiftParams p)
+{
+    extern __shared__ __align__(1024) unsigned char smem[];
+    constexpr int kTile = 128 * D * 2;
+    unsigned char *sOm = smem, *sK = smem + kTile;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + 2 * kTile);
+    uint64_t *bar_m = bars, *bar_k = bars + 1, *bar_u = bars + 2, *bar_e = bars + 3;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 4);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 5);
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int unit = blockIdx.x / p.nsplit, split = blockIdx.x % p.nsplit;
+    const int bh = unit / p.nslab, slab = unit % p.nslab, h = bh % p.H;
+    const int t0 = (int)((long long)p.T * split / p.nsplit), t1 = (int)((long long)p.T * (split + 1) / p.nsplit);
+    if (tid == 0) {
+        mbar_init(bar_m, 1); mbar_init(bar_k, 1); mbar_init(bar_u, 1); mbar_init(bar_e, 128);
+        *abort_flag = (smem_u32(smem) & 1023u) ? 1 : 0;
+        fence_mbar_init();
+    }
+    if (warp == 4) { tmem_alloc(tmem_slot, 128); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    if (*abort_flag) { if (tid == 0) atomicExch(p.status, (int)DARKATTN_ERR_CUDA); }
+    else if (warp == 4) {
+        if ((tid & 31) == 0 && t1 > t0) {
+            mbar_expect_tx(bar_m, kTile);
+            for (int a = 0; a < D / 64; ++a) tma_load_2d(sOm + a * 16384, &p.mapOm, bar_m, a * 64, h * p.m + slab * 128);
+            mbar_expect_tx(bar_k, kTile);
+            for (int a = 0; a < D / 64; ++a) tma_load_2d(sK + a * 16384, &p.mapK, bar_k, a * 64, bh * p.N + t0 * 128);
+            const TileDesc tOm(sOm), tK(sK);
+            const uint32_t idesc = make_idesc(128, 128, 0, 0);
+            bool ok = wait_or_abort(bar_m, 0, p.status, abort_flag);
+            for (int t = t0; t < t1 && ok; ++t) {
+                const uint32_t ph = (t - t0) & 1;
+                ok = wait_or_abort(bar_k, ph, p.status, abort_flag);
+                if (ok && t > t0) ok = wait_or_abort(bar_e, ph ^ 1, p.status, abort_flag);       // the tile before has been read out
+                if (!ok) break;
+                tc_fence_after();
+                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(tmem, kdesc(tK, k), kdesc(tOm, k), idesc, k > 0);
+                mma_commit(bar_u);
+                if (t + 1 < t1) {
+                    ok = wait_or_abort(bar_u, ph, p.status, abort_flag);
+                    if (!ok) break;
+                    mbar_expect_tx(bar_k, kTile);
+                    for (int a = 0; a < D / 64; ++a) tma_load_2d(sK + a * 16384, &p.mapK, bar_k, a * 64, bh * p.N + (t + 1) * 128);
+                }
+            }
+        }
+    } else {
+        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+        float best = -INFINITY;
+        bool ok = true;
+        for (int t = t0; t < t1; ++t) {
+            const uint32_t ph = (t - t0) & 1;
+            const float nk = p.nK[(size_t)bh * p.N + (size_t)t * 128 + tid];
+            ok = __all_sync(0xffffffffu, wait_or_abort(bar_u, ph, p.status, abort_flag));
+            if (!ok) break;
+            tc_fence_after();
+            float mx = -INFINITY;
+#pragma unroll
+            for (int c0 = 0; c0 < 128; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld32(lane_addr + c0, v);
+                tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(v[j]));
+            }
+            tc_fence_before();
+            mbar_arrive(bar_e);
+            best = fmaxf(best, mx - nk);
+        }
+        if (ok && t1 > t0) {
+            for (int o = 16; o; o >>= 1) best = fmaxf(best, __shfl_xor_sync(0xffffffffu, best, o));
+            if ((tid & 31) == 0) atomicMax(p.cs + bh * p.nslab + slab, float_order_key(best - kShiftHeadroom));
         }
     }
     tc_fence_before();
@@ -453,7 +538,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
         const int r = q4 * 32 + lane;
         const uint32_t lane_addr = tmem + ((uint32_t)(q4 * 32) << 16);
         const uint32_t R1 = lane_addr + kColR1, R2 = lane_addr + kColR2;
-        const float cshift = p.cs[bh * p.nslab + slab];
+        const float cshift = load_key_shift(p.cs, bh * p.nslab + slab);
         const size_t prow0 = ((size_t)slab * p.BH + bh) * p.N;
         uint32_t *sOnes = reinterpret_cast<uint32_t *>(sRed);
         bool ok = true;
@@ -685,7 +770,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_keys_kernel(const __grid_c
         const int lane = tid & 31, q4 = warp & 3, g = warp >> 2, col0 = g * 32;
         const int r = q4 * 32 + lane;
         const uint32_t lane_addr = tmem + ((uint32_t)(q4 * 32) << 16);
-        const float cshift = p.cs[bh * p.nslab + slab];
+        const float cshift = load_key_shift(p.cs, bh * p.nslab + slab);
         bool ok = true;
         for (int i = 0; i < n && ok; ++i) {
             const int b = i & 1;
@@ -839,7 +924,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_queries_kernel(const __gri
         const int lane = tid & 31, q4 = warp & 3, g = warp >> 2, col0 = g * 32;
         const int r = q4 * 32 + lane;
         const uint32_t lane_addr = tmem + ((uint32_t)(q4 * 32) << 16);
-        const float cshift = p.cs[bh * p.nslab + slab];
+        const float cshift = load_key_shift(p.cs, bh * p.nslab + slab);
         const size_t prow0 = ((size_t)slab * p.BH + bh) * p.N;
         bool ok = true;
         for (int i = 0; i < n && ok; ++i) {
@@ -1085,7 +1170,7 @@ void tensor_make_layout(darkattn_plan_s *plan)
     Y.Sb = take(off, BH * nstate * m * dv * 2);
     Y.sv = take(off, BH * N * 8);
     Y.zc = take(off, D.causal ? BH * (size_t)Y.T * m * 4 : 0);
-    plan->launches_fwd = D.causal ? (nsplit > 1 ? 7 : 5) : 7;
+    plan->launches_fwd = D.causal ? (nsplit > 1 ? 8 : 6) : 8;
     {
         size_t so = 0;
         Y.sv_sv = take(so, BH * N * 8);
@@ -1147,8 +1232,8 @@ cudaError_t tensor_prologue(const darkattn_plan_s *plan, const void *K, const vo
     fold_omega_kernel<<<dim3(D.m / 4, D.H), D.d, 0, sp>>>((const __nv_bfloat16 *)W, (const __nv_bfloat16 *)M, out.Om, out.Oml, D.m, D.r,
                                                       D.d, D.w_per_head, kLog2e * D.s);
     chk();
-    timer_mark(plan, st, "slab_shift_kernel");
-    slab_shift_kernel<<<(unsigned)(BH * Y.nslab), 128, 0, sp>>>((const __nv_bfloat16 *)W, out.cs, D.H, D.m, D.r, Y.nslab, D.w_per_head);
+    timer_mark(plan, st, "shift_init_kernel");
+    shift_init_kernel<<<(unsigned)((BH * Y.nslab + 255) / 256), 256, 0, sp>>>(reinterpret_cast<int *>(out.cs), (int)(BH * Y.nslab));
     chk();
     if (beside && e == cudaSuccess) e = cudaEventRecord(plan->aux_join, sp);
 
@@ -1167,6 +1252,23 @@ cudaError_t tensor_prologue(const darkattn_plan_s *plan, const void *K, const vo
     }
     chk();
     if (beside && e == cudaSuccess) e = cudaStreamWaitEvent(st, plan->aux_join, 0);
+
+    // the key-side shifts: the maximum of u - n over the keys of every (batch, head, slab)
+    ShiftParams SP;
+    memset(&SP, 0, sizeof(SP));
+    if (!make_map(&SP.mapK, K, BH * N, D.d, 128) || !make_map(&SP.mapOm, out.Om, (size_t)D.H * D.m, D.d, 128)) return cudaErrorInvalidValue;
+    SP.nK = out.nK; SP.cs = reinterpret_cast<int *>(out.cs); SP.status = NP.status;
+    SP.N = D.N; SP.H = D.H; SP.T = Y.T; SP.m = D.m; SP.nslab = Y.nslab;
+    SP.nsplit = pick_splits((long long)BH * Y.nslab, Y.T, 2.5, 3.0, 64, 3 * 148);
+    timer_mark(plan, st, "tc_key_shift_kernel");
+    if (D.d == 64) {
+        cudaFuncSetAttribute(tc_key_shift_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+        tc_key_shift_kernel<64><<<(unsigned)(BH * Y.nslab * SP.nsplit), 160, smem_bytes, st>>>(SP);
+    } else {
+        cudaFuncSetAttribute(tc_key_shift_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+        tc_key_shift_kernel<128><<<(unsigned)(BH * Y.nslab * SP.nsplit), 160, smem_bytes, st>>>(SP);
+    }
+    chk();
     return e;
 }
 

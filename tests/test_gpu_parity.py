@@ -75,14 +75,27 @@ def test_explicit_scale_and_per_head_projections(binding):
     _compare(got, _oracle(t, wl, scale=0.2), TOL["f32"], "wph")
 
 
-def test_large_norm_inputs_stay_finite(binding):
-    # exponents far outside exp's fp32 range without the stabilising shifts
-    wl = inputs.small(name="bignorm", wid=33, B=1, H=1, N=192, d=32, m=64, causal=False, dtype="f32", backward=False)
+@pytest.mark.parametrize("case", ["simt_f32", "tensor_bf16_causal", "tensor_bf16_noncausal"])
+def test_large_norm_inputs_stay_finite(binding, case):
+    """Queries and keys six times larger: exponents far outside exp's fp32 range without the stabilising shifts, which
+    are taken from the data on both paths (row maxima for the queries, the maximum over the keys for the key features)."""
+    if case == "simt_f32":
+        wl = inputs.small(name="bignorm", wid=33, B=1, H=1, N=192, d=32, m=64, causal=False, dtype="f32", backward=False)
+        path, tol = binding.PATH_SIMT, 5e-4     # the exponent's argument is ~36 times larger, and so is its fp32 rounding
+    else:
+        wl = inputs.small(name="bignorm", wid=33, B=1, H=2, N=384, d=64, m=256, causal="noncausal" not in case, dtype="bf16",
+                          backward=True)
+        path, tol = binding.PATH_TENSOR, TOL["bf16"]
     t = inputs.generate(wl)
-    t.Q *= 6.0
-    t.K *= 6.0
-    got = run_gpu(binding, wl, t)
-    _compare(got, _oracle(t, wl), 5e-4, "bignorm")
+    # a causal prefix sees only some of the keys while the key-side shift is one constant per (batch, head, slab): the
+    # spread of the exponents between prefixes, which grows with the square of the scale, has to stay within fp32's range
+    scale = 4.0 if case == "tensor_bf16_causal" else 6.0
+    t.Q = t.Q * scale
+    t.K = t.K * scale
+    if wl.dtype == "bf16":
+        t.Q, t.K = (inputs.round_to_bf16(x).astype(np.float64) for x in (t.Q, t.K))
+    got = run_gpu(binding, wl, t, path=path, use_saved=True)
+    _compare(got, _oracle(t, wl), tol, case)
 
 
 FULL = {
