@@ -217,6 +217,18 @@ def generate(wl: Workload, pairs=None, as_batch: bool = False) -> Tensors:
     return Tensors(wl, Q, K, V, M, W, dO, use)
 
 
+def parameters(wl: Workload):
+    """The parameters M [H, r, d] and W [m, r] of a workload alone (the same values generate() returns), rounded to the
+    workload's storage type: what every rank of a data-parallel job shares while it draws its own batch."""
+    B, H, N, d, r, m, dv = wl.dims()
+    G = _rng(wl.wid, "G").standard_normal((H, r, d)) / np.sqrt(d)
+    M = np.eye(r, d)[None, :, :] + 0.1 * G
+    W = _rng(wl.wid, "W").standard_normal((m, r))
+    if wl.dtype == "bf16":
+        return round_to_bf16(M).astype(np.float64), round_to_bf16(W).astype(np.float64)
+    return M.astype(np.float32).astype(np.float64), W.astype(np.float32).astype(np.float64)
+
+
 def small(name="tiny", wid=9, B=1, H=2, N=16, d=8, m=16, causal=False, dtype="f32", backward=True,
           rho=0.9, r=0, dv=0, top_scale=1.0) -> Workload:
     """A free-form small workload for tests."""

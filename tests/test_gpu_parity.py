@@ -298,6 +298,29 @@ def test_headline_backward_sampled_heads(binding, name):
     assert_close(got["dM"][h], want["dM"][0], TOL["bf16"], f"{name} head {h}: dM")
 
 
+SWEEP = [(wid, dict(B=2, H=2, N=512, d=64, m=256)) for wid in range(1, 11)] + \
+        [(wid, dict(B=1, H=2, N=1024, d=128, m=256)) for wid in (3, 7, 11)]
+
+
+@pytest.mark.parametrize("causal", [True, False], ids=["causal", "noncausal"])
+@pytest.mark.parametrize("wid,kw", SWEEP, ids=[f"id{w}_d{k['d']}" for w, k in SWEEP])
+def test_bf16_error_over_many_seeds(binding, wid, kw, causal):
+    """The bf16 bar must hold with margin whatever the random draw: ten workload ids at the smoke shape (among them
+    id 7, the draw on which one element of dQ once missed the bar) and three at d = 128, forward and backward. Every
+    tensor's largest deviation stays below 1.5e-2 of the tensor's largest value and its Frobenius-relative error below
+    1e-2; the worst element-wise relative error over the elements above 1 % of the maximum is printed."""
+    wl = inputs.small(name="sweep", wid=wid, dtype="bf16", causal=causal, backward=True, **kw)
+    t = inputs.generate(wl)
+    got = run_gpu(binding, wl, t, path=binding.PATH_TENSOR, use_saved=True)
+    want = _oracle(t, wl)
+    for k, w in want.items():
+        fro, mx = assert_close(got[k], w, TOL["bf16"], f"sweep id {wid} {k}")
+        big = np.abs(w) > 0.01 * np.abs(w).max()
+        ew = (np.abs(got[k] - w)[big] / np.abs(w)[big]).max()
+        print(f"sweep id {wid} d={kw['d']} causal={int(causal)} {k}: fro {fro:.2e} max {mx:.2e} worst element-wise {ew:.2e}")
+        assert fro < 1e-2 and mx < 1.5e-2, (wid, k, fro, mx)
+
+
 def test_tensor_path_is_deterministic(binding):
     """The scan kernels hand tiles between warps through shared and tensor memory; a missing wait shows up as rare,
     run-dependent errors of the size of the values themselves. O has a fixed summation order: repeated runs at the
