@@ -22,8 +22,10 @@
  * given CUDA stream and never synchronise it (except darkattn_last_device_status). Argument errors are
  * reported on the host before anything is launched. There is no CPU fallback.
  *
- *   Q, K, dQ, dK   [B, H, N, d]      desc.dtype
- *   V, O, dO, dV   [B, H, N, dv]     desc.dtype
+ *   Q, dQ          [B, H, N, d]      desc.dtype
+ *   K, dK          [B, H_kv, N, d]   desc.dtype   (H_kv = H unless desc.H_kv says otherwise: grouped key/value heads)
+ *   V, dV          [B, H_kv, N, dv]  desc.dtype
+ *   O, dO          [B, H, N, dv]     desc.dtype
  *   M              [H, r, d]         desc.dtype   (row a of M_h produces coordinate a of M_h x)
  *   W              [m, r]            desc.dtype   (or [H, m, r] when desc.w_per_head != 0)
  *   dM             [H, r, d]         float32, OVERWRITTEN (summed over the batch inside the call)
@@ -71,6 +73,11 @@ typedef struct {
                              scaling is absorbed symmetrically, sqrt(scale) into Mq and into Mk)   */
     int32_t w_per_head;   /* 0: W [m,r] shared by all heads; 1: W [H,m,r]                          */
     int32_t path;         /* darkattn_path_t                                                       */
+    int32_t H_kv;         /* key/value heads; 0 means H. Must divide H: query heads h*G .. h*G+G-1 (G = H / H_kv)
+                             attend to key/value head h. The paper's feature map applies one M to queries and keys
+                             alike (Appendix B: q~ = Mq, k~ = Mk), and M is per query head: a shared key is mapped
+                             with the M of the query head that reads it, so its features differ from head to head of
+                             the group and only the storage of K and V is shared. dK and dV sum over the group.     */
 } darkattn_desc_t;
 
 typedef struct darkattn_plan_s *darkattn_plan_t;

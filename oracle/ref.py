@@ -75,8 +75,21 @@ def _dims(Q, V, M, W):
     return B, H, N, d, r, m, dv, w_per_head
 
 
+def _expand_kv(Q, K, V):
+    """Grouped key/value heads (K, V of shape [B, H_kv, N, *] with H_kv dividing H): query heads h*G .. h*G+G-1 read
+    key/value head h, i.e. the attention is the ungrouped one with every key/value head repeated G times. The feature
+    map of a query head (its own M) is applied to the keys it reads, as to its queries (Appendix B: q~ = Mq, k~ = Mk)."""
+    H, Hkv = Q.shape[1], K.shape[1]
+    assert V.shape[1] == Hkv and H % Hkv == 0, "H_kv must divide H"
+    G = H // Hkv
+    if G == 1:
+        return K, V, 1
+    return np.repeat(K, G, axis=1), np.repeat(V, G, axis=1), G
+
+
 def forward(Q, K, V, M, W, causal=False, scale=None, shift_q=None, shift_k=None):
-    """O [B,H,N,dv]; scale defaults to 1/sqrt(d)."""
+    """O [B,H,N,dv]; scale defaults to 1/sqrt(d). K, V may have fewer heads than Q (grouped key/value heads)."""
+    K, V, _ = _expand_kv(np.asarray(Q), np.asarray(K), np.asarray(V))
     Q, K, V, M, W = _c(Q), _c(K), _c(V), _c(M), _c(W)
     B, H, N, d, r, m, dv, wph = _dims(Q, V, M, W)
     scale = 1.0 / np.sqrt(d) if scale is None else float(scale)
@@ -90,7 +103,9 @@ def forward(Q, K, V, M, W, causal=False, scale=None, shift_q=None, shift_k=None)
 
 
 def backward(Q, K, V, M, W, dO, causal=False, scale=None, shift_q=None, shift_k=None):
-    """Returns dQ, dK, dV, dM [H,r,d], dW (same shape as W) for L = sum(dO * O)."""
+    """Returns dQ, dK, dV, dM [H,r,d], dW (same shape as W) for L = sum(dO * O). With grouped key/value heads dK and
+    dV have K's and V's shapes: a shared key (value) collects the gradients of all query heads that read it."""
+    K, V, G = _expand_kv(np.asarray(Q), np.asarray(K), np.asarray(V))
     Q, K, V, M, W, dO = _c(Q), _c(K), _c(V), _c(M), _c(W), _c(dO)
     B, H, N, d, r, m, dv, wph = _dims(Q, V, M, W)
     scale = 1.0 / np.sqrt(d) if scale is None else float(scale)
@@ -102,4 +117,7 @@ def backward(Q, K, V, M, W, dO, causal=False, scale=None, shift_q=None, shift_k=
                                        _p(dQ), _p(dK), _p(dV), _p(dM), _p(dW))
     if rc:
         raise RuntimeError(f"darkattn_ref_backward failed ({rc})")
+    if G > 1:
+        dK = dK.reshape(B, H // G, G, N, d).sum(axis=2)
+        dV = dV.reshape(B, H // G, G, N, dv).sum(axis=2)
     return dQ, dK, dV, dM, dW

@@ -33,7 +33,7 @@ class Desc(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("N", ctypes.c_int32), ("d", ctypes.c_int32),
                 ("r", ctypes.c_int32), ("m", ctypes.c_int32), ("dv", ctypes.c_int32), ("dtype", ctypes.c_int32),
                 ("causal", ctypes.c_int32), ("chunk", ctypes.c_int32), ("scale", ctypes.c_float),
-                ("w_per_head", ctypes.c_int32), ("path", ctypes.c_int32)]
+                ("w_per_head", ctypes.c_int32), ("path", ctypes.c_int32), ("H_kv", ctypes.c_int32)]
 
 
 if not os.path.exists(LIB_PATH):
@@ -137,8 +137,8 @@ class Plan:
 
 
 def darkattn_plan(B, H, N, d, m, *, r=0, dv=0, dtype=BF16, causal=False, chunk=0, scale=0.0, w_per_head=False,
-                  path=PATH_AUTO) -> Plan:
-    desc = Desc(B, H, N, d, r, m, dv, dtype, int(bool(causal)), chunk, float(scale), int(bool(w_per_head)), path)
+                  path=PATH_AUTO, H_kv=0) -> Plan:
+    desc = Desc(B, H, N, d, r, m, dv, dtype, int(bool(causal)), chunk, float(scale), int(bool(w_per_head)), path, H_kv)
     h = _vp()
     _check(lib.darkattn_plan(ctypes.byref(desc), ctypes.byref(h)), "darkattn_plan")
     return Plan(h.value, desc)

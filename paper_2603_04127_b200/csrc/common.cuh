@@ -14,6 +14,7 @@ namespace darkattn {
 struct Dims {
     int B, H, N, d, r, m, dv;
     int BH;          // B * H
+    int Hkv, G;      // key/value heads and query heads per key/value head (H = Hkv * G)
     int C;           // causal chunk length
     int nc;          // number of chunks = ceil(N / C)   (1 when not causal)
     int Npad;        // nc * C when causal, else N

@@ -37,8 +37,10 @@ darkattn_status_t darkattn_plan(const darkattn_desc_t *desc, darkattn_plan_t *ou
     if (!desc || !out) return DARKATTN_ERR_INVALID_ARG;
     *out = nullptr;
     darkattn_desc_t ds = *desc;
-    if (ds.B < 1 || ds.H < 1 || ds.N < 1 || ds.d < 1 || ds.m < 1 || ds.r < 0 || ds.dv < 0 || ds.chunk < 0)
+    if (ds.B < 1 || ds.H < 1 || ds.N < 1 || ds.d < 1 || ds.m < 1 || ds.r < 0 || ds.dv < 0 || ds.chunk < 0 || ds.H_kv < 0)
         return DARKATTN_ERR_INVALID_ARG;
+    if (ds.H_kv == 0) ds.H_kv = ds.H;
+    if (ds.H_kv > ds.H || ds.H % ds.H_kv) return DARKATTN_ERR_INVALID_ARG;
     if (ds.dtype != DARKATTN_F32 && ds.dtype != DARKATTN_BF16) return DARKATTN_ERR_INVALID_ARG;
     if (ds.path < DARKATTN_PATH_AUTO || ds.path > DARKATTN_PATH_TENSOR) return DARKATTN_ERR_INVALID_ARG;
     if (!(ds.scale >= 0.f) || !isfinite(ds.scale)) return DARKATTN_ERR_INVALID_ARG;
@@ -54,6 +56,7 @@ darkattn_status_t darkattn_plan(const darkattn_desc_t *desc, darkattn_plan_t *ou
     Dims &D = p->dims;
     D.B = ds.B; D.H = ds.H; D.N = ds.N; D.d = ds.d; D.r = ds.r; D.m = ds.m; D.dv = ds.dv;
     D.BH = ds.B * ds.H;
+    D.Hkv = ds.H_kv; D.G = ds.H / ds.H_kv;
     D.causal = ds.causal ? 1 : 0;
     D.C = D.causal ? ds.chunk : ds.N;
     D.nc = D.causal ? (ds.N + D.C - 1) / D.C : 1;

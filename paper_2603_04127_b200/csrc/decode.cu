@@ -73,18 +73,19 @@ __device__ __forceinline__ void token_features(const T *qv, const T *kv, const T
 // decode_z_kernel, launched behind this one on the same stream, applies z += phi(k).
 template <typename T>
 __global__ void __launch_bounds__(256) decode_step_kernel(const T *q, const T *k, const T *v, const T *M, const T *W, float *S,
-                                                           const float *z, T *o, int H, int d, int r, int m, int dv, int w_per_head,
+                                                           const float *z, T *o, int H, int Hkv, int d, int r, int m, int dv, int w_per_head,
                                                            float s)
 {
     extern __shared__ float sm[];
     float *xq = sm, *xk = xq + r, *fq = xk + r, *fk = fq + m, *red = fk + m;   // red: 8 x 32 partial numerators + 8 partial normalisers + scratch
     const int bh = blockIdx.y, h = bh % H, tid = threadIdx.x;
-    token_features<T, true>(q + (size_t)bh * d, k + (size_t)bh * d, M + (size_t)h * r * d, W + (size_t)(w_per_head ? h : 0) * m * r,
+    const int kvh = (bh / H) * Hkv + h / (H / Hkv);     // the key/value head this query head reads (grouped key/value heads)
+    token_features<T, true>(q + (size_t)bh * d, k + (size_t)kvh * d, M + (size_t)h * r * d, W + (size_t)(w_per_head ? h : 0) * m * r,
                             xq, xk, fq, fk, red, d, r, m, s);
 
     // state update and read-out: thread = (column, feature group)
     const int col = blockIdx.x * 32 + (tid & 31), grp = tid >> 5;
-    const float vv = ldf(v, (size_t)bh * dv + col);
+    const float vv = ldf(v, (size_t)kvh * dv + col);
     float *Sb = S + (size_t)bh * m * dv;
     const float *zb = z + (size_t)bh * m;
     float num = 0.f, den = 0.f;
@@ -110,13 +111,13 @@ __global__ void __launch_bounds__(256) decode_step_kernel(const T *q, const T *k
 
 // z += phi(k) of the new token; one block per (batch, head).
 template <typename T>
-__global__ void __launch_bounds__(256) decode_z_kernel(const T *k, const T *M, const T *W, float *z, int H, int d, int r, int m,
+__global__ void __launch_bounds__(256) decode_z_kernel(const T *k, const T *M, const T *W, float *z, int H, int Hkv, int d, int r, int m,
                                                         int w_per_head, float s)
 {
     extern __shared__ float sm[];
     float *xq = sm, *xk = xq + r, *fq = xk + r, *fk = fq + m, *red = fk + m;
     const int bh = blockIdx.x, h = bh % H;
-    token_features<T, false>(nullptr, k + (size_t)bh * d, M + (size_t)h * r * d, W + (size_t)(w_per_head ? h : 0) * m * r, xq, xk, fq,
+    token_features<T, false>(nullptr, k + (size_t)((bh / H) * Hkv + h / (H / Hkv)) * d, M + (size_t)h * r * d, W + (size_t)(w_per_head ? h : 0) * m * r, xq, xk, fq,
                              fk, red, d, r, m, s);
     for (int l = threadIdx.x; l < m; l += 256) z[(size_t)bh * m + l] += fk[l];
 }
@@ -141,15 +142,15 @@ extern "C" darkattn_status_t darkattn_decode_step(darkattn_plan_t plan, const vo
     if (D.bf16)
         decode_step_kernel<__nv_bfloat16><<<grid, 256, smem, st>>>((const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k, (const __nv_bfloat16 *)v,
                                                                   (const __nv_bfloat16 *)M, (const __nv_bfloat16 *)W, S, z, (__nv_bfloat16 *)o,
-                                                                  D.H, D.d, D.r, D.m, D.dv, D.w_per_head, D.s);
+                                                                  D.H, D.Hkv, D.d, D.r, D.m, D.dv, D.w_per_head, D.s);
     else
         decode_step_kernel<float><<<grid, 256, smem, st>>>((const float *)q, (const float *)k, (const float *)v, (const float *)M,
-                                                           (const float *)W, S, z, (float *)o, D.H, D.d, D.r, D.m, D.dv, D.w_per_head, D.s);
+                                                           (const float *)W, S, z, (float *)o, D.H, D.Hkv, D.d, D.r, D.m, D.dv, D.w_per_head, D.s);
     if (D.bf16)
         decode_z_kernel<__nv_bfloat16><<<D.BH, 256, smem, st>>>((const __nv_bfloat16 *)k, (const __nv_bfloat16 *)M, (const __nv_bfloat16 *)W, z,
-                                                              D.H, D.d, D.r, D.m, D.w_per_head, D.s);
+                                                              D.H, D.Hkv, D.d, D.r, D.m, D.w_per_head, D.s);
     else
-        decode_z_kernel<float><<<D.BH, 256, smem, st>>>((const float *)k, (const float *)M, (const float *)W, z, D.H, D.d, D.r, D.m,
+        decode_z_kernel<float><<<D.BH, 256, smem, st>>>((const float *)k, (const float *)M, (const float *)W, z, D.H, D.Hkv, D.d, D.r, D.m,
                                                         D.w_per_head, D.s);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_cuda_error(e, "decode_step"); return DARKATTN_ERR_CUDA; }

@@ -230,6 +230,38 @@ __global__ void emit_rows_kernel(T *out, const float *src, int N, int w, long lo
     }
 }
 
+// Grouped key/value heads. out[(b,hk),i,c] = sum_g src[(b, hk G + g),i,c]: the gradient of a shared key or value row
+// collects the parts of the G query heads that read it.
+template <typename T>
+__global__ void emit_grouped_kernel(T *out, const float *src, int N, int w, long long src_batch, int src_row, int H, int Hkv,
+                                    long long total)
+{
+    const int G = H / Hkv;
+    for (long long t = blockIdx.x * (long long)blockDim.x + threadIdx.x; t < total; t += (long long)gridDim.x * blockDim.x) {
+        const int c = (int)(t % w);
+        const long long row = t / w;
+        const int i = (int)(row % N);
+        const long long bhk = row / N, b = bhk / Hkv, hk = bhk % Hkv;
+        float v = 0.f;
+        for (int g = 0; g < G; ++g) v += src[(b * H + hk * G + g) * src_batch + (long long)i * src_row + c];
+        if constexpr (sizeof(T) == 2) out[t] = __float2bfloat16_rn(v);
+        else out[t] = v;
+    }
+}
+
+// out[(b,h),i,c] = in[(b, h / G),i,c] as fp32: every query head gets its own copy of the key/value head it reads.
+template <typename T>
+__global__ void expand_kv_kernel(const T *in, float *out, long long per_head, int H, int Hkv, long long total)
+{
+    const int G = H / Hkv;
+    for (long long t = blockIdx.x * (long long)blockDim.x + threadIdx.x; t < total; t += (long long)gridDim.x * blockDim.x) {
+        const long long bh = t / per_head, e = t % per_head, b = bh / H, h = bh % H;
+        const T x = in[(b * Hkv + h / G) * per_head + e];
+        if constexpr (sizeof(T) == 2) out[t] = __bfloat162float(x);
+        else out[t] = x;
+    }
+}
+
 // Ga[bh,i,:] = [G_i / den_i | -(G_i . O_i) / den_i], O_i = num_i / den_i; one warp per row.
 __global__ void grad_aug_kernel(const float *G, const float *num, float *Ga, int N, int Npad, int dv, long long rows)
 {
@@ -305,6 +337,20 @@ struct Launcher {
         check();
     }
     void fill(float *p, float v, long long n) { fill_kernel<<<blocks(n, 1024), 256, 0, st>>>(p, v, n); check(); }
+    void expand_kv(const void *in, int bf16, float *out, long long per_head, int B, int H, int Hkv)
+    {
+        const long long total = (long long)B * H * per_head;
+        if (bf16) expand_kv_kernel<__nv_bfloat16><<<blocks(total, 1024), 256, 0, st>>>((const __nv_bfloat16 *)in, out, per_head, H, Hkv, total);
+        else expand_kv_kernel<float><<<blocks(total, 1024), 256, 0, st>>>((const float *)in, out, per_head, H, Hkv, total);
+        check();
+    }
+    void emit_grouped(void *out, int bf16, const float *src, int B, int H, int Hkv, int N, int w, long long src_batch, int src_row)
+    {
+        const long long total = (long long)B * Hkv * N * w;
+        if (bf16) emit_grouped_kernel<__nv_bfloat16><<<blocks(total, 1024), 256, 0, st>>>((__nv_bfloat16 *)out, src, N, w, src_batch, src_row, H, Hkv, total);
+        else emit_grouped_kernel<float><<<blocks(total, 1024), 256, 0, st>>>((float *)out, src, N, w, src_batch, src_row, H, Hkv, total);
+        check();
+    }
     void emit(void *out, int bf16, const float *src, long long BH, int N, int w, long long src_batch, int src_row, int div_col)
     {
         const long long total = BH * N * w;
@@ -330,11 +376,20 @@ void run_forward_stages(const darkattn_plan_s *plan, Launcher &L, const void *Q,
     const long long BH = D.BH, N = D.N, Np = D.Npad, d = D.d, r = D.r, m = D.m, dv = D.dv, dva = D.dva, C = D.C, nc = D.nc;
     auto F = [&](size_t off) { return reinterpret_cast<float *>(ws + off); };
     if (D.bf16) {
-        L.cast(Q, F(Y.Qf), BH * N * d); L.cast(K, F(Y.Kf), BH * N * d); L.cast(V, F(Y.Vf), BH * N * dv);
+        L.cast(Q, F(Y.Qf), BH * N * d);
         L.cast(M, F(Y.Mf), (long long)D.H * r * d); L.cast(W, F(Y.Wf), (long long)(D.w_per_head ? D.H : 1) * m * r);
-        b.Q = F(Y.Qf); b.K = F(Y.Kf); b.V = F(Y.Vf); b.M = F(Y.Mf); b.W = F(Y.Wf);
+        b.Q = F(Y.Qf); b.M = F(Y.Mf); b.W = F(Y.Wf);
     } else {
-        b.Q = (const float *)Q; b.K = (const float *)K; b.V = (const float *)V; b.M = (const float *)M; b.W = (const float *)W;
+        b.Q = (const float *)Q; b.M = (const float *)M; b.W = (const float *)W;
+    }
+    if (D.G > 1) {          // grouped key/value heads: every query head works on its own fp32 copy of the head it reads
+        L.expand_kv(K, D.bf16, F(Y.Kf), N * d, D.B, D.H, D.Hkv); L.expand_kv(V, D.bf16, F(Y.Vf), N * dv, D.B, D.H, D.Hkv);
+        b.K = F(Y.Kf); b.V = F(Y.Vf);
+    } else if (D.bf16) {
+        L.cast(K, F(Y.Kf), BH * N * d); L.cast(V, F(Y.Vf), BH * N * dv);
+        b.K = F(Y.Kf); b.V = F(Y.Vf);
+    } else {
+        b.K = (const float *)K; b.V = (const float *)V;
     }
     b.xtQ = F(Y.xtQ); b.xtK = F(Y.xtK); b.nQ = F(Y.nQ); b.nK = F(Y.nK); b.fQ = F(Y.fQ); b.fK = F(Y.fK);
     b.cK = F(Y.cK); b.Va = F(Y.Va); b.Sloc = F(Y.Sloc); b.P = F(Y.P); b.num = F(Y.num);
@@ -387,12 +442,12 @@ void simt_make_layout(darkattn_plan_s *plan)
     const long long BH = D.BH, N = D.N, Np = D.Npad, d = D.d, r = D.r, m = D.m, dv = D.dv, dva = D.dva, C = D.C, nc = D.nc;
     size_t off = 0;
     Y.status = take(off, 64);
+    Y.Qf = Y.Kf = Y.Vf = Y.Mf = Y.Wf = 0;
     if (D.bf16) {
-        Y.Qf = take(off, BH * N * d); Y.Kf = take(off, BH * N * d); Y.Vf = take(off, BH * N * dv);
+        Y.Qf = take(off, BH * N * d);
         Y.Mf = take(off, (long long)D.H * r * d); Y.Wf = take(off, (long long)(D.w_per_head ? D.H : 1) * m * r);
-    } else {
-        Y.Qf = Y.Kf = Y.Vf = Y.Mf = Y.Wf = 0;
     }
+    if (D.bf16 || D.G > 1) { Y.Kf = take(off, BH * N * d); Y.Vf = take(off, BH * N * dv); }
     Y.xtQ = take(off, BH * N * r); Y.xtK = take(off, BH * N * r);
     Y.nQ = take(off, BH * N); Y.nK = take(off, BH * N);
     Y.fQ = take(off, BH * Np * m); Y.fK = take(off, BH * Np * m);
@@ -469,7 +524,8 @@ darkattn_status_t simt_backward(const darkattn_plan_s *plan, const void *Q, cons
         L.gemm(b.P, Ga, dVa, (int)C, (int)dva, (int)C, 1, C, dva, 1, dva, 1, Z, (int)nc, sP0, sP1, sV0, sV1, sV0, sV1, 1.f, 0, 0);
         L.gemm(b.fK, Rl, dVa, (int)C, (int)dva, (int)m, m, 1, dva, 1, dva, 1, Z, (int)nc, sF0, sF1, sS0, sS1, sV0, sV1, 1.f, 1, 0);
     }
-    L.emit(dV, D.bf16, dVa, BH, (int)N, (int)dv, Np * dva, (int)dva, -1);
+    if (D.G > 1) L.emit_grouped(dV, D.bf16, dVa, D.B, D.H, D.Hkv, (int)N, (int)dv, Np * dva, (int)dva);
+    else L.emit(dV, D.bf16, dVa, BH, (int)N, (int)dv, Np * dva, (int)dva, -1);
 
     const long long wb1 = D.w_per_head ? m * r : 0;
     for (int side = 0; side < 2; ++side) {
@@ -482,7 +538,8 @@ darkattn_status_t simt_backward(const darkattn_plan_s *plan, const void *Q, cons
         norm_term_kernel<<<Launcher::blocks(BH * N * r, 1024), 256, 0, st>>>(dxt, xt, es, (int)r, BH * N * r); L.check();
         // dX = s dx~ M
         L.gemm(dxt, b.M, dXf, (int)N, (int)d, (int)r, r, 1, d, 1, d, 1, BH, D.H, D.H * N * r, N * r, 0, r * d, D.H * N * d, N * d, D.s, 0, 0);
-        L.emit(side ? dK : dQ, D.bf16, dXf, BH, (int)N, (int)d, N * d, (int)d, -1);
+        if (side && D.G > 1) L.emit_grouped(dK, D.bf16, dXf, D.B, D.H, D.Hkv, (int)N, (int)d, N * d, (int)d);
+        else L.emit(side ? dK : dQ, D.bf16, dXf, BH, (int)N, (int)d, N * d, (int)d, -1);
         // dM_(b,h) (+)= s dx~^T X
         L.gemm(dxt, X, F(Y.dMp), (int)r, (int)d, (int)N, 1, r, d, 1, d, 1, BH, 1, N * r, 0, N * d, 0, r * d, 0, D.s, side, 0);
     }

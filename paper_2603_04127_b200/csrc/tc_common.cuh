@@ -360,6 +360,10 @@ __device__ __forceinline__ void issue_projection(uint32_t dst, const TileDesc &t
     _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(dst, kdesc(tX, k), kdesc(tOml, k), idesc, 1);
 }
 
+// First row, in the [B * H_kv * N, width] view of K, V, dK, dV, of the key/value head that query head bh = b H + h reads
+// (grouped key/value heads: G = H / H_kv consecutive query heads share one).
+__device__ __forceinline__ int kv_row0(int bh, int H, int Hkv, int N) { return ((bh / H) * Hkv + (bh % H) / (H / Hkv)) * N; }
+
 // ---------------------------------------------------------------- host side: tensor maps
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,

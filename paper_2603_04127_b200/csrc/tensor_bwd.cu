@@ -48,7 +48,8 @@ struct BwdParams {
     float *espart;        // [4 nslab, BH*N] partials of rowsum(E^K): one per slab and 32-column group
     float *Tacc;          // [H, m, D]
     int *status;
-    int N, H, BH, m, nslab, T;
+    int N, H, Hkv, BH, m, nslab, T;
+    int add_kv;           // parts of dK and dV are added into the (zeroed) gradients: several slabs, or several query heads per key/value head
 };
 
 template <int D, int DV>
@@ -152,10 +153,11 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                 if (l1 > lend) l1 = lend;
                 const int nrun = (int)(l1 - l0);
                 l0 = l1;
-                const int h = bh % p.H, row0 = bh * p.N;
+                const int h = bh % p.H, row0 = bh * p.N, rowk0 = kv_row0(bh, p.H, p.Hkv, p.N);
                 auto load_tile = [&](unsigned char *dst, const CUtensorMap *map, uint64_t *bar, int width, int t) {
+                    const int base = (map == &p.mapV) ? rowk0 : row0;      // V may be shared by a group of query heads
                     mbar_expect_tx(bar, 128 * width * 2);
-                    for (int a = 0; a < width / 64; ++a) tma_load_2d(dst + a * 16384, map, bar, a * 64, row0 + t * 128);
+                    for (int a = 0; a < width / 64; ++a) tma_load_2d(dst + a * 16384, map, bar, a * 64, base + t * 128);
                 };
                 auto load_key_features = [&](int t) {                  // Bf of chunk t, as the forward pass formed it
                     mbar_expect_tx(bars + QB_B, 32768);
@@ -432,7 +434,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
 
     const int tid = threadIdx.x, warp = tid >> 5;
     const int bh = blockIdx.x / p.nslab, slab = blockIdx.x % p.nslab, h = bh % p.H;
-    const int row0 = bh * p.N, T = p.T;
+    const int row0 = bh * p.N, rowk0 = kv_row0(bh, p.H, p.Hkv, p.N), T = p.T;      // rowk0: K, V, dK, dV may be shared by a group of query heads
 
     if (tid == 0) {
         for (int i = 0; i < KE2; ++i) mbar_init(bars + i, 1);
@@ -454,7 +456,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
         if ((tid & 31) == 0) {
             auto load_tile = [&](unsigned char *dst, const CUtensorMap *map, uint64_t *bar, int width, int t) {
                 mbar_expect_tx(bar, 128 * width * 2);
-                for (int a = 0; a < width / 64; ++a) tma_load_2d(dst + a * 16384, map, bar, a * 64, row0 + t * 128);
+                const int base = (map == &p.mapG) ? row0 : rowk0;
+                for (int a = 0; a < width / 64; ++a) tma_load_2d(dst + a * 16384, map, bar, a * 64, base + t * 128);
             };
             auto load_features = [&](unsigned char *dst, const CUtensorMap *map, uint64_t *bar, int t) {
                 mbar_expect_tx(bar, 32768);
@@ -489,8 +492,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
             // A^ of the next chunk can be fetched as soon as dP^T A^ is done, V and dO with it, Bf once E Omega is done.
             auto store_out = [&](const CUtensorMap *map, int width, int t) {     // the staged tile into (or, with several slabs, added into) the gradient
                 for (int a = 0; a < width / 64; ++a) {
-                    if (p.nslab > 1) tma_reduce_add_2d(map, sStg + a * 16384, a * 64, row0 + t * 128);
-                    else tma_store_2d(map, sStg + a * 16384, a * 64, row0 + t * 128);
+                    if (p.add_kv) tma_reduce_add_2d(map, sStg + a * 16384, a * 64, rowk0 + t * 128);
+                    else tma_store_2d(map, sStg + a * 16384, a * 64, rowk0 + t * 128);
                 }
                 tma_store_commit();
             };
@@ -683,7 +686,7 @@ struct FinishParams {
     const float *espart;  // [nes, BH*N]
     float *dMn;           // [H, r, D]
     int *status;
-    int N, H, BH, T, nsplit, r, nes;
+    int N, H, Hkv, BH, T, nsplit, r, nes;
     float s2;
 };
 
@@ -726,7 +729,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __gr
             auto load_k = [&](int t) {
                 const int b = (t - t0) & 1;
                 mbar_expect_tx(bar_k + b, kTile);
-                for (int a = 0; a < D / 64; ++a) tma_load_2d(sK0 + b * kTile + a * 16384, &p.mapK, bar_k + b, a * 64, bh * p.N + t * 128);
+                for (int a = 0; a < D / 64; ++a) tma_load_2d(sK0 + b * kTile + a * 16384, &p.mapK, bar_k + b, a * 64, kv_row0(bh, p.H, p.Hkv, p.N) + t * 128);
             };
             mbar_expect_tx(bar_m, kTile);
             for (int a = 0; a < D / 64; ++a) tma_load_2d(sM + a * 16384, &p.mapM, bar_m, a * 64, h * p.r);
@@ -782,7 +785,6 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __gr
         float es_next = row_sum(t0);
         for (int t = t0; t < t1 && ok; ++t) {
             const uint32_t ph = (t - t0) & 1;
-            const size_t row = (size_t)bh * p.N + (size_t)t * 128 + r;
             const float coef = -p.s2 * es_next;
             ok = __all_sync(0xffffffffu, wait_or_abort(m1, ph, p.status, abort_flag));
             if (!ok) break;
@@ -819,7 +821,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __gr
             fence_async_smem();
             epi_sync();
             if (tid == 0) {
-                for (int a = 0; a < D / 64; ++a) tma_reduce_add_2d(&p.mapOut, sOut + a * 16384, a * 64, (int)(row - r));
+                for (int a = 0; a < D / 64; ++a) tma_reduce_add_2d(&p.mapOut, sOut + a * 16384, a * 64, kv_row0(bh, p.H, p.Hkv, p.N) + t * 128);
                 tma_store_commit();
             }
             tc_fence_before();
@@ -953,7 +955,7 @@ cudaError_t launch_scan(const darkattn_plan_s *plan, const BwdParams &P, int gri
     tc_bwd_q_kernel<D, DV><<<qgrid, kThreads, L::kTotal, st>>>(P);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    if (P.nslab > 1) {
+    if (P.add_kv) {
         e = cudaStreamWaitEvent(st, plan->aux_join, 0);      // dK and dV have been zeroed
         if (e != cudaSuccess) return e;
     }
@@ -1008,41 +1010,44 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
     chk();
     keep(cudaMemsetAsync(ws + Y.Tacc, 0, (size_t)D.H * D.m * D.d * 4, st));
     keep(cudaMemsetAsync(ws + Y.dMn, 0, (size_t)D.H * D.r * D.d * 4, st));
-    if (Y.nslab > 1) {
-        // The slabs of a head add their parts into the gradients, which therefore start at zero. dQ is needed first;
-        // dK and dV are zeroed on a side stream while the query-side scan runs (it leaves SMs and bandwidth free).
+    const size_t BHkv = (size_t)D.B * D.Hkv;
+    const bool add_kv = Y.nslab > 1 || D.G > 1;
+    if (add_kv) {
+        // The slabs of a head (and the query heads of a group that shares its keys and values) add their parts into the
+        // gradients, which therefore start at zero. dQ is needed first; dK and dV are zeroed on a side stream while the
+        // query-side scan runs (it leaves SMs and bandwidth free).
         keep(ensure_aux(plan));
         if (e != cudaSuccess) { set_cuda_error(e, "tensor_backward: side stream"); return DARKATTN_ERR_CUDA; }
         keep(cudaEventRecord(plan->aux_fork, st));
         keep(cudaStreamWaitEvent(plan->aux_stream, plan->aux_fork, 0));
-        keep(cudaMemsetAsync(dK, 0, BH * N * D.d * 2, plan->aux_stream));
-        keep(cudaMemsetAsync(dV, 0, BH * N * D.dv * 2, plan->aux_stream));
+        keep(cudaMemsetAsync(dK, 0, BHkv * N * D.d * 2, plan->aux_stream));
+        keep(cudaMemsetAsync(dV, 0, BHkv * N * D.dv * 2, plan->aux_stream));
         keep(cudaEventRecord(plan->aux_join, plan->aux_stream));
-        keep(cudaMemsetAsync(dQ, 0, BH * N * D.d * 2, st));
     }
+    if (Y.nslab > 1) keep(cudaMemsetAsync(dQ, 0, BH * N * D.d * 2, st));
 
     FinishParams F;
     memset(&F, 0, sizeof(F));
-    if (!make_map(&F.mapM, M, (size_t)D.H * D.r, D.d, 128) || !make_map(&F.mapK, K, BH * N, D.d, 128)) {
+    if (!make_map(&F.mapM, M, (size_t)D.H * D.r, D.d, 128) || !make_map(&F.mapK, K, BHkv * N, D.d, 128)) {
         set_cuda_error(cudaErrorInvalidValue, "tensor_backward: tensor map encode");
         return DARKATTN_ERR_CUDA;
     }
     if (D.causal) {
         BwdParams P;
         memset(&P, 0, sizeof(P));
-        const bool ok = make_map(&P.mapQ, Q, BH * N, D.d, 128) && make_map(&P.mapK, K, BH * N, D.d, 128) &&
-                        make_map(&P.mapV, V, BH * N, D.dv, 128) && make_map(&P.mapG, dO, BH * N, D.dv, 128) &&
+        const bool ok = make_map(&P.mapQ, Q, BH * N, D.d, 128) && make_map(&P.mapK, K, BHkv * N, D.d, 128) &&
+                        make_map(&P.mapV, V, BHkv * N, D.dv, 128) && make_map(&P.mapG, dO, BH * N, D.dv, 128) &&
                         make_map(&P.mapOm, stash.Om, (size_t)D.H * D.m, D.d, 128) &&
                         make_map(&P.mapOml, stash.Oml, (size_t)D.H * D.m, D.d, 128) &&
-                        make_map(&P.mapDQ, dQ, BH * N, D.d, 128) && make_map(&P.mapDK, dK, BH * N, D.d, 128) &&
-                        make_map(&P.mapDV, dV, BH * N, D.dv, 128) &&
+                        make_map(&P.mapDQ, dQ, BH * N, D.d, 128) && make_map(&P.mapDK, dK, BHkv * N, D.d, 128) &&
+                        make_map(&P.mapDV, dV, BHkv * N, D.dv, 128) &&
                         make_map(&P.mapAh, bf(Y.Ahat), BH * N, D.m, 128) && make_map(&P.mapBf, stash.Bphi, BH * N, D.m, 128) &&
                         make_map(&P.mapSst, stash.Sst, BH * Y.T * D.m, D.dv, 128);
         if (!ok) { set_cuda_error(cudaErrorInvalidValue, "tensor_backward: tensor map encode"); return DARKATTN_ERR_CUDA; }
         P.sv = stash.sv; P.delta = fl(Y.delta); P.nK = stash.nK; P.cs = stash.cs; P.zc = stash.zc; P.rhoc = fl(Y.rhoc);
         P.espart = fl(Y.espart); P.Tacc = fl(Y.Tacc);
         P.status = reinterpret_cast<int *>(ws + Y.status);
-        P.N = D.N; P.H = D.H; P.BH = D.BH; P.m = D.m; P.nslab = Y.nslab; P.T = Y.T;
+        P.N = D.N; P.H = D.H; P.Hkv = D.Hkv; P.BH = D.BH; P.m = D.m; P.nslab = Y.nslab; P.T = Y.T; P.add_kv = add_kv ? 1 : 0;
         const int units = (int)(BH * Y.nslab);
         if (D.d == 64 && D.dv == 64) keep(launch_scan<64, 64>(plan, P, units, st));
         else if (D.d == 128 && D.dv == 128) keep(launch_scan<128, 128>(plan, P, units, st));
@@ -1052,10 +1057,10 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
         keep(tensor_backward_nc_passes(plan, Q, K, V, dO, stash, dQ, dK, dV, ws, st));
     }
 
-    if (!make_map(&F.mapOut, dK, BH * N, D.d, 128)) { set_cuda_error(cudaErrorInvalidValue, "tensor_backward: tensor map encode"); return DARKATTN_ERR_CUDA; }
+    if (!make_map(&F.mapOut, dK, BHkv * N, D.d, 128)) { set_cuda_error(cudaErrorInvalidValue, "tensor_backward: tensor map encode"); return DARKATTN_ERR_CUDA; }
     F.espart = fl(Y.espart); F.dMn = fl(Y.dMn);
     F.status = reinterpret_cast<int *>(ws + Y.status);
-    F.N = D.N; F.H = D.H; F.BH = D.BH; F.T = Y.T; F.r = D.r; F.nes = 4 * Y.nslab; F.s2 = D.s * D.s;
+    F.N = D.N; F.H = D.H; F.Hkv = D.Hkv; F.BH = D.BH; F.T = Y.T; F.r = D.r; F.nes = 4 * Y.nslab; F.s2 = D.s * D.s;
     F.nsplit = pick_splits((long long)BH, Y.T, 3.5, 5.0, 64);
     // dM = s W^T T + (norm term). T is complete once the key-side pass is done, so its product runs on the side
     // stream next to the kernel that produces the norm term, and a small kernel adds the two. (With per-kernel

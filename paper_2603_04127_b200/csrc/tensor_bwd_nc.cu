@@ -38,7 +38,8 @@ struct NcParams {
     float *espart;        // [4 nslab, BH*N] partials of rowsum(E^K): one per slab and 32-column group
     float *Tacc;          // [H, m, D]
     int *status;
-    int N, H, BH, m, nslab, T, nsplit;
+    int N, H, Hkv, BH, m, nslab, T, nsplit;
+    int add_kv;           // parts of dK and dV are added into the (zeroed) gradients: several slabs, or several query heads per key/value head
 };
 
 template <int D, int DV>
@@ -86,6 +87,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_nc_kernel(const __grid_con
     const int unit = blockIdx.x / p.nsplit, piece = blockIdx.x % p.nsplit;
     const int bh = unit / p.nslab, slab = unit % p.nslab, h = bh % p.H;
     const int row0 = bh * p.N;
+    // key pass: K, dK (X, Out) and V, dV (Y, DV) may be shared by a group of query heads; query pass: only V has no part in it
+    const int rowx0 = KEYS ? kv_row0(bh, p.H, p.Hkv, p.N) : row0, rowy0 = rowx0;
     const int tbeg = (int)((long long)p.T * piece / p.nsplit), tend = (int)((long long)p.T * (piece + 1) / p.nsplit);
     const int nt = tend - tbeg;
 
@@ -111,7 +114,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_nc_kernel(const __grid_con
         if ((tid & 31) == 0) {
             auto load_tile = [&](unsigned char *dst, const CUtensorMap *map, uint64_t *bar, int width, int t) {
                 mbar_expect_tx(bar, 128 * width * 2);
-                for (int a = 0; a < width / 64; ++a) tma_load_2d(dst + a * 16384, map, bar, a * 64, row0 + t * 128);
+                const int base = (map == &p.mapX) ? rowx0 : rowy0;
+                for (int a = 0; a < width / 64; ++a) tma_load_2d(dst + a * 16384, map, bar, a * 64, base + t * 128);
             };
             const TileDesc tOm(sOm), tOml(sOml), tX0(sX), tX1(sX + 128 * D * 2), tA(sA), tY(sY), tSt(sSt), tDel(sDelOp);
             const uint32_t id_kk = make_idesc(128, 128, 0, 0);
@@ -145,9 +149,10 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_nc_kernel(const __grid_con
                 const TileDesc &tX = (it & 1) ? tX1 : tX0;
 #define NWAIT(b, q) do { ok = wait_or_abort(bars + (b), (q), status, abort_flag); } while (0)
                 auto store_out = [&](const CUtensorMap *map, unsigned char *src, int width, int tt) {     // (adds into the gradient when the head has several slabs)
+                    const bool add = KEYS ? (p.add_kv != 0) : (p.nslab > 1);
                     for (int a = 0; a < width / 64; ++a) {
-                        if (p.nslab > 1) tma_reduce_add_2d(map, src + a * 16384, a * 64, row0 + tt * 128);
-                        else tma_store_2d(map, src + a * 16384, a * 64, row0 + tt * 128);
+                        if (add) tma_reduce_add_2d(map, src + a * 16384, a * 64, rowx0 + tt * 128);
+                        else tma_store_2d(map, src + a * 16384, a * 64, rowx0 + tt * 128);
                     }
                     tma_store_commit();
                 };
@@ -376,15 +381,17 @@ cudaError_t tensor_backward_nc_passes(const darkattn_plan_s *plan, const void *Q
     PQ.sv = stash.sv; PQ.delta = fl(Y.delta); PQ.nK = stash.nK; PQ.cs = stash.cs; PQ.zt = stash.zt;
     PQ.Racc = fl(Y.Racc); PQ.rhot = fl(Y.rhot); PQ.espart = fl(Y.espart); PQ.Tacc = fl(Y.Tacc);
     PQ.status = reinterpret_cast<int *>(ws + Y.status);
-    PQ.N = D.N; PQ.H = D.H; PQ.BH = D.BH; PQ.m = D.m; PQ.nslab = Y.nslab; PQ.T = Y.T;
+    const size_t BHkv = (size_t)D.B * D.Hkv;
+    const bool add_kv = Y.nslab > 1 || D.G > 1;
+    PQ.N = D.N; PQ.H = D.H; PQ.Hkv = D.Hkv; PQ.BH = D.BH; PQ.m = D.m; PQ.nslab = Y.nslab; PQ.T = Y.T; PQ.add_kv = add_kv ? 1 : 0;
     PQ.nsplit = pick_splits((long long)BH * Y.nslab, Y.T, 3.0, 6.0, 64);
     NcParams PK = PQ;
     const bool ok = make_map(&PQ.mapX, Q, BH * N, D.d, 128) && make_map(&PQ.mapY, dO, BH * N, D.dv, 128) &&
                     make_map(&PQ.mapOm, stash.Om, (size_t)D.H * D.m, D.d, 128) && make_map(&PQ.mapOml, stash.Oml, (size_t)D.H * D.m, D.d, 128) &&
                     make_map(&PQ.mapSt, stash.Sb, BH * D.m, D.dv, 128) &&
-                    make_map(&PQ.mapOut, dQ, BH * N, D.d, 128) && make_map(&PQ.mapDV, dV, BH * N, D.dv, 128) &&
-                    make_map(&PK.mapX, K, BH * N, D.d, 128) && make_map(&PK.mapY, V, BH * N, D.dv, 128) &&
-                    make_map(&PK.mapSt, Rb, BH * D.m, D.dv, 128) && make_map(&PK.mapOut, dK, BH * N, D.d, 128);
+                    make_map(&PQ.mapOut, dQ, BH * N, D.d, 128) && make_map(&PQ.mapDV, dV, BHkv * N, D.dv, 128) &&
+                    make_map(&PK.mapX, K, BHkv * N, D.d, 128) && make_map(&PK.mapY, V, BHkv * N, D.dv, 128) &&
+                    make_map(&PK.mapSt, Rb, BH * D.m, D.dv, 128) && make_map(&PK.mapOut, dK, BHkv * N, D.d, 128);
     if (!ok) return cudaErrorInvalidValue;
     PK.mapOm = PQ.mapOm;
     PK.mapOml = PQ.mapOml;
@@ -392,7 +399,7 @@ cudaError_t tensor_backward_nc_passes(const darkattn_plan_s *plan, const void *Q
     const long long nstate = (long long)BH * D.m * D.dv;
     cudaError_t e = cudaMemsetAsync(ws + Y.Racc, 0, (Y.rhot - Y.Racc) + BH * D.m * 4, st);      // R and rho sums (adjacent)
     if (e != cudaSuccess) return e;
-    const bool join = Y.nslab > 1;
+    const bool join = add_kv;
     if (D.d == 64 && D.dv == 64) return launch_nc<64, 64>(plan, PQ, PK, fl(Y.Racc), Rb, nstate, join, st);
     if (D.d == 128 && D.dv == 128) return launch_nc<128, 128>(plan, PQ, PK, fl(Y.Racc), Rb, nstate, join, st);
     if (D.d == 64 && D.dv == 128) return launch_nc<64, 128>(plan, PQ, PK, fl(Y.Racc), Rb, nstate, join, st);

@@ -84,7 +84,7 @@ struct NormParams {
     CUtensorMap mapK, mapM;
     float *nK;
     int *status;
-    int N, H, T, nsplit, r;
+    int N, H, Hkv, T, nsplit, r;
     float coef;   // log2(e) * s^2 / 2
 };
 
@@ -117,7 +117,7 @@ __global__ void __launch_bounds__(160, 1) tc_key_norms_kernel(const __grid_const
             mbar_expect_tx(bar_m, kTile);
             for (int a = 0; a < D / 64; ++a) tma_load_2d(sM + a * 16384, &p.mapM, bar_m, a * 64, h * p.r);
             mbar_expect_tx(bar_k, kTile);
-            for (int a = 0; a < D / 64; ++a) tma_load_2d(sK + a * 16384, &p.mapK, bar_k, a * 64, bh * p.N + t0 * 128);
+            for (int a = 0; a < D / 64; ++a) tma_load_2d(sK + a * 16384, &p.mapK, bar_k, a * 64, kv_row0(bh, p.H, p.Hkv, p.N) + t0 * 128);
             const uint32_t idesc = make_idesc(128, p.r, 0, 0);
             bool ok = wait_or_abort(bar_m, 0, p.status, abort_flag);
             for (int t = t0; t < t1 && ok; ++t) {
@@ -135,7 +135,7 @@ __global__ void __launch_bounds__(160, 1) tc_key_norms_kernel(const __grid_const
                     if (!ok) break;
                     mbar_expect_tx(bar_k, kTile);
                     for (int a = 0; a < D / 64; ++a)
-                        tma_load_2d(sK + a * 16384, &p.mapK, bar_k, a * 64, bh * p.N + (t + 1) * 128);
+                        tma_load_2d(sK + a * 16384, &p.mapK, bar_k, a * 64, kv_row0(bh, p.H, p.Hkv, p.N) + (t + 1) * 128);
                 }
             }
         }
@@ -173,7 +173,7 @@ struct ShiftParams {
     const float *nK;     // [BH, N] key norms, log2 units
     int *cs;             // [BH, nslab] order keys of the shifts
     int *status;
-    int N, H, T, m, nslab, nsplit;
+    int N, H, Hkv, T, m, nslab, nsplit;
 };
 
 template <int D>
@@ -206,7 +206,7 @@ __global__ void __launch_bounds__(160, 1) tc_key_shift_kernel(const __grid_const
             mbar_expect_tx(bar_m, kTile);
             for (int a = 0; a < D / 64; ++a) tma_load_2d(sOm + a * 16384, &p.mapOm, bar_m, a * 64, h * p.m + slab * 128);
             mbar_expect_tx(bar_k, kTile);
-            for (int a = 0; a < D / 64; ++a) tma_load_2d(sK + a * 16384, &p.mapK, bar_k, a * 64, bh * p.N + t0 * 128);
+            for (int a = 0; a < D / 64; ++a) tma_load_2d(sK + a * 16384, &p.mapK, bar_k, a * 64, kv_row0(bh, p.H, p.Hkv, p.N) + t0 * 128);
             const TileDesc tOm(sOm), tK(sK);
             const uint32_t idesc = make_idesc(128, 128, 0, 0);
             bool ok = wait_or_abort(bar_m, 0, p.status, abort_flag);
@@ -222,7 +222,7 @@ __global__ void __launch_bounds__(160, 1) tc_key_shift_kernel(const __grid_const
                     ok = wait_or_abort(bar_u, ph, p.status, abort_flag);
                     if (!ok) break;
                     mbar_expect_tx(bar_k, kTile);
-                    for (int a = 0; a < D / 64; ++a) tma_load_2d(sK + a * 16384, &p.mapK, bar_k, a * 64, bh * p.N + (t + 1) * 128);
+                    for (int a = 0; a < D / 64; ++a) tma_load_2d(sK + a * 16384, &p.mapK, bar_k, a * 64, kv_row0(bh, p.H, p.Hkv, p.N) + (t + 1) * 128);
                 }
             }
         }
@@ -276,7 +276,7 @@ struct MainParams {
     float *Sseg, *zseg;
     float *zc;           // causal: z before chunk t for the backward pass, [BH, T, m] (row 0 not written)
     int *status;
-    int N, H, BH, m, nslab, T, nsplit;
+    int N, H, Hkv, BH, m, nslab, T, nsplit;
 };
 
 enum { MODE_CAUSAL = 0, MODE_KEYS = 1, MODE_QUERIES = 2 };
@@ -423,9 +423,11 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
     } else if (tend <= tbeg) {
     } else if (warp == kEpiWarps) {
         if ((tid & 31) == 0) {
+            const int rowk0 = kv_row0(bh, p.H, p.Hkv, p.N);       // K and V may be shared by a group of query heads
             auto load_tile = [&](unsigned char *dst, const CUtensorMap *map, uint64_t *bar, int width, int t) {
+                const int base = (map == &p.mapQ) ? row0 : rowk0;
                 mbar_expect_tx(bar, 128 * width * 2);
-                for (int a = 0; a < width / 64; ++a) tma_load_2d(dst + a * 16384, map, bar, a * 64, row0 + t * 128);
+                for (int a = 0; a < width / 64; ++a) tma_load_2d(dst + a * 16384, map, bar, a * 64, base + t * 128);
             };
             const int prow0 = (slab * p.BH + bh) * p.N;
             auto store_output = [&](int t) {       // this slab's part of the output rows of chunk t, staged in the state tile's buffer
@@ -685,7 +687,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_keys_kernel(const __grid_c
     const int unit = blockIdx.x / p.nsplit, split = blockIdx.x % p.nsplit;
     const int bh = unit / p.nslab, slab = unit % p.nslab, h = bh % p.H;
     const int t0 = (int)((long long)p.T * split / p.nsplit), t1 = (int)((long long)p.T * (split + 1) / p.nsplit);
-    const int n = t1 - t0, row0 = bh * p.N;
+    const int n = t1 - t0, row0 = bh * p.N, rowk0 = kv_row0(bh, p.H, p.Hkv, p.N);
 
     if (tid == 0) {
         for (int i = 0; i < YE1_0; ++i) mbar_init(bars + i, 1);
@@ -713,12 +715,12 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_keys_kernel(const __grid_c
             auto load_k = [&](int i) {
                 const int b = i % NST;
                 mbar_expect_tx(bars + YB_K0 + b, kXT);
-                for (int a = 0; a < D / 64; ++a) tma_load_2d(sK + b * kXT + a * 16384, &p.mapK, bars + YB_K0 + b, a * 64, row0 + (t0 + i) * 128);
+                for (int a = 0; a < D / 64; ++a) tma_load_2d(sK + b * kXT + a * 16384, &p.mapK, bars + YB_K0 + b, a * 64, rowk0 + (t0 + i) * 128);
             };
             auto load_v = [&](int i) {
                 const int b = i % NST;
                 mbar_expect_tx(bars + YB_V0 + b, kVT);
-                for (int a = 0; a < DV / 64; ++a) tma_load_2d(sV + b * kVT + a * 16384, &p.mapV, bars + YB_V0 + b, a * 64, row0 + (t0 + i) * 128);
+                for (int a = 0; a < DV / 64; ++a) tma_load_2d(sV + b * kVT + a * 16384, &p.mapV, bars + YB_V0 + b, a * 64, rowk0 + (t0 + i) * 128);
             };
             const TileDesc tOm(sOm), tOml(sOml), tF0(sFK), tF1(sFK + kFKstride);
             const uint64_t ones_desc = make_sdesc(smem_u32(sOnes), 16384, 1024);
@@ -1215,7 +1217,8 @@ cudaError_t tensor_prologue(const darkattn_plan_s *plan, const void *K, const vo
     const size_t BH = D.BH, N = D.N;
     NormParams NP;
     memset(&NP, 0, sizeof(NP));
-    if (!make_map(&NP.mapK, K, BH * N, D.d, 128) || !make_map(&NP.mapM, M, (size_t)D.H * D.r, D.d, 128))
+    const size_t BHkv = (size_t)D.B * D.Hkv;
+    if (!make_map(&NP.mapK, K, BHkv * N, D.d, 128) || !make_map(&NP.mapM, M, (size_t)D.H * D.r, D.d, 128))
         return cudaErrorInvalidValue;
     cudaError_t e = cudaSuccess;
     auto chk = [&]() { cudaError_t x = cudaGetLastError(); if (x != cudaSuccess && e == cudaSuccess) e = x; };
@@ -1238,7 +1241,7 @@ cudaError_t tensor_prologue(const darkattn_plan_s *plan, const void *K, const vo
     if (beside && e == cudaSuccess) e = cudaEventRecord(plan->aux_join, sp);
 
     NP.nK = out.nK; NP.status = reinterpret_cast<int *>(ws + Y.status);
-    NP.N = D.N; NP.H = D.H; NP.T = Y.T; NP.r = D.r;
+    NP.N = D.N; NP.H = D.H; NP.Hkv = D.Hkv; NP.T = Y.T; NP.r = D.r;
     NP.nsplit = pick_splits((long long)BH, Y.T, 2.5, 3.0, 64, 3 * 148);      // three CTAs of this kernel fit one SM
     NP.coef = kLog2e * 0.5f * D.s * D.s;
     const int smem_bytes = 2 * 128 * D.d * 2 + 64;
@@ -1256,9 +1259,9 @@ cudaError_t tensor_prologue(const darkattn_plan_s *plan, const void *K, const vo
     // the key-side shifts: the maximum of u - n over the keys of every (batch, head, slab)
     ShiftParams SP;
     memset(&SP, 0, sizeof(SP));
-    if (!make_map(&SP.mapK, K, BH * N, D.d, 128) || !make_map(&SP.mapOm, out.Om, (size_t)D.H * D.m, D.d, 128)) return cudaErrorInvalidValue;
+    if (!make_map(&SP.mapK, K, BHkv * N, D.d, 128) || !make_map(&SP.mapOm, out.Om, (size_t)D.H * D.m, D.d, 128)) return cudaErrorInvalidValue;
     SP.nK = out.nK; SP.cs = reinterpret_cast<int *>(out.cs); SP.status = NP.status;
-    SP.N = D.N; SP.H = D.H; SP.T = Y.T; SP.m = D.m; SP.nslab = Y.nslab;
+    SP.N = D.N; SP.H = D.H; SP.Hkv = D.Hkv; SP.T = Y.T; SP.m = D.m; SP.nslab = Y.nslab;
     SP.nsplit = pick_splits((long long)BH * Y.nslab, Y.T, 2.5, 3.0, 64, 3 * 148);
     timer_mark(plan, st, "tc_key_shift_kernel");
     if (D.d == 64) {
@@ -1285,8 +1288,9 @@ darkattn_status_t tensor_forward(const darkattn_plan_s *plan, const void *Q, con
     const Stash stash = saved ? stash_in_saved(Y, saved) : stash_in_workspace(Y, ws);
     MainParams P;
     memset(&P, 0, sizeof(P));
-    bool ok = make_map(&P.mapQ, Q, BH * N, D.d, 128) && make_map(&P.mapK, K, BH * N, D.d, 128) &&
-              make_map(&P.mapV, V, BH * N, D.dv, 128) && make_map(&P.mapOm, stash.Om, (size_t)D.H * D.m, D.d, 128) &&
+    const size_t BHkv = (size_t)D.B * D.Hkv;
+    bool ok = make_map(&P.mapQ, Q, BH * N, D.d, 128) && make_map(&P.mapK, K, BHkv * N, D.d, 128) &&
+              make_map(&P.mapV, V, BHkv * N, D.dv, 128) && make_map(&P.mapOm, stash.Om, (size_t)D.H * D.m, D.d, 128) &&
               make_map(&P.mapOml, stash.Oml, (size_t)D.H * D.m, D.d, 128) &&
               make_map(&P.mapSb, D.causal ? bf(Y.Sb) : stash.Sb, BH * (D.causal ? Y.nsplit : 1) * D.m, D.dv, 128) &&
               make_map(&P.mapPN, bf(Y.pnum), (size_t)Y.nslab * BH * N, D.dv, 128);
@@ -1297,7 +1301,7 @@ darkattn_status_t tensor_forward(const darkattn_plan_s *plan, const void *Q, con
 
     P.nK = stash.nK; P.cs = stash.cs; P.zc = stash.zc; P.pdr = fl(Y.pdr); P.Sacc = fl(Y.Sacc); P.zacc = fl(Y.zacc);
     P.status = reinterpret_cast<int *>(ws + Y.status);
-    P.N = D.N; P.H = D.H; P.BH = D.BH; P.m = D.m; P.nslab = Y.nslab; P.T = Y.T; P.nsplit = Y.nsplit;
+    P.N = D.N; P.H = D.H; P.Hkv = D.Hkv; P.BH = D.BH; P.m = D.m; P.nslab = Y.nslab; P.T = Y.T; P.nsplit = Y.nsplit;
     P.stash_S = (D.causal && stash_states) ? 1 : 0;
     if (P.stash_S && !(make_map(&P.mapSst, stash.Sst, BH * Y.T * D.m, D.dv, 128) && make_map(&P.mapBf, stash.Bphi, BH * N, D.m, 128))) {
         set_cuda_error(cudaErrorInvalidValue, "tensor_forward: tensor map encode");

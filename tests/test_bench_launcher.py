@@ -1,6 +1,6 @@
 """bench.py starts its own ranks: `--gpus N` without a launcher's environment re-runs the script under
 torch.distributed.run, one rank per GPU. Checked here without a GPU: the command it builds, and that on a machine
-without CUDA two ranks really start and each stops with a clear message instead of falling back to the CPU."""
+without CUDA two ranks really start and a rank stops with a clear message instead of falling back to the CPU."""
 import os
 import subprocess
 import sys
@@ -29,4 +29,6 @@ def test_two_ranks_start_and_refuse_to_run_without_cuda():
                        capture_output=True, text=True, timeout=300, env=env, cwd=ROOT)
     assert r.returncode != 0
     text = r.stdout + r.stderr
-    assert "rank 0 of 2: no CUDA device" in text and "rank 1 of 2: no CUDA device" in text, text[-2000:]
+    # the launcher ends the other rank as soon as the first one has failed, so only one of the two messages is certain;
+    # "of 2" shows that the rank ran inside a two-rank job
+    assert "rank 0 of 2: no CUDA device" in text or "rank 1 of 2: no CUDA device" in text, text[-2000:]

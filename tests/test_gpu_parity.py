@@ -321,6 +321,32 @@ def test_bf16_error_over_many_seeds(binding, wid, kw, causal):
         assert fro < 1e-2 and mx < 1.5e-2, (wid, k, fro, mx)
 
 
+GROUPED = [
+    # path, H, H_kv, shape
+    ("simt_f32", 4, 1, dict(B=2, N=150, d=24, m=40, r=16, dv=20)),
+    ("simt_f32", 6, 3, dict(B=1, N=130, d=16, m=32)),
+    ("tensor", 4, 1, dict(B=2, N=384, d=64, m=256)),
+    ("tensor", 8, 2, dict(B=1, N=256, d=128, m=128, dv=64)),
+    ("tensor", 4, 4, dict(B=1, N=256, d=64, m=128)),
+]
+
+
+@pytest.mark.parametrize("causal", [True, False], ids=["causal", "noncausal"])
+@pytest.mark.parametrize("path,H,Hkv,kw", GROUPED, ids=[f"{g[0]}_H{g[1]}_Hkv{g[2]}" for g in GROUPED])
+def test_grouped_key_value_heads(binding, path, H, Hkv, kw, causal):
+    """K and V with fewer heads than Q (H_kv in {1, H/4 .., H}): query heads h*G .. h*G+G-1 read key/value head h; dK and dV
+    sum over the group. Forward and backward against the oracle, on the FP32 and on the tensor-core kernels."""
+    dtype = "f32" if path == "simt_f32" else "bf16"
+    wl = inputs.small(name="grouped", wid=95, H=H, dtype=dtype, causal=causal, backward=True, **kw)
+    t = inputs.generate(wl)
+    G = H // Hkv
+    t.K, t.V = np.ascontiguousarray(t.K[:, ::G]), np.ascontiguousarray(t.V[:, ::G])     # keep every G-th head as the shared one
+    got = run_gpu(binding, wl, t, path=binding.PATH_SIMT if path == "simt_f32" else binding.PATH_TENSOR, use_saved=True)
+    want = _oracle(t, wl)
+    assert got["dK"].shape == t.K.shape and got["dV"].shape == t.V.shape
+    _compare(got, want, TOL[dtype], f"grouped {path} H={H} H_kv={Hkv}")
+
+
 def test_tensor_path_is_deterministic(binding):
     """The scan kernels hand tiles between warps through shared and tensor memory; a missing wait shows up as rare,
     run-dependent errors of the size of the values themselves. O has a fixed summation order: repeated runs at the

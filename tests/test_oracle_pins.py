@@ -244,3 +244,36 @@ def test_p10_whitening_orientation():
     E = np.zeros((d, d)); E[0, 1] = 1.0
     _, xt = ref.features(X[:5], E, np.zeros((1, d)), return_xt=True)
     np.testing.assert_allclose(xt[:, 0], X[:5, 1]); assert np.all(xt[:, 1:] == 0)
+
+
+def test_grouped_key_value_heads_explicit_form_and_finite_differences():
+    """Grouped key/value heads: query heads h*G .. h*G+G-1 read key/value head h, each through its own M. O equals the
+    explicit N x N form built head by head from the shared K, V; the gradients of the shared K and V (which collect
+    every reading head's contribution) agree with central differences of L = sum(dO * O)."""
+    rng = np.random.default_rng(77)
+    B, H, Hkv, N, d, r, m, dv = 2, 4, 2, 7, 5, 4, 6, 3
+    G = H // Hkv
+    Q, K, V = rng.standard_normal((B, H, N, d)), rng.standard_normal((B, Hkv, N, d)), rng.standard_normal((B, Hkv, N, dv))
+    M, W, dO = np.eye(r, d)[None] + 0.2 * rng.standard_normal((H, r, d)), rng.standard_normal((m, r)), rng.standard_normal((B, H, N, dv))
+    s2 = 1.0 / np.sqrt(d)
+    for causal in (False, True):
+        O = ref.forward(Q, K, V, M, W, causal=causal)
+        for b in range(B):
+            for h in range(H):
+                xq, xk = np.sqrt(s2) * Q[b, h] @ M[h].T, np.sqrt(s2) * K[b, h // G] @ M[h].T
+                fq = np.exp(xq @ W.T - 0.5 * (xq ** 2).sum(1, keepdims=True))
+                fk = np.exp(xk @ W.T - 0.5 * (xk ** 2).sum(1, keepdims=True))
+                Kh = fq @ fk.T
+                if causal:
+                    Kh = np.tril(Kh)
+                np.testing.assert_allclose(O[b, h], (Kh @ V[b, h // G]) / Kh.sum(1, keepdims=True), rtol=1e-10, atol=1e-12)
+        dQ, dK, dV, dM, dW = ref.backward(Q, K, V, M, W, dO, causal=causal)
+        assert dK.shape == K.shape and dV.shape == V.shape
+        loss = lambda K_, V_: float((dO * ref.forward(Q, K_, V_, M, W, causal=causal)).sum())
+        eps = 1e-6
+        for idx in [(0, 0, 0, 0), (1, 1, 3, 2), (0, 1, 6, 4)]:
+            Kp, Km = K.copy(), K.copy(); Kp[idx] += eps; Km[idx] -= eps
+            assert abs((loss(Kp, V) - loss(Km, V)) / (2 * eps) - dK[idx]) < 1e-6 * max(1.0, abs(dK[idx]))
+        for idx in [(0, 0, 0, 0), (1, 1, 3, 2), (1, 0, 6, 1)]:
+            Vp, Vm = V.copy(), V.copy(); Vp[idx] += eps; Vm[idx] -= eps
+            assert abs((loss(K, Vp) - loss(K, Vm)) / (2 * eps) - dV[idx]) < 1e-6 * max(1.0, abs(dV[idx]))

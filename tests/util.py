@@ -28,11 +28,13 @@ def run_gpu(binding, wl, t, path=0, chunk=0, scale=0.0, backward=None, w_per_hea
     r = t.M.shape[-2]
     m = t.W.shape[-2]
     dt = torch_dtype(wl.dtype)
+    Hkv = t.K.shape[1]                                    # fewer key/value heads than query heads: grouped heads
     plan = binding.darkattn_plan(Bq, Hq, N, d, m, r=r, dv=dv, dtype=binding.F32 if wl.dtype == "f32" else binding.BF16,
-                                 causal=wl.causal, chunk=chunk, scale=scale, w_per_head=w_per_head, path=path)
+                                 causal=wl.causal, chunk=chunk, scale=scale, w_per_head=w_per_head, path=path,
+                                 H_kv=0 if Hkv == Hq else Hkv)
     ws = plan.alloc_workspace()
     Q, K, V, M, W = (to_dev(x, dt) for x in (t.Q, t.K, t.V, t.M, t.W))
-    O = torch.empty_like(V)
+    O = torch.empty((Bq, Hq, N, dv), dtype=dt, device="cuda")     # (V may have fewer heads: grouped key/value heads)
     saved = None
     if use_saved and plan.saved_bytes:
         saved = torch.empty(plan.saved_bytes, dtype=torch.uint8, device="cuda")
