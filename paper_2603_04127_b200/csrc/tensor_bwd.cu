@@ -270,9 +270,11 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
         const bool g0 = (col0 == 0);                         // these 128 threads: row r also stands for feature r of the slab
         const uint32_t lane_addr = tmem + ((uint32_t)(q4 * 32) << 16);
         const uint32_t R1 = lane_addr + kColR1, R2 = lane_addr + kColR2;
+        // A wait that gave up (here or, seen through the abort flag, in another warp) switches the warp to a dry run: it skips
+        // every later wait but keeps walking the same chunks, so that every named barrier still gets all its arrivals.
         bool ok = true;
         int it = 0, run = 0;
-        for (long long l0 = lbeg; l0 < lend && ok; ++run) {
+        for (long long l0 = lbeg; l0 < lend; ++run) {
             const int bh = (int)(l0 / T), t0 = (int)(l0 % T);
             long long l1 = (long long)(bh + 1) * T;
             if (l1 > lend) l1 = lend;
@@ -282,12 +284,12 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
             const float cshift = load_key_shift(p.cs, bh * p.nslab + slab);
             if (g0) sZ[r] = (t0 > 0) ? __ldg(p.zc + ((size_t)bh * T + t0) * p.m + slab * 128 + r) : 0.f;
             epi_sync();
-            for (int c = 0; c < nrun && ok; ++c, ++it) {
+            for (int c = 0; c < nrun; ++c, ++it) {
                 const int t = t0 + c;
                 const uint32_t ph = it & 1;
                 const bool last = (c + 1 == nrun);
                 const size_t row = (size_t)row0 + (size_t)t * 128 + r;
-#define EWAIT(b) do { ok = __all_sync(0xffffffffu, wait_or_abort(bars + (b), ph, status, abort_flag)); } while (0)
+#define EWAIT(b) do { ok = ok && __all_sync(0xffffffffu, wait_or_abort(bars + (b), ph, status, abort_flag)); } while (0)
                 const float2 svv = p.sv[row];
                 const float del = p.delta[row];
                 const float aq = svv.y - cshift + log2f(svv.x);
@@ -299,7 +301,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                     for (int i = 0; i < 4; ++i) dtile[i] = -__ldg(p.delta + (size_t)row0 + (size_t)t * 128 + i * 32 + lane);
                 }
                 unsigned char *bX = ph ? sSt : sQA;          // this chunk's Q / A^ / E tile
-                EWAIT(QM1); if (!ok) break;
+                EWAIT(QM1);
                 tc_fence_after();
                 features_to_tile(lane_addr + kColState + col0, aq, bX, r, col0);           // A^
                 if (warp == 0) {
@@ -320,7 +322,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                 tc_fence_before();
                 mbar_arrive_warp(bars + QE1);
 
-                EWAIT(QM3); if (!ok) break;
+                EWAIT(QM3);
                 tc_fence_after();
                 {   // dP = tril(dO V^T - delta) as a bf16 operand in TMEM (packed over the fp32 tile)
                     uint32_t v[32], pk[16];
@@ -341,7 +343,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                 tc_fence_before();
                 mbar_arrive_warp(bars + QE2);
 
-                EWAIT(QM4); if (!ok) break;
+                EWAIT(QM4);
                 tc_fence_after();
                 if (g0) {       // rho_c of feature r (TMEM lane r; its MMAs ran ahead of dP Bf), for the key-side kernel
                     uint32_t v[16];
@@ -371,7 +373,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                 tc_fence_before();
                 mbar_arrive_warp(bars + QE3);
 
-                EWAIT(QM5); if (!ok) break;
+                EWAIT(QM5);
                 tc_fence_after();
                 {   // this slab's part of dQ: out of tensor memory, then (once T += E^T Q has read E) staged over E; the control
                     // thread adds the tile into dQ
@@ -380,7 +382,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                         tmem_ld32(R1 + col0, v);
                         tmem_wait_ld();
                     }
-                    EWAIT(QM6); if (!ok) break;
+                    EWAIT(QM6);
                     if (col0 < D) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(kLn2 * __uint_as_float(v[j]));
@@ -395,7 +397,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
 #undef EWAIT
             }
             // the run's T: every MMA of the run completed before its last T += E^T Q did
-            if (ok) ok = __all_sync(0xffffffffu, wait_or_abort(bars + QM6, (it - 1) & 1, status, abort_flag));
+            ok = ok && __all_sync(0xffffffffu, wait_or_abort(bars + QM6, (it - 1) & 1, status, abort_flag));
             if (ok) {
                 tc_fence_after();
                 if (col0 < D) {
@@ -570,19 +572,19 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
         const uint32_t lane_addr = tmem + ((uint32_t)(q4 * 32) << 16);
         const uint32_t R1 = lane_addr + kColR1, R2 = lane_addr + kColR2;
         const size_t rows = (size_t)p.BH * p.N;
-        bool ok = true;
-        for (int it = 0; it < T && ok; ++it) {
+        bool ok = true;     // (a wait that gave up switches the warp to a dry run over the remaining chunks: see the query-side kernel)
+        for (int it = 0; it < T; ++it) {
             const int t = T - 1 - it;
             const uint32_t ph = it & 1;
             const bool last = (it + 1 == T);
             const size_t row = (size_t)row0 + (size_t)t * 128 + r;
-#define EWAIT(b) do { ok = __all_sync(0xffffffffu, wait_or_abort(bars + (b), ph, status, abort_flag)); } while (0)
+#define EWAIT(b) do { ok = ok && __all_sync(0xffffffffu, wait_or_abort(bars + (b), ph, status, abort_flag)); } while (0)
             float rho_c = 0.f;
             if (g0) {
                 rho_c = p.rhoc[((size_t)bh * T + t) * p.m + slab * 128 + r];
                 sDel[r] = p.delta[row];
             }
-            EWAIT(KM3); if (!ok) break;
+            EWAIT(KM3);
             tc_fence_after();
             {   // dP^T = (V dO^T - delta_i) masked to queries i >= this key, packed over the fp32 tile
                 uint32_t v[32], pk[16];
@@ -598,7 +600,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
                 }
                 tmem_st16(R1 + col0 / 2, pk);
             }
-            EWAIT(KM4); if (!ok) break;
+            EWAIT(KM4);
             tc_fence_after();
             {   // P^^T masked the same way, packed behind dP^T
                 uint32_t v[32], pk[16];
@@ -616,14 +618,14 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
             tc_fence_before();
             mbar_arrive_warp(bars + KE2);
 
-            EWAIT(KM6); if (!ok) break;
+            EWAIT(KM6);
             tc_fence_after();
             if (col0 < DV) tmem_row_to_tile(R2 + col0, sStg, r, col0);      // this slab's part of dV, staged: the control thread adds it into dV
             fence_async_smem();
             tc_fence_before();
             mbar_arrive_warp(bars + KE3);
 
-            EWAIT(KM7); if (!ok) break;
+            EWAIT(KM7);
             tc_fence_after();
             {   // E = Bf .* (dP^T A^ + V R^T + rho^T), in place over Bf
                 float es = 0.f;
@@ -651,7 +653,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
             // while T += E^T K and E Omega run: R (updated behind the dV MMAs, its last reader V R^T done before E was formed) -> bf16 copy
             if (!last && col0 < DV) tmem_row_to_tile(lane_addr + kColState + col0, sSt, r, col0);
 
-            EWAIT(KM8); if (!ok) break;     // (T += E^T K, issued ahead of E Omega, has read the K tile in the spare tile)
+            EWAIT(KM8);     // (T += E^T K, issued ahead of E Omega, has read the K tile in the spare tile)
             tc_fence_after();
             if (col0 < D) tmem_row_to_tile(R2 + col0, sStg, r, col0, kLn2); // this slab's part of dK (without the norm term), staged: the control thread adds it into dK
             if (g0 && !last) sRho[r] += rho_c;      // rho_next for the chunk below (every reader of rho is past its E step)
@@ -660,7 +662,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
             mbar_arrive_warp(bars + KE5);
 #undef EWAIT
         }
-        if (ok) ok = wait_or_abort(bars + KM8, (T - 1) & 1, status, abort_flag);
+        ok = ok && wait_or_abort(bars + KM8, (T - 1) & 1, status, abort_flag);
         if (ok && col0 < D) {
             tc_fence_after();
             float *dst = p.Tacc + ((size_t)h * p.m + slab * 128 + r) * D + col0;
@@ -783,11 +785,11 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __gr
             return e;
         };
         float es_next = row_sum(t0);
-        for (int t = t0; t < t1 && ok; ++t) {
+        // (a wait that gave up switches the warp to a dry run over the remaining tiles, so that epi_sync still gets every arrival)
+        for (int t = t0; t < t1; ++t) {
             const uint32_t ph = (t - t0) & 1;
             const float coef = -p.s2 * es_next;
-            ok = __all_sync(0xffffffffu, wait_or_abort(m1, ph, p.status, abort_flag));
-            if (!ok) break;
+            ok = ok && __all_sync(0xffffffffu, wait_or_abort(m1, ph, p.status, abort_flag));
             tc_fence_after();
 #pragma unroll
             for (int hh = 0; hh < 2; ++hh) {
@@ -808,8 +810,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __gr
             mbar_arrive_warp(e1);
             if (t + 1 < t1) es_next = row_sum(t + 1);
 
-            ok = __all_sync(0xffffffffu, wait_or_abort(m2, ph, p.status, abort_flag));
-            if (!ok) break;
+            ok = ok && __all_sync(0xffffffffu, wait_or_abort(m2, ph, p.status, abort_flag));
             tc_fence_after();
             if (col0 < D) {
                 uint32_t v[32];

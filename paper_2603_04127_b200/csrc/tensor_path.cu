@@ -545,7 +545,10 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
         uint32_t *sOnes = reinterpret_cast<uint32_t *>(sRed);
         bool ok = true;
         float rmax = 0.f;                           // row maximum of the chunk whose phi(Q) was formed last
-#define EWAIT(b, q) do { ok = __all_sync(0xffffffffu, wait_or_abort(bars + (b), (q), status, abort_flag)); } while (0)
+// A wait that gave up (here or, seen through the abort flag, in another warp) switches the warp to a dry run: it skips
+// every later wait but keeps walking the same chunks, so that every named barrier below still gets all its arrivals and
+// no warp is left waiting for one that has gone (what it reads and writes from then on is garbage; the status word says so).
+#define EWAIT(b, q) do { ok = ok && __all_sync(0xffffffffu, wait_or_abort(bars + (b), (q), status, abort_flag)); } while (0)
         // phi(K): once the four warps of these rows are done with the exchanged maxima the array is filled with bf16 ones,
         // the B operand of z += phi(K)^T 1
         auto key_features = [&](float nk) {
@@ -565,32 +568,31 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
             mbar_arrive_warp(bars + CE0);
         };
         // the state through chunk t as the bf16 operand of phi(Q) S, once the staged output of chunk t has left the tile
-        auto copy_state = [&](int t) -> bool {
+        auto copy_state = [&](int t) {
             const uint32_t q = (t - tbeg) & 1;
-            EWAIT(CB_ST, q); if (!ok) return false;
-            EWAIT(CMS, q); if (!ok) return false;
+            EWAIT(CB_ST, q);
+            EWAIT(CMS, q);
             tc_fence_after();
             if (col0 < DV) tmem_row_to_tile(lane_addr + kColS + col0, sSb, r, col0);
             fence_async_smem();
             tc_fence_before();
             mbar_arrive_warp(bars + CE4);
-            return true;
         };
         EWAIT(CM1, 0);
-        if (ok) query_features();
+        query_features();
         float nk_next = p.nK[(size_t)row0 + (size_t)tbeg * 128 + r] + cshift;
-        for (int t = tbeg; t < tend && ok; ++t) {
+        for (int t = tbeg; t < tend; ++t) {
             const uint32_t ph = (t - tbeg) & 1;
             const bool last = (t + 1 == tend);
             const size_t prow = prow0 + (size_t)t * 128 + r;
             const float nk = nk_next;
             if (!last) nk_next = p.nK[(size_t)row0 + (size_t)(t + 1) * 128 + r] + cshift;     // needed a chunk from now
 
-            EWAIT(CM2, ph); if (!ok) break;
+            EWAIT(CM2, ph);
             key_features(nk);
-            if (t > tbeg && !copy_state(t - 1)) break;      // while P runs
+            if (t > tbeg) copy_state(t - 1);                // while P runs
 
-            EWAIT(CM3, ph); if (!ok) break;
+            EWAIT(CM3, ph);
             tc_fence_after();
             float rowsum = 0.f;
             {
@@ -611,7 +613,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
             tc_fence_before();
             mbar_arrive_warp(bars + CE2);
 
-            EWAIT(CM4, ph); if (!ok) break;         // the output tile; z through this chunk (its MMAs ran ahead of the output's)
+            EWAIT(CM4, ph);         // the output tile; z through this chunk (its MMAs ran ahead of the output's)
             tc_fence_after();
             if (col0 < DV) {
                 uint32_t v[32];
@@ -635,11 +637,11 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_causal_kernel(const __grid
             epi_sync();                             // every z is in place before anyone forms the next chunk's phi(Q)
 
             if (!last) {
-                EWAIT(CM1, ph ^ 1); if (!ok) break;
+                EWAIT(CM1, ph ^ 1);
                 query_features();
             }
         }
-        if (ok && copy_last) copy_state(tend - 1);
+        if (copy_last) copy_state(tend - 1);
 #undef EWAIT
     }
     if (*abort_flag) __nanosleep(200000);   // error path only: let copies and MMAs in flight drain
@@ -929,20 +931,19 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_queries_kernel(const __gri
         const float cshift = load_key_shift(p.cs, bh * p.nslab + slab);
         const size_t prow0 = ((size_t)slab * p.BH + bh) * p.N;
         bool ok = true;
-        for (int i = 0; i < n && ok; ++i) {
+        // (a wait that gave up switches the warp to a dry run over the remaining tiles: see the causal kernel)
+        for (int i = 0; i < n; ++i) {
             const int b = i & 1;
             const uint32_t phb = (i >> 1) & 1;
             const uint32_t R = lane_addr + (b ? kColR2 : kColR1);
             float rmax;
-            ok = __all_sync(0xffffffffu, wait_or_abort(bars + UM1_0 + b, phb, status, abort_flag));
-            if (!ok) break;
+            ok = ok && __all_sync(0xffffffffu, wait_or_abort(bars + UM1_0 + b, phb, status, abort_flag));
             tc_fence_after();
             const float dz = query_features_to_tmem<true>(R, lane_addr + b * 64, sRed, sZ, q4, g, r, col0, rmax);
             tc_fence_before();
             mbar_arrive_warp(bars + UE0_0 + b);
 
-            ok = __all_sync(0xffffffffu, wait_or_abort(bars + UM4_0 + b, phb, status, abort_flag));
-            if (!ok) break;
+            ok = ok && __all_sync(0xffffffffu, wait_or_abort(bars + UM4_0 + b, phb, status, abort_flag));
             tc_fence_after();
             uint32_t v[32];
             if (col0 < DV) {
