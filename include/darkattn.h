@@ -215,8 +215,14 @@ darkattn_status_t darkattn_kernel_times(darkattn_plan_t plan, int32_t max_entrie
  *    needs more than DARKATTN_STATIC_SCRATCH_BYTES is refused with DARKATTN_ERR_WORKSPACE before
  *    anything touches the GPU; use darkattn_forward with a workspace of your own for it.
  *  - The first call on each device looks up the array's device address (with that device current).
- *    Make that first call before any stream capture begins.
- *  - No cudaMalloc, cudaFree or other allocating routine is called, now or later.
+ *    Make that first call at start-up, before any stream capture begins and before the host's own pool
+ *    takes the rest of the GPU: under CUDA's default lazy module loading the driver only places the
+ *    array in device memory when its address is first asked for (or set CUDA_MODULE_LOADING=EAGER), so
+ *    this first call is the one that can still fail for lack of memory. The address is kept per
+ *    device; cudaDeviceReset invalidates it (the library is not meant to outlive a reset).
+ *  - No cudaMalloc, cudaFree or other allocating routine is called by the library, now or later.
+ *  - The status word of this call lives in the library's own array, out of reach of
+ *    darkattn_last_device_status: the FP32 kernels it runs never write one.
  *  - All calls on a device share the one array, and it keeps the previous call's contents; the call
  *    clears the words that must start at zero itself. Two calls whose GPU work overlaps (different
  *    streams, or different host threads) race on the array: serialise them on one stream.         */

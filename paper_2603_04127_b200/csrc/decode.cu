@@ -27,34 +27,43 @@ template <typename T, bool WITH_Q>
 __device__ __forceinline__ void token_features(const T *qv, const T *kv, const T *Mh, const T *Wh, float *xq, float *xk, float *fq,
                                                float *fk, float *red, int d, int r, int m, float s)
 {
-    const int tid = threadIdx.x;
-    for (int a = tid; a < r; a += 256) {            // x~ = s M x for the query and the key
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // x~ = s M x for the query and the key: one warp per row of M, its lanes along the row (coalesced), shuffle sum
+    for (int a = warp; a < r; a += 8) {
         float aq = 0.f, ak = 0.f;
-        for (int c = 0; c < d; ++c) {
+        for (int c = lane; c < d; c += 32) {
             const float mv = ldf(Mh, (size_t)a * d + c);
             if constexpr (WITH_Q) aq = fmaf(mv, ldf(qv, c), aq);
             ak = fmaf(mv, ldf(kv, c), ak);
         }
-        xq[a] = s * aq;
-        xk[a] = s * ak;
+        for (int off = 16; off; off >>= 1) {
+            if constexpr (WITH_Q) aq += __shfl_xor_sync(0xffffffffu, aq, off);
+            ak += __shfl_xor_sync(0xffffffffu, ak, off);
+        }
+        if (lane == 0) { xq[a] = s * aq; xk[a] = s * ak; }
     }
     __syncthreads();
     float nk = 0.f;
-    for (int a = 0; a < r; ++a) nk = fmaf(xk[a], xk[a], nk);
+    for (int a = lane; a < r; a += 32) nk = fmaf(xk[a], xk[a], nk);
+    for (int off = 16; off; off >>= 1) nk += __shfl_xor_sync(0xffffffffu, nk, off);
     nk *= 0.5f;
     float mx = -INFINITY;
-    for (int l = tid; l < m; l += 256) {            // exponents of the features
+    for (int l = warp; l < m; l += 8) {             // exponents of the features: one warp per row of W
         float uq = 0.f, uk = 0.f, c = 0.f;
-        for (int a = 0; a < r; ++a) {
+        for (int a = lane; a < r; a += 32) {
             const float w = ldf(Wh, (size_t)l * r + a);
             if constexpr (WITH_Q) uq = fmaf(w, xq[a], uq);
             uk = fmaf(w, xk[a], uk);
             c = fmaf(w, w, c);
         }
+        for (int off = 16; off; off >>= 1) {
+            if constexpr (WITH_Q) uq += __shfl_xor_sync(0xffffffffu, uq, off);
+            uk += __shfl_xor_sync(0xffffffffu, uk, off);
+            c += __shfl_xor_sync(0xffffffffu, c, off);
+        }
         c *= 0.5f;
-        fk[l] = __expf(uk - nk - c);
-        fq[l] = uq + c;
-        mx = fmaxf(mx, fq[l]);
+        if (lane == 0) { fk[l] = __expf(uk - nk - c); fq[l] = uq + c; }
+        mx = fmaxf(mx, uq + c);
     }
     if constexpr (WITH_Q) {
         for (int off = 16; off; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));

@@ -3,8 +3,8 @@
 A serving process that handed the whole GPU to its own memory pool, or a plug-in that only ever sees
 input and output buffers, has no workspace to give and must not call cudaMalloc. The static entry
 point keeps its intermediates in an array inside the library instead. These tests call it through
-the C ABI and hold it to the ordinary entry point's result, twice in a row because the array keeps
-the previous call's contents. The file sorts last on purpose, so a run that stops at the first
+the C ABI and hold it to the ordinary entry point's result and to the float64 oracle, twice in a row
+because the array keeps the previous call's contents. The file sorts last on purpose, so a run that stops at the first
 failure has already been through every other test.
 """
 import numpy as np
@@ -23,6 +23,14 @@ def binding():
     return b
 
 
+def _have_library():
+    import os
+    import shutil
+    here = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    return os.path.exists(os.path.join(here, "paper_2603_04127_b200", "libdarkattn.so")) or shutil.which("nvcc") or os.path.exists("/usr/local/cuda/bin/nvcc")
+
+
+@pytest.mark.skipif(not _have_library(), reason="neither libdarkattn.so nor nvcc to build it")
 def test_oversized_problem_is_refused_on_the_host(binding):
     plan = binding.darkattn_plan(4, 16, 8192, 128, 256, dtype=binding.BF16, causal=True)
     assert binding.darkattn_static_scratch_needed(plan) > binding.STATIC_SCRATCH_BYTES
@@ -48,6 +56,8 @@ def test_static_scratch_forward_matches_workspace_forward(binding, dtype, causal
     binding.darkattn_forward(plan, Q, K, V, M, W, want, ws)
     torch.cuda.synchronize()
     want = want.float().cpu().numpy()
+    from oracle import ref
+    exact = ref.forward(t.Q, t.K, t.V, t.M, t.W, causal=causal)
     for call in range(2):
         # the second call runs on a different problem's leftovers: swap queries and keys in between
         if call == 1:
@@ -60,4 +70,6 @@ def test_static_scratch_forward_matches_workspace_forward(binding, dtype, causal
         assert np.isfinite(got).all()
         fro, mx = rel_errors(got.astype(np.float64), want.astype(np.float64))
         assert fro < TOL[dtype] and mx < TOL[dtype], (call, fro, mx)
+        fro, mx = rel_errors(got.astype(np.float64), exact)          # and against the oracle, like every other entry point
+        assert fro < TOL[dtype] and mx < TOL[dtype], ("oracle", call, fro, mx)
     plan.destroy()
