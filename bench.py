@@ -313,7 +313,11 @@ def main():
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
     from paper_2603_04127_b200 import inputs
-    wl = inputs.WORKLOADS[args.workload]
+    workloads = dict(inputs.WORKLOADS)
+    # for profiler captures: the headline's per-head shape on fewer, shorter sequences, one CTA per SM (2 * 37 heads * 2 slabs
+    # = 148), inputs still larger than L2, small enough for a full counter capture
+    workloads["profile_small"] = inputs.Workload("profile_small", 3, 2, 37, 2048, 128, 256, "bf16", True, backward=True, rho=0.95)
+    wl = workloads[args.workload]
     if args.impl == "reference":
         run_reference(args, wl)
         return

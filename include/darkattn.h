@@ -100,11 +100,6 @@ size_t darkattn_saved_bytes(darkattn_plan_t plan);
 /* The path (DARKATTN_PATH_SIMT or DARKATTN_PATH_TENSOR) the plan resolved to.                   */
 int32_t darkattn_plan_path(darkattn_plan_t plan);
 
-/* Number of kernel launches one forward (which = 0) or one backward (which = 1) call enqueues
- * (backward: when it is given O and `saved`; otherwise the forward launches come on top), in the
- * plan's current mode: with per-kernel timing on, the tensor-core backward launches one fewer.   */
-int32_t darkattn_plan_launches(darkattn_plan_t plan, int32_t which);
-
 /* O = normalised random-feature attention (formulas at the top of this file).                   */
 darkattn_status_t darkattn_forward(darkattn_plan_t plan, const void *Q, const void *K, const void *V,
                                    const void *M, const void *W, void *O, void *saved /* nullable */,
@@ -165,38 +160,12 @@ const char *darkattn_last_cuda_error(void);
 darkattn_status_t darkattn_measure_alu_peak(int32_t which, int32_t iters, double *ops_per_second,
                                             void *cuda_stream);
 
-/* Measure what one tcgen05.mma (bf16, M = 128, K = 16) costs on this GPU in the forms the scan kernels
- * issue, so that their tensor-pipe time can be told apart from the hand-over between MMA batches and
- * the warps that consume them. variant: 0 both operands in shared memory, K-major, N = 128; 1 B MN-major;
- * 2 A and B MN-major; 3 A in tensor memory, B K-major; 4 A in tensor memory, B MN-major; 5 as 0 with
- * N = 256; 6 as 0 with N = 64; 7 A MN-major, N = 16. One CTA per SM issues two batches of dependent MMAs
- * (32 and 288) and waits for each batch's commit with a bounded wait; busy_epilogue != 0 makes the 16
- * other warps read tensor memory and write shared memory meanwhile. Writes the SM-clock cycles per MMA
- * (slope) and the fixed cycles per batch (intercept) to the two host pointers. Synchronises the
- * stream. DARKATTN_ERR_TIMEOUT if a commit did not arrive within the wait's limit.                 */
-darkattn_status_t darkattn_measure_mma_cycles(int32_t variant, int32_t busy_epilogue, double *cycles_per_mma,
-                                              double *batch_overhead_cycles, void *cuda_stream);
-
 /* Self-test of the bounded device-side wait the scan kernels rely on: launches one small kernel whose
  * only thread waits on a barrier nobody arrives on. The wait must give up after its limit (2 s),
  * record DARKATTN_ERR_TIMEOUT in a device status word and let the kernel end normally. Writes that
  * status word and the kernel's device time in seconds to the two host pointers; synchronises the
  * stream. Nothing faults, the context stays usable. Returns DARKATTN_OK when the launch itself ran. */
 darkattn_status_t darkattn_selftest_wait_limit(int32_t *device_status, double *seconds, void *cuda_stream);
-
-/* Per-kernel device times, for benchmarks. While enabled, forward and backward record a CUDA event on
- * the call's stream in front of every kernel they launch and one behind the last (events are host
- * objects created by the first enabling call; no device memory is involved). Enabling also clears the
- * accumulated times. Leave it off when measuring whole-call throughput.                           */
-darkattn_status_t darkattn_kernel_timing(darkattn_plan_t plan, int32_t enable);
-
-/* Wait for the events recorded since the last harvest, add the elapsed time between consecutive events
- * to the kernel in front of which the first was recorded, and report the totals since timing was
- * enabled: names (HOST buffer of 64 * max_entries bytes, one NUL-terminated name per 64 bytes),
- * total_ms and launches (HOST arrays of max_entries), *count = entries written. Call it at least once
- * per 96 kernels, since only that many events are kept.                                            */
-darkattn_status_t darkattn_kernel_times(darkattn_plan_t plan, int32_t max_entries, char *names, float *total_ms,
-                                        int32_t *launches, int32_t *count);
 
 /* Forward pass that needs no workspace from the caller and allocates nothing.
  *

@@ -21,11 +21,13 @@ PATH_AUTO, PATH_SIMT, PATH_TENSOR = 0, 1, 2
 
 EXPORTS = [
     "darkattn_plan", "darkattn_workspace_bytes", "darkattn_saved_bytes", "darkattn_plan_path",
-    "darkattn_plan_launches", "darkattn_forward", "darkattn_backward", "darkattn_last_device_status",
+    "darkattn_forward", "darkattn_backward", "darkattn_last_device_status",
     "darkattn_destroy", "darkattn_status_string", "darkattn_last_cuda_error", "darkattn_measure_alu_peak",
-    "darkattn_static_scratch_needed", "darkattn_forward_static", "darkattn_kernel_timing", "darkattn_kernel_times",
-    "darkattn_backward_dw", "darkattn_decode_step", "darkattn_measure_mma_cycles", "darkattn_selftest_wait_limit",
+    "darkattn_static_scratch_needed", "darkattn_forward_static",
+    "darkattn_backward_dw", "darkattn_decode_step", "darkattn_selftest_wait_limit",
 ]
+# instruments of the benchmark, in a library of their own (include/darkattn_bench.h)
+BENCH_EXPORTS = ["darkattn_plan_launches", "darkattn_kernel_timing", "darkattn_kernel_times", "darkattn_measure_mma_cycles"]
 STATIC_SCRATCH_BYTES = 16 << 20
 
 
@@ -50,8 +52,6 @@ lib.darkattn_saved_bytes.argtypes = [_vp]
 lib.darkattn_saved_bytes.restype = ctypes.c_size_t
 lib.darkattn_plan_path.argtypes = [_vp]
 lib.darkattn_plan_path.restype = ctypes.c_int32
-lib.darkattn_plan_launches.argtypes = [_vp, ctypes.c_int32]
-lib.darkattn_plan_launches.restype = ctypes.c_int32
 lib.darkattn_forward.argtypes = [_vp] * 10
 lib.darkattn_forward.restype = ctypes.c_int
 lib.darkattn_backward.argtypes = [_vp] * 15
@@ -70,20 +70,37 @@ lib.darkattn_last_cuda_error.argtypes = []
 lib.darkattn_last_cuda_error.restype = ctypes.c_char_p
 lib.darkattn_measure_alu_peak.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(ctypes.c_double), _vp]
 lib.darkattn_measure_alu_peak.restype = ctypes.c_int
-lib.darkattn_measure_mma_cycles.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(ctypes.c_double),
-                                            ctypes.POINTER(ctypes.c_double), _vp]
-lib.darkattn_measure_mma_cycles.restype = ctypes.c_int
 lib.darkattn_selftest_wait_limit.argtypes = [ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_double), _vp]
 lib.darkattn_selftest_wait_limit.restype = ctypes.c_int
-lib.darkattn_kernel_timing.argtypes = [_vp, ctypes.c_int32]
-lib.darkattn_kernel_timing.restype = ctypes.c_int
-lib.darkattn_kernel_times.argtypes = [_vp, ctypes.c_int32, ctypes.c_char_p, ctypes.POINTER(ctypes.c_float),
-                                      ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]
-lib.darkattn_kernel_times.restype = ctypes.c_int
 lib.darkattn_static_scratch_needed.argtypes = [_vp]
 lib.darkattn_static_scratch_needed.restype = ctypes.c_size_t
 lib.darkattn_forward_static.argtypes = [_vp] * 8
 lib.darkattn_forward_static.restype = ctypes.c_int
+
+
+BENCH_LIB_PATH = os.path.join(_HERE, "libdarkattn_bench.so")
+_benchlib = None
+
+
+def benchlib():
+    """The instruments' library (loaded on first use; the product calls above never need it)."""
+    global _benchlib
+    if _benchlib is None:
+        if not os.path.exists(BENCH_LIB_PATH):
+            raise ImportError(f"{BENCH_LIB_PATH} is missing: build it with `python -m paper_2603_04127_b200.build`")
+        b = ctypes.CDLL(BENCH_LIB_PATH)
+        b.darkattn_plan_launches.argtypes = [_vp, ctypes.c_int32]
+        b.darkattn_plan_launches.restype = ctypes.c_int32
+        b.darkattn_measure_mma_cycles.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(ctypes.c_double),
+                                                  ctypes.POINTER(ctypes.c_double), _vp]
+        b.darkattn_measure_mma_cycles.restype = ctypes.c_int
+        b.darkattn_kernel_timing.argtypes = [_vp, ctypes.c_int32]
+        b.darkattn_kernel_timing.restype = ctypes.c_int
+        b.darkattn_kernel_times.argtypes = [_vp, ctypes.c_int32, ctypes.c_char_p, ctypes.POINTER(ctypes.c_float),
+                                            ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]
+        b.darkattn_kernel_times.restype = ctypes.c_int
+        _benchlib = b
+    return _benchlib
 
 
 class DarkAttnError(RuntimeError):
@@ -119,7 +136,7 @@ class Plan:
         return int(lib.darkattn_plan_path(self.handle))
 
     def launches(self, backward: bool = False) -> int:
-        return int(lib.darkattn_plan_launches(self.handle, 1 if backward else 0))
+        return int(benchlib().darkattn_plan_launches(self.handle, 1 if backward else 0))
 
     def alloc_workspace(self, device="cuda") -> torch.Tensor:
         return torch.empty(max(self.workspace_bytes, 256), dtype=torch.uint8, device=device)
@@ -200,7 +217,7 @@ def darkattn_measure_alu_peak(which: int, iters: int = 20, stream=None) -> float
 def darkattn_measure_mma_cycles(variant: int, busy_epilogue: bool = False, stream=None):
     """(cycles per MMA, fixed cycles per batch) of one tcgen05.mma form; see the header for the variants."""
     per, fixed = ctypes.c_double(0.0), ctypes.c_double(0.0)
-    _check(lib.darkattn_measure_mma_cycles(variant, int(bool(busy_epilogue)), ctypes.byref(per), ctypes.byref(fixed),
+    _check(benchlib().darkattn_measure_mma_cycles(variant, int(bool(busy_epilogue)), ctypes.byref(per), ctypes.byref(fixed),
                                            _stream(stream)), "darkattn_measure_mma_cycles")
     return per.value, fixed.value
 
@@ -213,7 +230,7 @@ def darkattn_selftest_wait_limit(stream=None):
 
 
 def darkattn_kernel_timing(plan: Plan, enable: bool):
-    _check(lib.darkattn_kernel_timing(plan.handle, int(bool(enable))), "darkattn_kernel_timing")
+    _check(benchlib().darkattn_kernel_timing(plan.handle, int(bool(enable))), "darkattn_kernel_timing")
 
 
 def darkattn_kernel_times(plan: Plan, max_entries: int = 32) -> dict:
@@ -222,7 +239,7 @@ def darkattn_kernel_times(plan: Plan, max_entries: int = 32) -> dict:
     ms = (ctypes.c_float * max_entries)()
     cnt = (ctypes.c_int32 * max_entries)()
     n = ctypes.c_int32(0)
-    _check(lib.darkattn_kernel_times(plan.handle, max_entries, names, ms, cnt, ctypes.byref(n)), "darkattn_kernel_times")
+    _check(benchlib().darkattn_kernel_times(plan.handle, max_entries, names, ms, cnt, ctypes.byref(n)), "darkattn_kernel_times")
     out = {}
     for i in range(n.value):
         out[names.raw[64 * i:64 * (i + 1)].split(b"\0", 1)[0].decode()] = (float(ms[i]), int(cnt[i]))

@@ -9,15 +9,18 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 LIB = os.path.join(HERE, "libdarkattn.so")
+BENCH_LIB = os.path.join(HERE, "libdarkattn_bench.so")     # instruments of the benchmark (per-kernel times, MMA probe)
 SOURCES = sorted(glob.glob(os.path.join(HERE, "csrc", "*.cu")))
-HEADERS = sorted(glob.glob(os.path.join(HERE, "csrc", "*.cuh"))) + [os.path.join(ROOT, "include", "darkattn.h")]
+BENCH_SOURCES = sorted(glob.glob(os.path.join(HERE, "csrc_bench", "*.cu")))
+HEADERS = sorted(glob.glob(os.path.join(HERE, "csrc", "*.cuh"))) + [os.path.join(ROOT, "include", "darkattn.h"),
+                                                                     os.path.join(ROOT, "include", "darkattn_bench.h")]
 
 
 def stale() -> bool:
-    if not os.path.exists(LIB):
+    if not os.path.exists(LIB) or not os.path.exists(BENCH_LIB):
         return True
-    t = os.path.getmtime(LIB)
-    return any(os.path.getmtime(f) > t for f in SOURCES + HEADERS)
+    t = min(os.path.getmtime(LIB), os.path.getmtime(BENCH_LIB))
+    return any(os.path.getmtime(f) > t for f in SOURCES + BENCH_SOURCES + HEADERS)
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
@@ -31,17 +34,21 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if verbose:
         flags += ["-Xptxas", "-v"]
     # one object per translation unit, compiled side by side (only the stale ones), then one link
-    jobs, objs = [], []
+    jobs, objs, bench_objs = [], [], []
     newest_header = max(os.path.getmtime(h) for h in HEADERS)
-    for src in SOURCES:
-        obj = os.path.join(objdir, os.path.basename(src)[:-3] + ".o")
-        objs.append(obj)
+    for src in SOURCES + BENCH_SOURCES:
+        bench = src in BENCH_SOURCES
+        obj = os.path.join(objdir, ("bench_" if bench else "") + os.path.basename(src)[:-3] + ".o")
+        (bench_objs if bench else objs).append(obj)
         if force or not os.path.exists(obj) or os.path.getmtime(obj) < max(os.path.getmtime(src), newest_header):
             jobs.append((src, subprocess.Popen([nvcc] + flags + ["-c", src, "-o", obj])))
     failed = [src for src, pr in jobs if pr.wait() != 0]
     if failed:
         raise RuntimeError("nvcc failed for " + ", ".join(failed))
-    subprocess.run([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-Xcompiler", "-fPIC", "-o", LIB] + objs, check=True)
+    link = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-Xcompiler", "-fPIC"]
+    subprocess.run(link + ["-o", LIB] + objs, check=True)
+    # the instruments use the product's plan object and error reporting: linked against it, found beside it at run time
+    subprocess.run(link + ["-o", BENCH_LIB] + bench_objs + ["-L", HERE, "-l:libdarkattn.so", "-Xlinker", "-rpath=$ORIGIN"], check=True)
     return LIB
 
 

@@ -2,8 +2,9 @@
 // for the operand placements that occur (both operands in shared memory, K- or MN-major; A in tensor memory),
 // optionally with the 16 epilogue warps reading tensor memory and writing shared memory beside the MMAs.
 // One CTA per SM; one thread issues reps * 8 MMAs onto one accumulator, commits, and waits (bounded) for the commit.
-#include "common.cuh"
-#include "tc_common.cuh"
+#include "../csrc/common.cuh"
+#include "../csrc/tc_common.cuh"
+#include "darkattn_bench.h"
 
 namespace darkattn {
 

@@ -50,9 +50,6 @@ WORKLOADS = {
     "headline": Workload("headline", 3, 4, 16, 8192, 128, 256, "bf16", True, backward=True, rho=0.95),
     # the headline shape without the causal mask (bidirectional attention), forward + backward
     "headline_nc": Workload("headline_nc", 6, 4, 16, 8192, 128, 256, "bf16", False, backward=True, rho=0.95),
-    # the headline's per-head shape on fewer, shorter sequences: one CTA per SM (2 * 37 heads * 2 slabs = 148),
-    # inputs still larger than L2; small enough for a full profiler capture
-    "profile_small": Workload("profile_small", 3, 2, 37, 2048, 128, 256, "bf16", True, backward=True, rho=0.95),
 }
 
 

@@ -17,8 +17,8 @@ def binding():
     return b
 
 
-def _declared_symbols():
-    text = open(os.path.join(ROOT, "include", "darkattn.h")).read()
+def _declared_symbols(header="darkattn.h"):
+    text = open(os.path.join(ROOT, "include", header)).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     return sorted(set(re.findall(r"\b(darkattn_[a-z_0-9]+)\s*\(", text)))
 
@@ -30,6 +30,11 @@ def test_every_declared_symbol_is_exported(binding):
         assert hasattr(binding.lib, n), n
     assert sorted(binding.EXPORTS) == [n for n in names if n in binding.EXPORTS]
     assert set(names) == set(binding.EXPORTS)
+    # the instruments of the benchmark: their own header, their own library
+    bench = [n for n in _declared_symbols("darkattn_bench.h")]
+    assert set(bench) == set(binding.BENCH_EXPORTS)
+    for n in bench:
+        assert hasattr(binding.benchlib(), n) and not hasattr(binding.lib, n), n
 
 
 def test_plan_defaults_and_sizes(binding):
