@@ -14,12 +14,14 @@
 // (chain rule through the definitions of the feature map and of the attention; every stabilising
 // shift is a constant because the output does not depend on it).
 //
-// Two scan kernels walk the chunks of a sequence, one CTA per (batch, head, slab): the query-side
-// kernel forwards (state S in TMEM), the key-side kernel backwards (state R in TMEM). Features are
-// recomputed from Q, K and the folded projections and never leave the SM. The 128 x 128 tiles dP
-// (query side) and P^^T, dP^T (key side) are written back to tensor memory as bf16 and used as the
-// A operand of the next MMA directly from there. Slab partials of dQ, dK, dV go to the workspace in
-// bf16 and are summed by small kernels; the key-side one also applies the norm term with three MMAs.
+// Two scan kernels. The query-side kernel takes the state S before every chunk and the key features Bf from the
+// forward pass (bf16, through the stash), so its chunks are independent and spread evenly over the SMs; it forms
+// A^ again from Q and both halves of the folded projections and leaves it in the workspace for the key-side kernel,
+// which walks each (batch, head, slab) backwards with the state R in TMEM and reads A^ and Bf back. The 128 x 128
+// tiles dP (query side) and P^^T, dP^T (key side) are written back to tensor memory as bf16 and used as the A operand
+// of the next MMA directly from there. Each slab's parts of dQ, dK, dV are staged in a tile buffer that is free at
+// that point and added into the (zeroed) gradients by TMA reduce-add stores; a finishing kernel applies the norm
+// term of dK with three MMAs per tile.
 #include "common.cuh"
 #include "tc_common.cuh"
 
