@@ -134,18 +134,15 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
             const uint32_t id_dx = make_idesc(128, D, 0, 1);
             const uint32_t id_t = make_idesc(128, D, 1, 1);
             const uint32_t R1 = tmem + kColR1, R2 = tmem + kColR2;
-            // The Q tile that T += E^T Q needs is fetched again into the V tile's buffer as soon as dO V^T is done (where
-            // it fits), so that dO of the next chunk can follow early into its own buffer; otherwise into dO's buffer.
-            constexpr bool kQinV = (D <= DV);
-
-            // Schedule of one chunk (R1, R2, R3: scratch regions of TMEM). U_Q of the next chunk is issued in the tail of
-            // the current one, dO V^T runs while the epilogue warps are busy with A^, dO S^T while they mask dP.
+            // Schedule of one chunk (R1, R2, R3: scratch regions of TMEM). U_Q and dO V^T of the next chunk are issued in the
+            // tail of the current one.
             //   R3: U_Q -> (A^ read) -> U_Q of the next chunk
-            //   R2: dO V^T -> packed dP in [0,64) (A operand of dP Bf), rho_c in [64,80)
-            //   R1: dO S^T + dP Bf -> (E read) -> E Omega -> (dQ read)
-            // Two tile buffers swap roles from chunk to chunk: X holds Q, then A^, then E, then the staged dQ tile; S holds
-            // the state before the chunk. S is free first (after dO S^T) and takes the next chunk's Q, so that its
-            // projection can be issued in the tail; X is free last and takes the next chunk's state, which is needed late.
+            //   R2: dO V^T -> packed dP in [0,64) (A operand of dP Bf), rho_c in [64,80) -> dO V^T of the next chunk
+            //   R1: dP Bf + dO S^T -> (E read) -> E Omega -> (dQ read)
+            // Shared memory: X holds Q, then A^, then E, then the staged dQ tile, then the next chunk's state; S holds the
+            // state, then the next chunk's Q (the two swap roles from chunk to chunk); the Bf tile's buffer takes the Q tile
+            // again once dP Bf is done (T += E^T Q needs it) and the next chunk's Bf after that; V is free as soon as dO V^T
+            // has been read out, so the next chunk's V tile, the first thing that chunk needs, loads earliest.
             const uint32_t R3 = tmem + kColState;
             bool ok = true;
             int it = 0, run = 0;        // chunks and runs done so far: the parities of the barriers
@@ -183,12 +180,18 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                 load_state((it & 1) ? sQA : sSt, t0);
                 ok = wait_or_abort(bars + QB_OM, run & 1, status, abort_flag);
                 if (ok) ok = wait_or_abort(bars + QB_Q, it & 1, status, abort_flag);
-                if (ok && run > 0) ok = wait_or_abort(bars + QET, (run - 1) & 1, status, abort_flag);       // T of the previous run has been read out
                 if (ok) {
                     tc_fence_after();
                     const TileDesc &tX0 = (it & 1) ? tSt : tQA;
                     issue_projection<D>(R3, tX0, tOm, tOml, id_kk);                                              // U_Q of the run's first chunk
                     mma_commit(bars + QM1);
+                    ok = wait_or_abort(bars + QB_V, it & 1, status, abort_flag);
+                    if (ok) ok = wait_or_abort(bars + QB_G, it & 1, status, abort_flag);
+                }
+                if (ok) {
+                    tc_fence_after();
+                    _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R2, kdesc(tG, k), kdesc(tV, k), id_kk, k > 0);     // dO V^T of the run's first chunk
+                    mma_commit(bars + QM3);
                 }
                 for (int c = 0; c < nrun && ok; ++c, ++it) {
                     const int t = t0 + c;
@@ -197,46 +200,44 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                     unsigned char *bX = ph ? sSt : sQA, *bS = ph ? sQA : sSt;
                     const TileDesc &tX = ph ? tSt : tQA, &tS = ph ? tQA : tSt;
 #define QWAIT(b) do { ok = wait_or_abort(bars + (b), ph, status, abort_flag); } while (0)
-                    QWAIT(QB_V); if (!ok) break;
-                    QWAIT(QB_G); if (!ok) break;
-                    tc_fence_after();
-                    _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R2, kdesc(tG, k), kdesc(tV, k), id_kk, k > 0);     // dO V^T
-                    mma_commit(bars + QM3);
-                    if (!first) {
-                        QWAIT(QB_S); if (!ok) break;
-                        tc_fence_after();
-                        _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R1, kdesc(tG, k), kdesc(tS, k), id_kk, k > 0); // dO S_prev^T
-                    }
                     QWAIT(QE1); if (!ok) break;                                                                  // A^ in X, R3 read, -delta operand written
                     tma_store_2d(&p.mapAh, bX, slab * 128, row0 + t * 128);                                      // A^ kept for the key-side kernel
                     tma_store_2d(&p.mapAh, bX + 16384, slab * 128 + 64, row0 + t * 128);
                     tma_store_commit();
-                    QWAIT(QE2A); if (!ok) break;                                                                 // dO V^T read out of R2
-                    if (kQinV) load_tile(sV, &p.mapQ, bars + QB_X2, D, t);                                      // V is done with: Q again, for T
+                    QWAIT(QE2A); if (!ok) break;                                                                 // dO V^T read out of R2: V is done with
+                    if (!last) load_tile(sV, &p.mapV, bars + QB_V, DV, t + 1);
                     tc_fence_after();
                     _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R2 + 64, mndesc(tX, k), vecdesc(tDel, k), id_vec, k > 0);  // rho_c = -A^^T delta (columns 0, 1)
                     QWAIT(QE2); if (!ok) break;                                                                  // dP packed in R2
-                    if (first) { QWAIT(QB_S); if (!ok) break; }                                                  // (keeps the barrier's phases in step)
                     QWAIT(QB_B); if (!ok) break;
                     tc_fence_after();
-                    _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R1, R2 + k * 8, mndesc(tKB, k), id_tm, (!first) || k > 0);   // + dP Bf
+                    _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ts(R1, R2 + k * 8, mndesc(tKB, k), id_tm, k > 0);           // dP Bf
+                    QWAIT(QB_S); if (!ok) break;                                                                 // (for the first chunk the tile is loaded but not used)
+                    if (!first) {
+                        tc_fence_after();
+                        _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R1, kdesc(tG, k), kdesc(tS, k), id_kk, 1);     // + dO S_prev^T
+                    }
                     tma_store_wait_read();      // the A^ tile has left shared memory: E may overwrite it
                     mma_commit(bars + QM4);
-                    QWAIT(QM4); if (!ok) break;                                                                  // Bf, V, dO and S of this chunk are done with
-                    if (!kQinV) load_tile(sG, &p.mapQ, bars + QB_X2, D, t);                                     // Q again, for T
+                    QWAIT(QM4); if (!ok) break;                                                                  // Bf, dO and S of this chunk are done with
+                    load_tile(sKB, &p.mapQ, bars + QB_X2, D, t);                                                // Q again, for T, where Bf was
                     if (!last) {
-                        if (kQinV) load_tile(sG, &p.mapG, bars + QB_G, DV, t + 1);
-                        else load_tile(sV, &p.mapV, bars + QB_V, DV, t + 1);
-                        load_key_features(t + 1);
+                        load_tile(sG, &p.mapG, bars + QB_G, DV, t + 1);
                         load_tile(bS, &p.mapQ, bars + QB_Q, D, t + 1);                                          // the state tile is done with: the next chunk's Q
+                        for (int a = 0; a < DV / 64; ++a)                                                        // into L2 now: the next state's load can only be issued at the chunk's very end
+                            tma_prefetch_l2_2d(&p.mapSst, a * 64, (bh * T + t + 1) * p.m + slab * 128);
                     }
                     QWAIT(QE3); if (!ok) break;
                     tc_fence_after();
                     _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(R1, kdesc(tX, k), mndesc(tOm, k), id_dx, k > 0);         // E Omega
                     mma_commit(bars + QM5);
                     QWAIT(QB_X2); if (!ok) break;
+                    if (c == 0 && run > 0) {                                                                     // T of the previous run has been read out
+                        ok = wait_or_abort(bars + QET, (run - 1) & 1, status, abort_flag);
+                        if (!ok) break;
+                    }
                     tc_fence_after();
-                    _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColT, mndesc(tX, k), mndesc(kQinV ? tV : tG, k), id_t, (c > 0) || k > 0);   // T += E^T Q
+                    _Pragma("unroll") for (int k = 0; k < 8; ++k) mma_ss(tmem + kColT, mndesc(tX, k), mndesc(tKB, k), id_t, (c > 0) || k > 0);   // T += E^T Q
                     mma_commit(bars + QM6);
                     if (!last) {
                         ok = wait_or_abort(bars + QB_Q, ph ^ 1, status, abort_flag);
@@ -244,12 +245,15 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                         tc_fence_after();
                         issue_projection<D>(R3, tS, tOm, tOml, id_kk);                                           // U_Q of the next chunk (its Q sits in S)
                         mma_commit(bars + QM1);
+                        ok = wait_or_abort(bars + QB_V, ph ^ 1, status, abort_flag);
+                        if (ok) ok = wait_or_abort(bars + QB_G, ph ^ 1, status, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        _Pragma("unroll") for (int k = 0; k < DV / 16; ++k) mma_ss(R2, kdesc(tG, k), kdesc(tV, k), id_kk, k > 0); // dO V^T of the next chunk
+                        mma_commit(bars + QM3);
                     }
-                    QWAIT(QM6); if (!ok) break;
-                    if (!last) {
-                        if (kQinV) load_tile(sV, &p.mapV, bars + QB_V, DV, t + 1);
-                        else load_tile(sG, &p.mapG, bars + QB_G, DV, t + 1);
-                    }
+                    QWAIT(QM6); if (!ok) break;                                                                  // the Q tile is done with:
+                    if (!last) load_key_features(t + 1);                                                         // the next chunk's Bf
                     QWAIT(QE4); if (!ok) break;                                                                  // this slab's part of dQ is staged where E was
                     for (int a = 0; a < D / 64; ++a) {
                         if (p.nslab > 1) tma_reduce_add_2d(&p.mapDQ, bX + a * 16384, a * 64, row0 + t * 128);
@@ -285,6 +289,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
             const int h = bh % p.H, row0 = bh * p.N;
             const float cshift = load_key_shift(p.cs, bh * p.nslab + slab);
             if (g0) sZ[r] = (t0 > 0) ? __ldg(p.zc + ((size_t)bh * T + t0) * p.m + slab * 128 + r) : 0.f;
+            float2 svv_next = p.sv[(size_t)row0 + (size_t)t0 * 128 + r];
+            float del_next = p.delta[(size_t)row0 + (size_t)t0 * 128 + r];
             epi_sync();
             for (int c = 0; c < nrun; ++c, ++it) {
                 const int t = t0 + c;
@@ -292,8 +298,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_q_kernel(const __grid_cons
                 const bool last = (c + 1 == nrun);
                 const size_t row = (size_t)row0 + (size_t)t * 128 + r;
 #define EWAIT(b) do { ok = ok && __all_sync(0xffffffffu, wait_or_abort(bars + (b), ph, status, abort_flag)); } while (0)
-                const float2 svv = p.sv[row];
-                const float del = p.delta[row];
+                const float2 svv = svv_next;                 // (loaded a chunk ahead: their latency is off the chunk's critical path)
+                const float del = del_next;
+                if (!last) { svv_next = p.sv[row + 128]; del_next = p.delta[row + 128]; }
                 const float aq = svv.y - cshift + log2f(svv.x);
                 // z before the next chunk, from the forward pass (loaded early, used at the end of the chunk)
                 const float znext = (g0 && !last) ? __ldg(p.zc + ((size_t)bh * T + t + 1) * p.m + slab * 128 + r) : 0.f;
