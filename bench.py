@@ -88,8 +88,7 @@ def kernel_work(d, r, m, dv, C, nslab, causal):
         "tc_bwd_nc_q_kernel": (feat // 2 + 4 * m * dv + 2 * m * r + 4 * r * d, m, (2 * d + dv) * e, "tensor"),
         "tc_bwd_nc_k_kernel": (feat // 2 + 4 * m * dv + 2 * m * r + 4 * r * d, m, (2 * d + 2 * dv) * e, "tensor"),
         "tc_bwd_finish_k_kernel": (6 * r * d, 0, 3 * d * e, "hbm"),
-        "tc_key_norms_kernel": (2 * r * d, 0, d * e + 4, "hbm"),
-        "tc_key_shift_kernel": (2 * d * m, 0, d * e + 4, "hbm"),
+        "tc_key_prepass_kernel": (2 * r * d + 2 * d * m, 0, d * e + 4, "hbm"),
         "combine_kernel": (0, 0, (nslab * dv + dv) * e + nslab * 32, "hbm"),
         "delta_kernel": (0, 0, 2 * dv * e + 4, "hbm"),
     }

@@ -36,18 +36,21 @@ constexpr float kShiftHeadroom = 64.f;
 
 // ------------------------------------------------------------------ prologue kernels (SIMT, tiny)
 // Omega[h,l,c] = log2(e) * s * sum_a W[l,a] M[h,a,c], stored as its bf16 rounding Om and the bf16 rounding Oml of what
-// that left out (Om + Oml carries 16 bits of Omega). One block per (head, 4 rows l), one thread per column c
+// that left out (Om + Oml carries 16 bits of Omega). One block per (head, 16 rows l), one thread per column c
 // (the block has d threads); many small blocks, because the kernel is bound by the latency of its loads.
 __global__ void fold_omega_kernel(const __nv_bfloat16 *W, const __nv_bfloat16 *M, __nv_bfloat16 *Om, __nv_bfloat16 *Oml, int m, int r,
                                   int d, int w_per_head, float coef)
 {
-    __shared__ __align__(16) float sw[4][128];
-    const int h = blockIdx.y, l0 = blockIdx.x * 4, c = threadIdx.x;
+    constexpr int R = 16;                           // rows l per block: every loaded element of M serves 16 products
+    __shared__ __align__(16) float sw[R][128];
+    const int h = blockIdx.y, l0 = blockIdx.x * R, c = threadIdx.x;
     const __nv_bfloat16 *w = W + ((size_t)(w_per_head ? h : 0) * m + l0) * r;
-    for (int i = threadIdx.x; i < 4 * r; i += blockDim.x) sw[i / r][i % r] = __bfloat162float(w[i]);
+    for (int i = threadIdx.x; i < R * r; i += blockDim.x) sw[i / r][i % r] = __bfloat162float(w[i]);
     __syncthreads();
     const __nv_bfloat16 *Mh = M + (size_t)h * r * d;
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    float acc[R];
+#pragma unroll
+    for (int i = 0; i < R; ++i) acc[i] = 0.f;
     for (int a0 = 0; a0 < r; a0 += 16) {            // r is a multiple of 16; 16 independent loads in flight
         __nv_bfloat16 mv[16];
 #pragma unroll
@@ -57,14 +60,14 @@ __global__ void fold_omega_kernel(const __nv_bfloat16 *W, const __nv_bfloat16 *M
             const float x0 = __bfloat162float(mv[j]), x1 = __bfloat162float(mv[j + 1]);
             const float x2 = __bfloat162float(mv[j + 2]), x3 = __bfloat162float(mv[j + 3]);
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
+            for (int i = 0; i < R; ++i) {
                 const float4 wv = *reinterpret_cast<const float4 *>(&sw[i][a0 + j]);   // one broadcast load per four products
                 acc[i] = fmaf(wv.x, x0, fmaf(wv.y, x1, fmaf(wv.z, x2, fmaf(wv.w, x3, acc[i]))));
             }
         }
     }
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < R; ++i) {
         const float om = coef * acc[i];
         const __nv_bfloat16 hi = __float2bfloat16_rn(om);
         Om[((size_t)h * m + l0 + i) * d + c] = hi;
@@ -72,191 +75,163 @@ __global__ void fold_omega_kernel(const __nv_bfloat16 *W, const __nv_bfloat16 *M
     }
 }
 
-// Start value of the key-side shifts, which tc_key_shift_kernel raises to the maximum over the keys: the smallest order key.
+// Start value of the key-side shifts, which tc_key_prepass_kernel raises to the maximum over the keys: the smallest order key.
 __global__ void shift_init_kernel(int *cs, int n)
 {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) cs[i] = (int)0x80000000u;
 }
 
-// ------------------------------------------------------------------ key norms: n[bh,j] = coef * |M_h k_j|^2
-struct NormParams {
-    CUtensorMap mapK, mapM;
-    float *nK;
+// ------------------------------------------------------------------ key prepass: norms and key-side shifts in one pass over K
+//   n[bh,j]     = coef * |M_h k_j|^2                                   (log2 units; written by the CTAs of the first slab pair)
+//   c[bh,slab]  = max_j max_{l in slab} (u_jl - n_j) - kShiftHeadroom   u = K Omega_hi^T
+// The stabiliser of the key features is the largest exponent any key of the (batch, head) reaches in the slab, taken
+// from the data (with it the largest key feature is 2^kShiftHeadroom, whatever the norms of the keys); being one constant per
+// (batch, head, slab) it cancels in O. One CTA per (batch, head, pair of slabs, piece of the sequence): K tiles by TMA into
+// two buffers, x~ = K M^T and U = K Omega_slab^T on the tensor cores, squared norms and row maxima read out of tensor memory
+// by four warps (x~ of tile t + 1 is computed while U of tile t is read), the piece's maxima by atomicMax on order keys.
+struct PrepassParams {
+    CUtensorMap mapK, mapM, mapOm;
+    float *nK;           // [BH, N] key norms, log2 units
+    int *cs;             // [BH, nslab] order keys of the shifts
     int *status;
-    int N, H, Hkv, T, nsplit, r;
-    float coef;   // log2(e) * s^2 / 2
+    int N, H, Hkv, T, m, r, nslab, npair, nsplit;
+    float coef;          // log2(e) * s^2 / 2
 };
 
+enum PBars { PB_M, PB_K0, PB_K1, PMX, PMU, PEX, PEU, PNBARS };
+
 template <int D>
-__global__ void __launch_bounds__(160, 1) tc_key_norms_kernel(const __grid_constant__ NormParams p)
+__global__ void __launch_bounds__(160, 1) tc_key_prepass_kernel(const __grid_constant__ PrepassParams p)
 {
     extern __shared__ __align__(1024) unsigned char smem[];
     constexpr int kTile = 128 * D * 2;
-    unsigned char *sM = smem, *sK = smem + kTile;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + 2 * kTile);
-    uint64_t *bar_m = bars, *bar_k = bars + 1, *bar_u = bars + 2, *bar_e = bars + 3;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 4);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 5);
+    unsigned char *sM = smem, *sOm = smem + kTile, *sK = smem + 3 * kTile;       // M, two slabs of Omega, two K buffers
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + 5 * kTile);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + PNBARS);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + PNBARS + 1);
     const int tid = threadIdx.x, warp = tid >> 5;
-    const int bh = blockIdx.x / p.nsplit, split = blockIdx.x % p.nsplit, h = bh % p.H;
+    const int unit = blockIdx.x / p.nsplit, split = blockIdx.x % p.nsplit;
+    const int bh = unit / p.npair, pair = unit % p.npair, h = bh % p.H;
+    const int slab0 = 2 * pair, ns = (slab0 + 1 < p.nslab) ? 2 : 1;           // this CTA's one or two slabs
     const int t0 = (int)((long long)p.T * split / p.nsplit), t1 = (int)((long long)p.T * (split + 1) / p.nsplit);
+    const int rowk0 = kv_row0(bh, p.H, p.Hkv, p.N);
     if (tid == 0) {
-        mbar_init(bar_m, 1); mbar_init(bar_k, 1); mbar_init(bar_u, 1); mbar_init(bar_e, 128);
+        for (int i = 0; i < PEX; ++i) mbar_init(bars + i, 1);
+        mbar_init(bars + PEX, 128); mbar_init(bars + PEU, 128);
         *abort_flag = (smem_u32(smem) & 1023u) ? 1 : 0;
         fence_mbar_init();
     }
-    if (warp == 4) { tmem_alloc(tmem_slot, 128); tmem_relinquish(); }
+    if (warp == 4) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    constexpr uint32_t kColX = 0, kColU = 128;      // x~ at 0, U of the two slabs at 128 and 256
     if (*abort_flag) { if (tid == 0) atomicExch(p.status, (int)DARKATTN_ERR_CUDA); }
     else if (warp == 4) {
         if ((tid & 31) == 0 && t1 > t0) {
-            mbar_expect_tx(bar_m, kTile);
-            for (int a = 0; a < D / 64; ++a) tma_load_2d(sM + a * 16384, &p.mapM, bar_m, a * 64, h * p.r);
-            mbar_expect_tx(bar_k, kTile);
-            for (int a = 0; a < D / 64; ++a) tma_load_2d(sK + a * 16384, &p.mapK, bar_k, a * 64, kv_row0(bh, p.H, p.Hkv, p.N) + t0 * 128);
-            const uint32_t idesc = make_idesc(128, p.r, 0, 0);
-            bool ok = wait_or_abort(bar_m, 0, p.status, abort_flag);
+            auto load_k = [&](int t) {
+                const int b = (t - t0) & 1;
+                mbar_expect_tx(bars + PB_K0 + b, kTile);
+                for (int a = 0; a < D / 64; ++a) tma_load_2d(sK + b * kTile + a * 16384, &p.mapK, bars + PB_K0 + b, a * 64, rowk0 + t * 128);
+            };
+            mbar_expect_tx(bars + PB_M, kTile * (1 + ns));
+            for (int a = 0; a < D / 64; ++a) {
+                tma_load_2d(sM + a * 16384, &p.mapM, bars + PB_M, a * 64, h * p.r);
+                for (int s = 0; s < ns; ++s) tma_load_2d(sOm + s * kTile + a * 16384, &p.mapOm, bars + PB_M, a * 64, h * p.m + (slab0 + s) * 128);
+            }
+            load_k(t0);
+            if (t0 + 1 < t1) load_k(t0 + 1);
+            const TileDesc tM(sM), tOm0(sOm), tOm1(sOm + kTile), tK0(sK), tK1(sK + kTile);
+            const uint32_t id_x = make_idesc(128, p.r, 0, 0), id_u = make_idesc(128, 128, 0, 0);
+            bool ok = wait_or_abort(bars + PB_M, 0, p.status, abort_flag);
             for (int t = t0; t < t1 && ok; ++t) {
-                const uint32_t ph = (t - t0) & 1;
-                ok = wait_or_abort(bar_k, ph, p.status, abort_flag);
-                if (ok && t > t0) ok = wait_or_abort(bar_e, ph ^ 1, p.status, abort_flag);
+                const int i = t - t0, b = i & 1;
+                const uint32_t ph = i & 1, phk = (i >> 1) & 1;
+                const TileDesc &tK = b ? tK1 : tK0;
+                ok = wait_or_abort(bars + PB_K0 + b, phk, p.status, abort_flag);
+                if (ok && i > 0) ok = wait_or_abort(bars + PEX, ph ^ 1, p.status, abort_flag);       // x~ of the tile before has been read
                 if (!ok) break;
                 tc_fence_after();
-                for (int k = 0; k < D / 16; ++k)
-                    mma_ss(tmem, make_sdesc(smem_u32(sK) + (k / 4) * 16384 + (k % 4) * 32, 16, 1024),
-                           make_sdesc(smem_u32(sM) + (k / 4) * 16384 + (k % 4) * 32, 16, 1024), idesc, k > 0);
-                mma_commit(bar_u);
-                if (t + 1 < t1) {
-                    ok = wait_or_abort(bar_u, ph, p.status, abort_flag);
+                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(tmem + kColX, kdesc(tK, k), kdesc(tM, k), id_x, k > 0);
+                mma_commit(bars + PMX);
+                if (i > 0) { ok = wait_or_abort(bars + PEU, ph ^ 1, p.status, abort_flag); if (!ok) break; }      // U of the tile before has been read
+                tc_fence_after();
+                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(tmem + kColU, kdesc(tK, k), kdesc(tOm0, k), id_u, k > 0);
+                if (ns == 2)
+                    _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(tmem + kColU + 128, kdesc(tK, k), kdesc(tOm1, k), id_u, k > 0);
+                mma_commit(bars + PMU);
+                if (t + 2 < t1) {       // this tile's buffer is free once its MMAs are done
+                    ok = wait_or_abort(bars + PMU, ph, p.status, abort_flag);
                     if (!ok) break;
-                    mbar_expect_tx(bar_k, kTile);
-                    for (int a = 0; a < D / 64; ++a)
-                        tma_load_2d(sK + a * 16384, &p.mapK, bar_k, a * 64, kv_row0(bh, p.H, p.Hkv, p.N) + (t + 1) * 128);
+                    load_k(t + 2);
                 }
             }
         }
     } else {
         const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+        float best0 = -INFINITY, best1 = -INFINITY;
+        bool ok = true;
         for (int t = t0; t < t1; ++t) {
             const uint32_t ph = (t - t0) & 1;
-            if (!wait_or_abort(bar_u, ph, p.status, abort_flag)) break;
+            ok = __all_sync(0xffffffffu, wait_or_abort(bars + PMX, ph, p.status, abort_flag));
+            if (!ok) break;
             tc_fence_after();
             float acc = 0.f;
             for (int c0 = 0; c0 < p.r; c0 += 16) {
                 uint32_t v[16];
-                tmem_ld16(lane_addr + c0, v);
+                tmem_ld16(lane_addr + kColX + c0, v);
                 tmem_wait_ld();
 #pragma unroll
                 for (int j = 0; j < 16; ++j) { const float x = __uint_as_float(v[j]); acc = fmaf(x, x, acc); }
             }
             tc_fence_before();
-            mbar_arrive(bar_e);
-            p.nK[(size_t)bh * p.N + (size_t)t * 128 + tid] = p.coef * acc;
-        }
-    }
-    tc_fence_before();
-    __syncthreads();
-    if (warp == 4) tmem_dealloc(tmem, 128);
-}
-
-// ------------------------------------------------------------------ key-side shift: c[bh,slab] = max_j max_{l in slab} (u_jl - n_j)
-// The stabiliser of the key features is the largest exponent any key of the (batch, head) reaches in the slab, taken
-// from the data (with it the largest key feature is 2^kShiftHeadroom, whatever the norms of the keys); being one constant per
-// (batch, head, slab) it cancels in O. One CTA per (batch, head, slab, piece of the sequence): K tile by TMA,
-// U = K Omega_slab^T on the tensor cores, row maxima read out of tensor memory, the piece's maximum by atomicMax.
-struct ShiftParams {
-    CUtensorMap mapK, mapOm;
-    const float *nK;     // [BH, N] key norms, log2 units
-    int *cs;             // [BH, nslab] order keys of the shifts
-    int *status;
-    int N, H, Hkv, T, m, nslab, nsplit;
-};
-
-template <int D>
-__global__ void __launch_bounds__(160, 1) tc_key_shift_kernel(const __grid_constant__ ShiftParams p)
-{
-    extern __shared__ __align__(1024) unsigned char smem[];
-    constexpr int kTile = 128 * D * 2;
-    unsigned char *sOm = smem, *sK = smem + kTile;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + 2 * kTile);
-    uint64_t *bar_m = bars, *bar_k = bars + 1, *bar_u = bars + 2, *bar_e = bars + 3;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 4);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 5);
-    const int tid = threadIdx.x, warp = tid >> 5;
-    const int unit = blockIdx.x / p.nsplit, split = blockIdx.x % p.nsplit;
-    const int bh = unit / p.nslab, slab = unit % p.nslab, h = bh % p.H;
-    const int t0 = (int)((long long)p.T * split / p.nsplit), t1 = (int)((long long)p.T * (split + 1) / p.nsplit);
-    if (tid == 0) {
-        mbar_init(bar_m, 1); mbar_init(bar_k, 1); mbar_init(bar_u, 1); mbar_init(bar_e, 128);
-        *abort_flag = (smem_u32(smem) & 1023u) ? 1 : 0;
-        fence_mbar_init();
-    }
-    if (warp == 4) { tmem_alloc(tmem_slot, 128); tmem_relinquish(); }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem = *tmem_slot;
-    if (*abort_flag) { if (tid == 0) atomicExch(p.status, (int)DARKATTN_ERR_CUDA); }
-    else if (warp == 4) {
-        if ((tid & 31) == 0 && t1 > t0) {
-            mbar_expect_tx(bar_m, kTile);
-            for (int a = 0; a < D / 64; ++a) tma_load_2d(sOm + a * 16384, &p.mapOm, bar_m, a * 64, h * p.m + slab * 128);
-            mbar_expect_tx(bar_k, kTile);
-            for (int a = 0; a < D / 64; ++a) tma_load_2d(sK + a * 16384, &p.mapK, bar_k, a * 64, kv_row0(bh, p.H, p.Hkv, p.N) + t0 * 128);
-            const TileDesc tOm(sOm), tK(sK);
-            const uint32_t idesc = make_idesc(128, 128, 0, 0);
-            bool ok = wait_or_abort(bar_m, 0, p.status, abort_flag);
-            for (int t = t0; t < t1 && ok; ++t) {
-                const uint32_t ph = (t - t0) & 1;
-                ok = wait_or_abort(bar_k, ph, p.status, abort_flag);
-                if (ok && t > t0) ok = wait_or_abort(bar_e, ph ^ 1, p.status, abort_flag);       // the tile before has been read out
-                if (!ok) break;
-                tc_fence_after();
-                _Pragma("unroll") for (int k = 0; k < D / 16; ++k) mma_ss(tmem, kdesc(tK, k), kdesc(tOm, k), idesc, k > 0);
-                mma_commit(bar_u);
-                if (t + 1 < t1) {
-                    ok = wait_or_abort(bar_u, ph, p.status, abort_flag);
-                    if (!ok) break;
-                    mbar_expect_tx(bar_k, kTile);
-                    for (int a = 0; a < D / 64; ++a) tma_load_2d(sK + a * 16384, &p.mapK, bar_k, a * 64, kv_row0(bh, p.H, p.Hkv, p.N) + (t + 1) * 128);
-                }
-            }
-        }
-    } else {
-        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
-        float best = -INFINITY;
-        bool ok = true;
-        for (int t = t0; t < t1; ++t) {
-            const uint32_t ph = (t - t0) & 1;
-            const float nk = p.nK[(size_t)bh * p.N + (size_t)t * 128 + tid];
-            ok = __all_sync(0xffffffffu, wait_or_abort(bar_u, ph, p.status, abort_flag));
+            mbar_arrive(bars + PEX);
+            const float nk = p.coef * acc;
+            if (pair == 0) p.nK[(size_t)bh * p.N + (size_t)t * 128 + tid] = nk;
+            ok = __all_sync(0xffffffffu, wait_or_abort(bars + PMU, ph, p.status, abort_flag));
             if (!ok) break;
             tc_fence_after();
-            float mx = -INFINITY;
+            float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
             for (int c0 = 0; c0 < 128; c0 += 32) {
                 uint32_t v[32];
-                tmem_ld32(lane_addr + c0, v);
+                tmem_ld32(lane_addr + kColU + c0, v);
                 tmem_wait_ld();
 #pragma unroll
-                for (int j = 0; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(v[j]));
+                for (int j = 0; j < 32; ++j) mx0 = fmaxf(mx0, __uint_as_float(v[j]));
+            }
+            if (ns == 2) {
+#pragma unroll
+                for (int c0 = 0; c0 < 128; c0 += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(lane_addr + kColU + 128 + c0, v);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) mx1 = fmaxf(mx1, __uint_as_float(v[j]));
+                }
             }
             tc_fence_before();
-            mbar_arrive(bar_e);
-            best = fmaxf(best, mx - nk);
+            mbar_arrive(bars + PEU);
+            best0 = fmaxf(best0, mx0 - nk);
+            best1 = fmaxf(best1, mx1 - nk);
         }
         if (ok && t1 > t0) {
-            for (int o = 16; o; o >>= 1) best = fmaxf(best, __shfl_xor_sync(0xffffffffu, best, o));
-            if ((tid & 31) == 0) atomicMax(p.cs + bh * p.nslab + slab, float_order_key(best - kShiftHeadroom));
+            for (int o = 16; o; o >>= 1) {
+                best0 = fmaxf(best0, __shfl_xor_sync(0xffffffffu, best0, o));
+                best1 = fmaxf(best1, __shfl_xor_sync(0xffffffffu, best1, o));
+            }
+            if ((tid & 31) == 0) {
+                atomicMax(p.cs + bh * p.nslab + slab0, float_order_key(best0 - kShiftHeadroom));
+                if (ns == 2) atomicMax(p.cs + bh * p.nslab + slab0 + 1, float_order_key(best1 - kShiftHeadroom));
+            }
         }
     }
+    if (*abort_flag) __nanosleep(200000);
     tc_fence_before();
     __syncthreads();
-    if (warp == 4) tmem_dealloc(tmem, 128);
+    if (warp == 4) tmem_dealloc(tmem, 512);
 }
 
 // ------------------------------------------------------------------ the main kernel
@@ -1173,7 +1148,7 @@ void tensor_make_layout(darkattn_plan_s *plan)
     Y.Sb = take(off, BH * nstate * m * dv * 2);
     Y.sv = take(off, BH * N * 8);
     Y.zc = take(off, D.causal ? BH * (size_t)Y.T * m * 4 : 0);
-    plan->launches_fwd = D.causal ? (nsplit > 1 ? 8 : 6) : 8;
+    plan->launches_fwd = D.causal ? (nsplit > 1 ? 7 : 5) : 7;
     {
         size_t so = 0;
         Y.sv_sv = take(so, BH * N * 8);
@@ -1216,16 +1191,17 @@ cudaError_t tensor_prologue(const darkattn_plan_s *plan, const void *K, const vo
     const Dims &D = plan->dims;
     const TensorLayout &Y = plan->tensor;
     const size_t BH = D.BH, N = D.N;
-    NormParams NP;
-    memset(&NP, 0, sizeof(NP));
+    PrepassParams PP;
+    memset(&PP, 0, sizeof(PP));
     const size_t BHkv = (size_t)D.B * D.Hkv;
-    if (!make_map(&NP.mapK, K, BHkv * N, D.d, 128) || !make_map(&NP.mapM, M, (size_t)D.H * D.r, D.d, 128))
+    if (!make_map(&PP.mapK, K, BHkv * N, D.d, 128) || !make_map(&PP.mapM, M, (size_t)D.H * D.r, D.d, 128) ||
+        !make_map(&PP.mapOm, out.Om, (size_t)D.H * D.m, D.d, 128))
         return cudaErrorInvalidValue;
     cudaError_t e = cudaSuccess;
     auto chk = [&]() { cudaError_t x = cudaGetLastError(); if (x != cudaSuccess && e == cudaSuccess) e = x; };
 
-    // The two small kernels that read only M and W run on the side stream next to the key-norm kernel (with
-    // per-kernel timing on, everything stays on one stream).
+    // The two small kernels that read only M and W run on the plan's side stream (with per-kernel timing on,
+    // everything stays on one stream).
     const bool beside = !plan->timer.on && ensure_aux(plan) == cudaSuccess;
     cudaStream_t sp = beside ? plan->aux_stream : st;
     if (beside) {
@@ -1233,7 +1209,7 @@ cudaError_t tensor_prologue(const darkattn_plan_s *plan, const void *K, const vo
         if (e == cudaSuccess) e = cudaStreamWaitEvent(sp, plan->aux_fork, 0);
     }
     timer_mark(plan, st, "fold_omega_kernel");
-    fold_omega_kernel<<<dim3(D.m / 4, D.H), D.d, 0, sp>>>((const __nv_bfloat16 *)W, (const __nv_bfloat16 *)M, out.Om, out.Oml, D.m, D.r,
+    fold_omega_kernel<<<dim3(D.m / 16, D.H), D.d, 0, sp>>>((const __nv_bfloat16 *)W, (const __nv_bfloat16 *)M, out.Om, out.Oml, D.m, D.r,
                                                       D.d, D.w_per_head, kLog2e * D.s);
     chk();
     timer_mark(plan, st, "shift_init_kernel");
@@ -1241,36 +1217,22 @@ cudaError_t tensor_prologue(const darkattn_plan_s *plan, const void *K, const vo
     chk();
     if (beside && e == cudaSuccess) e = cudaEventRecord(plan->aux_join, sp);
 
-    NP.nK = out.nK; NP.status = reinterpret_cast<int *>(ws + Y.status);
-    NP.N = D.N; NP.H = D.H; NP.Hkv = D.Hkv; NP.T = Y.T; NP.r = D.r;
-    NP.nsplit = pick_splits((long long)BH, Y.T, 2.5, 3.0, 64, 3 * 148);      // three CTAs of this kernel fit one SM
-    NP.coef = kLog2e * 0.5f * D.s * D.s;
-    const int smem_bytes = 2 * 128 * D.d * 2 + 64;
-    timer_mark(plan, st, "tc_key_norms_kernel");
-    if (D.d == 64) {
-        cudaFuncSetAttribute(tc_key_norms_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
-        tc_key_norms_kernel<64><<<(unsigned)(BH * NP.nsplit), 160, smem_bytes, st>>>(NP);
-    } else {
-        cudaFuncSetAttribute(tc_key_norms_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
-        tc_key_norms_kernel<128><<<(unsigned)(BH * NP.nsplit), 160, smem_bytes, st>>>(NP);
-    }
-    chk();
     if (beside && e == cudaSuccess) e = cudaStreamWaitEvent(st, plan->aux_join, 0);
 
-    // the key-side shifts: the maximum of u - n over the keys of every (batch, head, slab)
-    ShiftParams SP;
-    memset(&SP, 0, sizeof(SP));
-    if (!make_map(&SP.mapK, K, BHkv * N, D.d, 128) || !make_map(&SP.mapOm, out.Om, (size_t)D.H * D.m, D.d, 128)) return cudaErrorInvalidValue;
-    SP.nK = out.nK; SP.cs = reinterpret_cast<int *>(out.cs); SP.status = NP.status;
-    SP.N = D.N; SP.H = D.H; SP.Hkv = D.Hkv; SP.T = Y.T; SP.m = D.m; SP.nslab = Y.nslab;
-    SP.nsplit = pick_splits((long long)BH * Y.nslab, Y.T, 2.5, 3.0, 64, 3 * 148);
-    timer_mark(plan, st, "tc_key_shift_kernel");
+    // key norms and key-side shifts in one pass over K
+    PP.nK = out.nK; PP.cs = reinterpret_cast<int *>(out.cs); PP.status = reinterpret_cast<int *>(ws + Y.status);
+    PP.N = D.N; PP.H = D.H; PP.Hkv = D.Hkv; PP.T = Y.T; PP.m = D.m; PP.r = D.r; PP.nslab = Y.nslab; PP.npair = (Y.nslab + 1) / 2;
+    PP.coef = kLog2e * 0.5f * D.s * D.s;
+    const int per_sm = D.d == 64 ? 2 : 1;                           // CTAs of this kernel that fit one SM
+    PP.nsplit = pick_splits((long long)BH * PP.npair, Y.T, 1.5, 3.0, 64, per_sm * 148);
+    const int smem_bytes = 5 * 128 * D.d * 2 + 128;
+    timer_mark(plan, st, "tc_key_prepass_kernel");
     if (D.d == 64) {
-        cudaFuncSetAttribute(tc_key_shift_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
-        tc_key_shift_kernel<64><<<(unsigned)(BH * Y.nslab * SP.nsplit), 160, smem_bytes, st>>>(SP);
+        cudaFuncSetAttribute(tc_key_prepass_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+        tc_key_prepass_kernel<64><<<(unsigned)(BH * PP.npair * PP.nsplit), 160, smem_bytes, st>>>(PP);
     } else {
-        cudaFuncSetAttribute(tc_key_shift_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
-        tc_key_shift_kernel<128><<<(unsigned)(BH * Y.nslab * SP.nsplit), 160, smem_bytes, st>>>(SP);
+        cudaFuncSetAttribute(tc_key_prepass_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+        tc_key_prepass_kernel<128><<<(unsigned)(BH * PP.npair * PP.nsplit), 160, smem_bytes, st>>>(PP);
     }
     chk();
     return e;
