@@ -36,42 +36,59 @@ constexpr float kShiftHeadroom = 64.f;
 
 // ------------------------------------------------------------------ prologue kernels (SIMT, tiny)
 // Omega[h,l,c] = log2(e) * s * sum_a W[l,a] M[h,a,c], stored as its bf16 rounding Om and the bf16 rounding Oml of what
-// that left out (Om + Oml carries 16 bits of Omega). One block per (head, 16 rows l), one thread per column c
-// (the block has d threads); many small blocks, because the kernel is bound by the latency of its loads.
-__global__ void fold_omega_kernel(const __nv_bfloat16 *W, const __nv_bfloat16 *M, __nv_bfloat16 *Om, __nv_bfloat16 *Oml, int m, int r,
-                                  int d, int w_per_head, float coef)
+// that left out (Om + Oml carries 16 bits of Omega). One block per (head, 16 rows l); its four warps split the sum over a and add up through
+// shared memory; d / 32 columns per lane: a thread's 16 x d/32 tile of outputs takes one broadcast load of four W values per
+// 4 d/32 products.
+template <int TC>
+__global__ void __launch_bounds__(128) fold_omega_kernel(const __nv_bfloat16 *W, const __nv_bfloat16 *M, __nv_bfloat16 *Om, __nv_bfloat16 *Oml,
+                                                         int m, int r, int w_per_head, float coef)
 {
-    constexpr int R = 16;                           // rows l per block: every loaded element of M serves 16 products
+    constexpr int R = 16, d = 32 * TC;
     __shared__ __align__(16) float sw[R][128];
-    const int h = blockIdx.y, l0 = blockIdx.x * R, c = threadIdx.x;
+    __shared__ float part[3][R * TC][32];           // the partial sums of warps 1..3
+    const int h = blockIdx.y, l0 = blockIdx.x * R, lane = threadIdx.x & 31, wq = threadIdx.x >> 5;
     const __nv_bfloat16 *w = W + ((size_t)(w_per_head ? h : 0) * m + l0) * r;
-    for (int i = threadIdx.x; i < R * r; i += blockDim.x) sw[i / r][i % r] = __bfloat162float(w[i]);
+    for (int i = threadIdx.x; i < R * r; i += 128) sw[i / r][i % r] = __bfloat162float(w[i]);
     __syncthreads();
-    const __nv_bfloat16 *Mh = M + (size_t)h * r * d;
-    float acc[R];
+    const __nv_bfloat16 *Mh = M + (size_t)h * r * d + lane;
+    float acc[R][TC];
 #pragma unroll
-    for (int i = 0; i < R; ++i) acc[i] = 0.f;
-    for (int a0 = 0; a0 < r; a0 += 16) {            // r is a multiple of 16; 16 independent loads in flight
-        __nv_bfloat16 mv[16];
+    for (int i = 0; i < R; ++i)
 #pragma unroll
-        for (int j = 0; j < 16; ++j) mv[j] = Mh[(size_t)(a0 + j) * d + c];
+        for (int q = 0; q < TC; ++q) acc[i][q] = 0.f;
+#pragma unroll 2
+    for (int a0 = 4 * wq; a0 < r; a0 += 16) {       // r is a multiple of 16: warp wq takes a = 4 wq .. 4 wq + 3 of every 16
+        float x[4][TC];
 #pragma unroll
-        for (int j = 0; j < 16; j += 4) {
-            const float x0 = __bfloat162float(mv[j]), x1 = __bfloat162float(mv[j + 1]);
-            const float x2 = __bfloat162float(mv[j + 2]), x3 = __bfloat162float(mv[j + 3]);
+        for (int jj = 0; jj < 4; ++jj)
 #pragma unroll
-            for (int i = 0; i < R; ++i) {
-                const float4 wv = *reinterpret_cast<const float4 *>(&sw[i][a0 + j]);   // one broadcast load per four products
-                acc[i] = fmaf(wv.x, x0, fmaf(wv.y, x1, fmaf(wv.z, x2, fmaf(wv.w, x3, acc[i]))));
-            }
+            for (int q = 0; q < TC; ++q) x[jj][q] = __bfloat162float(Mh[(size_t)(a0 + jj) * d + 32 * q]);
+#pragma unroll
+        for (int i = 0; i < R; ++i) {
+            const float4 wv = *reinterpret_cast<const float4 *>(&sw[i][a0]);
+#pragma unroll
+            for (int q = 0; q < TC; ++q)
+                acc[i][q] = fmaf(wv.x, x[0][q], fmaf(wv.y, x[1][q], fmaf(wv.z, x[2][q], fmaf(wv.w, x[3][q], acc[i][q]))));
         }
     }
+    if (wq > 0) {
 #pragma unroll
-    for (int i = 0; i < R; ++i) {
-        const float om = coef * acc[i];
-        const __nv_bfloat16 hi = __float2bfloat16_rn(om);
-        Om[((size_t)h * m + l0 + i) * d + c] = hi;
-        Oml[((size_t)h * m + l0 + i) * d + c] = __float2bfloat16_rn(om - __bfloat162float(hi));
+        for (int i = 0; i < R; ++i)
+#pragma unroll
+            for (int q = 0; q < TC; ++q) part[wq - 1][i * TC + q][lane] = acc[i][q];
+    }
+    __syncthreads();
+    if (wq == 0) {
+#pragma unroll
+        for (int i = 0; i < R; ++i)
+#pragma unroll
+            for (int q = 0; q < TC; ++q) {
+                const float om = coef * (acc[i][q] + part[0][i * TC + q][lane] + part[1][i * TC + q][lane] + part[2][i * TC + q][lane]);
+                const __nv_bfloat16 hi = __float2bfloat16_rn(om);
+                const size_t o = ((size_t)h * m + l0 + i) * d + lane + 32 * q;
+                Om[o] = hi;
+                Oml[o] = __float2bfloat16_rn(om - __bfloat162float(hi));
+            }
     }
 }
 
@@ -1209,8 +1226,12 @@ cudaError_t tensor_prologue(const darkattn_plan_s *plan, const void *K, const vo
         if (e == cudaSuccess) e = cudaStreamWaitEvent(sp, plan->aux_fork, 0);
     }
     timer_mark(plan, st, "fold_omega_kernel");
-    fold_omega_kernel<<<dim3(D.m / 16, D.H), D.d, 0, sp>>>((const __nv_bfloat16 *)W, (const __nv_bfloat16 *)M, out.Om, out.Oml, D.m, D.r,
-                                                      D.d, D.w_per_head, kLog2e * D.s);
+    if (D.d == 64)
+        fold_omega_kernel<2><<<dim3(D.m / 16, D.H), 128, 0, sp>>>((const __nv_bfloat16 *)W, (const __nv_bfloat16 *)M, out.Om, out.Oml, D.m, D.r,
+                                                               D.w_per_head, kLog2e * D.s);
+    else
+        fold_omega_kernel<4><<<dim3(D.m / 16, D.H), 128, 0, sp>>>((const __nv_bfloat16 *)W, (const __nv_bfloat16 *)M, out.Om, out.Oml, D.m, D.r,
+                                                               D.w_per_head, kLog2e * D.s);
     chk();
     timer_mark(plan, st, "shift_init_kernel");
     shift_init_kernel<<<(unsigned)((BH * Y.nslab + 255) / 256), 256, 0, sp>>>(reinterpret_cast<int *>(out.cs), (int)(BH * Y.nslab));
