@@ -21,26 +21,60 @@ __device__ __forceinline__ float ldf(const T *p, size_t i)
     else return p[i];
 }
 
-// Features of one (batch, head)'s new token, by a block of 256 threads: fk[l] = phi(k)_l and, when WITH_Q, fq[l] = phi(q)_l
-// (shared memory: xq[r], xk[r], fq[m], fk[m], red[...]).
-template <typename T, bool WITH_Q>
-__device__ __forceinline__ void token_features(const T *qv, const T *kv, const T *Mh, const T *Wh, float *xq, float *xk, float *fq,
-                                               float *fk, float *red, int d, int r, int m, float s)
+// Dot products of one row of a matrix with up to two vectors held in shared memory, and the row's squared norm: one thread
+// per row, the row read with 16-byte loads that do not depend on one another (the kernel is bound by the latency of its
+// loads, so each thread keeps a whole row in flight).
+template <typename T, bool TWO>
+__device__ __forceinline__ void row_dots(const T *row, const float *x0, const float *x1, int n, float &d0, float &d1, float &nn)
 {
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    // x~ = s M x for the query and the key: one warp per row of M, its lanes along the row (coalesced), shuffle sum
-    for (int a = warp; a < r; a += 8) {
-        float aq = 0.f, ak = 0.f;
-        for (int c = lane; c < d; c += 32) {
-            const float mv = ldf(Mh, (size_t)a * d + c);
-            if constexpr (WITH_Q) aq = fmaf(mv, ldf(qv, c), aq);
-            ak = fmaf(mv, ldf(kv, c), ak);
+    d0 = d1 = nn = 0.f;
+    constexpr int V = 16 / (int)sizeof(T);          // elements per 16-byte load
+    if (n % V == 0 && (reinterpret_cast<uintptr_t>(row) & 15) == 0) {
+#pragma unroll 4
+        for (int c = 0; c < n; c += V) {
+            float w[V];
+            if constexpr (sizeof(T) == 2) {         // eight bf16: the upper half of an fp32 each
+                const uint4 raw = *reinterpret_cast<const uint4 *>(row + c);
+                const uint32_t u[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) { w[2 * j] = __uint_as_float(u[j] << 16); w[2 * j + 1] = __uint_as_float(u[j] & 0xffff0000u); }
+            }
+            else { const float4 f = *reinterpret_cast<const float4 *>(row + c); w[0] = f.x; w[1] = f.y; w[2] = f.z; w[3] = f.w; }
+#pragma unroll
+            for (int j = 0; j < V; ++j) {
+                d0 = fmaf(w[j], x0[c + j], d0);
+                if constexpr (TWO) d1 = fmaf(w[j], x1[c + j], d1);
+                nn = fmaf(w[j], w[j], nn);
+            }
         }
-        for (int off = 16; off; off >>= 1) {
-            if constexpr (WITH_Q) aq += __shfl_xor_sync(0xffffffffu, aq, off);
-            ak += __shfl_xor_sync(0xffffffffu, ak, off);
+    } else {
+        for (int c = 0; c < n; ++c) {
+            const float w = ldf(row, c);
+            d0 = fmaf(w, x0[c], d0);
+            if constexpr (TWO) d1 = fmaf(w, x1[c], d1);
+            nn = fmaf(w, w, nn);
         }
-        if (lane == 0) { xq[a] = s * aq; xk[a] = s * ak; }
+    }
+}
+
+// Features of one (batch, head)'s new token, by a block of 256 threads: fk[l] = phi(k)_l and, when WITH_Q, fq[l] = phi(q)_l
+// (shared memory: vq[d], vk[d], xq[r], xk[r], fq[m], fk[m], red[...]).
+template <typename T, bool WITH_Q>
+__device__ __forceinline__ void token_features(const T *qv, const T *kv, const T *Mh, const T *Wh, float *vq, float *vk, float *xq,
+                                               float *xk, float *fq, float *fk, float *red, int d, int r, int m, float s)
+{
+    const int tid = threadIdx.x, lane = tid & 31;
+    for (int c = tid; c < d; c += 256) {
+        vk[c] = ldf(kv, c);
+        if constexpr (WITH_Q) vq[c] = ldf(qv, c);
+    }
+    __syncthreads();
+    // x~ = s M x for the query and the key: one thread per row of M
+    for (int a = tid; a < r; a += 256) {
+        float aq, ak, nn;
+        row_dots<T, WITH_Q>(Mh + (size_t)a * d, WITH_Q ? vq : vk, vk, d, aq, ak, nn);
+        if constexpr (WITH_Q) { xq[a] = s * aq; xk[a] = s * ak; }
+        else xk[a] = s * aq;
     }
     __syncthreads();
     float nk = 0.f;
@@ -48,26 +82,17 @@ __device__ __forceinline__ void token_features(const T *qv, const T *kv, const T
     for (int off = 16; off; off >>= 1) nk += __shfl_xor_sync(0xffffffffu, nk, off);
     nk *= 0.5f;
     float mx = -INFINITY;
-    for (int l = warp; l < m; l += 8) {             // exponents of the features: one warp per row of W
-        float uq = 0.f, uk = 0.f, c = 0.f;
-        for (int a = lane; a < r; a += 32) {
-            const float w = ldf(Wh, (size_t)l * r + a);
-            if constexpr (WITH_Q) uq = fmaf(w, xq[a], uq);
-            uk = fmaf(w, xk[a], uk);
-            c = fmaf(w, w, c);
-        }
-        for (int off = 16; off; off >>= 1) {
-            if constexpr (WITH_Q) uq += __shfl_xor_sync(0xffffffffu, uq, off);
-            uk += __shfl_xor_sync(0xffffffffu, uk, off);
-            c += __shfl_xor_sync(0xffffffffu, c, off);
-        }
+    for (int l = tid; l < m; l += 256) {            // exponents of the features: one thread per row of W
+        float uq, uk, c;
+        row_dots<T, WITH_Q>(Wh + (size_t)l * r, WITH_Q ? xq : xk, xk, r, uq, uk, c);
+        if constexpr (!WITH_Q) uk = uq;
         c *= 0.5f;
-        if (lane == 0) { fk[l] = __expf(uk - nk - c); fq[l] = uq + c; }
-        mx = fmaxf(mx, uq + c);
+        fk[l] = __expf(uk - nk - c);
+        if constexpr (WITH_Q) { fq[l] = uq + c; mx = fmaxf(mx, uq + c); }
     }
     if constexpr (WITH_Q) {
         for (int off = 16; off; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-        if ((tid & 31) == 0) red[tid >> 5] = mx;
+        if (lane == 0) red[tid >> 5] = mx;
         __syncthreads();
         mx = red[0];
         for (int w = 1; w < 8; ++w) mx = fmaxf(mx, red[w]);
@@ -86,28 +111,39 @@ __global__ void __launch_bounds__(256) decode_step_kernel(const T *q, const T *k
                                                            float s)
 {
     extern __shared__ float sm[];
-    float *xq = sm, *xk = xq + r, *fq = xk + r, *fk = fq + m, *red = fk + m;   // red: 8 x 32 partial numerators + 8 partial normalisers + scratch
-    const int bh = blockIdx.y, h = bh % H, tid = threadIdx.x;
+    float *vq = sm, *vk = vq + d, *xq = vk + d, *xk = xq + r, *fq = xk + r, *fk = fq + m, *red = fk + m;   // red: 8 x 32 partial numerators + 8 partial normalisers
+    const int bh = blockIdx.y, h = bh % H, tid = threadIdx.x, lane = tid & 31;
     const int kvh = (bh / H) * Hkv + h / (H / Hkv);     // the key/value head this query head reads (grouped key/value heads)
     token_features<T, true>(q + (size_t)bh * d, k + (size_t)kvh * d, M + (size_t)h * r * d, W + (size_t)(w_per_head ? h : 0) * m * r,
-                            xq, xk, fq, fk, red, d, r, m, s);
+                            vq, vk, xq, xk, fq, fk, red, d, r, m, s);
 
-    // state update and read-out: thread = (column, feature group)
-    const int col = blockIdx.x * 32 + (tid & 31), grp = tid >> 5;
-    const float vv = ldf(v, (size_t)kvh * dv + col);
-    float *Sb = S + (size_t)bh * m * dv;
+    // normaliser phi(q) . (z + phi(k)): one feature per thread, summed over the block
     const float *zb = z + (size_t)bh * m;
-    float num = 0.f, den = 0.f;
-    for (int l = grp; l < m; l += 8) {
-        const float snew = fmaf(fk[l], vv, Sb[(size_t)l * dv + col]);
-        Sb[(size_t)l * dv + col] = snew;
-        num = fmaf(fq[l], snew, num);
-        if ((tid & 31) == 0) {                       // one lane per group carries the normaliser
-            den = fmaf(fq[l], zb[l] + fk[l], den);
+    float den = 0.f;
+    for (int l = tid; l < m; l += 256) den = fmaf(fq[l], zb[l] + fk[l], den);
+    for (int off = 16; off; off >>= 1) den += __shfl_xor_sync(0xffffffffu, den, off);
+
+    // state update and read-out: thread = (column, feature group); 16 rows of the state in flight per thread
+    const int col = blockIdx.x * 32 + lane, grp = tid >> 5;
+    const float vv = ldf(v, (size_t)kvh * dv + col);
+    float *Sb = S + (size_t)bh * m * dv + col;
+    float num = 0.f;
+    for (int l0 = grp; l0 < m; l0 += 128) {
+        float sv[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) { const int l = l0 + 8 * j; sv[j] = (l < m) ? Sb[(size_t)l * dv] : 0.f; }
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const int l = l0 + 8 * j;
+            if (l < m) {
+                const float snew = fmaf(fk[l], vv, sv[j]);
+                Sb[(size_t)l * dv] = snew;
+                num = fmaf(fq[l], snew, num);
+            }
         }
     }
-    red[grp * 32 + (tid & 31)] = num;
-    if ((tid & 31) == 0) red[256 + grp] = den;
+    red[grp * 32 + lane] = num;
+    if (lane == 0) red[256 + grp] = den;
     __syncthreads();
     if (tid < 32) {
         float n = 0.f, dn = 0.f;
@@ -124,10 +160,10 @@ __global__ void __launch_bounds__(256) decode_z_kernel(const T *k, const T *M, c
                                                         int w_per_head, float s)
 {
     extern __shared__ float sm[];
-    float *xq = sm, *xk = xq + r, *fq = xk + r, *fk = fq + m, *red = fk + m;
+    float *vq = sm, *vk = vq + d, *xq = vk + d, *xk = xq + r, *fq = xk + r, *fk = fq + m, *red = fk + m;
     const int bh = blockIdx.x, h = bh % H;
-    token_features<T, false>(nullptr, k + (size_t)((bh / H) * Hkv + h / (H / Hkv)) * d, M + (size_t)h * r * d, W + (size_t)(w_per_head ? h : 0) * m * r, xq, xk, fq,
-                             fk, red, d, r, m, s);
+    token_features<T, false>(nullptr, k + (size_t)((bh / H) * Hkv + h / (H / Hkv)) * d, M + (size_t)h * r * d, W + (size_t)(w_per_head ? h : 0) * m * r, vq, vk,
+                             xq, xk, fq, fk, red, d, r, m, s);
     for (int l = threadIdx.x; l < m; l += 256) z[(size_t)bh * m + l] += fk[l];
 }
 
@@ -145,7 +181,7 @@ extern "C" darkattn_status_t darkattn_decode_step(darkattn_plan_t plan, const vo
     if (!D.causal) return DARKATTN_ERR_UNSUPPORTED;          // the recurrent form is the causal one
     if (D.dv % 32) return DARKATTN_ERR_UNSUPPORTED;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    const size_t smem = (size_t)(2 * D.r + 2 * D.m + 256 + 16) * sizeof(float);
+    const size_t smem = (size_t)(2 * D.d + 2 * D.r + 2 * D.m + 256 + 16) * sizeof(float);
     if (smem > 48 * 1024) return DARKATTN_ERR_UNSUPPORTED;
     const dim3 grid(D.dv / 32, D.BH);
     if (D.bf16)
