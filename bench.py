@@ -290,7 +290,7 @@ def decode_benchmark(torch, binding, inputs, peaks, B=4, H=16, d=128, m=256, dv=
     us = 1e3 * e0.elapsed_time(e1) / steps
     nbytes = B * H * (2 * m * dv * 4 + 2 * m * 4) + (H * d * d + m * d) * 2
     plan.destroy()
-    return {"workload": f"decode step: B={B} H={H} d={d} m={m} dv={dv} bf16, state fp32", "us_per_step": us, "launches_per_step": 2,
+    return {"workload": f"decode step: B={B} H={H} d={d} m={m} dv={dv} bf16, state fp32", "us_per_step": us, "launches_per_step": 1,
             "bound": "hbm (state read and written once; at this size the state, 8 MB, stays in L2: launch- and latency-bound)",
             "achieved": nbytes / (us * 1e-6) / 1e9, "unit": "GB/s", "peak": peaks["hbm_gbs"],
             "frac": nbytes / (us * 1e-6) / 1e9 / peaks["hbm_gbs"], "tokens_per_s": B / (us * 1e-6)}

@@ -137,7 +137,8 @@ darkattn_status_t darkattn_backward_dw(darkattn_plan_t plan, const void *M, floa
  * updated in place: zero them before the first token. The features are scaled by exp(-|w_l|^2/2) (keys) and its
  * inverse (queries), which cancels in o, is the same at every step and keeps every key feature <= 1; the state is
  * therefore only meaningful to this call. Needs a causal plan (B, H, d, r, m, dv, dtype, scale, w_per_head are taken
- * from it; N is not used) with dv a multiple of 32. No workspace. Asynchronous on `cuda_stream`.                  */
+ * from it; N is not used) with dv a multiple of 32, at most 512 (else DARKATTN_ERR_UNSUPPORTED). No workspace. One
+ * kernel launch, asynchronous on `cuda_stream`.                                                                   */
 darkattn_status_t darkattn_decode_step(darkattn_plan_t plan, const void *q, const void *k, const void *v, const void *M,
                                        const void *W, float *S, float *z, void *o, void *cuda_stream);
 

@@ -30,7 +30,7 @@ __device__ __forceinline__ void row_dots(const T *row, const float *x0, const fl
     d0 = d1 = nn = 0.f;
     constexpr int V = 16 / (int)sizeof(T);          // elements per 16-byte load
     if (n % V == 0 && (reinterpret_cast<uintptr_t>(row) & 15) == 0) {
-#pragma unroll 4
+#pragma unroll 8
         for (int c = 0; c < n; c += V) {
             float w[V];
             if constexpr (sizeof(T) == 2) {         // eight bf16: the upper half of an fp32 each
@@ -57,20 +57,21 @@ __device__ __forceinline__ void row_dots(const T *row, const float *x0, const fl
     }
 }
 
-// Features of one (batch, head)'s new token, by a block of 256 threads: fk[l] = phi(k)_l and, when WITH_Q, fq[l] = phi(q)_l
+// Features of one (batch, head)'s new token, by the whole block (a multiple of 32 threads, at most 1024): fk[l] = phi(k)_l and, when WITH_Q, fq[l] = phi(q)_l
 // (shared memory: vq[d], vk[d], xq[r], xk[r], fq[m], fk[m], red[...]).
 template <typename T, bool WITH_Q>
 __device__ __forceinline__ void token_features(const T *qv, const T *kv, const T *Mh, const T *Wh, float *vq, float *vk, float *xq,
                                                float *xk, float *fq, float *fk, float *red, int d, int r, int m, float s)
 {
     const int tid = threadIdx.x, lane = tid & 31;
-    for (int c = tid; c < d; c += 256) {
+    const int nt = blockDim.x;
+    for (int c = tid; c < d; c += nt) {
         vk[c] = ldf(kv, c);
         if constexpr (WITH_Q) vq[c] = ldf(qv, c);
     }
     __syncthreads();
     // x~ = s M x for the query and the key: one thread per row of M
-    for (int a = tid; a < r; a += 256) {
+    for (int a = tid; a < r; a += nt) {
         float aq, ak, nn;
         row_dots<T, WITH_Q>(Mh + (size_t)a * d, WITH_Q ? vq : vk, vk, d, aq, ak, nn);
         if constexpr (WITH_Q) { xq[a] = s * aq; xk[a] = s * ak; }
@@ -82,7 +83,7 @@ __device__ __forceinline__ void token_features(const T *qv, const T *kv, const T
     for (int off = 16; off; off >>= 1) nk += __shfl_xor_sync(0xffffffffu, nk, off);
     nk *= 0.5f;
     float mx = -INFINITY;
-    for (int l = tid; l < m; l += 256) {            // exponents of the features: one thread per row of W
+    for (int l = tid; l < m; l += nt) {             // exponents of the features: one thread per row of W
         float uq, uk, c;
         row_dots<T, WITH_Q>(Wh + (size_t)l * r, WITH_Q ? xq : xk, xk, r, uq, uk, c);
         if constexpr (!WITH_Q) uk = uq;
@@ -95,76 +96,69 @@ __device__ __forceinline__ void token_features(const T *qv, const T *kv, const T
         if (lane == 0) red[tid >> 5] = mx;
         __syncthreads();
         mx = red[0];
-        for (int w = 1; w < 8; ++w) mx = fmaxf(mx, red[w]);
+        for (int w = 1; w < nt / 32; ++w) mx = fmaxf(mx, red[w]);
         __syncthreads();
-        for (int l = tid; l < m; l += 256) fq[l] = __expf(fq[l] - mx);
+        for (int l = tid; l < m; l += nt) fq[l] = __expf(fq[l] - mx);
     }
     __syncthreads();
 }
 
-// grid = (dv / 32 column blocks, B*H); block = 256 threads = 32 columns x 8 groups of features. Every column block of a
-// (batch, head) needs z + phi(k) for the normaliser; none of them stores it (the blocks are not ordered among themselves):
-// decode_z_kernel, launched behind this one on the same stream, applies z += phi(k).
+// One block of 512 threads per (batch, head): thread = (column of the state, feature group), 512 / dv groups. The block owns
+// the head's z, so it reads z for the normaliser and stores z + phi(k) itself.
 template <typename T>
-__global__ void __launch_bounds__(256) decode_step_kernel(const T *q, const T *k, const T *v, const T *M, const T *W, float *S,
-                                                           const float *z, T *o, int H, int Hkv, int d, int r, int m, int dv, int w_per_head,
+__global__ void __launch_bounds__(512) decode_step_kernel(const T *q, const T *k, const T *v, const T *M, const T *W, float *S,
+                                                           float *z, T *o, int H, int Hkv, int d, int r, int m, int dv, int w_per_head,
                                                            float s)
 {
     extern __shared__ float sm[];
-    float *vq = sm, *vk = vq + d, *xq = vk + d, *xk = xq + r, *fq = xk + r, *fk = fq + m, *red = fk + m;   // red: 8 x 32 partial numerators + 8 partial normalisers
-    const int bh = blockIdx.y, h = bh % H, tid = threadIdx.x, lane = tid & 31;
+    float *vq = sm, *vk = vq + d, *xq = vk + d, *xk = xq + r, *fq = xk + r, *fk = fq + m, *red = fk + m;   // red: 512 partial numerators + 16 partial normalisers
+    const int bh = blockIdx.x, h = bh % H, tid = threadIdx.x, lane = tid & 31;
     const int kvh = (bh / H) * Hkv + h / (H / Hkv);     // the key/value head this query head reads (grouped key/value heads)
     token_features<T, true>(q + (size_t)bh * d, k + (size_t)kvh * d, M + (size_t)h * r * d, W + (size_t)(w_per_head ? h : 0) * m * r,
                             vq, vk, xq, xk, fq, fk, red, d, r, m, s);
 
-    // normaliser phi(q) . (z + phi(k)): one feature per thread, summed over the block
-    const float *zb = z + (size_t)bh * m;
+    // normaliser phi(q) . (z + phi(k)) and the new z: one feature per thread
+    float *zb = z + (size_t)bh * m;
     float den = 0.f;
-    for (int l = tid; l < m; l += 256) den = fmaf(fq[l], zb[l] + fk[l], den);
+    for (int l = tid; l < m; l += 512) {
+        const float zn = zb[l] + fk[l];
+        zb[l] = zn;
+        den = fmaf(fq[l], zn, den);
+    }
     for (int off = 16; off; off >>= 1) den += __shfl_xor_sync(0xffffffffu, den, off);
 
-    // state update and read-out: thread = (column, feature group); 16 rows of the state in flight per thread
-    const int col = blockIdx.x * 32 + lane, grp = tid >> 5;
-    const float vv = ldf(v, (size_t)kvh * dv + col);
-    float *Sb = S + (size_t)bh * m * dv + col;
+    // state update and read-out; 16 rows of the state in flight per thread
+    const int ngrp = 512 / dv, col = tid % dv, grp = tid / dv;
     float num = 0.f;
-    for (int l0 = grp; l0 < m; l0 += 128) {
-        float sv[16];
+    if (grp < ngrp) {
+        const float vv = ldf(v, (size_t)kvh * dv + col);
+        float *Sb = S + (size_t)bh * m * dv + col;
+        for (int l0 = grp; l0 < m; l0 += 16 * ngrp) {
+            float sv[16];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) { const int l = l0 + 8 * j; sv[j] = (l < m) ? Sb[(size_t)l * dv] : 0.f; }
+            for (int j = 0; j < 16; ++j) { const int l = l0 + ngrp * j; sv[j] = (l < m) ? Sb[(size_t)l * dv] : 0.f; }
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-            const int l = l0 + 8 * j;
-            if (l < m) {
-                const float snew = fmaf(fk[l], vv, sv[j]);
-                Sb[(size_t)l * dv] = snew;
-                num = fmaf(fq[l], snew, num);
+            for (int j = 0; j < 16; ++j) {
+                const int l = l0 + ngrp * j;
+                if (l < m) {
+                    const float snew = fmaf(fk[l], vv, sv[j]);
+                    Sb[(size_t)l * dv] = snew;
+                    num = fmaf(fq[l], snew, num);
+                }
             }
         }
     }
-    red[grp * 32 + lane] = num;
-    if (lane == 0) red[256 + grp] = den;
+    red[tid] = num;
+    if (lane == 0) red[512 + (tid >> 5)] = den;
     __syncthreads();
-    if (tid < 32) {
+    if (tid < dv) {
         float n = 0.f, dn = 0.f;
-        for (int g = 0; g < 8; ++g) { n += red[g * 32 + tid]; dn += red[256 + g]; }
+        for (int g = 0; g < ngrp; ++g) n += red[g * dv + tid];
+        for (int w = 0; w < 16; ++w) dn += red[512 + w];
         const float out = n / dn;
-        if constexpr (sizeof(T) == 2) o[(size_t)bh * dv + blockIdx.x * 32 + tid] = __float2bfloat16_rn(out);
-        else o[(size_t)bh * dv + blockIdx.x * 32 + tid] = out;
+        if constexpr (sizeof(T) == 2) o[(size_t)bh * dv + tid] = __float2bfloat16_rn(out);
+        else o[(size_t)bh * dv + tid] = out;
     }
-}
-
-// z += phi(k) of the new token; one block per (batch, head).
-template <typename T>
-__global__ void __launch_bounds__(256) decode_z_kernel(const T *k, const T *M, const T *W, float *z, int H, int Hkv, int d, int r, int m,
-                                                        int w_per_head, float s)
-{
-    extern __shared__ float sm[];
-    float *vq = sm, *vk = vq + d, *xq = vk + d, *xk = xq + r, *fq = xk + r, *fk = fq + m, *red = fk + m;
-    const int bh = blockIdx.x, h = bh % H;
-    token_features<T, false>(nullptr, k + (size_t)((bh / H) * Hkv + h / (H / Hkv)) * d, M + (size_t)h * r * d, W + (size_t)(w_per_head ? h : 0) * m * r, vq, vk,
-                             xq, xk, fq, fk, red, d, r, m, s);
-    for (int l = threadIdx.x; l < m; l += 256) z[(size_t)bh * m + l] += fk[l];
 }
 
 }  // namespace
@@ -181,22 +175,16 @@ extern "C" darkattn_status_t darkattn_decode_step(darkattn_plan_t plan, const vo
     if (!D.causal) return DARKATTN_ERR_UNSUPPORTED;          // the recurrent form is the causal one
     if (D.dv % 32) return DARKATTN_ERR_UNSUPPORTED;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    const size_t smem = (size_t)(2 * D.d + 2 * D.r + 2 * D.m + 256 + 16) * sizeof(float);
+    if (D.dv > 512) return DARKATTN_ERR_UNSUPPORTED;
+    const size_t smem = (size_t)(2 * D.d + 2 * D.r + 2 * D.m + 512 + 16) * sizeof(float);
     if (smem > 48 * 1024) return DARKATTN_ERR_UNSUPPORTED;
-    const dim3 grid(D.dv / 32, D.BH);
     if (D.bf16)
-        decode_step_kernel<__nv_bfloat16><<<grid, 256, smem, st>>>((const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k, (const __nv_bfloat16 *)v,
-                                                                  (const __nv_bfloat16 *)M, (const __nv_bfloat16 *)W, S, z, (__nv_bfloat16 *)o,
-                                                                  D.H, D.Hkv, D.d, D.r, D.m, D.dv, D.w_per_head, D.s);
+        decode_step_kernel<__nv_bfloat16><<<(unsigned)D.BH, 512, smem, st>>>((const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k, (const __nv_bfloat16 *)v,
+                                                                           (const __nv_bfloat16 *)M, (const __nv_bfloat16 *)W, S, z, (__nv_bfloat16 *)o,
+                                                                           D.H, D.Hkv, D.d, D.r, D.m, D.dv, D.w_per_head, D.s);
     else
-        decode_step_kernel<float><<<grid, 256, smem, st>>>((const float *)q, (const float *)k, (const float *)v, (const float *)M,
-                                                           (const float *)W, S, z, (float *)o, D.H, D.Hkv, D.d, D.r, D.m, D.dv, D.w_per_head, D.s);
-    if (D.bf16)
-        decode_z_kernel<__nv_bfloat16><<<D.BH, 256, smem, st>>>((const __nv_bfloat16 *)k, (const __nv_bfloat16 *)M, (const __nv_bfloat16 *)W, z,
-                                                              D.H, D.Hkv, D.d, D.r, D.m, D.w_per_head, D.s);
-    else
-        decode_z_kernel<float><<<D.BH, 256, smem, st>>>((const float *)k, (const float *)M, (const float *)W, z, D.H, D.Hkv, D.d, D.r, D.m,
-                                                        D.w_per_head, D.s);
+        decode_step_kernel<float><<<(unsigned)D.BH, 512, smem, st>>>((const float *)q, (const float *)k, (const float *)v, (const float *)M,
+                                                                    (const float *)W, S, z, (float *)o, D.H, D.Hkv, D.d, D.r, D.m, D.dv, D.w_per_head, D.s);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_cuda_error(e, "decode_step"); return DARKATTN_ERR_CUDA; }
     return DARKATTN_OK;
