@@ -250,8 +250,13 @@ def test_gradient_of_the_projection_rows(binding, case):
 
 DECODE = [
     ("few_heads", dict(B=2, H=3, N=40, d=32, m=96, r=16, dv=64)),
-    # several thousand (batch, head) pairs with four column blocks each: the blocks of one pair land in different waves
+    # several thousand (batch, head) pairs: more blocks than one wave of the GPU holds
     ("many_heads_dv128", dict(B=64, H=48, N=5, d=32, m=64, r=16, dv=128)),
+    # dv = 96: 512 / 96 = 5 feature groups and 32 idle threads; m = 640 > 512: more than one feature per thread in the
+    # normaliser; rows of M (d = 48) are read with 16-byte loads, rows of W (r = 20) are not multiples of 16 bytes and take
+    # the element-wise loop
+    ("dv96_m640", dict(B=1, H=2, N=12, d=48, m=640, r=20, dv=96)),
+    ("dv512", dict(B=1, H=1, N=6, d=64, m=128, r=64, dv=512)),
 ]
 
 
