@@ -21,17 +21,20 @@ __device__ __forceinline__ float ldf(const T *p, size_t i)
     else return p[i];
 }
 
-// Dot products of one row of a matrix with up to two vectors held in shared memory, and the row's squared norm: one thread
-// per row, the row read with 16-byte loads that do not depend on one another (the kernel is bound by the latency of its
-// loads, so each thread keeps a whole row in flight).
+// Dot products of one row of a matrix with up to two vectors held in shared memory, and the row's squared norm. Eight lanes
+// share a row: lane `sub` of the eight takes every eighth 16-byte piece of it, so a warp's load covers four rows in pieces
+// of 128 contiguous bytes (every sector it fetches is used), and three shuffle steps add the eight parts up (all eight
+// lanes end with the sums). Rows whose length is not a multiple of 16 bytes are read element by element, eight apart.
+// Every lane of the warp must call this (the shuffles name the full warp).
 template <typename T, bool TWO>
-__device__ __forceinline__ void row_dots(const T *row, const float *x0, const float *x1, int n, float &d0, float &d1, float &nn)
+__device__ __forceinline__ void row_dots(const T *row, const float *x0, const float *x1, int n, int sub, bool vec, float &d0, float &d1,
+                                         float &nn)
 {
     d0 = d1 = nn = 0.f;
     constexpr int V = 16 / (int)sizeof(T);          // elements per 16-byte load
-    if (n % V == 0 && (reinterpret_cast<uintptr_t>(row) & 15) == 0) {
-#pragma unroll 8
-        for (int c = 0; c < n; c += V) {
+    if (vec) {
+#pragma unroll 4
+        for (int c = sub * V; c < n; c += 8 * V) {
             float w[V];
             if constexpr (sizeof(T) == 2) {         // eight bf16: the upper half of an fp32 each
                 const uint4 raw = *reinterpret_cast<const uint4 *>(row + c);
@@ -48,12 +51,18 @@ __device__ __forceinline__ void row_dots(const T *row, const float *x0, const fl
             }
         }
     } else {
-        for (int c = 0; c < n; ++c) {
+        for (int c = sub; c < n; c += 8) {
             const float w = ldf(row, c);
             d0 = fmaf(w, x0[c], d0);
             if constexpr (TWO) d1 = fmaf(w, x1[c], d1);
             nn = fmaf(w, w, nn);
         }
+    }
+#pragma unroll
+    for (int off = 1; off < 8; off <<= 1) {
+        d0 += __shfl_xor_sync(0xffffffffu, d0, off);
+        if constexpr (TWO) d1 += __shfl_xor_sync(0xffffffffu, d1, off);
+        nn += __shfl_xor_sync(0xffffffffu, nn, off);
     }
 }
 
@@ -64,18 +73,24 @@ __device__ __forceinline__ void token_features(const T *qv, const T *kv, const T
                                                float *xk, float *fq, float *fk, float *red, int d, int r, int m, float s)
 {
     const int tid = threadIdx.x, lane = tid & 31;
-    const int nt = blockDim.x;
+    const int nt = blockDim.x, sub = tid & 7, grp = tid >> 3, ngrp = nt >> 3;
+    constexpr int V = 16 / (int)sizeof(T);
     for (int c = tid; c < d; c += nt) {
         vk[c] = ldf(kv, c);
         if constexpr (WITH_Q) vq[c] = ldf(qv, c);
     }
     __syncthreads();
-    // x~ = s M x for the query and the key: one thread per row of M
-    for (int a = tid; a < r; a += nt) {
+    // x~ = s M x for the query and the key: eight lanes per row of M (whole warps walk the loop: rows past the end are read
+    // from the last row and not stored)
+    const bool vec_m = (d % V == 0) && (reinterpret_cast<uintptr_t>(Mh) & 15) == 0;
+    for (int a0 = 0; a0 < r; a0 += ngrp) {
+        const int a = a0 + grp, ac = a < r ? a : r - 1;
         float aq, ak, nn;
-        row_dots<T, WITH_Q>(Mh + (size_t)a * d, WITH_Q ? vq : vk, vk, d, aq, ak, nn);
-        if constexpr (WITH_Q) { xq[a] = s * aq; xk[a] = s * ak; }
-        else xk[a] = s * aq;
+        row_dots<T, WITH_Q>(Mh + (size_t)ac * d, WITH_Q ? vq : vk, vk, d, sub, vec_m, aq, ak, nn);
+        if (a < r && sub == 0) {
+            if constexpr (WITH_Q) { xq[a] = s * aq; xk[a] = s * ak; }
+            else xk[a] = s * aq;
+        }
     }
     __syncthreads();
     float nk = 0.f;
@@ -83,13 +98,20 @@ __device__ __forceinline__ void token_features(const T *qv, const T *kv, const T
     for (int off = 16; off; off >>= 1) nk += __shfl_xor_sync(0xffffffffu, nk, off);
     nk *= 0.5f;
     float mx = -INFINITY;
-    for (int l = tid; l < m; l += nt) {             // exponents of the features: one thread per row of W
+    const bool vec_w = (r % V == 0) && (reinterpret_cast<uintptr_t>(Wh) & 15) == 0;
+    for (int l0 = 0; l0 < m; l0 += ngrp) {          // exponents of the features: eight lanes per row of W
+        const int l = l0 + grp, lc = l < m ? l : m - 1;
         float uq, uk, c;
-        row_dots<T, WITH_Q>(Wh + (size_t)l * r, WITH_Q ? xq : xk, xk, r, uq, uk, c);
+        row_dots<T, WITH_Q>(Wh + (size_t)lc * r, WITH_Q ? xq : xk, xk, r, sub, vec_w, uq, uk, c);
         if constexpr (!WITH_Q) uk = uq;
         c *= 0.5f;
-        fk[l] = __expf(uk - nk - c);
-        if constexpr (WITH_Q) { fq[l] = uq + c; mx = fmaxf(mx, uq + c); }
+        if (l < m) {
+            if (sub == 0) {
+                fk[l] = __expf(uk - nk - c);
+                if constexpr (WITH_Q) fq[l] = uq + c;
+            }
+            if constexpr (WITH_Q) mx = fmaxf(mx, uq + c);
+        }
     }
     if constexpr (WITH_Q) {
         for (int off = 16; off; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
