@@ -125,7 +125,7 @@ __device__ __forceinline__ void token_features(const T *qv, const T *kv, const T
     __syncthreads();
 }
 
-// One block of 512 threads per (batch, head): thread = (column of the state, feature group), 512 / dv groups. The block owns
+// One block of 512 threads per (batch, head): thread = (four columns of the state, group of rows). The block owns
 // the head's z, so it reads z for the normaliser and stores z + phi(k) itself.
 template <typename T>
 __global__ void __launch_bounds__(512) decode_step_kernel(const T *q, const T *k, const T *v, const T *M, const T *W, float *S,
@@ -133,7 +133,7 @@ __global__ void __launch_bounds__(512) decode_step_kernel(const T *q, const T *k
                                                            float s)
 {
     extern __shared__ float sm[];
-    float *vq = sm, *vk = vq + d, *xq = vk + d, *xk = xq + r, *fq = xk + r, *fk = fq + m, *red = fk + m;   // red: 512 partial numerators + 16 partial normalisers
+    float *vq = sm, *vk = vq + d, *xq = vk + d, *xk = xq + r, *fq = xk + r, *fk = fq + m, *red = fk + m;   // red: up to 2048 partial numerators + 16 partial normalisers
     const int bh = blockIdx.x, h = bh % H, tid = threadIdx.x, lane = tid & 31;
     const int kvh = (bh / H) * Hkv + h / (H / Hkv);     // the key/value head this query head reads (grouped key/value heads)
     token_features<T, true>(q + (size_t)bh * d, k + (size_t)kvh * d, M + (size_t)h * r * d, W + (size_t)(w_per_head ? h : 0) * m * r,
@@ -149,34 +149,38 @@ __global__ void __launch_bounds__(512) decode_step_kernel(const T *q, const T *k
     }
     for (int off = 16; off; off >>= 1) den += __shfl_xor_sync(0xffffffffu, den, off);
 
-    // state update and read-out; 16 rows of the state in flight per thread
-    const int ngrp = 512 / dv, col = tid % dv, grp = tid / dv;
-    float num = 0.f;
-    if (grp < ngrp) {
-        const float vv = ldf(v, (size_t)kvh * dv + col);
-        float *Sb = S + (size_t)bh * m * dv + col;
-        for (int l0 = grp; l0 < m; l0 += 16 * ngrp) {
-            float sv[16];
+    // state update and read-out: a thread owns four neighbouring columns of every (512 / (dv / 4))-th row and keeps 16 of
+    // its rows (256 bytes) in flight
+    const int tpr = dv / 4, nrg = 512 / tpr, c4 = (tid % tpr) * 4, rg = tid / tpr;
+    float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (rg < nrg) {
+        const float4 vv = make_float4(ldf(v, (size_t)kvh * dv + c4), ldf(v, (size_t)kvh * dv + c4 + 1), ldf(v, (size_t)kvh * dv + c4 + 2),
+                                      ldf(v, (size_t)kvh * dv + c4 + 3));
+        float4 *Sb = reinterpret_cast<float4 *>(S + (size_t)bh * m * dv + c4);
+        for (int l0 = rg; l0 < m; l0 += 16 * nrg) {
+            float4 sv[16];
 #pragma unroll
-            for (int j = 0; j < 16; ++j) { const int l = l0 + ngrp * j; sv[j] = (l < m) ? Sb[(size_t)l * dv] : 0.f; }
+            for (int j = 0; j < 16; ++j) { const int l = l0 + nrg * j; sv[j] = (l < m) ? Sb[(size_t)l * tpr] : make_float4(0.f, 0.f, 0.f, 0.f); }
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
-                const int l = l0 + ngrp * j;
+                const int l = l0 + nrg * j;
                 if (l < m) {
-                    const float snew = fmaf(fk[l], vv, sv[j]);
-                    Sb[(size_t)l * dv] = snew;
-                    num = fmaf(fq[l], snew, num);
+                    const float f = fk[l], g = fq[l];
+                    const float4 sn = make_float4(fmaf(f, vv.x, sv[j].x), fmaf(f, vv.y, sv[j].y), fmaf(f, vv.z, sv[j].z), fmaf(f, vv.w, sv[j].w));
+                    Sb[(size_t)l * tpr] = sn;
+                    num.x = fmaf(g, sn.x, num.x); num.y = fmaf(g, sn.y, num.y); num.z = fmaf(g, sn.z, num.z); num.w = fmaf(g, sn.w, num.w);
                 }
             }
         }
+        float *rd = red + rg * dv + c4;
+        rd[0] = num.x; rd[1] = num.y; rd[2] = num.z; rd[3] = num.w;
     }
-    red[tid] = num;
-    if (lane == 0) red[512 + (tid >> 5)] = den;
+    if (lane == 0) red[2048 + (tid >> 5)] = den;
     __syncthreads();
     if (tid < dv) {
         float n = 0.f, dn = 0.f;
-        for (int g = 0; g < ngrp; ++g) n += red[g * dv + tid];
-        for (int w = 0; w < 16; ++w) dn += red[512 + w];
+        for (int g = 0; g < nrg; ++g) n += red[g * dv + tid];
+        for (int w = 0; w < 16; ++w) dn += red[2048 + w];
         const float out = n / dn;
         if constexpr (sizeof(T) == 2) o[(size_t)bh * dv + tid] = __float2bfloat16_rn(out);
         else o[(size_t)bh * dv + tid] = out;
@@ -198,7 +202,7 @@ extern "C" darkattn_status_t darkattn_decode_step(darkattn_plan_t plan, const vo
     if (D.dv % 32) return DARKATTN_ERR_UNSUPPORTED;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     if (D.dv > 512) return DARKATTN_ERR_UNSUPPORTED;
-    const size_t smem = (size_t)(2 * D.d + 2 * D.r + 2 * D.m + 512 + 16) * sizeof(float);
+    const size_t smem = (size_t)(2 * D.d + 2 * D.r + 2 * D.m + 2048 + 16) * sizeof(float);
     if (smem > 48 * 1024) return DARKATTN_ERR_UNSUPPORTED;
     if (D.bf16)
         decode_step_kernel<__nv_bfloat16><<<(unsigned)D.BH, 512, smem, st>>>((const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k, (const __nv_bfloat16 *)v,
