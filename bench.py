@@ -290,8 +290,11 @@ def decode_benchmark(torch, binding, inputs, peaks, B=4, H=16, d=128, m=256, dv=
     us = 1e3 * e0.elapsed_time(e1) / steps
     nbytes = B * H * (2 * m * dv * 4 + 2 * m * 4) + (H * d * d + m * d) * 2
     plan.destroy()
+    state_mb = B * H * m * dv * 4 / 1e6
+    note = ("at this size the state, %.0f MB, stays in L2: launch- and latency-bound" % state_mb if state_mb < 100
+            else "state of %.0f MB, larger than L2" % state_mb)
     return {"workload": f"decode step: B={B} H={H} d={d} m={m} dv={dv} bf16, state fp32", "us_per_step": us, "launches_per_step": 1,
-            "bound": "hbm (state read and written once; at this size the state, 8 MB, stays in L2: launch- and latency-bound)",
+            "bound": "hbm (state read and written once; " + note + ")",
             "achieved": nbytes / (us * 1e-6) / 1e9, "unit": "GB/s", "peak": peaks["hbm_gbs"],
             "frac": nbytes / (us * 1e-6) / 1e9 / peaks["hbm_gbs"], "tokens_per_s": B / (us * 1e-6)}
 
@@ -552,6 +555,7 @@ def main():
         torch.cuda.empty_cache()
         roofline["configs"] = extra_configs(torch, binding, inputs, peaks, tensor_peak, exclude=args.workload)
         roofline["decode_step"] = decode_benchmark(torch, binding, inputs, peaks)
+        roofline["decode_step_large_batch"] = decode_benchmark(torch, binding, inputs, peaks, B=64)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         from oracle import ref
         sub, use, cores = oracle_sample(wl, inputs, ref)
