@@ -125,10 +125,12 @@ __device__ __forceinline__ void token_features(const T *qv, const T *kv, const T
     __syncthreads();
 }
 
-// One block of 512 threads per (batch, head): thread = (four columns of the state, group of rows). The block owns
-// the head's z, so it reads z for the normaliser and stores z + phi(k) itself.
-template <typename T>
-__global__ void __launch_bounds__(512) decode_step_kernel(const T *q, const T *k, const T *v, const T *M, const T *W, float *S,
+// One block of NT threads per (batch, head): thread = (four columns of the state, group of rows). The block owns
+// the head's z, so it reads z for the normaliser and stores z + phi(k) itself. NT = 512 when the blocks are few (each is
+// a chain of load latencies: more threads shorten it); NT = 256 when there are several per SM, so that two share an SM
+// and one's feature phase, which moves no state, runs under the other's state traffic.
+template <typename T, int NT>
+__global__ void __launch_bounds__(NT, 512 / NT) decode_step_kernel(const T *q, const T *k, const T *v, const T *M, const T *W, float *S,
                                                            float *z, T *o, int H, int Hkv, int d, int r, int m, int dv, int w_per_head,
                                                            float s)
 {
@@ -142,16 +144,16 @@ __global__ void __launch_bounds__(512) decode_step_kernel(const T *q, const T *k
     // normaliser phi(q) . (z + phi(k)) and the new z: one feature per thread
     float *zb = z + (size_t)bh * m;
     float den = 0.f;
-    for (int l = tid; l < m; l += 512) {
+    for (int l = tid; l < m; l += NT) {
         const float zn = zb[l] + fk[l];
         zb[l] = zn;
         den = fmaf(fq[l], zn, den);
     }
     for (int off = 16; off; off >>= 1) den += __shfl_xor_sync(0xffffffffu, den, off);
 
-    // state update and read-out: a thread owns four neighbouring columns of every (512 / (dv / 4))-th row and keeps 16 of
+    // state update and read-out: a thread owns four neighbouring columns of every (NT / (dv / 4))-th row and keeps 16 of
     // its rows (256 bytes) in flight
-    const int tpr = dv / 4, nrg = 512 / tpr, c4 = (tid % tpr) * 4, rg = tid / tpr;
+    const int tpr = dv / 4, nrg = NT / tpr, c4 = (tid % tpr) * 4, rg = tid / tpr;
     float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
     if (rg < nrg) {
         const float4 vv = make_float4(ldf(v, (size_t)kvh * dv + c4), ldf(v, (size_t)kvh * dv + c4 + 1), ldf(v, (size_t)kvh * dv + c4 + 2),
@@ -180,7 +182,7 @@ __global__ void __launch_bounds__(512) decode_step_kernel(const T *q, const T *k
     if (tid < dv) {
         float n = 0.f, dn = 0.f;
         for (int g = 0; g < nrg; ++g) n += red[g * dv + tid];
-        for (int w = 0; w < 16; ++w) dn += red[2048 + w];
+        for (int w = 0; w < NT / 32; ++w) dn += red[2048 + w];
         const float out = n / dn;
         if constexpr (sizeof(T) == 2) o[(size_t)bh * dv + tid] = __float2bfloat16_rn(out);
         else o[(size_t)bh * dv + tid] = out;
@@ -204,13 +206,13 @@ extern "C" darkattn_status_t darkattn_decode_step(darkattn_plan_t plan, const vo
     if (D.dv > 512) return DARKATTN_ERR_UNSUPPORTED;
     const size_t smem = (size_t)(2 * D.d + 2 * D.r + 2 * D.m + 2048 + 16) * sizeof(float);
     if (smem > 48 * 1024) return DARKATTN_ERR_UNSUPPORTED;
-    if (D.bf16)
-        decode_step_kernel<__nv_bfloat16><<<(unsigned)D.BH, 512, smem, st>>>((const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k, (const __nv_bfloat16 *)v,
-                                                                           (const __nv_bfloat16 *)M, (const __nv_bfloat16 *)W, S, z, (__nv_bfloat16 *)o,
-                                                                           D.H, D.Hkv, D.d, D.r, D.m, D.dv, D.w_per_head, D.s);
-    else
-        decode_step_kernel<float><<<(unsigned)D.BH, 512, smem, st>>>((const float *)q, (const float *)k, (const float *)v, (const float *)M,
-                                                                    (const float *)W, S, z, (float *)o, D.H, D.Hkv, D.d, D.r, D.m, D.dv, D.w_per_head, D.s);
+    const bool many = D.BH >= 2 * 148 && D.dv <= 256;      // several blocks per SM: two smaller blocks share one
+#define DARKATTN_DECODE_LAUNCH(T, NT)                                                                                              \
+    decode_step_kernel<T, NT><<<(unsigned)D.BH, NT, smem, st>>>((const T *)q, (const T *)k, (const T *)v, (const T *)M, (const T *)W, S, z, \
+                                                                (T *)o, D.H, D.Hkv, D.d, D.r, D.m, D.dv, D.w_per_head, D.s)
+    if (D.bf16) { if (many) DARKATTN_DECODE_LAUNCH(__nv_bfloat16, 256); else DARKATTN_DECODE_LAUNCH(__nv_bfloat16, 512); }
+    else { if (many) DARKATTN_DECODE_LAUNCH(float, 256); else DARKATTN_DECODE_LAUNCH(float, 512); }
+#undef DARKATTN_DECODE_LAUNCH
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_cuda_error(e, "decode_step"); return DARKATTN_ERR_CUDA; }
     return DARKATTN_OK;
