@@ -72,6 +72,7 @@ struct TensorLayout {
     size_t espart;  // partials of rowsum(E_K) per slab and 32-column group, fp32 [4 nslab, BH, N]
     size_t Tacc;    // sum_i E_i^T x_i over both sides and the batch, fp32 [H, m, d]
     size_t dMn;     // gradient of M through the key norm term, fp32 [H, r, d]
+    size_t dKh, dVh; // grouped key/value heads: dK and dV per query head, bf16 [BH, N, d] and [BH, N, dv], summed over each group in fp32 at the end
     size_t Sst;     // workspace copy of the stash's per-chunk S (causal): bf16 [BH, T, m, dv], S before chunk t (t = 0 not written)
     size_t Ahat;    // causal backward: A^ of every (token, feature), bf16 [BH, N, m] (query-side kernel -> key-side kernel)
     size_t Bphi;    // workspace copy of the stash's key features Bf (causal), bf16 [BH, N, m]: forward scan -> both backward kernels
@@ -187,7 +188,7 @@ cudaError_t tensor_prologue(const darkattn_plan_s *plan, const void *K, const vo
 // dW from what the last backward call left in the workspace
 darkattn_status_t simt_backward_dw(const darkattn_plan_s *plan, float *dW, char *ws, cudaStream_t st);
 cudaError_t tensor_backward_nc_passes(const darkattn_plan_s *plan, const void *Q, const void *K, const void *V, const void *dO,
-                                      const Stash &stash, void *dQ, void *dK, void *dV, char *ws, cudaStream_t st);
+                                      const Stash &stash, void *dQ, void *dK, void *dV, bool per_head, char *ws, cudaStream_t st);
 darkattn_status_t tensor_backward_dw(const darkattn_plan_s *plan, const void *M, float *dW, char *ws, cudaStream_t st);
 darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, const void *K, const void *V,
                                   const void *M, const void *W, const void *O, const void *dO, const void *saved,

@@ -51,7 +51,8 @@ struct BwdParams {
     float *Tacc;          // [H, m, D]
     int *status;
     int N, H, Hkv, BH, m, nslab, T;
-    int add_kv;           // parts of dK and dV are added into the (zeroed) gradients: several slabs, or several query heads per key/value head
+    int add_kv;           // parts of dK and dV are added into the (zeroed) gradients: several slabs
+    int out_per_head;     // grouped key/value heads: dK and dV rows are indexed by the query head (a later kernel sums each group)
 };
 
 template <int D, int DV>
@@ -445,7 +446,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
 
     const int tid = threadIdx.x, warp = tid >> 5;
     const int bh = blockIdx.x / p.nslab, slab = blockIdx.x % p.nslab, h = bh % p.H;
-    const int row0 = bh * p.N, rowk0 = kv_row0(bh, p.H, p.Hkv, p.N), T = p.T;      // rowk0: K, V, dK, dV may be shared by a group of query heads
+    const int row0 = bh * p.N, rowk0 = kv_row0(bh, p.H, p.Hkv, p.N), T = p.T;      // rowk0: K and V may be shared by a group of query heads
+    const int rowo0 = p.out_per_head ? row0 : rowk0;                                 // rows of dK and dV
 
     if (tid == 0) {
         for (int i = 0; i < KE2; ++i) mbar_init(bars + i, 1);
@@ -503,8 +505,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_k_kernel(const __grid_cons
             // A^ of the next chunk can be fetched as soon as dP^T A^ is done, V and dO with it, Bf once E Omega is done.
             auto store_out = [&](const CUtensorMap *map, int width, int t) {     // the staged tile into (or, with several slabs, added into) the gradient
                 for (int a = 0; a < width / 64; ++a) {
-                    if (p.add_kv) tma_reduce_add_2d(map, sStg + a * 16384, a * 64, rowk0 + t * 128);
-                    else tma_store_2d(map, sStg + a * 16384, a * 64, rowk0 + t * 128);
+                    if (p.add_kv) tma_reduce_add_2d(map, sStg + a * 16384, a * 64, rowo0 + t * 128);
+                    else tma_store_2d(map, sStg + a * 16384, a * 64, rowo0 + t * 128);
                 }
                 tma_store_commit();
             };
@@ -698,6 +700,7 @@ struct FinishParams {
     float *dMn;           // [H, r, D]
     int *status;
     int N, H, Hkv, BH, T, nsplit, r, nes;
+    int out_per_head;     // dK rows are indexed by the query head (grouped key/value heads)
     float s2;
 };
 
@@ -831,7 +834,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __gr
             fence_async_smem();
             epi_sync();
             if (tid == 0) {
-                for (int a = 0; a < D / 64; ++a) tma_reduce_add_2d(&p.mapOut, sOut + a * 16384, a * 64, kv_row0(bh, p.H, p.Hkv, p.N) + t * 128);
+                for (int a = 0; a < D / 64; ++a)
+                    tma_reduce_add_2d(&p.mapOut, sOut + a * 16384, a * 64, (p.out_per_head ? bh * p.N : kv_row0(bh, p.H, p.Hkv, p.N)) + t * 128);
                 tma_store_commit();
             }
             tc_fence_before();
@@ -858,6 +862,30 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_finish_k_kernel(const __gr
 }
 
 // ------------------------------------------------------------------ small SIMT kernels
+// Grouped key/value heads: out[(b,hk),i,:] = sum_g src[(b, hk G + g),i,:], added up in fp32 and rounded once; eight
+// elements per thread.
+__global__ void group_sum_kernel(const __nv_bfloat16 *src, __nv_bfloat16 *out, int N, int w, int H, int Hkv, long long total8)
+{
+    const long long t = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+    if (t >= total8) return;
+    const int per_row = w / 8, G = H / Hkv;
+    const int c8 = (int)(t % per_row);
+    const long long row = t / per_row;
+    const int i = (int)(row % N);
+    const long long bhk = row / N, b = bhk / Hkv, hk = bhk % Hkv;
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    for (int g = 0; g < G; ++g) {
+        float x[8];
+        unpack8(*reinterpret_cast<const uint4 *>(src + (((b * H + hk * G + g) * N + i) * (long long)w + c8 * 8)), x);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[j] += x[j];
+    }
+    uint32_t pk[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) pk[j] = __float_as_uint(acc[j]);
+    *reinterpret_cast<uint4 *>(out + t * 8) = pack8(pk);
+}
+
 // delta[row] = dO[row,:] . O[row,:]; dv/8 threads per row, 16 bytes of each tensor per thread.
 __global__ void delta_kernel(const __nv_bfloat16 *G, const __nv_bfloat16 *O, float *delta, long long rows, int dv)
 {
@@ -1021,17 +1049,21 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
     keep(cudaMemsetAsync(ws + Y.Tacc, 0, (size_t)D.H * D.m * D.d * 4, st));
     keep(cudaMemsetAsync(ws + Y.dMn, 0, (size_t)D.H * D.r * D.d * 4, st));
     const size_t BHkv = (size_t)D.B * D.Hkv;
-    const bool add_kv = Y.nslab > 1 || D.G > 1;
+    // Grouped key/value heads: every query head's part of dK and dV goes to rows of its own in the workspace (so that an
+    // element is rounded to bf16 as often as without groups), and a last kernel adds each group up in fp32.
+    const bool per_head = D.G > 1;
+    void *dKo = per_head ? (void *)bf(Y.dKh) : dK, *dVo = per_head ? (void *)bf(Y.dVh) : dV;
+    const size_t BHo = per_head ? BH : BHkv;
+    const bool add_kv = Y.nslab > 1;
     if (add_kv) {
-        // The slabs of a head (and the query heads of a group that shares its keys and values) add their parts into the
-        // gradients, which therefore start at zero. dQ is needed first; dK and dV are zeroed on a side stream while the
-        // query-side scan runs (it leaves SMs and bandwidth free).
+        // The slabs of a head add their parts into the gradients, which therefore start at zero. dQ is needed first; dK and
+        // dV are zeroed on a side stream while the query-side scan runs (it leaves SMs and bandwidth free).
         keep(ensure_aux(plan));
         if (e != cudaSuccess) { set_cuda_error(e, "tensor_backward: side stream"); return DARKATTN_ERR_CUDA; }
         keep(cudaEventRecord(plan->aux_fork, st));
         keep(cudaStreamWaitEvent(plan->aux_stream, plan->aux_fork, 0));
-        keep(cudaMemsetAsync(dK, 0, BHkv * N * D.d * 2, plan->aux_stream));
-        keep(cudaMemsetAsync(dV, 0, BHkv * N * D.dv * 2, plan->aux_stream));
+        keep(cudaMemsetAsync(dKo, 0, BHo * N * D.d * 2, plan->aux_stream));
+        keep(cudaMemsetAsync(dVo, 0, BHo * N * D.dv * 2, plan->aux_stream));
         keep(cudaEventRecord(plan->aux_join, plan->aux_stream));
     }
     if (Y.nslab > 1) keep(cudaMemsetAsync(dQ, 0, BH * N * D.d * 2, st));
@@ -1049,8 +1081,8 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
                         make_map(&P.mapV, V, BHkv * N, D.dv, 128) && make_map(&P.mapG, dO, BH * N, D.dv, 128) &&
                         make_map(&P.mapOm, stash.Om, (size_t)D.H * D.m, D.d, 128) &&
                         make_map(&P.mapOml, stash.Oml, (size_t)D.H * D.m, D.d, 128) &&
-                        make_map(&P.mapDQ, dQ, BH * N, D.d, 128) && make_map(&P.mapDK, dK, BHkv * N, D.d, 128) &&
-                        make_map(&P.mapDV, dV, BHkv * N, D.dv, 128) &&
+                        make_map(&P.mapDQ, dQ, BH * N, D.d, 128) && make_map(&P.mapDK, dKo, BHo * N, D.d, 128) &&
+                        make_map(&P.mapDV, dVo, BHo * N, D.dv, 128) &&
                         make_map(&P.mapAh, bf(Y.Ahat), BH * N, D.m, 128) && make_map(&P.mapBf, stash.Bphi, BH * N, D.m, 128) &&
                         make_map(&P.mapSst, stash.Sst, BH * Y.T * D.m, D.dv, 128);
         if (!ok) { set_cuda_error(cudaErrorInvalidValue, "tensor_backward: tensor map encode"); return DARKATTN_ERR_CUDA; }
@@ -1058,19 +1090,20 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
         P.espart = fl(Y.espart); P.Tacc = fl(Y.Tacc);
         P.status = reinterpret_cast<int *>(ws + Y.status);
         P.N = D.N; P.H = D.H; P.Hkv = D.Hkv; P.BH = D.BH; P.m = D.m; P.nslab = Y.nslab; P.T = Y.T; P.add_kv = add_kv ? 1 : 0;
+        P.out_per_head = per_head ? 1 : 0;
         const int units = (int)(BH * Y.nslab);
         if (D.d == 64 && D.dv == 64) keep(launch_scan<64, 64>(plan, P, units, st));
         else if (D.d == 128 && D.dv == 128) keep(launch_scan<128, 128>(plan, P, units, st));
         else if (D.d == 64 && D.dv == 128) keep(launch_scan<64, 128>(plan, P, units, st));
         else keep(launch_scan<128, 64>(plan, P, units, st));
     } else {
-        keep(tensor_backward_nc_passes(plan, Q, K, V, dO, stash, dQ, dK, dV, ws, st));
+        keep(tensor_backward_nc_passes(plan, Q, K, V, dO, stash, dQ, dKo, dVo, per_head, ws, st));
     }
 
-    if (!make_map(&F.mapOut, dK, BHkv * N, D.d, 128)) { set_cuda_error(cudaErrorInvalidValue, "tensor_backward: tensor map encode"); return DARKATTN_ERR_CUDA; }
+    if (!make_map(&F.mapOut, dKo, BHo * N, D.d, 128)) { set_cuda_error(cudaErrorInvalidValue, "tensor_backward: tensor map encode"); return DARKATTN_ERR_CUDA; }
     F.espart = fl(Y.espart); F.dMn = fl(Y.dMn);
     F.status = reinterpret_cast<int *>(ws + Y.status);
-    F.N = D.N; F.H = D.H; F.Hkv = D.Hkv; F.BH = D.BH; F.T = Y.T; F.r = D.r; F.nes = 4 * Y.nslab; F.s2 = D.s * D.s;
+    F.N = D.N; F.H = D.H; F.Hkv = D.Hkv; F.BH = D.BH; F.T = Y.T; F.r = D.r; F.nes = 4 * Y.nslab; F.s2 = D.s * D.s; F.out_per_head = per_head ? 1 : 0;
     F.nsplit = pick_splits((long long)BH, Y.T, 3.5, 5.0, 64);
     // dM = s W^T T + (norm term). T is complete once the key-side pass is done, so its product runs on the side
     // stream next to the kernel that produces the norm term, and a small kernel adds the two. (With per-kernel
@@ -1098,6 +1131,15 @@ darkattn_status_t tensor_backward(const darkattn_plan_s *plan, const void *Q, co
         timer_mark(plan, st, "dm_kernel");
         keep(cudaMemsetAsync(dM, 0, (size_t)D.H * D.r * D.d * 4, st));
         dm_kernel<<<dm_grid, D.d, 0, st>>>((const __nv_bfloat16 *)W, fl(Y.Tacc), fl(Y.dMn), dM, D.m, D.r, D.d, D.w_per_head, D.s);
+        chk();
+    }
+    if (per_head) {
+        const long long nk = (long long)BHkv * N * D.d / 8, nv = (long long)BHkv * N * D.dv / 8;
+        timer_mark(plan, st, "group_sum_kernel (dK)");
+        group_sum_kernel<<<(unsigned)((nk + 255) / 256), 256, 0, st>>>(bf(Y.dKh), (__nv_bfloat16 *)dK, D.N, D.d, D.H, D.Hkv, nk);
+        chk();
+        timer_mark(plan, st, "group_sum_kernel (dV)");
+        group_sum_kernel<<<(unsigned)((nv + 255) / 256), 256, 0, st>>>(bf(Y.dVh), (__nv_bfloat16 *)dV, D.N, D.dv, D.H, D.Hkv, nv);
         chk();
     }
     if (e != cudaSuccess) { set_cuda_error(e, "tensor_backward"); return DARKATTN_ERR_CUDA; }

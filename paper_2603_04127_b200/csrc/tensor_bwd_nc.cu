@@ -39,7 +39,8 @@ struct NcParams {
     float *Tacc;          // [H, m, D]
     int *status;
     int N, H, Hkv, BH, m, nslab, T, nsplit;
-    int add_kv;           // parts of dK and dV are added into the (zeroed) gradients: several slabs, or several query heads per key/value head
+    int add_kv;           // parts of dK and dV are added into the (zeroed) gradients: several slabs
+    int out_per_head;     // grouped key/value heads: dK and dV rows are indexed by the query head (a later kernel sums each group)
 };
 
 template <int D, int DV>
@@ -89,6 +90,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_nc_kernel(const __grid_con
     const int row0 = bh * p.N;
     // key pass: K, dK (X, Out) and V, dV (Y, DV) may be shared by a group of query heads; query pass: only V has no part in it
     const int rowx0 = KEYS ? kv_row0(bh, p.H, p.Hkv, p.N) : row0, rowy0 = rowx0;
+    const int rowo0 = (KEYS && !p.out_per_head) ? rowx0 : row0;       // rows of the gradient tiles this pass writes
     const int tbeg = (int)((long long)p.T * piece / p.nsplit), tend = (int)((long long)p.T * (piece + 1) / p.nsplit);
     const int nt = tend - tbeg;
 
@@ -151,8 +153,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_nc_kernel(const __grid_con
                 auto store_out = [&](const CUtensorMap *map, unsigned char *src, int width, int tt) {     // (adds into the gradient when the head has several slabs)
                     const bool add = KEYS ? (p.add_kv != 0) : (p.nslab > 1);
                     for (int a = 0; a < width / 64; ++a) {
-                        if (add) tma_reduce_add_2d(map, src + a * 16384, a * 64, rowx0 + tt * 128);
-                        else tma_store_2d(map, src + a * 16384, a * 64, rowx0 + tt * 128);
+                        if (add) tma_reduce_add_2d(map, src + a * 16384, a * 64, rowo0 + tt * 128);
+                        else tma_store_2d(map, src + a * 16384, a * 64, rowo0 + tt * 128);
                     }
                     tma_store_commit();
                 };
@@ -366,9 +368,10 @@ cudaError_t launch_nc(const darkattn_plan_s *plan, const NcParams &PQ, const NcP
 }  // namespace
 
 // The two passes of the non-causal backward. Expects delta computed, Tacc zeroed and (with several
-// slabs) dQ zeroed on `st`, dK and dV zeroed behind plan->aux_join.
+// slabs) dQ zeroed on `st`, dK and dV zeroed behind plan->aux_join. With `per_head`, dK and dV are the per-query-head
+// buffers of grouped key/value heads ([BH, N, *]).
 cudaError_t tensor_backward_nc_passes(const darkattn_plan_s *plan, const void *Q, const void *K, const void *V, const void *dO,
-                                      const Stash &stash, void *dQ, void *dK, void *dV, char *ws, cudaStream_t st)
+                                      const Stash &stash, void *dQ, void *dK, void *dV, bool per_head, char *ws, cudaStream_t st)
 {
     const Dims &D = plan->dims;
     const TensorLayout &Y = plan->tensor;
@@ -382,16 +385,18 @@ cudaError_t tensor_backward_nc_passes(const darkattn_plan_s *plan, const void *Q
     PQ.Racc = fl(Y.Racc); PQ.rhot = fl(Y.rhot); PQ.espart = fl(Y.espart); PQ.Tacc = fl(Y.Tacc);
     PQ.status = reinterpret_cast<int *>(ws + Y.status);
     const size_t BHkv = (size_t)D.B * D.Hkv;
-    const bool add_kv = Y.nslab > 1 || D.G > 1;
+    const bool add_kv = Y.nslab > 1;
+    const size_t BHo = per_head ? BH : BHkv;          // rows of dK and dV (per query head with grouped key/value heads)
+    PQ.out_per_head = per_head ? 1 : 0;
     PQ.N = D.N; PQ.H = D.H; PQ.Hkv = D.Hkv; PQ.BH = D.BH; PQ.m = D.m; PQ.nslab = Y.nslab; PQ.T = Y.T; PQ.add_kv = add_kv ? 1 : 0;
     PQ.nsplit = pick_splits((long long)BH * Y.nslab, Y.T, 3.0, 6.0, 64);
     NcParams PK = PQ;
     const bool ok = make_map(&PQ.mapX, Q, BH * N, D.d, 128) && make_map(&PQ.mapY, dO, BH * N, D.dv, 128) &&
                     make_map(&PQ.mapOm, stash.Om, (size_t)D.H * D.m, D.d, 128) && make_map(&PQ.mapOml, stash.Oml, (size_t)D.H * D.m, D.d, 128) &&
                     make_map(&PQ.mapSt, stash.Sb, BH * D.m, D.dv, 128) &&
-                    make_map(&PQ.mapOut, dQ, BH * N, D.d, 128) && make_map(&PQ.mapDV, dV, BHkv * N, D.dv, 128) &&
+                    make_map(&PQ.mapOut, dQ, BH * N, D.d, 128) && make_map(&PQ.mapDV, dV, BHo * N, D.dv, 128) &&
                     make_map(&PK.mapX, K, BHkv * N, D.d, 128) && make_map(&PK.mapY, V, BHkv * N, D.dv, 128) &&
-                    make_map(&PK.mapSt, Rb, BH * D.m, D.dv, 128) && make_map(&PK.mapOut, dK, BHkv * N, D.d, 128);
+                    make_map(&PK.mapSt, Rb, BH * D.m, D.dv, 128) && make_map(&PK.mapOut, dK, BHo * N, D.d, 128);
     if (!ok) return cudaErrorInvalidValue;
     PK.mapOm = PQ.mapOm;
     PK.mapOml = PQ.mapOml;

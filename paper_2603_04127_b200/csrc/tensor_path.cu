@@ -1188,6 +1188,8 @@ void tensor_make_layout(darkattn_plan_s *plan)
     Y.espart = take(off, (size_t)4 * Y.nslab * BH * N * 4);
     Y.Tacc = take(off, (size_t)D.H * m * d * 4);
     Y.dMn = take(off, (size_t)D.H * D.r * d * 4);
+    Y.dKh = take(off, D.G > 1 ? BH * N * d * 2 : 0);
+    Y.dVh = take(off, D.G > 1 ? BH * N * dv * 2 : 0);
     Y.Sst = take(off, D.causal ? BH * (size_t)Y.T * m * dv * 2 : 0);
     Y.Ahat = take(off, D.causal ? BH * N * m * 2 : 0);
     Y.Bphi = take(off, D.causal ? BH * N * m * 2 : 0);
@@ -1197,7 +1199,7 @@ void tensor_make_layout(darkattn_plan_s *plan)
     // with `saved`; without it the forward launches come on top. Causal: delta, two scan kernels, dK finishing, the
     // dM product and the small kernel that adds the norm term's part; non-causal: one more for the rounding of R
     // between the two passes. (With per-kernel timing on, dM is one kernel.)
-    plan->launches_bwd = D.causal ? 6 : 7;
+    plan->launches_bwd = (D.causal ? 6 : 7) + (D.G > 1 ? 2 : 0);      // (+ the two sums over the groups of query heads)
     Y.total_bytes = off;
     plan->workspace_bytes = Y.total_bytes;
 }

@@ -334,6 +334,9 @@ GROUPED = [
     ("tensor", 4, 1, dict(B=2, N=384, d=64, m=256)),
     ("tensor", 8, 2, dict(B=1, N=256, d=128, m=128, dv=64)),
     ("tensor", 4, 4, dict(B=1, N=256, d=64, m=128)),
+    # four slabs and two query heads per key/value head: eight parts per element of dK and dV. Added straight into the shared
+    # bf16 rows they put dK over the bar; each query head's parts go to rows of its own and the group is summed in fp32
+    ("tensor", 2, 1, dict(B=2, N=384, d=128, m=512, r=48, dv=128)),
 ]
 
 
